@@ -1,0 +1,249 @@
+"""CPU oracle for the SegLinear + DualScale quantized linear layer.
+
+TEST INFRASTRUCTURE ONLY.  This package wraps ``segquant_oracle.c`` (plain C
+loops, gcc) with numpy marshalling.  It shares no code with the CUDA library and
+must never be imported by it; only the test-suite, the smoke check and the
+``cpu_baseline`` / ``--impl reference`` legs of the benchmark may call it.
+
+Every function follows one step of the method, in the paper's order:
+calibration (Sec. 4.3.2 scale formula), weight and activation codes (Sec. 3
+quantizer, Sec. 4.3.2 Q_dual and the polarity split), per-K-segment
+accumulation (Sec. 4.2.2, Sec. 4.3.2), and the dequantizing recombination
+(Sec. 4.3.2 last display, App. A symmetric recovery).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "segquant_oracle.c")
+_LIB = os.path.join(_HERE, "libsegquant_oracle.so")
+
+INT8_QMAX = 127.0      # positive bound of the int8 range
+INT8_QMIN_ABS = 128.0  # magnitude of the negative bound used by the dual quantizer
+E4M3_MAX = 448.0
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (building the checker is not using it)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(
+            ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-o", _LIB, _SRC, "-lm"])
+    return _LIB
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        # SEGQUANT_ORACLE_LIB lets the mutation test load a deliberately broken build of the oracle
+        _lib = C.CDLL(os.environ.get("SEGQUANT_ORACLE_LIB") or build())
+        _lib.sqo_e4m3_decode.restype = C.c_double
+        _lib.sqo_e4m3_decode.argtypes = [C.c_uint8]
+        _lib.sqo_e4m3_encode.restype = C.c_uint8
+        _lib.sqo_e4m3_encode.argtypes = [C.c_float]
+        _lib.sqo_bf16_from_f64.restype = C.c_uint16
+        _lib.sqo_bf16_from_f64.argtypes = [C.c_double]
+        _lib.sqo_accumulate_i8.restype = C.c_int64
+        _lib.sqo_num_threads.restype = C.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().sqo_num_threads())
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _f32(a):
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def _i32(a):
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+@dataclass
+class SegTable:
+    """K-partition kb[0..P] and N-partition nb[0..Q] (Sec. 4.2.2)."""
+    kb: np.ndarray
+    nb: np.ndarray
+
+    def __post_init__(self):
+        self.kb = _i32(self.kb)
+        self.nb = _i32(self.nb)
+
+    @property
+    def P(self):
+        return len(self.kb) - 1
+
+    @property
+    def Q(self):
+        return len(self.nb) - 1
+
+
+# ------------------------------------------------------------------ step 1
+
+def calib_act(X, kb, dual, q_max=INT8_QMAX, q_min_abs=INT8_QMIN_ABS):
+    """Min/max activation scales per K-segment.  Returns (s_pos, s_neg|None)."""
+    X = _f32(X)
+    kb = _i32(kb)
+    P = len(kb) - 1
+    s_pos = np.zeros(P, np.float32)
+    s_neg = np.zeros(P, np.float32)
+    lib().sqo_calib_act(_p(X), C.c_int64(X.shape[0]), C.c_int64(X.shape[1]), C.c_int64(X.shape[1]),
+                        C.c_int(P), _p(kb), C.c_int(int(dual)),
+                        C.c_float(q_max), C.c_float(q_min_abs), _p(s_pos), _p(s_neg))
+    return s_pos, (s_neg if dual else None)
+
+
+def calib_weight(W, kb, nb, w_max=INT8_QMAX):
+    """Abs-max weight scales per (K-segment, N-segment) block, shape [P,Q]."""
+    W = _f32(W)
+    kb, nb = _i32(kb), _i32(nb)
+    P, Q = len(kb) - 1, len(nb) - 1
+    s_w = np.zeros((P, Q), np.float32)
+    lib().sqo_calib_weight(_p(W), C.c_int64(W.shape[0]), C.c_int64(W.shape[1]), C.c_int64(W.shape[1]),
+                           C.c_int(P), _p(kb), C.c_int(Q), _p(nb), C.c_float(w_max), _p(s_w))
+    return s_w
+
+
+# ------------------------------------------------------------- steps 2, 3
+
+def quantize_act(X, kb, s_pos, s_neg=None, code="int8",
+                 q_max=INT8_QMAX, q_min_abs=INT8_QMIN_ABS):
+    """Activation codes.  Dual (s_neg given): returns (c_pos, c_neg); else (c, None)."""
+    X = _f32(X)
+    kb = _i32(kb)
+    M, K = X.shape
+    P = len(kb) - 1
+    s_pos = _f32(s_pos)
+    s_neg = None if s_neg is None else _f32(s_neg)
+    dt = np.int8 if code == "int8" else np.uint8
+    c_pos = np.zeros((M, K), dt)
+    c_neg = np.zeros((M, K), dt) if s_neg is not None else None
+    if code == "int8":
+        lib().sqo_quantize_act_i8(_p(X), C.c_int64(M), C.c_int64(K), C.c_int64(K), C.c_int(P), _p(kb),
+                                  _p(s_pos), _p(s_neg), C.c_float(q_max), C.c_float(q_min_abs),
+                                  _p(c_pos), _p(c_neg), C.c_int64(K))
+    elif code == "e4m3":
+        lib().sqo_quantize_act_e4m3(_p(X), C.c_int64(M), C.c_int64(K), C.c_int64(K), C.c_int(P), _p(kb),
+                                    _p(s_pos), _p(s_neg), _p(c_pos), _p(c_neg), C.c_int64(K))
+    else:
+        raise ValueError(code)
+    return c_pos, c_neg
+
+
+def quantize_weight(W, kb, nb, s_w, code="int8", w_max=INT8_QMAX):
+    W = _f32(W)
+    kb, nb = _i32(kb), _i32(nb)
+    N, K = W.shape
+    P, Q = len(kb) - 1, len(nb) - 1
+    s_w = _f32(s_w).reshape(P, Q)
+    if code == "int8":
+        Wq = np.zeros((N, K), np.int8)
+        lib().sqo_quantize_weight_i8(_p(W), C.c_int64(N), C.c_int64(K), C.c_int64(K), C.c_int(P), _p(kb),
+                                     C.c_int(Q), _p(nb), _p(s_w), C.c_float(w_max), _p(Wq), C.c_int64(K))
+    elif code == "e4m3":
+        Wq = np.zeros((N, K), np.uint8)
+        lib().sqo_quantize_weight_e4m3(_p(W), C.c_int64(N), C.c_int64(K), C.c_int64(K), C.c_int(P), _p(kb),
+                                       C.c_int(Q), _p(nb), _p(s_w), _p(Wq), C.c_int64(K))
+    else:
+        raise ValueError(code)
+    return Wq
+
+
+# ------------------------------------------------------------------ step 4
+
+def accumulate(Xq, Wq, kb, code="int8"):
+    """acc[p,m,n] = sum over K-segment p of Xq[m,k]*Wq[n,k].  int32 (int8 codes) or fp64 (e4m3)."""
+    kb = _i32(kb)
+    P = len(kb) - 1
+    M, K = Xq.shape
+    N = Wq.shape[0]
+    assert Wq.shape[1] == K
+    if code == "int8":
+        Xq = np.ascontiguousarray(Xq, np.int8)
+        Wq = np.ascontiguousarray(Wq, np.int8)
+        acc = np.zeros((P, M, N), np.int32)
+        ovf = lib().sqo_accumulate_i8(_p(Xq), C.c_int64(K), _p(Wq), C.c_int64(K), C.c_int64(M),
+                                      C.c_int64(N), C.c_int64(K), C.c_int(P), _p(kb), _p(acc))
+        if ovf:
+            raise OverflowError(f"{ovf} accumulators exceed int32")
+    else:
+        Xq = np.ascontiguousarray(Xq, np.uint8)
+        Wq = np.ascontiguousarray(Wq, np.uint8)
+        acc = np.zeros((P, M, N), np.float64)
+        lib().sqo_accumulate_e4m3(_p(Xq), C.c_int64(K), _p(Wq), C.c_int64(K), C.c_int64(M),
+                                  C.c_int64(N), C.c_int64(K), C.c_int(P), _p(kb), _p(acc))
+    return acc
+
+
+# ------------------------------------------------------------------ step 5
+
+def dequant(acc_pos, acc_neg, nb, s_pos, s_neg, s_w, bias=None, with_abs=False):
+    """fp64 recombination  sum_p (s_pos s_w acc_pos + s_neg s_w acc_neg) + bias."""
+    nb = _i32(nb)
+    P, M, N = acc_pos.shape
+    Q = len(nb) - 1
+    a_pos = np.ascontiguousarray(acc_pos, np.float64)
+    a_neg = None if acc_neg is None else np.ascontiguousarray(acc_neg, np.float64)
+    s_pos = _f32(s_pos)
+    s_neg = None if s_neg is None else _f32(s_neg)
+    s_w = _f32(s_w).reshape(P, Q)
+    bias = None if bias is None else _f32(bias)
+    y = np.zeros((M, N), np.float64)
+    ya = np.zeros((M, N), np.float64) if with_abs else None
+    lib().sqo_dequant(_p(a_pos), _p(a_neg), C.c_int64(M), C.c_int64(N), C.c_int(P), C.c_int(Q), _p(nb),
+                      _p(s_pos), _p(s_neg), _p(s_w), _p(bias), _p(y), _p(ya))
+    return (y, ya) if with_abs else y
+
+
+def bf16_bits(y64):
+    """Round fp64 values to bf16 (nearest-even, directly from fp64); returns uint16 bit patterns."""
+    y64 = np.ascontiguousarray(y64, np.float64)
+    out = np.zeros(y64.shape, np.uint16)
+    lib().sqo_bf16_from_f64_array(_p(y64), C.c_int64(y64.size), _p(out))
+    return out
+
+
+def e4m3_decode(codes):
+    lut = np.array([lib().sqo_e4m3_decode(c) for c in range(256)], np.float64)
+    return lut[np.asarray(codes, np.uint8)]
+
+
+def e4m3_encode(values):
+    v = _f32(values)
+    f = lib().sqo_e4m3_encode
+    return np.array([f(float(x)) for x in v.ravel()], np.uint8).reshape(v.shape)
+
+
+# ----------------------------------------------------------- whole layer
+
+@dataclass
+class LayerResult:
+    c_pos: np.ndarray
+    c_neg: np.ndarray | None
+    acc_pos: np.ndarray
+    acc_neg: np.ndarray | None
+    y64: np.ndarray
+    y_abs: np.ndarray
+
+
+def layer_forward(X, Wq, seg: SegTable, s_pos, s_neg, s_w, bias=None, code="int8",
+                  q_max=INT8_QMAX, q_min_abs=INT8_QMIN_ABS) -> LayerResult:
+    """Steps 3-5 for one layer (weights already quantized)."""
+    c_pos, c_neg = quantize_act(X, seg.kb, s_pos, s_neg, code, q_max, q_min_abs)
+    acc_pos = accumulate(c_pos, Wq, seg.kb, code)
+    acc_neg = accumulate(c_neg, Wq, seg.kb, code) if c_neg is not None else None
+    y64, y_abs = dequant(acc_pos, acc_neg, seg.nb, s_pos, s_neg, s_w, bias, with_abs=True)
+    return LayerResult(c_pos, c_neg, acc_pos, acc_neg, y64, y_abs)
