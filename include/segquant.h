@@ -1,0 +1,176 @@
+/*
+ * segquant.h -- C ABI of the B200 (sm_100a) SegLinear + DualScale W8A8 linear layer.
+ *
+ * The layer computes  Y = X W^T + b  with 8-bit codes:
+ *   SegLinear (Sec. 4.2.2): the K axis (input-segmented mode, fed by a concat / stack /
+ *   reshape) and the N axis (output-segmented mode, consumed by a chunk / split) are
+ *   partitioned into segments and every segment is quantized with its own scale.
+ *   DualScale (Sec. 4.3.2): a polarity-asymmetric activation is split into
+ *   X_+ = max(X,0) and X_- = min(X,0), each quantized with its own scale s_+ / s_-,
+ *   both multiplied with the same quantized weight and recombined as
+ *   s_+ s_w (X^_+ W^) + s_- s_w (X^_- W^).
+ *
+ * Conventions for every entry point
+ *   - Matrices are row-major with an explicit leading dimension in ELEMENTS.
+ *     X [M,K] activations, W [N,K] weights (nn.Linear order), Y [M,N].
+ *   - "dev" pointers are CUDA device pointers of the current device, "host" pointers are
+ *     ordinary host memory that is only read during the call.
+ *   - The caller owns every buffer.  The library allocates no device memory and keeps no
+ *     state between calls other than cached driver entry points and per-device attributes.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream) and return without synchronizing, except segquant_last_device_status.
+ *   - Every entry point returns an sq_status.  Anything checkable on the host is rejected
+ *     before any launch; nothing aborts or throws.  There is no CPU fallback.
+ */
+#ifndef SEGQUANT_H_
+#define SEGQUANT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SQ_OK = 0,
+    SQ_ERR_NULL = 1,        /* a required pointer is NULL */
+    SQ_ERR_SHAPE = 2,       /* M/N/K/ld out of range (<= 0, ld < extent, K too large for int32 sums) */
+    SQ_ERR_SEGTABLE = 3,    /* segment bounds not ascending / not starting at 0 / not ending at K or N */
+    SQ_ERR_ALIGN = 4,       /* pointer, leading dimension or segment bound violates an alignment rule */
+    SQ_ERR_UNSUPPORTED = 5, /* unknown code / dtype, or more segments than the kernels support */
+    SQ_ERR_CUDA = 6,        /* a CUDA runtime / driver call failed (launch, tensor-map encode, ...) */
+    SQ_ERR_TIMEOUT = 7,     /* a bounded device-side wait expired (read back by segquant_last_device_status) */
+    SQ_ERR_WORKSPACE = 8    /* workspace NULL or smaller than segquant_workspace_bytes() */
+} sq_status;
+
+typedef enum { SQ_CODE_INT8 = 0, SQ_CODE_E4M3 = 1 } sq_code;   /* 8-bit code type */
+typedef enum { SQ_F32 = 0, SQ_BF16 = 1 } sq_dtype;             /* real-valued element type */
+
+/* flags */
+#define SQ_FLAG_QMIN_SYM 1u  /* int8 DualScale: clamp the negative path to -127 instead of -128 */
+
+/* limits */
+#define SQ_MAX_P 16   /* K-segments per layer */
+#define SQ_MAX_Q 64   /* N-segments per layer */
+
+/* Segment table (the output of the paper's graph pattern detection, App. B Alg. 1):
+ * K-partition kb[0..P] with kb[0]=0, kb[P]=K and N-partition nb[0..Q] with nb[0]=0, nb[Q]=N,
+ * both strictly ascending, in HOST memory (copied during the call). */
+typedef struct {
+    int32_t P;
+    const int32_t *kb;
+    int32_t Q;
+    const int32_t *nb;
+} sq_segtable;
+
+/* Bytes of device scratch every call below accepts as `workspace` (a small constant; it holds
+ * device status words and reduction partials).  The buffer must be 256-byte aligned and zero-filled
+ * once by the caller after allocating it.  Two calls that may run concurrently need two workspaces. */
+size_t segquant_workspace_bytes(void);
+
+/* Step "calibration" -- Sec. 4.3.2 scale formula (s_- = |min x| / |q_min|, s_+ = max x / q_max),
+ * strict min/max (App. B, Dual Scale Sensitivity Analysis), one scalar per segment (App. B,
+ * per-tensor 8-bit scheme; Sec. 4.2.2 "independently within each segment").
+ *   is_weight = 0: X is a calibration batch [rows,K] (dev, dtype dt, leading dimension ld).
+ *       dual != 0: s_pos[p] = max(max x,0)/q_max and s_neg[p] = max(-min x,0)/|q_min| per K-segment p.
+ *       dual == 0: s_pos[p] = max|x|/q_max; s_neg is ignored (may be NULL).
+ *   is_weight = 1: X is the weight matrix [rows=N,K]; s_pos[p*Q+q] = max|W block(p,q)|/q_max.
+ *   q_max = 127 (int8) or 448 (e4m3); |q_min| = 128 (int8; 127 with SQ_FLAG_QMIN_SYM) or 448.
+ *   A segment whose extremum is 0 gets scale 1.  Inputs must be finite.
+ *   s_pos / s_neg: dev float arrays written by the call.  Alignment: X 16 bytes, ld*sizeof(dt)
+ *   a multiple of 16 bytes. */
+sq_status segquant_calib_scales(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld,
+                                const sq_segtable *seg, sq_code code, int is_weight, int dual,
+                                uint32_t flags, float *s_pos, float *s_neg,
+                                void *workspace, size_t ws_bytes, void *stream);
+
+/* Step "activation quantization" -- Sec. 4.3.2 Q_dual with the polarity split X_+ / X_-, plus the
+ * clip of the Sec. 3 uniform quantizer; x/s is one IEEE fp32 division, rounding is half-to-even.
+ *   s_neg != NULL (dual): x >= 0 -> c_pos = clip(round(x/s_pos[p]), 0, q_max), c_neg = 0;
+ *                         x <  0 -> c_neg = clip(round(x/s_neg[p]), q_min, 0), c_pos = 0.
+ *   s_neg == NULL (single scale): c_pos = clip(round(x/s_pos[p]), -q_max, q_max); c_neg unused.
+ *   e4m3 codes: "round" is the round-to-nearest-even cast to e4m3 (finite, max 448, subnormals
+ *   kept), saturating; a result of -0 is stored as +0.
+ *   X [M,K] dev (dtype dt, ld elements); c_pos, c_neg [M,K] dev, 1 byte per code, leading dimension
+ *   ldc bytes.  Alignment: X, c_pos, c_neg 16 bytes; ld*sizeof(dt) and ldc multiples of 16 bytes. */
+sq_status segquant_quantize_act(const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld,
+                                const sq_segtable *seg, const float *s_pos, const float *s_neg,
+                                sq_code code, uint32_t flags, void *c_pos, void *c_neg, int64_t ldc,
+                                void *stream);
+
+/* Step "weight quantization" (offline) -- Sec. 4.2.2: every block W(p,q) is quantized separately,
+ * W^ = clip(round(W / s_w[p*Q+q]), -q_max, q_max) (App. A symmetric case).
+ *   W [N,K] dev (dtype dt, ld elements); s_w dev [P*Q]; Wq [N,K] dev codes, leading dimension ldq bytes. */
+sq_status segquant_quantize_weight(const void *W, sq_dtype dt, int64_t N, int64_t K, int64_t ld,
+                                   const sq_segtable *seg, const float *s_w, sq_code code,
+                                   uint32_t flags, void *Wq, int64_t ldq, void *stream);
+
+/* Steps "low-bit GEMM" + "dequantizing epilogue", single activation scale per K-segment --
+ * Sec. 4.2.2 (output-segmented: Y^ = [X^ W^_1, ..., X^ W^_N]; input-segmented: Y^ = sum_i X^_i W^_i)
+ * with the App. A symmetric recovery Y = s_X s_W Y^ applied per segment pair:
+ *   y[m][n] = sum_p s_x[p] * s_w[p*Q+q(n)] * acc[p][m][n] + bias[n],
+ *   acc[p][m][n] = sum_{k in K-segment p} Xq[m][k] * Wq[n][k]   (int32 for int8 codes, exact;
+ *   fp32 tensor-core accumulation for e4m3 codes).
+ *   Xq [M,K], Wq [N,K] dev codes (ldx, ldw in bytes); s_x dev [P]; s_w dev [P*Q]; bias dev [N] fp32 or
+ *   NULL; Y [M,N] dev of y_dtype (bf16 round-to-nearest-even, or fp32), ldy in elements.
+ *   acc_dump: NULL, or a dev buffer [P][M][N] (int32 for int8, fp32 for e4m3) that receives the raw
+ *   accumulators (used by parity tests).
+ *   Alignment: Xq, Wq, Y 16 bytes; ldx, ldw multiples of 16; ldy*sizeof(y_dtype) a multiple of 16;
+ *   N a multiple of 8; interior K-segment bounds multiples of 32, K a multiple of 16.
+ *   Limits: P <= SQ_MAX_P, Q <= SQ_MAX_Q, K <= 131072 (int8: |acc| stays below 2^31).
+ *   The epilogue multiplies c = s_x*s_w in fp32 and accumulates with fp32 FMAs in ascending p. */
+sq_status segquant_seglinear_gemm(const void *Xq, int64_t ldx, const void *Wq, int64_t ldw,
+                                  int64_t M, int64_t N, int64_t K, const sq_segtable *seg, sq_code code,
+                                  const float *s_x, const float *s_w, const float *bias,
+                                  void *Y, sq_dtype y_dtype, int64_t ldy, void *acc_dump,
+                                  void *workspace, size_t ws_bytes, void *stream);
+
+/* The same two steps for a DualScale layer -- Sec. 4.3.2 last display, combined with segments:
+ *   y[m][n] = sum_p ( s_pos[p]*s_w[p*Q+q(n)]*acc_pos[p][m][n] + s_neg[p]*s_w[p*Q+q(n)]*acc_neg[p][m][n] ) + bias[n]
+ *   where acc_pos / acc_neg are the contractions of Xq_pos / Xq_neg with the SAME weight tile.
+ *   acc_dump (optional): [P][2][M][N], polarity 0 = positive path.
+ *   A layer needs P*2 accumulators of the tile width in tensor memory: P <= 8 here. */
+sq_status segquant_dualscale_gemm(const void *Xq_pos, const void *Xq_neg, int64_t ldx,
+                                  const void *Wq, int64_t ldw, int64_t M, int64_t N, int64_t K,
+                                  const sq_segtable *seg, sq_code code,
+                                  const float *s_pos, const float *s_neg, const float *s_w,
+                                  const float *bias, void *Y, sq_dtype y_dtype, int64_t ldy,
+                                  void *acc_dump, void *workspace, size_t ws_bytes, void *stream);
+
+/* Bytes of device scratch segquant_layer_forward needs for the code matrices of an [M,K] input. */
+size_t segquant_layer_scratch_bytes(int64_t M, int64_t K, int dual);
+
+/* The whole per-call path of one layer -- quantize (Sec. 4.3.2 Q_dual) -> GEMM -> epilogue -- as
+ * one call: X [M,K] of dtype dt in -> Y [M,N] out.  s_neg == NULL selects the single-scale layer.
+ *   x_on_host / y_on_host != 0: X / Y are HOST buffers (pinned memory recommended); the call copies
+ *   X to `x_stage` (dev, M*ld*sizeof(dt) bytes) before and Y from `y_stage` (dev, M*ldy*sizeof(y_dtype)
+ *   bytes) after the kernels, on `stream`.  With device X / Y the stage pointers are ignored.
+ *   scratch: dev, segquant_layer_scratch_bytes(M,K,dual) bytes, 256-byte aligned (code matrices). */
+sq_status segquant_layer_forward(const void *X, int x_on_host, void *x_stage, sq_dtype dt,
+                                 int64_t M, int64_t K, int64_t ld,
+                                 const void *Wq, int64_t ldw, int64_t N, const sq_segtable *seg, sq_code code,
+                                 const float *s_pos, const float *s_neg, const float *s_w, const float *bias,
+                                 uint32_t flags, void *Y, int y_on_host, void *y_stage, sq_dtype y_dtype, int64_t ldy,
+                                 void *scratch, size_t scratch_bytes,
+                                 void *workspace, size_t ws_bytes, void *stream);
+
+/* Synchronizes `stream`, reads the device status word of `workspace` and clears it.  Returns SQ_OK,
+ * SQ_ERR_TIMEOUT (a bounded wait inside a kernel expired; *detail, if not NULL, receives a code that
+ * names the wait) or SQ_ERR_CUDA. */
+sq_status segquant_last_device_status(void *workspace, void *stream, uint32_t *detail);
+
+/* Tile plan of the GEMM kernel: tile_n in {0 (automatic), 32, 64, 128, 256}; stages 0 (automatic) or
+ * 2..8.  Process-wide; meant for benchmarking sweeps.  Values the layer cannot use are replaced by
+ * the automatic choice. */
+sq_status segquant_set_tuning(int tile_n, int stages);
+
+/* Number of kernels the library has launched in this process (all entry points). */
+uint64_t segquant_launch_count(void);
+
+const char *segquant_status_string(sq_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SEGQUANT_H_ */

@@ -1,0 +1,242 @@
+"""Thin ctypes binding over libsegquant.so: argument marshalling only.
+
+Function names mirror the C ABI (include/segquant.h).  Tensors are torch CUDA tensors used as
+device memory; every step of the path runs inside the library's kernels.  There is no fallback:
+if the library is missing or a call returns an error status, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsegquant.so")
+
+SQ_OK = 0
+SQ_CODE = {"int8": 0, "e4m3": 1}
+SQ_F32, SQ_BF16 = 0, 1
+SQ_FLAG_QMIN_SYM = 1
+STATUS_NAMES = {0: "SQ_OK", 1: "SQ_ERR_NULL", 2: "SQ_ERR_SHAPE", 3: "SQ_ERR_SEGTABLE", 4: "SQ_ERR_ALIGN",
+                5: "SQ_ERR_UNSUPPORTED", 6: "SQ_ERR_CUDA", 7: "SQ_ERR_TIMEOUT", 8: "SQ_ERR_WORKSPACE"}
+
+EXPORTS = [
+    "segquant_workspace_bytes", "segquant_calib_scales", "segquant_quantize_act", "segquant_quantize_weight",
+    "segquant_seglinear_gemm", "segquant_dualscale_gemm", "segquant_layer_scratch_bytes",
+    "segquant_layer_forward", "segquant_last_device_status", "segquant_set_tuning", "segquant_launch_count",
+    "segquant_status_string",
+]
+
+
+class SegquantError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}")
+
+
+class _SegTable(C.Structure):
+    _fields_ = [("P", C.c_int32), ("kb", C.POINTER(C.c_int32)), ("Q", C.c_int32), ("nb", C.POINTER(C.c_int32))]
+
+
+_lib = None
+
+
+def lib():
+    """Loads the shared library; raises if it has not been built (no silent fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} not found: build it with `python -m paper_2507_14811_b200.build`")
+        L = C.CDLL(LIB_PATH)
+        L.segquant_workspace_bytes.restype = C.c_size_t
+        L.segquant_layer_scratch_bytes.restype = C.c_size_t
+        L.segquant_layer_scratch_bytes.argtypes = [C.c_int64, C.c_int64, C.c_int]
+        L.segquant_launch_count.restype = C.c_uint64
+        L.segquant_status_string.restype = C.c_char_p
+        L.segquant_status_string.argtypes = [C.c_int]
+        _lib = L
+    return _lib
+
+
+class SegTable:
+    """Host-side segment table: kb[0..P], nb[0..Q]."""
+
+    def __init__(self, kb, nb):
+        self.kb = np.ascontiguousarray(kb, np.int32)
+        self.nb = np.ascontiguousarray(nb, np.int32)
+        self._c = _SegTable(len(self.kb) - 1, self.kb.ctypes.data_as(C.POINTER(C.c_int32)),
+                            len(self.nb) - 1, self.nb.ctypes.data_as(C.POINTER(C.c_int32)))
+
+    @property
+    def P(self):
+        return len(self.kb) - 1
+
+    @property
+    def Q(self):
+        return len(self.nb) - 1
+
+    def ref(self):
+        return C.byref(self._c)
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return SQ_F32
+    if t.dtype == torch.bfloat16:
+        return SQ_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _ptr(t):
+    return C.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(status, where):
+    if status != SQ_OK:
+        raise SegquantError(status, where)
+
+
+def workspace_bytes() -> int:
+    return int(lib().segquant_workspace_bytes())
+
+
+def new_workspace(device="cuda") -> torch.Tensor:
+    """Zero-filled, 256-byte aligned device scratch for the calls below."""
+    return torch.zeros(workspace_bytes(), dtype=torch.uint8, device=device)
+
+
+def segquant_calib_scales(X: torch.Tensor, seg: SegTable, code: str, is_weight: bool, dual: bool,
+                          workspace: torch.Tensor, flags: int = 0):
+    """Returns (s_pos, s_neg|None) for activations, (s_w [P*Q], None) for weights."""
+    rows, K = X.shape
+    n = seg.P * (seg.Q if is_weight else 1)
+    s_pos = torch.empty(n, dtype=torch.float32, device=X.device)
+    s_neg = torch.empty(n, dtype=torch.float32, device=X.device) if (dual and not is_weight) else None
+    st = lib().segquant_calib_scales(_ptr(X), C.c_int(_dt(X)), C.c_int64(rows), C.c_int64(K), C.c_int64(X.stride(0)),
+                                     seg.ref(), C.c_int(SQ_CODE[code]), C.c_int(int(is_weight)), C.c_int(int(dual)),
+                                     C.c_uint32(flags), _ptr(s_pos), _ptr(s_neg), _ptr(workspace),
+                                     C.c_size_t(workspace.numel()), _stream())
+    _check(st, "segquant_calib_scales")
+    return s_pos, s_neg
+
+
+def _ldc(K: int) -> int:
+    return (K + 127) // 128 * 128
+
+
+def new_codes(M: int, K: int, device) -> torch.Tensor:
+    """Code matrix [M,K] with a 128-byte padded row pitch (view of a [M, ldc] buffer)."""
+    return torch.empty((M, _ldc(K)), dtype=torch.uint8, device=device)[:, :K]
+
+
+def segquant_quantize_act(X: torch.Tensor, seg: SegTable, s_pos, s_neg, code: str, flags: int = 0,
+                          c_pos=None, c_neg=None):
+    M, K = X.shape
+    if c_pos is None:
+        c_pos = new_codes(M, K, X.device)
+    if s_neg is not None and c_neg is None:
+        c_neg = new_codes(M, K, X.device)
+    st = lib().segquant_quantize_act(_ptr(X), C.c_int(_dt(X)), C.c_int64(M), C.c_int64(K), C.c_int64(X.stride(0)),
+                                     seg.ref(), _ptr(s_pos), _ptr(s_neg), C.c_int(SQ_CODE[code]), C.c_uint32(flags),
+                                     _ptr(c_pos), _ptr(c_neg), C.c_int64(c_pos.stride(0)), _stream())
+    _check(st, "segquant_quantize_act")
+    return c_pos, (c_neg if s_neg is not None else None)
+
+
+def segquant_quantize_weight(W: torch.Tensor, seg: SegTable, s_w, code: str, flags: int = 0, Wq=None):
+    N, K = W.shape
+    if Wq is None:
+        Wq = new_codes(N, K, W.device)
+    st = lib().segquant_quantize_weight(_ptr(W), C.c_int(_dt(W)), C.c_int64(N), C.c_int64(K), C.c_int64(W.stride(0)),
+                                        seg.ref(), _ptr(s_w), C.c_int(SQ_CODE[code]), C.c_uint32(flags),
+                                        _ptr(Wq), C.c_int64(Wq.stride(0)), _stream())
+    _check(st, "segquant_quantize_weight")
+    return Wq
+
+
+def _new_y(M, N, y_dtype, device):
+    return torch.empty((M, N), dtype=y_dtype, device=device)
+
+
+def _new_dump(nacc, M, N, code, device):
+    return torch.zeros((nacc, M, N), dtype=torch.int32 if code == "int8" else torch.float32, device=device)
+
+
+def segquant_seglinear_gemm(Xq, Wq, seg: SegTable, code: str, s_x, s_w, bias, workspace,
+                            y_dtype=torch.bfloat16, Y=None, dump_acc=False):
+    M, K = Xq.shape
+    N = Wq.shape[0]
+    if Y is None:
+        Y = _new_y(M, N, y_dtype, Xq.device)
+    dump = _new_dump(seg.P, M, N, code, Xq.device) if dump_acc else None
+    st = lib().segquant_seglinear_gemm(_ptr(Xq), C.c_int64(Xq.stride(0)), _ptr(Wq), C.c_int64(Wq.stride(0)),
+                                       C.c_int64(M), C.c_int64(N), C.c_int64(K), seg.ref(), C.c_int(SQ_CODE[code]),
+                                       _ptr(s_x), _ptr(s_w), _ptr(bias), _ptr(Y), C.c_int(_dt(Y)),
+                                       C.c_int64(Y.stride(0)), _ptr(dump), _ptr(workspace),
+                                       C.c_size_t(workspace.numel()), _stream())
+    _check(st, "segquant_seglinear_gemm")
+    return (Y, dump) if dump_acc else Y
+
+
+def segquant_dualscale_gemm(Xq_pos, Xq_neg, Wq, seg: SegTable, code: str, s_pos, s_neg, s_w, bias, workspace,
+                            y_dtype=torch.bfloat16, Y=None, dump_acc=False):
+    M, K = Xq_pos.shape
+    N = Wq.shape[0]
+    assert Xq_neg.stride(0) == Xq_pos.stride(0)
+    if Y is None:
+        Y = _new_y(M, N, y_dtype, Xq_pos.device)
+    dump = _new_dump(seg.P * 2, M, N, code, Xq_pos.device) if dump_acc else None
+    st = lib().segquant_dualscale_gemm(_ptr(Xq_pos), _ptr(Xq_neg), C.c_int64(Xq_pos.stride(0)), _ptr(Wq),
+                                       C.c_int64(Wq.stride(0)), C.c_int64(M), C.c_int64(N), C.c_int64(K), seg.ref(),
+                                       C.c_int(SQ_CODE[code]), _ptr(s_pos), _ptr(s_neg), _ptr(s_w), _ptr(bias),
+                                       _ptr(Y), C.c_int(_dt(Y)), C.c_int64(Y.stride(0)), _ptr(dump), _ptr(workspace),
+                                       C.c_size_t(workspace.numel()), _stream())
+    _check(st, "segquant_dualscale_gemm")
+    return (Y, dump) if dump_acc else Y
+
+
+def layer_scratch_bytes(M: int, K: int, dual: bool) -> int:
+    return int(lib().segquant_layer_scratch_bytes(M, K, int(dual)))
+
+
+def segquant_layer_forward(X, Wq, seg: SegTable, code: str, s_pos, s_neg, s_w, bias, Y, scratch, workspace,
+                           x_stage=None, y_stage=None, flags: int = 0):
+    """Quantize -> GEMM -> epilogue in one call.  X / Y may be (pinned) host tensors, in which case
+    x_stage / y_stage are device buffers of the same shape and the copies are part of the call."""
+    M, K = X.shape
+    N = Wq.shape[0]
+    x_host, y_host = not X.is_cuda, not Y.is_cuda
+    st = lib().segquant_layer_forward(
+        _ptr(X), C.c_int(int(x_host)), _ptr(x_stage), C.c_int(_dt(X)), C.c_int64(M), C.c_int64(K),
+        C.c_int64(X.stride(0)), _ptr(Wq), C.c_int64(Wq.stride(0)), C.c_int64(N), seg.ref(), C.c_int(SQ_CODE[code]),
+        _ptr(s_pos), _ptr(s_neg), _ptr(s_w), _ptr(bias), C.c_uint32(flags), _ptr(Y), C.c_int(int(y_host)),
+        _ptr(y_stage), C.c_int(_dt(Y)), C.c_int64(Y.stride(0)), _ptr(scratch), C.c_size_t(scratch.numel()),
+        _ptr(workspace), C.c_size_t(workspace.numel()), _stream())
+    _check(st, "segquant_layer_forward")
+    return Y
+
+
+def segquant_last_device_status(workspace) -> tuple[int, int]:
+    detail = C.c_uint32(0)
+    st = lib().segquant_last_device_status(_ptr(workspace), _stream(), C.byref(detail))
+    return int(st), int(detail.value)
+
+
+def check_device_status(workspace):
+    st, detail = segquant_last_device_status(workspace)
+    if st != SQ_OK:
+        raise SegquantError(st, f"device status (detail 0x{detail:x})")
+
+
+def segquant_set_tuning(tile_n: int = 0, stages: int = 0):
+    _check(lib().segquant_set_tuning(C.c_int(tile_n), C.c_int(stages)), "segquant_set_tuning")
+
+
+def segquant_launch_count() -> int:
+    return int(lib().segquant_launch_count())

@@ -1,0 +1,247 @@
+// C ABI: host-side validation and dispatch.  Every argument error is reported before any launch.
+#include <atomic>
+#include "sq_common.cuh"
+
+namespace sq {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(uint64_t(n), std::memory_order_relaxed); }
+
+HostSeg load_segtable(const sq_segtable *seg, int64_t K, int64_t N)
+{
+    HostSeg h{};
+    h.status = SQ_OK;
+    if (!seg || !seg->kb || !seg->nb) { h.status = SQ_ERR_NULL; return h; }
+    if (seg->P < 1 || seg->Q < 1) { h.status = SQ_ERR_SEGTABLE; return h; }
+    if (seg->P > SQ_MAX_P || seg->Q > SQ_MAX_Q) { h.status = SQ_ERR_UNSUPPORTED; return h; }
+    h.b.P = seg->P;
+    h.b.Q = seg->Q;
+    for (int i = 0; i <= seg->P; i++) h.b.kb[i] = seg->kb[i];
+    for (int i = 0; i <= seg->Q; i++) h.b.nb[i] = seg->nb[i];
+    if (h.b.kb[0] != 0 || h.b.kb[seg->P] != K || h.b.nb[0] != 0 || h.b.nb[seg->Q] != N) {
+        h.status = SQ_ERR_SEGTABLE;
+        return h;
+    }
+    for (int i = 0; i < seg->P; i++)
+        if (h.b.kb[i + 1] <= h.b.kb[i]) { h.status = SQ_ERR_SEGTABLE; return h; }
+    for (int i = 0; i < seg->Q; i++)
+        if (h.b.nb[i + 1] <= h.b.nb[i]) { h.status = SQ_ERR_SEGTABLE; return h; }
+    return h;
+}
+
+static size_t dt_size(sq_dtype dt) { return dt == SQ_F32 ? 4 : 2; }
+static bool valid_dt(sq_dtype dt) { return dt == SQ_F32 || dt == SQ_BF16; }
+static bool valid_code(sq_code c) { return c == SQ_CODE_INT8 || c == SQ_CODE_E4M3; }
+constexpr int64_t kMaxDim = 1 << 30;
+constexpr int64_t kMaxK = 131072;   // int8: 131072 * 128 * 127 < 2^31
+
+static sq_status check_ws(void *ws, size_t bytes)
+{
+    if (!ws || bytes < kWsBytes) return SQ_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(ws) & 255u) return SQ_ERR_ALIGN;
+    return SQ_OK;
+}
+
+static sq_status check_matrix(const void *p, int64_t rows, int64_t cols, int64_t ld, size_t elem)
+{
+    if (!p) return SQ_ERR_NULL;
+    if (rows <= 0 || cols <= 0 || rows > kMaxDim || cols > kMaxDim || ld < cols) return SQ_ERR_SHAPE;
+    if (!aligned16(p) || (size_t(ld) * elem) % 16 != 0) return SQ_ERR_ALIGN;
+    return SQ_OK;
+}
+
+static sq_status gemm_common(const void *a_pos, const void *a_neg, int dual, int64_t ldx, const void *Wq, int64_t ldw,
+                             int64_t M, int64_t N, int64_t K, const sq_segtable *seg, sq_code code,
+                             const float *s_pos, const float *s_neg, const float *s_w, const float *bias, void *Y,
+                             sq_dtype y_dtype, int64_t ldy, void *acc_dump, void *workspace, size_t ws_bytes,
+                             void *stream)
+{
+    if (!s_pos || !s_w || (dual && (!a_neg || !s_neg))) return SQ_ERR_NULL;
+    if (!valid_code(code) || !valid_dt(y_dtype)) return SQ_ERR_UNSUPPORTED;
+    sq_status st;
+    if ((st = check_matrix(a_pos, M, K, ldx, 1)) != SQ_OK) return st;
+    if (dual && (st = check_matrix(a_neg, M, K, ldx, 1)) != SQ_OK) return st;
+    if ((st = check_matrix(Wq, N, K, ldw, 1)) != SQ_OK) return st;
+    if ((st = check_matrix(Y, M, N, ldy, dt_size(y_dtype))) != SQ_OK) return st;
+    if (K > kMaxK) return SQ_ERR_SHAPE;
+    if (K % 16 != 0 || N % 8 != 0) return SQ_ERR_ALIGN;
+    if (acc_dump && !aligned16(acc_dump)) return SQ_ERR_ALIGN;
+    HostSeg hs = load_segtable(seg, K, N);
+    if (hs.status != SQ_OK) return hs.status;
+    for (int p = 1; p < hs.b.P; p++)
+        if (hs.b.kb[p] % 32 != 0) return SQ_ERR_ALIGN;
+    if (hs.b.P * (dual ? 2 : 1) > 16) return SQ_ERR_UNSUPPORTED;   // accumulators of >= 32 columns in 512
+    if ((st = check_ws(workspace, ws_bytes)) != SQ_OK) return st;
+
+    GemmArgs g{};
+    g.a_pos = a_pos; g.a_neg = dual ? a_neg : nullptr; g.lda = ldx;
+    g.b = Wq; g.ldb = ldw;
+    g.M = M; g.N = N; g.K = K;
+    g.sb = hs.b;
+    g.code = code;
+    g.s_pos = s_pos; g.s_neg = dual ? s_neg : nullptr; g.s_w = s_w; g.bias = bias;
+    g.Y = Y; g.y_dtype = y_dtype; g.ldy = ldy;
+    g.acc_dump = acc_dump;
+    g.status = static_cast<uint32_t *>(workspace);
+    return launch_gemm(g, static_cast<cudaStream_t>(stream));
+}
+
+}  // namespace sq
+
+using namespace sq;
+
+extern "C" {
+
+size_t segquant_workspace_bytes(void) { return kWsBytes; }
+
+sq_status segquant_calib_scales(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld,
+                                const sq_segtable *seg, sq_code code, int is_weight, int dual, uint32_t flags,
+                                float *s_pos, float *s_neg, void *workspace, size_t ws_bytes, void *stream)
+{
+    if (!s_pos || (!is_weight && dual && !s_neg)) return SQ_ERR_NULL;
+    if (!valid_dt(dt) || !valid_code(code)) return SQ_ERR_UNSUPPORTED;
+    sq_status st = check_matrix(X, rows, K, ld, dt_size(dt));
+    if (st != SQ_OK) return st;
+    HostSeg hs = load_segtable(seg, K, is_weight ? rows : (seg && seg->nb && seg->Q >= 1 ? seg->nb[seg->Q] : 0));
+    if (hs.status != SQ_OK) return hs.status;
+    if ((st = check_ws(workspace, ws_bytes)) != SQ_OK) return st;
+    uint32_t *partials = reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(workspace) + kWsStatusBytes);
+    return launch_calib(X, dt, rows, K, ld, hs.b, is_weight, dual, code_qmax(code), code_qmin_abs(code, flags),
+                        s_pos, s_neg, partials, static_cast<cudaStream_t>(stream));
+}
+
+sq_status segquant_quantize_act(const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld,
+                                const sq_segtable *seg, const float *s_pos, const float *s_neg, sq_code code,
+                                uint32_t flags, void *c_pos, void *c_neg, int64_t ldc, void *stream)
+{
+    if (!s_pos || (s_neg && !c_neg)) return SQ_ERR_NULL;
+    if (!valid_dt(dt) || !valid_code(code)) return SQ_ERR_UNSUPPORTED;
+    sq_status st;
+    if ((st = check_matrix(X, M, K, ld, dt_size(dt))) != SQ_OK) return st;
+    if ((st = check_matrix(c_pos, M, K, ldc, 1)) != SQ_OK) return st;
+    if (s_neg && (st = check_matrix(c_neg, M, K, ldc, 1)) != SQ_OK) return st;
+    HostSeg hs = load_segtable(seg, K, seg && seg->nb && seg->Q >= 1 ? seg->nb[seg->Q] : 0);
+    if (hs.status != SQ_OK) return hs.status;
+    return launch_quantize(X, dt, M, K, ld, hs.b, s_pos, s_neg, 0, code, code_qmax(code),
+                           code_qmin_abs(code, flags), c_pos, c_neg, ldc, static_cast<cudaStream_t>(stream));
+}
+
+sq_status segquant_quantize_weight(const void *W, sq_dtype dt, int64_t N, int64_t K, int64_t ld,
+                                   const sq_segtable *seg, const float *s_w, sq_code code, uint32_t flags,
+                                   void *Wq, int64_t ldq, void *stream)
+{
+    (void)flags;
+    if (!s_w) return SQ_ERR_NULL;
+    if (!valid_dt(dt) || !valid_code(code)) return SQ_ERR_UNSUPPORTED;
+    sq_status st;
+    if ((st = check_matrix(W, N, K, ld, dt_size(dt))) != SQ_OK) return st;
+    if ((st = check_matrix(Wq, N, K, ldq, 1)) != SQ_OK) return st;
+    HostSeg hs = load_segtable(seg, K, N);
+    if (hs.status != SQ_OK) return hs.status;
+    return launch_quantize(W, dt, N, K, ld, hs.b, s_w, nullptr, 1, code, code_qmax(code), code_qmax(code), Wq,
+                           nullptr, ldq, static_cast<cudaStream_t>(stream));
+}
+
+sq_status segquant_seglinear_gemm(const void *Xq, int64_t ldx, const void *Wq, int64_t ldw, int64_t M, int64_t N,
+                                  int64_t K, const sq_segtable *seg, sq_code code, const float *s_x,
+                                  const float *s_w, const float *bias, void *Y, sq_dtype y_dtype, int64_t ldy,
+                                  void *acc_dump, void *workspace, size_t ws_bytes, void *stream)
+{
+    return gemm_common(Xq, nullptr, 0, ldx, Wq, ldw, M, N, K, seg, code, s_x, nullptr, s_w, bias, Y, y_dtype, ldy,
+                       acc_dump, workspace, ws_bytes, stream);
+}
+
+sq_status segquant_dualscale_gemm(const void *Xq_pos, const void *Xq_neg, int64_t ldx, const void *Wq, int64_t ldw,
+                                  int64_t M, int64_t N, int64_t K, const sq_segtable *seg, sq_code code,
+                                  const float *s_pos, const float *s_neg, const float *s_w, const float *bias,
+                                  void *Y, sq_dtype y_dtype, int64_t ldy, void *acc_dump, void *workspace,
+                                  size_t ws_bytes, void *stream)
+{
+    return gemm_common(Xq_pos, Xq_neg, 1, ldx, Wq, ldw, M, N, K, seg, code, s_pos, s_neg, s_w, bias, Y, y_dtype,
+                       ldy, acc_dump, workspace, ws_bytes, stream);
+}
+
+size_t segquant_layer_scratch_bytes(int64_t M, int64_t K, int dual)
+{
+    if (M <= 0 || K <= 0) return 0;
+    const size_t ldc = (size_t(K) + 127) & ~size_t(127);
+    const size_t one = (size_t(M) * ldc + 255) & ~size_t(255);
+    return one * (dual ? 2 : 1);
+}
+
+sq_status segquant_layer_forward(const void *X, int x_on_host, void *x_stage, sq_dtype dt, int64_t M, int64_t K,
+                                 int64_t ld, const void *Wq, int64_t ldw, int64_t N, const sq_segtable *seg,
+                                 sq_code code, const float *s_pos, const float *s_neg, const float *s_w,
+                                 const float *bias, uint32_t flags, void *Y, int y_on_host, void *y_stage,
+                                 sq_dtype y_dtype, int64_t ldy, void *scratch, size_t scratch_bytes,
+                                 void *workspace, size_t ws_bytes, void *stream)
+{
+    if (!X || !Y || !scratch || (x_on_host && !x_stage) || (y_on_host && !y_stage)) return SQ_ERR_NULL;
+    if (!valid_dt(dt) || !valid_dt(y_dtype)) return SQ_ERR_UNSUPPORTED;
+    if (M <= 0 || K <= 0 || N <= 0 || ld < K || ldy < N) return SQ_ERR_SHAPE;
+    const int dual = s_neg != nullptr;
+    if (scratch_bytes < segquant_layer_scratch_bytes(M, K, dual)) return SQ_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(scratch) & 255u) return SQ_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const void *xd = X;
+    if (x_on_host) {
+        if (cudaMemcpyAsync(x_stage, X, size_t(M) * ld * dt_size(dt), cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return SQ_ERR_CUDA;
+        xd = x_stage;
+    }
+    const int64_t ldc = (K + 127) & ~int64_t(127);
+    uint8_t *c_pos = static_cast<uint8_t *>(scratch);
+    uint8_t *c_neg = dual ? c_pos + ((size_t(M) * ldc + 255) & ~size_t(255)) : nullptr;
+    sq_status r = segquant_quantize_act(xd, dt, M, K, ld, seg, s_pos, s_neg, code, flags, c_pos, c_neg, ldc, stream);
+    if (r != SQ_OK) return r;
+    void *yd = y_on_host ? y_stage : Y;
+    r = dual ? segquant_dualscale_gemm(c_pos, c_neg, ldc, Wq, ldw, M, N, K, seg, code, s_pos, s_neg, s_w, bias, yd,
+                                       y_dtype, ldy, nullptr, workspace, ws_bytes, stream)
+             : segquant_seglinear_gemm(c_pos, ldc, Wq, ldw, M, N, K, seg, code, s_pos, s_w, bias, yd, y_dtype, ldy,
+                                       nullptr, workspace, ws_bytes, stream);
+    if (r != SQ_OK) return r;
+    if (y_on_host &&
+        cudaMemcpyAsync(Y, y_stage, size_t(M) * ldy * dt_size(y_dtype), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return SQ_ERR_CUDA;
+    return SQ_OK;
+}
+
+sq_status segquant_last_device_status(void *workspace, void *stream, uint32_t *detail)
+{
+    if (!workspace) return SQ_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint32_t word = 0;
+    if (cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess) return SQ_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SQ_ERR_CUDA;
+    if (detail) *detail = word;
+    if (word == 0) return SQ_OK;
+    if (cudaMemsetAsync(workspace, 0, sizeof(word), st) != cudaSuccess) return SQ_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SQ_ERR_CUDA;
+    return SQ_ERR_TIMEOUT;
+}
+
+sq_status segquant_set_tuning(int tile_n, int stages)
+{
+    set_gemm_tuning(tile_n, stages);
+    return SQ_OK;
+}
+
+uint64_t segquant_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char *segquant_status_string(sq_status s)
+{
+    switch (s) {
+        case SQ_OK: return "ok";
+        case SQ_ERR_NULL: return "null pointer";
+        case SQ_ERR_SHAPE: return "bad shape";
+        case SQ_ERR_SEGTABLE: return "bad segment table";
+        case SQ_ERR_ALIGN: return "alignment";
+        case SQ_ERR_UNSUPPORTED: return "unsupported";
+        case SQ_ERR_CUDA: return "cuda error";
+        case SQ_ERR_TIMEOUT: return "device wait timed out";
+        case SQ_ERR_WORKSPACE: return "workspace missing or too small";
+    }
+    return "unknown";
+}
+
+}  // extern "C"

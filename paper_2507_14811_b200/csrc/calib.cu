@@ -1,0 +1,123 @@
+// Min/max calibration (Sec. 4.3.2 scale formula; strict min/max, App. B sensitivity analysis):
+// per K-segment extrema of a calibration batch, or per (K-segment, N-segment) abs-max of a weight
+// matrix, reduced through ordered-integer atomics into workspace partials, then one IEEE division
+// per scale.
+#include <cuda_bf16.h>
+#include "sq_common.cuh"
+
+namespace sq {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kRowsPerBlock = 64;
+
+// monotone map float -> uint32 (a < b  <=>  enc(a) < enc(b)); 0 and 0xFFFFFFFF are never produced
+// by finite inputs and serve as the "nothing seen" marks of the max / min slots.
+__device__ __forceinline__ uint32_t enc(float f)
+{
+    uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float dec(uint32_t u)
+{
+    return __uint_as_float((u & 0x80000000u) ? (u & 0x7FFFFFFFu) : ~u);
+}
+
+__device__ __forceinline__ float ld1(const float *p) { return __ldg(p); }
+__device__ __forceinline__ float ld1(const __nv_bfloat16 *p)
+{
+    return __uint_as_float(uint32_t(__ldg(reinterpret_cast<const unsigned short *>(p))) << 16);
+}
+
+__global__ void calib_init_kernel(uint32_t *partials, int nblocks)
+{
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < nblocks) { partials[2 * i] = 0u; partials[2 * i + 1] = 0xFFFFFFFFu; }
+}
+
+// grid.x covers columns (one column per thread), grid.y covers chunks of kRowsPerBlock rows.
+// Consecutive threads read consecutive columns of the same row: coalesced.
+template <typename Tin>
+__global__ void __launch_bounds__(kThreads)
+calib_reduce_kernel(const Tin *__restrict__ X, int64_t rows, int K, int64_t ld, SegBounds sb, int is_weight,
+                    uint32_t *__restrict__ partials)
+{
+    __shared__ uint32_t sh_max[kMaxBlocks];
+    __shared__ uint32_t sh_min[kMaxBlocks];
+    const int Qs = is_weight ? sb.Q : 1;
+    const int nblk = sb.P * Qs;
+    for (int i = threadIdx.x; i < nblk; i += kThreads) { sh_max[i] = 0u; sh_min[i] = 0xFFFFFFFFu; }
+    __syncthreads();
+
+    const int k = blockIdx.x * kThreads + threadIdx.x;
+    const int64_t r0 = int64_t(blockIdx.y) * kRowsPerBlock;
+    const int64_t r1 = min(rows, r0 + kRowsPerBlock);
+    if (k < K && r0 < r1) {
+        int p = 0;
+        while (p + 1 < sb.P && k >= sb.kb[p + 1]) p++;
+        int q = 0;
+        if (is_weight) while (q + 1 < sb.Q && r0 >= sb.nb[q + 1]) q++;
+        float mx = -INFINITY, mn = INFINITY;
+        for (int64_t r = r0; r < r1; r++) {
+            if (is_weight && q + 1 < sb.Q && r >= sb.nb[q + 1]) {       // row enters the next N-segment
+                atomicMax(&sh_max[p * Qs + q], enc(mx));
+                atomicMin(&sh_min[p * Qs + q], enc(mn));
+                mx = -INFINITY; mn = INFINITY;
+                while (q + 1 < sb.Q && r >= sb.nb[q + 1]) q++;
+            }
+            float x = ld1(X + r * ld + k);
+            mx = fmaxf(mx, x);
+            mn = fminf(mn, x);
+        }
+        atomicMax(&sh_max[p * Qs + q], enc(mx));
+        atomicMin(&sh_min[p * Qs + q], enc(mn));
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < nblk; i += kThreads) {
+        if (sh_max[i] != 0u) atomicMax(&partials[2 * i], sh_max[i]);
+        if (sh_min[i] != 0xFFFFFFFFu) atomicMin(&partials[2 * i + 1], sh_min[i]);
+    }
+}
+
+__global__ void calib_finalize_kernel(const uint32_t *__restrict__ partials, int nblocks, int is_weight, int dual,
+                                      float q_max, float q_min_abs, float *__restrict__ s_pos,
+                                      float *__restrict__ s_neg)
+{
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= nblocks) return;
+    const uint32_t emx = partials[2 * i], emn = partials[2 * i + 1];
+    const float mx = (emx == 0u || emx == enc(-INFINITY)) ? 0.0f : dec(emx);
+    const float mn = (emn == 0xFFFFFFFFu || emn == enc(INFINITY)) ? 0.0f : dec(emn);
+    if (!is_weight && dual) {
+        const float hi = fmaxf(mx, 0.0f), lo = fmaxf(-mn, 0.0f);
+        s_pos[i] = hi > 0.0f ? __fdiv_rn(hi, q_max) : 1.0f;
+        s_neg[i] = lo > 0.0f ? __fdiv_rn(lo, q_min_abs) : 1.0f;
+    } else {
+        const float a = fmaxf(fabsf(mx), fabsf(mn));
+        s_pos[i] = a > 0.0f ? __fdiv_rn(a, q_max) : 1.0f;
+    }
+}
+
+}  // namespace
+
+sq_status launch_calib(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld, const SegBounds &sb,
+                       int is_weight, int dual, float q_max, float q_min_abs, float *s_pos, float *s_neg,
+                       uint32_t *partials, cudaStream_t st)
+{
+    const int nblocks = sb.P * (is_weight ? sb.Q : 1);
+    calib_init_kernel<<<(nblocks + 255) / 256, 256, 0, st>>>(partials, nblocks);
+    dim3 grid(unsigned((K + kThreads - 1) / kThreads), unsigned((rows + kRowsPerBlock - 1) / kRowsPerBlock));
+    if (grid.y > 65535) return SQ_ERR_SHAPE;
+    if (dt == SQ_F32)
+        calib_reduce_kernel<float><<<grid, kThreads, 0, st>>>(static_cast<const float *>(X), rows, int(K), ld, sb,
+                                                              is_weight, partials);
+    else
+        calib_reduce_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(static_cast<const __nv_bfloat16 *>(X), rows,
+                                                                      int(K), ld, sb, is_weight, partials);
+    calib_finalize_kernel<<<(nblocks + 255) / 256, 256, 0, st>>>(partials, nblocks, is_weight, dual, q_max, q_min_abs,
+                                                                 s_pos, s_neg);
+    count_launch(3);
+    return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
+}
+
+}  // namespace sq

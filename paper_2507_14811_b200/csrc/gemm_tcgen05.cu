@@ -1,0 +1,518 @@
+// W8A8 GEMM + dequantizing epilogue for sm_100a (Sec. 4.2.2 segment-wise products, Sec. 4.3.2 dual
+// path recombination, App. A symmetric recovery).
+//
+// One persistent CTA per SM, 192 threads:
+//   warp 0      TMA producer: per 128-byte K-block, one tile of each activation code matrix
+//               (128 rows) and ONE weight tile (TILE_N rows) into a shared-memory ring
+//   warp 1      tcgen05.mma issuer (one elected lane): for every 32-byte K-step, one MMA per polarity
+//               against the same weight tile, each polarity and each K-segment into its own
+//               accumulator in tensor memory (TMEM)
+//   warps 2..5  epilogue: tcgen05.ld of all accumulators of a 32-column slab, fp32 FMA with the
+//               per-(segment, polarity, column) scale, + bias, -> bf16 / fp32 store
+// Accumulators: NACC = P * npol, each 128 lanes x TILE_N columns; NACC * TILE_N <= 512 columns.
+// If they use at most half of TMEM the accumulator set is double-buffered so that the epilogue of
+// one tile overlaps the main loop of the next.
+// Every wait on an mbarrier is bounded (wall-clock limit); on expiry the CTA records which wait gave
+// up in the status word, stops issuing work, lets its own copies land and leaves normally.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include "sq_common.cuh"
+
+namespace sq {
+namespace {
+
+constexpr int TILE_M = 128;
+constexpr int BLOCK_K = 128;          // bytes (= codes) per K-block: one 128B swizzle row
+constexpr int MMA_K = 32;             // codes per tcgen05.mma of an 8-bit kind
+constexpr int kThreads = 192;
+constexpr int kEpiThreads = 128;
+constexpr int kMaxStages = 8;
+constexpr int kTmemCols = 512;
+constexpr uint32_t kSmemBudget = 227 * 1024;
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
+
+struct KernelParams {
+    int M, N, K;
+    int npol;          // 1 or 2 activation code matrices
+    int nacc;          // P * npol
+    int acc_stages;    // 1 or 2 accumulator sets in TMEM
+    int stages;        // shared-memory ring depth
+    int num_m_tiles, num_n_tiles;
+    SegBounds sb;
+    const float *s_pos, *s_neg, *s_w, *bias;
+    void *Y;
+    long long ldy;
+    int y_is_f32;
+    void *acc_dump;
+    uint32_t *status;
+};
+
+// ----------------------------------------------------------------------------- PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return uint32_t(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+__device__ __forceinline__ uint64_t globaltimer_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait.  Returns false if the wait expired or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                          uint32_t *status, uint32_t where)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = globaltimer_ns();
+    uint32_t polls = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++polls & 255u) == 0) {
+            if (*abort_flag) return false;
+            if (globaltimer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicCAS(status, 0u, where);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+template <int KIND>   // 0: kind::i8, 1: kind::f8f6f4
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t accumulate)
+{
+    if (KIND == 0)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// 32 lanes x 32 consecutive 32-bit columns: thread t of the warp receives lane (base_lane + t).
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile stored as 128-byte rows with the 128B swizzle
+// (the layout a 2-D TMA load with CU_TENSOR_MAP_SWIZZLE_128B writes): start address >> 4 in bits
+// 0-13, stride between 8-row groups (1024 B) >> 4 in bits 32-45, descriptor version 1 in bits 46-47,
+// swizzle mode 2 (128B) in bits 61-63.  The leading-dimension offset is unused for this layout.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= uint64_t((smem_addr & 0x3FFFFu) >> 4);
+    d |= uint64_t(1024u >> 4) << 32;
+    d |= uint64_t(1) << 46;
+    d |= uint64_t(2) << 61;
+    return d;
+}
+
+// Instruction descriptor: D format bits 4-5 (1 = f32, 2 = s32), A format bits 7-9, B format bits
+// 10-12 (kind::i8: 1 = signed 8-bit; kind::f8f6f4: 0 = e4m3), A and B K-major (bits 15, 16 = 0),
+// N >> 3 in bits 17-22, M >> 4 in bits 24-28.
+__host__ __device__ constexpr uint32_t make_idesc(int kind, int tile_n)
+{
+    return (kind == 0 ? (2u << 4) | (1u << 7) | (1u << 10) : (1u << 4)) |
+           (uint32_t(tile_n >> 3) << 17) | (uint32_t(TILE_M >> 4) << 24);
+}
+
+// ----------------------------------------------------------------------------- the kernel
+
+struct SharedHeader {
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+
+// where-codes written to the status word when a wait expires
+enum : uint32_t { kWhereProducer = 0x100, kWhereMmaFull = 0x200, kWhereMmaTmem = 0x300, kWhereEpilogue = 0x400 };
+
+template <int KIND, int TILE_N>
+__global__ void __launch_bounds__(kThreads, 1)
+segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_constant__ CUtensorMap tm_a_neg,
+                     const __grid_constant__ CUtensorMap tm_b, const KernelParams prm)
+{
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    // layout: [ring: stages x (npol A tiles of 16 KiB, B tile of TILE_N*128 B)] [scales] [header]
+    const uint32_t a_bytes = TILE_M * BLOCK_K;
+    const uint32_t b_bytes = TILE_N * BLOCK_K;
+    const uint32_t stage_bytes = prm.npol * a_bytes + b_bytes;
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    float *sh_scale = reinterpret_cast<float *>(smem + size_t(prm.stages) * stage_bytes);   // [nacc][TILE_N]
+    float *sh_bias = sh_scale + prm.nacc * TILE_N;                                           // [TILE_N]
+    SharedHeader *hdr = reinterpret_cast<SharedHeader *>(sh_bias + TILE_N);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int num_tiles = prm.num_m_tiles * prm.num_n_tiles;
+    volatile uint32_t *abort_flag = &hdr->abort_flag;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < prm.stages; s++) {
+            mbar_init(smem_u32(&hdr->full[s]), 1);
+            mbar_init(smem_u32(&hdr->empty[s]), 1);
+        }
+        for (int s = 0; s < 2; s++) {
+            mbar_init(smem_u32(&hdr->tmem_full[s]), 1);
+            mbar_init(smem_u32(&hdr->tmem_empty[s]), kEpiThreads);
+        }
+        hdr->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&hdr->tmem_base)), "r"(uint32_t(kTmemCols)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = hdr->tmem_base;
+    const int acc_cols = prm.nacc * TILE_N;     // TMEM columns of one accumulator set
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_a_pos)) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_b)) : "memory");
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile / prm.num_n_tiles) * TILE_M;
+                const int n0 = (tile % prm.num_n_tiles) * TILE_N;
+                for (int p = 0; p < prm.sb.P && ok; p++) {
+                    for (int k = prm.sb.kb[p]; k < prm.sb.kb[p + 1]; k += BLOCK_K, it++) {
+                        const uint32_t s = it % prm.stages, ph = (it / prm.stages) & 1;
+                        if (!mbar_wait(smem_u32(&hdr->empty[s]), ph ^ 1, abort_flag, prm.status, kWhereProducer)) {
+                            ok = false;
+                            break;
+                        }
+                        const uint32_t bar = smem_u32(&hdr->full[s]);
+                        const uint32_t dst = smem_u32(smem + size_t(s) * stage_bytes);
+                        mbar_expect_tx(bar, stage_bytes);
+                        tma_load_2d(dst, &tm_a_pos, bar, k, m0);
+                        if (prm.npol == 2) tma_load_2d(dst + a_bytes, &tm_a_neg, bar, k, m0);
+                        tma_load_2d(dst + prm.npol * a_bytes, &tm_b, bar, k, n0);
+                    }
+                }
+            }
+            if (!ok) {
+                // let the copies this thread issued land before the CTA's shared memory goes away
+                const uint32_t pending = it < uint32_t(prm.stages) ? it : uint32_t(prm.stages);
+                for (uint32_t j = 0; j < pending; j++) {
+                    const uint32_t i2 = it - 1 - j, s = i2 % prm.stages, ph = (i2 / prm.stages) & 1;
+                    const uint64_t t0 = globaltimer_ns();
+                    while (!mbar_try_wait(smem_u32(&hdr->full[s]), ph) && globaltimer_ns() - t0 < 100000000ull) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(KIND, TILE_N);
+            uint32_t it = 0, tile_iter = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, tile_iter++) {
+                const uint32_t as = tile_iter % prm.acc_stages, aph = (tile_iter / prm.acc_stages) & 1;
+                if (!mbar_wait(smem_u32(&hdr->tmem_empty[as]), aph ^ 1, abort_flag, prm.status, kWhereMmaTmem)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                for (int p = 0; p < prm.sb.P && ok; p++) {
+                    const uint32_t d0 = tmem_base + as * acc_cols + uint32_t(p * prm.npol) * TILE_N;
+                    uint32_t accumulate = 0;
+                    for (int k = prm.sb.kb[p]; k < prm.sb.kb[p + 1]; k += BLOCK_K, it++) {
+                        const uint32_t s = it % prm.stages, ph = (it / prm.stages) & 1;
+                        if (!mbar_wait(smem_u32(&hdr->full[s]), ph, abort_flag, prm.status, kWhereMmaFull)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint32_t base = smem_u32(smem + size_t(s) * stage_bytes);
+                        const uint64_t da0 = make_smem_desc(base);
+                        const uint64_t da1 = make_smem_desc(base + a_bytes);
+                        const uint64_t db = make_smem_desc(base + prm.npol * a_bytes);
+                        const int rem = prm.sb.kb[p + 1] - k;
+                        const int nk = rem >= BLOCK_K ? BLOCK_K / MMA_K : (rem + MMA_K - 1) / MMA_K;
+                        for (int kk = 0; kk < nk; kk++) {
+                            const uint64_t koff = uint64_t((kk * MMA_K) >> 4);   // +32 B inside the swizzle row
+                            tc_mma<KIND>(d0, da0 + koff, db + koff, idesc, accumulate);
+                            if (prm.npol == 2) tc_mma<KIND>(d0 + TILE_N, da1 + koff, db + koff, idesc, accumulate);
+                            accumulate = 1;
+                        }
+                        tc_commit(smem_u32(&hdr->empty[s]));      // frees the ring slot when these MMAs retire
+                    }
+                }
+                if (ok) tc_commit(smem_u32(&hdr->tmem_full[as]));  // accumulators of this tile complete
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int et = threadIdx.x - 64;           // 0..127
+        const int lane_grp = warp & 3;             // TMEM lanes 32*lane_grp .. +31 are this warp's
+        uint32_t tile_iter = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, tile_iter++) {
+            const int m0 = (tile / prm.num_n_tiles) * TILE_M;
+            const int n0 = (tile % prm.num_n_tiles) * TILE_N;
+            const uint32_t as = tile_iter % prm.acc_stages, aph = (tile_iter / prm.acc_stages) & 1;
+
+            // per-column dequantization factors of this tile: c[a][j] = s_act[p][pol] * s_w[p][q(n0+j)]
+            asm volatile("bar.sync 1, 128;" ::: "memory");       // previous tile's readers are done
+            for (int j = et; j < TILE_N; j += kEpiThreads) {
+                const int n = n0 + j;
+                int q = 0;
+                while (q + 1 < prm.sb.Q && n >= prm.sb.nb[q + 1]) q++;
+                for (int p = 0; p < prm.sb.P; p++) {
+                    const float sw = n < prm.N ? prm.s_w[p * prm.sb.Q + q] : 0.0f;
+                    sh_scale[(p * prm.npol) * TILE_N + j] = prm.s_pos[p] * sw;
+                    if (prm.npol == 2) sh_scale[(p * prm.npol + 1) * TILE_N + j] = prm.s_neg[p] * sw;
+                }
+                sh_bias[j] = (prm.bias && n < prm.N) ? prm.bias[n] : 0.0f;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+
+            if (ok) ok = mbar_wait(smem_u32(&hdr->tmem_full[as]), aph, abort_flag, prm.status, kWhereEpilogue);
+            if (!ok) continue;                      // keep the named barriers balanced, do no more work
+            tc_fence_after();
+
+            const int row = m0 + lane_grp * 32 + lane;
+            const uint32_t t_row = tmem_base + (uint32_t(lane_grp * 32) << 16) + as * acc_cols;
+#pragma unroll 1
+            for (int c0 = 0; c0 < TILE_N; c0 += 32) {
+                float y[32];
+#pragma unroll
+                for (int j = 0; j < 32; j++) y[j] = 0.0f;
+#pragma unroll 1
+                for (int a = 0; a < prm.nacc; a++) {
+                    uint32_t r[32];
+                    tc_ld32(t_row + uint32_t(a * TILE_N + c0), r);
+                    tc_wait_ld();
+                    const float *sc = sh_scale + a * TILE_N + c0;
+#pragma unroll
+                    for (int j = 0; j < 32; j++) {
+                        const float v = KIND == 0 ? __int2float_rn(int(r[j])) : __uint_as_float(r[j]);
+                        y[j] = fmaf(sc[j], v, y[j]);
+                    }
+                    if (prm.acc_dump && row < prm.M) {
+                        uint32_t *dump = static_cast<uint32_t *>(prm.acc_dump) +
+                                         (size_t(a) * prm.M + row) * size_t(prm.N) + n0 + c0;
+#pragma unroll
+                        for (int j = 0; j < 32; j++)
+                            if (n0 + c0 + j < prm.N) dump[j] = r[j];
+                    }
+                }
+                if (row < prm.M) {
+#pragma unroll
+                    for (int j = 0; j < 32; j++) y[j] += sh_bias[c0 + j];
+                    const int ncol = prm.N - (n0 + c0);          // valid columns in this slab (multiple of 8)
+                    if (prm.y_is_f32) {
+                        float *dst = static_cast<float *>(prm.Y) + size_t(row) * prm.ldy + n0 + c0;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            if (j < ncol) *reinterpret_cast<float4 *>(dst + j) = make_float4(y[j], y[j + 1], y[j + 2], y[j + 3]);
+                    } else {
+                        __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(prm.Y) + size_t(row) * prm.ldy + n0 + c0;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            if (j < ncol) {
+                                uint32_t w[4];
+#pragma unroll
+                                for (int t = 0; t < 4; t++) {
+                                    __nv_bfloat162 h = __floats2bfloat162_rn(y[j + 2 * t], y[j + 2 * t + 1]);
+                                    w[t] = *reinterpret_cast<uint32_t *>(&h);
+                                }
+                                *reinterpret_cast<uint4 *>(dst + j) = make_uint4(w[0], w[1], w[2], w[3]);
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(smem_u32(&hdr->tmem_empty[as]));
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(uint32_t(kTmemCols)) : "memory");
+    }
+}
+
+// ----------------------------------------------------------------------------- host side
+
+using EncodeFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                              const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn get_encode_fn()
+{
+    static EncodeFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeFn>(p);
+    }
+    return fn;
+}
+
+// 2-D map over a row-major byte matrix [rows, cols] with row pitch ld: box = 128 bytes x box_rows,
+// 128B swizzle, out-of-range elements read as zero.
+bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, int64_t ld, int box_rows)
+{
+    EncodeFn enc = get_encode_fn();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {cuuint64_t(cols), cuuint64_t(rows)};
+    cuuint64_t strides[1] = {cuuint64_t(ld)};
+    cuuint32_t box[2] = {cuuint32_t(BLOCK_K), cuuint32_t(box_rows)};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+int g_tune_tile_n = 0, g_tune_stages = 0;
+
+template <int KIND, int TILE_N>
+sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cudaStream_t st)
+{
+    CUtensorMap ta, tn, tb;
+    if (!make_map(&ta, g.a_pos, g.M, g.K, g.lda, TILE_M)) return SQ_ERR_CUDA;
+    if (!make_map(&tn, g.a_neg ? g.a_neg : g.a_pos, g.M, g.K, g.lda, TILE_M)) return SQ_ERR_CUDA;
+    if (!make_map(&tb, g.b, g.N, g.K, g.ldb, TILE_N)) return SQ_ERR_CUDA;
+
+    const uint32_t stage_bytes = prm.npol * TILE_M * BLOCK_K + TILE_N * BLOCK_K;
+    const uint32_t tail = uint32_t(prm.nacc + 1) * TILE_N * 4 + sizeof(SharedHeader);
+    int stages = int((kSmemBudget - 1024 - tail) / stage_bytes);
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (g_tune_stages >= 2 && g_tune_stages < stages) stages = g_tune_stages;
+    if (stages < 2) return SQ_ERR_UNSUPPORTED;
+    prm.stages = stages;
+    prm.num_m_tiles = int((g.M + TILE_M - 1) / TILE_M);
+    prm.num_n_tiles = int((g.N + TILE_N - 1) / TILE_N);
+    const size_t smem = 1024 + size_t(stages) * stage_bytes + tail;
+
+    auto kern = segquant_gemm_kernel<KIND, TILE_N>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
+        return SQ_ERR_CUDA;
+    const int tiles = prm.num_m_tiles * prm.num_n_tiles;
+    const int grid = tiles < sm_count ? tiles : sm_count;
+    kern<<<grid, kThreads, smem, st>>>(ta, tn, tb, prm);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
+}
+
+template <int KIND>
+sq_status launch_kind(const GemmArgs &g, KernelParams &prm, int tile_n, int sm_count, cudaStream_t st)
+{
+    switch (tile_n) {
+        case 256: return launch_variant<KIND, 256>(g, prm, sm_count, st);
+        case 128: return launch_variant<KIND, 128>(g, prm, sm_count, st);
+        case 64: return launch_variant<KIND, 64>(g, prm, sm_count, st);
+        case 32: return launch_variant<KIND, 32>(g, prm, sm_count, st);
+    }
+    return SQ_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+void set_gemm_tuning(int tile_n, int stages)
+{
+    g_tune_tile_n = tile_n;
+    g_tune_stages = stages;
+}
+
+sq_status launch_gemm(const GemmArgs &g, cudaStream_t st)
+{
+    KernelParams prm{};
+    prm.M = int(g.M); prm.N = int(g.N); prm.K = int(g.K);
+    prm.npol = g.a_neg ? 2 : 1;
+    prm.nacc = g.sb.P * prm.npol;
+    prm.sb = g.sb;
+    prm.s_pos = g.s_pos; prm.s_neg = g.s_neg; prm.s_w = g.s_w; prm.bias = g.bias;
+    prm.Y = g.Y; prm.ldy = g.ldy; prm.y_is_f32 = g.y_dtype == SQ_F32;
+    prm.acc_dump = g.acc_dump;
+    prm.status = g.status;
+
+    // widest tile whose accumulators fit the 512 TMEM columns
+    int tile_n = 256;
+    while (tile_n * prm.nacc > kTmemCols) tile_n >>= 1;
+    if (tile_n < 32) return SQ_ERR_UNSUPPORTED;
+    if (g_tune_tile_n >= 32 && g_tune_tile_n <= tile_n && (g_tune_tile_n & (g_tune_tile_n - 1)) == 0)
+        tile_n = g_tune_tile_n;
+    prm.acc_stages = (2 * tile_n * prm.nacc <= kTmemCols) ? 2 : 1;
+
+    int dev = 0, sm_count = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SQ_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
+        return SQ_ERR_CUDA;
+
+    return g.code == SQ_CODE_INT8 ? launch_kind<0>(g, prm, tile_n, sm_count, st)
+                                  : launch_kind<1>(g, prm, tile_n, sm_count, st);
+}
+
+}  // namespace sq

@@ -1,0 +1,71 @@
+// Internal declarations shared by the CUDA translation units of the library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include "segquant.h"
+
+namespace sq {
+
+// Workspace layout (device, 256-byte aligned):
+//   [0,256)        status words: word 0 = first expired wait (0 = none)
+//   [256, 256+32K) calibration partials: 2 ordered-uint words per (p,q) block
+constexpr size_t kWsStatusBytes = 256;
+constexpr int kMaxBlocks = SQ_MAX_P * SQ_MAX_Q;               // 1024 (p,q) blocks
+constexpr size_t kWsCalibBytes = size_t(kMaxBlocks) * 2 * 4;  // 8 KiB
+constexpr size_t kWsBytes = kWsStatusBytes + kWsCalibBytes;
+
+// Segment bounds by value in kernel parameters (constant bank).
+struct SegBounds {
+    int P, Q;
+    int kb[SQ_MAX_P + 1];
+    int nb[SQ_MAX_Q + 1];
+};
+
+struct HostSeg {
+    SegBounds b;
+    sq_status status;
+};
+
+// Validates a segment table against K and N and copies it (host side).
+HostSeg load_segtable(const sq_segtable *seg, int64_t K, int64_t N);
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+void count_launch(int n = 1);
+
+// per-code ranges
+inline float code_qmax(sq_code c) { return c == SQ_CODE_INT8 ? 127.0f : 448.0f; }
+inline float code_qmin_abs(sq_code c, uint32_t flags)
+{
+    if (c == SQ_CODE_INT8) return (flags & SQ_FLAG_QMIN_SYM) ? 127.0f : 128.0f;
+    return 448.0f;
+}
+
+// kernels' host launchers (defined in the .cu files)
+sq_status launch_calib(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld, const SegBounds &sb,
+                       int is_weight, int dual, float q_max, float q_min_abs, float *s_pos, float *s_neg,
+                       uint32_t *partials, cudaStream_t st);
+
+sq_status launch_quantize(const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld, const SegBounds &sb,
+                          const float *s_pos, const float *s_neg, int row_segments, sq_code code,
+                          float q_max, float q_min_abs, void *c_pos, void *c_neg, int64_t ldc, cudaStream_t st);
+
+struct GemmArgs {
+    const void *a_pos, *a_neg;   // code matrices [M,K]; a_neg == nullptr: single path
+    int64_t lda;
+    const void *b;               // weight codes [N,K]
+    int64_t ldb;
+    int64_t M, N, K;
+    SegBounds sb;
+    sq_code code;
+    const float *s_pos, *s_neg, *s_w, *bias;
+    void *Y;
+    sq_dtype y_dtype;
+    int64_t ldy;
+    void *acc_dump;
+    uint32_t *status;
+};
+sq_status launch_gemm(const GemmArgs &g, cudaStream_t st);
+void set_gemm_tuning(int tile_n, int stages);
+
+}  // namespace sq

@@ -1,0 +1,221 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs.
+Bit-exact scales, codes and int32 accumulators; fp32 epilogue within 1e-5 relative; bf16 within
+1 ulp; e4m3 accumulators within 1e-3 relative."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from paper_2507_14811_b200 import binding as B
+from paper_2507_14811_b200 import workloads as WL
+from paper_2507_14811_b200.layer import SegQuantLinear
+
+from parity_util import (QRANGE, check_bf16_output, check_fp32_output, oracle_scales, to_f32_np)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def custom_spec(name, M, K, N, kb, nb, dual, code, x_dtype="bf16", x_kind="normal+gelu", seed=7, cal_rows=32,
+                x_seg_std=None, w_kind="plain"):
+    return WL.LayerSpec(name=name, M=M, K=K, N=N, kb=kb, nb=nb, dual=dual, code=code, x_dtype=x_dtype,
+                        x_kind=x_kind, w_kind=w_kind, seed=seed, cal_rows=cal_rows, x_seg_std=x_seg_std or [])
+
+
+def run_parity(spec, rows=None, flags=0, tile_n=0):
+    """Full element-by-element parity of one layer.  rows: optional subset of rows the oracle computes."""
+    data = WL.make_layer(spec)
+    qmin_sym = bool(flags & B.SQ_FLAG_QMIN_SYM)
+    s_pos, s_neg, s_w, Wq, (qmax, qmin_abs) = oracle_scales(data, qmin_sym)
+
+    B.segquant_set_tuning(tile_n, 0)
+    try:
+        layer = SegQuantLinear(data.W, data.bias, spec.kb, spec.nb, spec.dual, spec.code, DEV, flags)
+        g_pos, g_neg = layer.calibrate(data.X_cal)
+        # --- scales: bit-exact
+        assert np.array_equal(layer.s_w.cpu().numpy().reshape(spec.P, spec.Q), s_w)
+        assert np.array_equal(g_pos.cpu().numpy(), s_pos)
+        if spec.dual:
+            assert np.array_equal(g_neg.cpu().numpy(), s_neg)
+        # --- weight codes: bit-exact
+        assert np.array_equal(layer.Wq.cpu().numpy().view(Wq.dtype), Wq)
+
+        Xd = data.X.to(DEV)
+        Y32, c_pos, c_neg, dump = layer.forward_steps(Xd, y_dtype=torch.float32, dump_acc=True)
+        Ybf = layer.forward(Xd)                       # the one-call path, bf16 output
+        layer.check_status()
+        torch.cuda.synchronize()
+    finally:
+        B.segquant_set_tuning(0, 0)
+
+    sel = np.arange(spec.M) if rows is None else np.asarray(rows)
+    Xs = to_f32_np(data.X)[sel]
+    res = O.layer_forward(Xs, Wq, O.SegTable(spec.kb, spec.nb), s_pos, s_neg, s_w, to_f32_np(data.bias),
+                          code=spec.code, q_max=qmax, q_min_abs=qmin_abs)
+    # --- activation codes: bit-exact
+    dt = np.int8 if spec.code == "int8" else np.uint8
+    assert np.array_equal(c_pos.cpu().numpy().view(dt)[sel], res.c_pos)
+    if spec.dual:
+        assert np.array_equal(c_neg.cpu().numpy().view(dt)[sel], res.c_neg)
+    # --- accumulators
+    npol = 2 if spec.dual else 1
+    acc = dump.cpu().numpy().reshape(spec.P, npol, spec.M, spec.N)[:, :, sel]
+    nacc = spec.P * npol
+    if spec.code == "int8":
+        assert np.array_equal(acc[:, 0], res.acc_pos)
+        if spec.dual:
+            assert np.array_equal(acc[:, 1], res.acc_neg)
+        y64, y_abs = res.y64, res.y_abs
+    else:
+        # e4m3: tensor-core fp32 accumulation against exact sums; judged against the sum of |products|
+        mag = lambda c: (np.asarray(c, np.uint8) & 0x7F)
+        for pol, (cx, ref) in enumerate([(res.c_pos, res.acc_pos), (res.c_neg, res.acc_neg)][:npol]):
+            abs_sum = O.accumulate(mag(cx), mag(Wq), spec.kb, code="e4m3")
+            err = np.abs(acc[:, pol].astype(np.float64) - ref)
+            assert np.all(err <= 1e-3 * np.abs(ref) + 1e-5 * abs_sum), \
+                f"e4m3 accumulator error {np.max(err / np.maximum(abs_sum, 1e-30)):.3g} of sum|prod|"
+        # epilogue is judged on the accumulators the GPU produced
+        a_pos = acc[:, 0].astype(np.float64)
+        a_neg = acc[:, 1].astype(np.float64) if spec.dual else None
+        y64, y_abs = O.dequant(a_pos, a_neg, spec.nb, s_pos, s_neg, s_w, to_f32_np(data.bias), with_abs=True)
+    # --- epilogue
+    check_fp32_output(Y32[torch.as_tensor(sel, device=DEV)], y64, y_abs, nacc)
+    check_bf16_output(Ybf[torch.as_tensor(sel, device=DEV)], y64, y_abs, nacc)
+    return res
+
+
+# ------------------------------------------------------------------ small shapes, every element
+
+def test_config_tiny_qkv_full_parity():
+    run_parity(WL.WORKLOADS["tiny_qkv"][0])
+
+
+@pytest.mark.parametrize("case", [
+    # name, M, K, N, kb, nb, dual, code
+    ("ragged_m_single", 300, 256, 256, [0, 256], [0, 256], False, "int8"),
+    ("ragged_everything_dual", 129, 208, 200, [0, 96, 208], [0, 64, 200], True, "int8"),
+    ("one_row", 1, 128, 64, [0, 128], [0, 64], True, "int8"),
+    ("k_tail_16", 70, 48, 40, [0, 48], [0, 8, 40], True, "int8"),
+    ("four_k_segments_dual", 260, 512, 192, [0, 128, 224, 384, 512], [0, 192], True, "int8"),
+    ("eight_k_segments_dual", 150, 512, 96, [0, 64, 128, 192, 256, 320, 384, 448, 512], [0, 96], True, "int8"),
+    ("sixteen_k_segments_single", 140, 1024, 72, list(range(0, 1025, 64)), [0, 72], False, "int8"),
+    ("six_n_segments", 257, 384, 768, [0, 384], [0, 128, 256, 384, 512, 640, 768], True, "int8"),
+    ("uneven_n_segments", 200, 256, 520, [0, 256], [0, 8, 264, 520], False, "int8"),
+    ("multi_tile_long_k", 384, 2304, 512, [0, 2304], [0, 512], True, "int8"),
+    ("e4m3_single", 200, 256, 256, [0, 256], [0, 256], False, "e4m3"),
+    ("e4m3_dual_seg", 260, 384, 320, [0, 128, 384], [0, 64, 320], True, "e4m3"),
+])
+def test_small_shapes_full_parity(case):
+    name, M, K, N, kb, nb, dual, code = case
+    run_parity(custom_spec(name, M, K, N, kb, nb, dual, code, x_seg_std=[1.0 + 2 * i for i in range(len(kb) - 1)]))
+
+
+@pytest.mark.parametrize("tile_n", [32, 64, 128, 256])
+def test_every_tile_width(tile_n):
+    run_parity(custom_spec("tile", 200, 384, 520, [0, 384], [0, 256, 520], False, "int8"), tile_n=tile_n)
+
+
+@pytest.mark.parametrize("tile_n", [64, 128, 256])
+def test_every_tile_width_dual(tile_n):
+    run_parity(custom_spec("tile_dual", 300, 640, 776, [0, 640], [0, 776], True, "int8"), tile_n=tile_n)
+
+
+def test_fp32_input_and_student_t():
+    run_parity(custom_spec("f32_in", 160, 256, 128, [0, 128, 256], [0, 128], True, "int8", x_dtype="f32",
+                           x_kind="student_t4+silu"))
+
+
+def test_symmetric_negative_bound_flag():
+    spec = custom_spec("qmin_sym", 130, 128, 64, [0, 128], [0, 64], True, "int8")
+    res = run_parity(spec, flags=B.SQ_FLAG_QMIN_SYM)
+    assert res.c_neg.min() >= -127
+
+
+def test_runtime_values_beyond_calibrated_range_are_clamped():
+    spec = custom_spec("clamp", 256, 128, 64, [0, 128], [0, 64], True, "int8", cal_rows=4, x_kind="student_t4+gelu")
+    res = run_parity(spec)
+    assert (res.c_pos == 127).sum() > 1
+
+
+def test_degenerate_all_nonnegative_input():
+    # ReLU-like input: the negative path is all zeros and its scale degenerates to 1
+    spec = custom_spec("relu_like", 140, 128, 64, [0, 128], [0, 64], True, "int8", x_kind="normal")
+    data = WL.make_layer(spec)
+    data.X = data.X.abs(); data.X_cal = data.X_cal.abs()
+    s_pos, s_neg, s_w, Wq, (qmax, qmin_abs) = oracle_scales(data)
+    layer = SegQuantLinear(data.W, data.bias, spec.kb, spec.nb, True, "int8", DEV)
+    g_pos, g_neg = layer.calibrate(data.X_cal)
+    assert g_neg.cpu().numpy()[0] == 1.0 and np.array_equal(g_pos.cpu().numpy(), s_pos)
+    Y, c_pos, c_neg, dump = layer.forward_steps(data.X.to(DEV), y_dtype=torch.float32, dump_acc=True)
+    assert int(c_neg.cpu().numpy().view(np.int8).astype(np.int32).__abs__().max()) == 0
+    res = O.layer_forward(to_f32_np(data.X), Wq, O.SegTable(spec.kb, spec.nb), s_pos, s_neg, s_w, to_f32_np(data.bias))
+    assert np.array_equal(dump.cpu().numpy()[0], res.acc_pos[0])
+    assert np.all(dump.cpu().numpy()[1] == 0)
+    check_fp32_output(Y, res.y64, res.y_abs, 2)
+
+
+def test_repeated_calls_are_deterministic():
+    spec = custom_spec("det", 300, 512, 384, [0, 256, 512], [0, 384], True, "int8")
+    data = WL.make_layer(spec)
+    layer = SegQuantLinear(data.W, data.bias, spec.kb, spec.nb, True, "int8", DEV)
+    layer.calibrate(data.X_cal)
+    Xd = data.X.to(DEV)
+    y1 = layer.forward(Xd).clone()
+    y2 = layer.forward(Xd).clone()
+    assert torch.equal(y1, y2)
+
+
+# ------------------------------------------------------------------ reduced copies of the benchmark layers
+
+@pytest.mark.parametrize("wl,idx,M,K,N", [
+    ("dit_xl2", 0, 300, 384, 768 * 3),      # 6 N-segments, ladder weights, SiLU, dual
+    ("dit_xl2", 1, 300, 1536, 384),         # GELU dual, long K
+    ("sd3_mmdit", 0, 333, 512, 768),        # 2 K-segments x 3 N-segments, single scale
+    ("sd3_mmdit", 2, 270, 2048, 512),
+    ("flux", 0, 280, 512, 1024),            # e4m3 single, heavy tails
+    ("flux", 1, 280, 2048, 512),            # e4m3 dual
+    ("flux", 2, 280, 512, 768 * 3),         # e4m3 dual, 6 N-segments
+    ("sdxl_skip", 0, 1000, 1280, 640),      # 2 K-segments, dual, full K and N
+])
+def test_reduced_benchmark_layers(wl, idx, M, K, N):
+    run_parity(WL.small_variant(WL.WORKLOADS[wl][idx], M, K, N))
+
+
+# ------------------------------------------------------------------ full benchmark sizes, sampled rows
+
+@pytest.mark.parametrize("wl,idx", [("dit_xl2", 0), ("dit_xl2", 1), ("sd3_mmdit", 0), ("sd3_mmdit", 1),
+                                    ("sd3_mmdit", 2), ("flux", 0), ("flux", 1), ("flux", 2), ("sdxl_skip", 0)])
+def test_full_size_layers_sampled_rows(wl, idx):
+    spec = WL.WORKLOADS[wl][idx]
+    rs = np.random.default_rng(99)
+    # first and last tile rows (ragged tail) plus random rows in between
+    rows = np.unique(np.concatenate([[0, 127, 128, spec.M - 1, spec.M - 2], rs.integers(0, spec.M, 19)]))
+    run_parity(spec, rows=rows)
+
+
+# ------------------------------------------------------------------ host-side errors through the loaded library
+
+def test_argument_errors_are_reported_before_launch():
+    spec = custom_spec("err", 64, 128, 64, [0, 128], [0, 64], True, "int8")
+    data = WL.make_layer(spec)
+    layer = SegQuantLinear(data.W, data.bias, spec.kb, spec.nb, True, "int8", DEV)
+    layer.calibrate(data.X_cal)
+    Xd = data.X.to(DEV)
+    n0 = B.segquant_launch_count()
+    bad_seg = B.SegTable([0, 64, 32, 128], [0, 64])
+    with pytest.raises(B.SegquantError) as e:
+        B.segquant_quantize_act(Xd, bad_seg, layer.s_pos, layer.s_neg, "int8")
+    assert e.value.status == 3
+    unaligned = B.SegTable([0, 40, 128], [0, 64])
+    c_pos, c_neg = B.segquant_quantize_act(Xd, layer.seg, layer.s_pos, layer.s_neg, "int8")
+    n1 = B.segquant_launch_count()
+    sp2 = torch.ones(2, device=DEV)
+    with pytest.raises(B.SegquantError) as e:
+        B.segquant_dualscale_gemm(c_pos, c_neg, layer.Wq, unaligned, "int8", sp2, sp2, torch.ones(2, device=DEV),
+                                  None, layer.workspace)
+    assert e.value.status == 4
+    with pytest.raises(B.SegquantError) as e:
+        B.segquant_dualscale_gemm(c_pos, c_neg, layer.Wq, layer.seg, "int8", layer.s_pos, layer.s_neg, layer.s_w,
+                                  None, torch.zeros(16, dtype=torch.uint8, device=DEV))
+    assert e.value.status == 8
+    assert B.segquant_launch_count() == n1 and n1 == n0 + 1
