@@ -12,7 +12,7 @@
 // Accumulators: NACC = P * npol, each 128 lanes x TILE_N columns; NACC * TILE_N <= 512 columns.
 // If they use at most half of TMEM the accumulator set is double-buffered so that the epilogue of
 // one tile overlaps the main loop of the next.
-// Every wait on an mbarrier is bounded (wall-clock limit); on expiry the CTA records which wait gave
+// Every wait on an mbarrier is bounded (SM cycle-counter limit, about 2 s); on expiry the CTA records which wait gave
 // up in the status word, stops issuing work, lets its own copies land and leaves normally.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -29,7 +29,7 @@ constexpr int kEpiThreads = 128;
 constexpr int kMaxStages = 8;
 constexpr int kTmemCols = 512;
 constexpr uint32_t kSmemBudget = 227 * 1024;
-constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
+constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s
 
 struct KernelParams {
     int M, N, K;
@@ -45,6 +45,7 @@ struct KernelParams {
     int y_is_f32;
     void *acc_dump;
     uint32_t *status;
+    int debug;         // timing experiments only: 1 = no TMA loads, 2 = no MMAs, 4 = no epilogue work
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -73,24 +74,20 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok;
 }
-__device__ __forceinline__ uint64_t globaltimer_ns()
-{
-    uint64_t t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-
-// Bounded wait.  Returns false if the wait expired or another role already gave up.
+// Bounded wait.  Returns false if the wait expired or another role already gave up.  The limit is
+// counted on the SM cycle counter; kWaitLimitCycles is about 2 s at the maximum SM clock.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
                                           uint32_t *status, uint32_t where)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = globaltimer_ns();
+    long long t0 = 0;
     uint32_t polls = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++polls & 255u) == 0) {
+        if ((++polls & 63u) == 0) {
             if (*abort_flag) return false;
-            if (globaltimer_ns() - t0 > kWaitLimitNs) {
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > kWaitLimitCycles) {
                 *abort_flag = 1;
                 atomicCAS(status, 0u, where);
                 return false;
@@ -183,16 +180,42 @@ struct SharedHeader {
 // where-codes written to the status word when a wait expires
 enum : uint32_t { kWhereProducer = 0x100, kWhereMmaFull = 0x200, kWhereMmaTmem = 0x300, kWhereEpilogue = 0x400 };
 
-template <int KIND, int TILE_N>
+// One K-block worth of MMAs: nk K-steps of 32 codes, each against every activation tile.
+template <int KIND, int NPOL, int TILE_N>
+__device__ __forceinline__ void issue_kblock(uint32_t d0, uint64_t da, uint64_t db, uint32_t idesc, int nk,
+                                             uint32_t accumulate)
+{
+    constexpr uint64_t kATileDesc = uint64_t(TILE_M * BLOCK_K) >> 4;   // next activation tile in the stage
+    if (nk == BLOCK_K / MMA_K) {
+#pragma unroll
+        for (int kk = 0; kk < BLOCK_K / MMA_K; kk++) {
+            const uint64_t koff = uint64_t((kk * MMA_K) >> 4);           // +32 B inside the swizzle row
+#pragma unroll
+            for (int pol = 0; pol < NPOL; pol++)
+                tc_mma<KIND>(d0 + pol * TILE_N, da + pol * kATileDesc + koff, db + koff, idesc,
+                             kk == 0 ? accumulate : 1u);
+        }
+    } else {
+        for (int kk = 0; kk < nk; kk++) {
+            const uint64_t koff = uint64_t((kk * MMA_K) >> 4);
+#pragma unroll
+            for (int pol = 0; pol < NPOL; pol++)
+                tc_mma<KIND>(d0 + pol * TILE_N, da + pol * kATileDesc + koff, db + koff, idesc,
+                             kk == 0 ? accumulate : 1u);
+        }
+    }
+}
+
+template <int KIND, int NPOL, int TILE_N>
 __global__ void __launch_bounds__(kThreads, 1)
 segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_constant__ CUtensorMap tm_a_neg,
                      const __grid_constant__ CUtensorMap tm_b, const KernelParams prm)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    // layout: [ring: stages x (npol A tiles of 16 KiB, B tile of TILE_N*128 B)] [scales] [header]
-    const uint32_t a_bytes = TILE_M * BLOCK_K;
-    const uint32_t b_bytes = TILE_N * BLOCK_K;
-    const uint32_t stage_bytes = prm.npol * a_bytes + b_bytes;
+    // layout: [ring: stages x (NPOL A tiles of 16 KiB, B tile of TILE_N*128 B)] [scales] [header]
+    constexpr uint32_t a_bytes = TILE_M * BLOCK_K;
+    constexpr uint32_t b_bytes = TILE_N * BLOCK_K;
+    constexpr uint32_t stage_bytes = NPOL * a_bytes + b_bytes;
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     float *sh_scale = reinterpret_cast<float *>(smem + size_t(prm.stages) * stage_bytes);   // [nacc][TILE_N]
     float *sh_bias = sh_scale + prm.nacc * TILE_N;                                           // [TILE_N]
@@ -227,39 +250,52 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     const uint32_t tmem_base = hdr->tmem_base;
     const int acc_cols = prm.nacc * TILE_N;     // TMEM columns of one accumulator set
 
+    // The producer and the MMA issuer are single threads: their loops are kept to a few dozen
+    // instructions per K-block (ring slot and phase advance incrementally, descriptors by addition).
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_a_pos)) : "memory");
+            if (NPOL == 2) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_a_neg)) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_b)) : "memory");
-            uint32_t it = 0;
+            const uint32_t stages = prm.stages, P = prm.sb.P, debug = prm.debug;
+            const uint32_t full0 = smem_u32(&hdr->full[0]), empty0 = smem_u32(&hdr->empty[0]);
+            const uint32_t ring0 = smem_u32(smem);
+            uint32_t s = 0, ph = 0, issued = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 const int m0 = (tile / prm.num_n_tiles) * TILE_M;
                 const int n0 = (tile % prm.num_n_tiles) * TILE_N;
-                for (int p = 0; p < prm.sb.P && ok; p++) {
-                    for (int k = prm.sb.kb[p]; k < prm.sb.kb[p + 1]; k += BLOCK_K, it++) {
-                        const uint32_t s = it % prm.stages, ph = (it / prm.stages) & 1;
-                        if (!mbar_wait(smem_u32(&hdr->empty[s]), ph ^ 1, abort_flag, prm.status, kWhereProducer)) {
+                for (uint32_t p = 0; p < P && ok; p++) {
+                    const int k_end = prm.sb.kb[p + 1];
+                    for (int k = prm.sb.kb[p]; k < k_end; k += BLOCK_K) {
+                        if (!mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag, prm.status, kWhereProducer)) {
                             ok = false;
                             break;
                         }
-                        const uint32_t bar = smem_u32(&hdr->full[s]);
-                        const uint32_t dst = smem_u32(smem + size_t(s) * stage_bytes);
-                        mbar_expect_tx(bar, stage_bytes);
-                        tma_load_2d(dst, &tm_a_pos, bar, k, m0);
-                        if (prm.npol == 2) tma_load_2d(dst + a_bytes, &tm_a_neg, bar, k, m0);
-                        tma_load_2d(dst + prm.npol * a_bytes, &tm_b, bar, k, n0);
+                        const uint32_t bar = full0 + 8 * s;
+                        const uint32_t dst = ring0 + s * stage_bytes;
+                        if (debug & 1) {
+                            mbar_arrive(bar);
+                        } else {
+                            mbar_expect_tx(bar, stage_bytes);
+                            tma_load_2d(dst, &tm_a_pos, bar, k, m0);
+                            if (NPOL == 2) tma_load_2d(dst + a_bytes, &tm_a_neg, bar, k, m0);
+                            tma_load_2d(dst + NPOL * a_bytes, &tm_b, bar, k, n0);
+                        }
+                        issued++;
+                        if (++s == stages) { s = 0; ph ^= 1; }
                     }
                 }
             }
             if (!ok) {
                 // let the copies this thread issued land before the CTA's shared memory goes away
-                const uint32_t pending = it < uint32_t(prm.stages) ? it : uint32_t(prm.stages);
+                const uint32_t pending = issued < stages ? issued : stages;
                 for (uint32_t j = 0; j < pending; j++) {
-                    const uint32_t i2 = it - 1 - j, s = i2 % prm.stages, ph = (i2 / prm.stages) & 1;
-                    const uint64_t t0 = globaltimer_ns();
-                    while (!mbar_try_wait(smem_u32(&hdr->full[s]), ph) && globaltimer_ns() - t0 < 100000000ull) {}
+                    if (s == 0) { s = stages; ph ^= 1; }
+                    s--;
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(full0 + 8 * s, ph) && clock64() - t0 < 200000000ll) {}
                 }
             }
         }
@@ -267,53 +303,70 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc(KIND, TILE_N);
-            uint32_t it = 0, tile_iter = 0;
+            const uint32_t stages = prm.stages, P = prm.sb.P, debug = prm.debug, acc_stages = prm.acc_stages;
+            const uint32_t full0 = smem_u32(&hdr->full[0]), empty0 = smem_u32(&hdr->empty[0]);
+            const uint64_t desc0 = make_smem_desc(smem_u32(smem));
+            constexpr uint64_t kStageDesc = uint64_t(stage_bytes) >> 4;
+            constexpr uint64_t kBDesc = uint64_t(NPOL * a_bytes) >> 4;
+            uint32_t s = 0, ph = 0, as = 0, aph = 0;
+            long long prof[4] = {0, 0, 0, 0};
+            uint32_t prof_n = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, tile_iter++) {
-                const uint32_t as = tile_iter % prm.acc_stages, aph = (tile_iter / prm.acc_stages) & 1;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 if (!mbar_wait(smem_u32(&hdr->tmem_empty[as]), aph ^ 1, abort_flag, prm.status, kWhereMmaTmem)) {
                     ok = false;
                     break;
                 }
                 tc_fence_after();
-                for (int p = 0; p < prm.sb.P && ok; p++) {
-                    const uint32_t d0 = tmem_base + as * acc_cols + uint32_t(p * prm.npol) * TILE_N;
+                for (uint32_t p = 0; p < P && ok; p++) {
+                    const uint32_t d0 = tmem_base + as * acc_cols + p * (NPOL * TILE_N);
+                    const int k_end = prm.sb.kb[p + 1];
                     uint32_t accumulate = 0;
-                    for (int k = prm.sb.kb[p]; k < prm.sb.kb[p + 1]; k += BLOCK_K, it++) {
-                        const uint32_t s = it % prm.stages, ph = (it / prm.stages) & 1;
-                        if (!mbar_wait(smem_u32(&hdr->full[s]), ph, abort_flag, prm.status, kWhereMmaFull)) {
+                    for (int k = prm.sb.kb[p]; k < k_end; k += BLOCK_K) {
+                        long long t0 = 0, t1 = 0, t2 = 0, t3 = 0;
+                        if (debug & 32) t0 = clock64();
+                        if (!mbar_wait(full0 + 8 * s, ph, abort_flag, prm.status, kWhereMmaFull)) {
                             ok = false;
                             break;
                         }
+                        if (debug & 32) t1 = clock64();
                         tc_fence_after();
-                        const uint32_t base = smem_u32(smem + size_t(s) * stage_bytes);
-                        const uint64_t da0 = make_smem_desc(base);
-                        const uint64_t da1 = make_smem_desc(base + a_bytes);
-                        const uint64_t db = make_smem_desc(base + prm.npol * a_bytes);
-                        const int rem = prm.sb.kb[p + 1] - k;
+                        if (debug & 32) t2 = clock64();
+                        const uint64_t da = desc0 + s * kStageDesc;
+                        const int rem = k_end - k;
                         const int nk = rem >= BLOCK_K ? BLOCK_K / MMA_K : (rem + MMA_K - 1) / MMA_K;
-                        for (int kk = 0; kk < nk; kk++) {
-                            const uint64_t koff = uint64_t((kk * MMA_K) >> 4);   // +32 B inside the swizzle row
-                            tc_mma<KIND>(d0, da0 + koff, db + koff, idesc, accumulate);
-                            if (prm.npol == 2) tc_mma<KIND>(d0 + TILE_N, da1 + koff, db + koff, idesc, accumulate);
-                            accumulate = 1;
+                        if (!(debug & 2)) issue_kblock<KIND, NPOL, TILE_N>(d0, da, da + kBDesc, idesc, nk, accumulate);
+                        accumulate = 1;
+                        if (debug & 32) t3 = clock64();
+                        tc_commit(empty0 + 8 * s);                 // frees the ring slot when these MMAs retire
+                        if (debug & 32) {
+                            const long long t4 = clock64();
+                            prof[0] += t1 - t0; prof[1] += t2 - t1; prof[2] += t3 - t2; prof[3] += t4 - t3;
+                            prof_n++;
                         }
-                        tc_commit(smem_u32(&hdr->empty[s]));      // frees the ring slot when these MMAs retire
+                        if (++s == stages) { s = 0; ph ^= 1; }
                     }
                 }
                 if (ok) tc_commit(smem_u32(&hdr->tmem_full[as]));  // accumulators of this tile complete
+                if (++as == acc_stages) { as = 0; aph ^= 1; }
+            }
+            if ((debug & 32) && blockIdx.x == 0) {
+                // timing experiment: average cycles of wait / fence / MMA issue / commit per K-block
+                for (int i = 0; i < 4; i++) prm.status[16 + i] = uint32_t(prof[i] / (prof_n ? prof_n : 1));
+                prm.status[20] = prof_n;
             }
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
         const int et = threadIdx.x - 64;           // 0..127
         const int lane_grp = warp & 3;             // TMEM lanes 32*lane_grp .. +31 are this warp's
-        uint32_t tile_iter = 0;
+        uint32_t as = 0, aph = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, tile_iter++) {
+        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
             const int m0 = (tile / prm.num_n_tiles) * TILE_M;
             const int n0 = (tile % prm.num_n_tiles) * TILE_N;
-            const uint32_t as = tile_iter % prm.acc_stages, aph = (tile_iter / prm.acc_stages) & 1;
+            const uint32_t cur_as = as, cur_aph = aph;
+            if (++as == uint32_t(prm.acc_stages)) { as = 0; aph ^= 1; }
 
             // per-column dequantization factors of this tile: c[a][j] = s_act[p][pol] * s_w[p][q(n0+j)]
             asm volatile("bar.sync 1, 128;" ::: "memory");       // previous tile's readers are done
@@ -323,19 +376,20 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                 while (q + 1 < prm.sb.Q && n >= prm.sb.nb[q + 1]) q++;
                 for (int p = 0; p < prm.sb.P; p++) {
                     const float sw = n < prm.N ? prm.s_w[p * prm.sb.Q + q] : 0.0f;
-                    sh_scale[(p * prm.npol) * TILE_N + j] = prm.s_pos[p] * sw;
-                    if (prm.npol == 2) sh_scale[(p * prm.npol + 1) * TILE_N + j] = prm.s_neg[p] * sw;
+                    sh_scale[(p * NPOL) * TILE_N + j] = prm.s_pos[p] * sw;
+                    if (NPOL == 2) sh_scale[(p * NPOL + 1) * TILE_N + j] = prm.s_neg[p] * sw;
                 }
                 sh_bias[j] = (prm.bias && n < prm.N) ? prm.bias[n] : 0.0f;
             }
             asm volatile("bar.sync 1, 128;" ::: "memory");
 
-            if (ok) ok = mbar_wait(smem_u32(&hdr->tmem_full[as]), aph, abort_flag, prm.status, kWhereEpilogue);
+            if (ok) ok = mbar_wait(smem_u32(&hdr->tmem_full[cur_as]), cur_aph, abort_flag, prm.status, kWhereEpilogue);
             if (!ok) continue;                      // keep the named barriers balanced, do no more work
             tc_fence_after();
+            if (prm.debug & 4) { tc_fence_before(); mbar_arrive(smem_u32(&hdr->tmem_empty[cur_as])); continue; }
 
             const int row = m0 + lane_grp * 32 + lane;
-            const uint32_t t_row = tmem_base + (uint32_t(lane_grp * 32) << 16) + as * acc_cols;
+            const uint32_t t_row = tmem_base + (uint32_t(lane_grp * 32) << 16) + cur_as * acc_cols;
 #pragma unroll 1
             for (int c0 = 0; c0 < TILE_N; c0 += 32) {
                 float y[32];
@@ -387,7 +441,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                 }
             }
             tc_fence_before();
-            mbar_arrive(smem_u32(&hdr->tmem_empty[as]));
+            mbar_arrive(smem_u32(&hdr->tmem_empty[cur_as]));
         }
     }
 
@@ -435,9 +489,9 @@ bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, in
     return r == CUDA_SUCCESS;
 }
 
-int g_tune_tile_n = 0, g_tune_stages = 0;
+int g_tune_tile_n = 0, g_tune_stages = 0, g_tune_debug = 0;
 
-template <int KIND, int TILE_N>
+template <int KIND, int NPOL, int TILE_N>
 sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cudaStream_t st)
 {
     CUtensorMap ta, tn, tb;
@@ -456,7 +510,7 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
     prm.num_n_tiles = int((g.N + TILE_N - 1) / TILE_N);
     const size_t smem = 1024 + size_t(stages) * stage_bytes + tail;
 
-    auto kern = segquant_gemm_kernel<KIND, TILE_N>;
+    auto kern = segquant_gemm_kernel<KIND, NPOL, TILE_N>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
         return SQ_ERR_CUDA;
     const int tiles = prm.num_m_tiles * prm.num_n_tiles;
@@ -469,11 +523,20 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
 template <int KIND>
 sq_status launch_kind(const GemmArgs &g, KernelParams &prm, int tile_n, int sm_count, cudaStream_t st)
 {
-    switch (tile_n) {
-        case 256: return launch_variant<KIND, 256>(g, prm, sm_count, st);
-        case 128: return launch_variant<KIND, 128>(g, prm, sm_count, st);
-        case 64: return launch_variant<KIND, 64>(g, prm, sm_count, st);
-        case 32: return launch_variant<KIND, 32>(g, prm, sm_count, st);
+    if (prm.npol == 2) {
+        switch (tile_n) {
+            case 256: return launch_variant<KIND, 2, 256>(g, prm, sm_count, st);
+            case 128: return launch_variant<KIND, 2, 128>(g, prm, sm_count, st);
+            case 64: return launch_variant<KIND, 2, 64>(g, prm, sm_count, st);
+            case 32: return launch_variant<KIND, 2, 32>(g, prm, sm_count, st);
+        }
+    } else {
+        switch (tile_n) {
+            case 256: return launch_variant<KIND, 1, 256>(g, prm, sm_count, st);
+            case 128: return launch_variant<KIND, 1, 128>(g, prm, sm_count, st);
+            case 64: return launch_variant<KIND, 1, 64>(g, prm, sm_count, st);
+            case 32: return launch_variant<KIND, 1, 32>(g, prm, sm_count, st);
+        }
     }
     return SQ_ERR_UNSUPPORTED;
 }
@@ -483,7 +546,8 @@ sq_status launch_kind(const GemmArgs &g, KernelParams &prm, int tile_n, int sm_c
 void set_gemm_tuning(int tile_n, int stages)
 {
     g_tune_tile_n = tile_n;
-    g_tune_stages = stages;
+    g_tune_stages = stages & 0xFF;
+    g_tune_debug = stages >> 8;
 }
 
 sq_status launch_gemm(const GemmArgs &g, cudaStream_t st)
@@ -497,6 +561,7 @@ sq_status launch_gemm(const GemmArgs &g, cudaStream_t st)
     prm.Y = g.Y; prm.ldy = g.ldy; prm.y_is_f32 = g.y_dtype == SQ_F32;
     prm.acc_dump = g.acc_dump;
     prm.status = g.status;
+    prm.debug = g_tune_debug;
 
     // widest tile whose accumulators fit the 512 TMEM columns
     int tile_n = 256;
