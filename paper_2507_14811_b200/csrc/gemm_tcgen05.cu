@@ -45,7 +45,6 @@ struct KernelParams {
     int y_is_f32;
     void *acc_dump;
     uint32_t *status;
-    int debug;         // timing experiments only: 1 = no TMA loads, 2 = no MMAs, 4 = no epilogue work
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -258,7 +257,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_a_pos)) : "memory");
             if (NPOL == 2) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_a_neg)) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_b)) : "memory");
-            const uint32_t stages = prm.stages, P = prm.sb.P, debug = prm.debug;
+            const uint32_t stages = prm.stages, P = prm.sb.P;
             const uint32_t full0 = smem_u32(&hdr->full[0]), empty0 = smem_u32(&hdr->empty[0]);
             const uint32_t ring0 = smem_u32(smem);
             uint32_t s = 0, ph = 0, issued = 0;
@@ -275,14 +274,10 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                         }
                         const uint32_t bar = full0 + 8 * s;
                         const uint32_t dst = ring0 + s * stage_bytes;
-                        if (debug & 1) {
-                            mbar_arrive(bar);
-                        } else {
-                            mbar_expect_tx(bar, stage_bytes);
-                            tma_load_2d(dst, &tm_a_pos, bar, k, m0);
-                            if (NPOL == 2) tma_load_2d(dst + a_bytes, &tm_a_neg, bar, k, m0);
-                            tma_load_2d(dst + NPOL * a_bytes, &tm_b, bar, k, n0);
-                        }
+                        mbar_expect_tx(bar, stage_bytes);
+                        tma_load_2d(dst, &tm_a_pos, bar, k, m0);
+                        if (NPOL == 2) tma_load_2d(dst + a_bytes, &tm_a_neg, bar, k, m0);
+                        tma_load_2d(dst + NPOL * a_bytes, &tm_b, bar, k, n0);
                         issued++;
                         if (++s == stages) { s = 0; ph ^= 1; }
                     }
@@ -303,14 +298,12 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc(KIND, TILE_N);
-            const uint32_t stages = prm.stages, P = prm.sb.P, debug = prm.debug, acc_stages = prm.acc_stages;
+            const uint32_t stages = prm.stages, P = prm.sb.P, acc_stages = prm.acc_stages;
             const uint32_t full0 = smem_u32(&hdr->full[0]), empty0 = smem_u32(&hdr->empty[0]);
             const uint64_t desc0 = make_smem_desc(smem_u32(smem));
             constexpr uint64_t kStageDesc = uint64_t(stage_bytes) >> 4;
             constexpr uint64_t kBDesc = uint64_t(NPOL * a_bytes) >> 4;
             uint32_t s = 0, ph = 0, as = 0, aph = 0;
-            long long prof[4] = {0, 0, 0, 0};
-            uint32_t prof_n = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 if (!mbar_wait(smem_u32(&hdr->tmem_empty[as]), aph ^ 1, abort_flag, prm.status, kWhereMmaTmem)) {
@@ -323,37 +316,22 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                     const int k_end = prm.sb.kb[p + 1];
                     uint32_t accumulate = 0;
                     for (int k = prm.sb.kb[p]; k < k_end; k += BLOCK_K) {
-                        long long t0 = 0, t1 = 0, t2 = 0, t3 = 0;
-                        if (debug & 32) t0 = clock64();
                         if (!mbar_wait(full0 + 8 * s, ph, abort_flag, prm.status, kWhereMmaFull)) {
                             ok = false;
                             break;
                         }
-                        if (debug & 32) t1 = clock64();
                         tc_fence_after();
-                        if (debug & 32) t2 = clock64();
                         const uint64_t da = desc0 + s * kStageDesc;
                         const int rem = k_end - k;
                         const int nk = rem >= BLOCK_K ? BLOCK_K / MMA_K : (rem + MMA_K - 1) / MMA_K;
-                        if (!(debug & 2)) issue_kblock<KIND, NPOL, TILE_N>(d0, da, da + kBDesc, idesc, nk, accumulate);
+                        issue_kblock<KIND, NPOL, TILE_N>(d0, da, da + kBDesc, idesc, nk, accumulate);
                         accumulate = 1;
-                        if (debug & 32) t3 = clock64();
                         tc_commit(empty0 + 8 * s);                 // frees the ring slot when these MMAs retire
-                        if (debug & 32) {
-                            const long long t4 = clock64();
-                            prof[0] += t1 - t0; prof[1] += t2 - t1; prof[2] += t3 - t2; prof[3] += t4 - t3;
-                            prof_n++;
-                        }
                         if (++s == stages) { s = 0; ph ^= 1; }
                     }
                 }
                 if (ok) tc_commit(smem_u32(&hdr->tmem_full[as]));  // accumulators of this tile complete
                 if (++as == acc_stages) { as = 0; aph ^= 1; }
-            }
-            if ((debug & 32) && blockIdx.x == 0) {
-                // timing experiment: average cycles of wait / fence / MMA issue / commit per K-block
-                for (int i = 0; i < 4; i++) prm.status[16 + i] = uint32_t(prof[i] / (prof_n ? prof_n : 1));
-                prm.status[20] = prof_n;
             }
         }
     } else {
@@ -386,7 +364,6 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
             if (ok) ok = mbar_wait(smem_u32(&hdr->tmem_full[cur_as]), cur_aph, abort_flag, prm.status, kWhereEpilogue);
             if (!ok) continue;                      // keep the named barriers balanced, do no more work
             tc_fence_after();
-            if (prm.debug & 4) { tc_fence_before(); mbar_arrive(smem_u32(&hdr->tmem_empty[cur_as])); continue; }
 
             const int row = m0 + lane_grp * 32 + lane;
             const uint32_t t_row = tmem_base + (uint32_t(lane_grp * 32) << 16) + cur_as * acc_cols;
@@ -489,7 +466,7 @@ bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, in
     return r == CUDA_SUCCESS;
 }
 
-int g_tune_tile_n = 0, g_tune_stages = 0, g_tune_debug = 0;
+int g_tune_tile_n = 0, g_tune_stages = 0;
 
 template <int KIND, int NPOL, int TILE_N>
 sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cudaStream_t st)
@@ -546,8 +523,7 @@ sq_status launch_kind(const GemmArgs &g, KernelParams &prm, int tile_n, int sm_c
 void set_gemm_tuning(int tile_n, int stages)
 {
     g_tune_tile_n = tile_n;
-    g_tune_stages = stages & 0xFF;
-    g_tune_debug = stages >> 8;
+    g_tune_stages = stages;
 }
 
 sq_status launch_gemm(const GemmArgs &g, cudaStream_t st)
@@ -561,7 +537,6 @@ sq_status launch_gemm(const GemmArgs &g, cudaStream_t st)
     prm.Y = g.Y; prm.ldy = g.ldy; prm.y_is_f32 = g.y_dtype == SQ_F32;
     prm.acc_dump = g.acc_dump;
     prm.status = g.status;
-    prm.debug = g_tune_debug;
 
     // widest tile whose accumulators fit the 512 TMEM columns
     int tile_n = 256;
