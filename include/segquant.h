@@ -161,9 +161,10 @@ sq_status segquant_layer_forward(const void *X, int x_on_host, void *x_stage, sq
 sq_status segquant_last_device_status(void *workspace, void *stream, uint32_t *detail);
 
 /* Tile plan of the GEMM kernel: tile_n in {0 (automatic), 32, 64, 128, 256}; stages 0 (automatic) or
- * 2..8.  Process-wide; meant for benchmarking sweeps.  Values the layer cannot use are replaced by
- * the automatic choice. */
-sq_status segquant_set_tuning(int tile_n, int stages);
+ * 2..8 (shared-memory ring depth); cta_group 0 (automatic: CTA pairs on 256-row tiles when M > 128),
+ * 1 (one CTA per 128-row tile) or 2.  Process-wide; meant for benchmarking sweeps and tests.  Values
+ * the layer cannot use are replaced by the automatic choice. */
+sq_status segquant_set_tuning(int tile_n, int stages, int cta_group);
 
 /* Number of kernels the library has launched in this process (all entry points). */
 uint64_t segquant_launch_count(void);

@@ -220,9 +220,9 @@ sq_status segquant_last_device_status(void *workspace, void *stream, uint32_t *d
     return SQ_ERR_TIMEOUT;
 }
 
-sq_status segquant_set_tuning(int tile_n, int stages)
+sq_status segquant_set_tuning(int tile_n, int stages, int cta_group)
 {
-    set_gemm_tuning(tile_n, stages);
+    set_gemm_tuning(tile_n, stages, cta_group);
     return SQ_OK;
 }
 

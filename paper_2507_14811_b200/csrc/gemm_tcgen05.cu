@@ -1,19 +1,25 @@
 // W8A8 GEMM + dequantizing epilogue for sm_100a (Sec. 4.2.2 segment-wise products, Sec. 4.3.2 dual
 // path recombination, App. A symmetric recovery).
 //
-// One persistent CTA per SM, 192 threads:
-//   warp 0      TMA producer: per 128-byte K-block, one tile of each activation code matrix
-//               (128 rows) and ONE weight tile (TILE_N rows) into a shared-memory ring
-//   warp 1      tcgen05.mma issuer (one elected lane): for every 32-byte K-step, one MMA per polarity
-//               against the same weight tile, each polarity and each K-segment into its own
-//               accumulator in tensor memory (TMEM)
-//   warps 2..5  epilogue: tcgen05.ld of all accumulators of a 32-column slab, fp32 FMA with the
-//               per-(segment, polarity, column) scale, + bias, -> bf16 / fp32 store
+// Persistent kernel, one CTA per SM, 320 threads.  With CG = 2 two neighbouring CTAs (a cluster of
+// two) work on one 256-row output tile with tcgen05 cta_group::2: each CTA loads its own 128
+// activation rows and HALF of the weight tile, the pair's leader issues every MMA, and each CTA
+// holds the accumulators of its own 128 rows in its tensor memory (TMEM).  CG = 1 is the same
+// kernel with one CTA per 128-row tile (used when M <= 128).
+//   warp 0      TMA producer (one lane): per 128-byte K-block, one tile of each activation code
+//               matrix and this CTA's part of ONE weight tile into a shared-memory ring
+//   warp 1      tcgen05.mma issuer (one lane, leader CTA only): for every 32-byte K-step one MMA per
+//               polarity against the same weight tile; every (K-segment, polarity) has its own
+//               accumulator in TMEM
+//   warps 2..9  epilogue: tcgen05.ld of all accumulators of a 32-column slab, fp32 FMA with the
+//               per-(segment, polarity, column) scale, + bias, -> bf16 / fp32, staged in shared
+//               memory and written by TMA stores (whole sectors, clipped at the matrix edge)
 // Accumulators: NACC = P * npol, each 128 lanes x TILE_N columns; NACC * TILE_N <= 512 columns.
 // If they use at most half of TMEM the accumulator set is double-buffered so that the epilogue of
 // one tile overlaps the main loop of the next.
-// Every wait on an mbarrier is bounded (SM cycle-counter limit, about 2 s); on expiry the CTA records which wait gave
-// up in the status word, stops issuing work, lets its own copies land and leaves normally.
+// Every wait on an mbarrier is bounded (SM cycle counter, about 2 s); on expiry the CTA records
+// which wait gave up in the status word, stops issuing work, lets its own copies land and leaves
+// normally.  No load uses cluster multicast.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include "sq_common.cuh"
@@ -21,27 +27,27 @@
 namespace sq {
 namespace {
 
-constexpr int TILE_M = 128;
+constexpr int TILE_M = 128;           // rows per CTA (TMEM lanes)
 constexpr int BLOCK_K = 128;          // bytes (= codes) per K-block: one 128B swizzle row
 constexpr int MMA_K = 32;             // codes per tcgen05.mma of an 8-bit kind
-constexpr int kThreads = 192;
-constexpr int kEpiThreads = 128;
+constexpr int kEpiWarps = 8;
+constexpr int kEpiThreads = kEpiWarps * 32;
+constexpr int kThreads = 64 + kEpiThreads;
 constexpr int kMaxStages = 8;
 constexpr int kTmemCols = 512;
 constexpr uint32_t kSmemBudget = 227 * 1024;
+constexpr uint32_t kStageBufBytes = 32 * 64;            // output staging: 32 rows x 64 bytes
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s
 
 struct KernelParams {
     int M, N, K;
-    int npol;          // 1 or 2 activation code matrices
     int nacc;          // P * npol
     int acc_stages;    // 1 or 2 accumulator sets in TMEM
     int stages;        // shared-memory ring depth
+    int out_bufs;      // 1 or 2 output staging buffers per epilogue warp
     int num_m_tiles, num_n_tiles;
     SegBounds sb;
     const float *s_pos, *s_neg, *s_w, *bias;
-    void *Y;
-    long long ldy;
     int y_is_f32;
     void *acc_dump;
     uint32_t *status;
@@ -50,6 +56,25 @@ struct KernelParams {
 // ----------------------------------------------------------------------------- PTX wrappers
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return uint32_t(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
@@ -62,6 +87,11 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// arrive on a barrier given by a shared::cluster address (possibly in the peer CTA)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 {
@@ -96,34 +126,71 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return true;
 }
 
+// 2-D tiled TMA load into this CTA's shared memory; completion bytes go to `bar`, which for CG = 2
+// is a shared::cluster address (the leader CTA's barrier).
+template <int CG>
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
 {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y) : "memory");
+    if (CG == 1)
+        asm volatile(
+            "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+            ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y) : "memory");
+    else
+        asm volatile(
+            "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+            ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y) : "memory");
 }
+
+// 2-D tiled TMA store of a staged box from this CTA's shared memory (bulk async-group completion).
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// Arrives on `bar` once every MMA issued so far by this thread has retired.  CG = 2: the arrival is
+// delivered to the barrier at the same shared-memory offset in both CTAs of the pair.
+template <int CG>
 __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    if (CG == 1)
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    else
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(bar), "h"(uint16_t(3)) : "memory");
 }
 
-template <int KIND>   // 0: kind::i8, 1: kind::f8f6f4
+template <int KIND, int CG>   // KIND 0: kind::i8, 1: kind::f8f6f4
 __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                        uint32_t accumulate)
 {
-    if (KIND == 0)
+    if (KIND == 0 && CG == 1)
         asm volatile(
             "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
             "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
             ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-    else
+    else if (KIND == 0)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    else if (CG == 1)
         asm volatile(
             "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
             "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
             ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
@@ -158,11 +225,11 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr)
 
 // Instruction descriptor: D format bits 4-5 (1 = f32, 2 = s32), A format bits 7-9, B format bits
 // 10-12 (kind::i8: 1 = signed 8-bit; kind::f8f6f4: 0 = e4m3), A and B K-major (bits 15, 16 = 0),
-// N >> 3 in bits 17-22, M >> 4 in bits 24-28.
-__host__ __device__ constexpr uint32_t make_idesc(int kind, int tile_n)
+// N >> 3 in bits 17-22, M >> 4 in bits 24-28 (M = 128 per CTA, 256 for a CTA pair).
+__host__ __device__ constexpr uint32_t make_idesc(int kind, int tile_n, int mma_m)
 {
     return (kind == 0 ? (2u << 4) | (1u << 7) | (1u << 10) : (1u << 4)) |
-           (uint32_t(tile_n >> 3) << 17) | (uint32_t(TILE_M >> 4) << 24);
+           (uint32_t(tile_n >> 3) << 17) | (uint32_t(mma_m >> 4) << 24);
 }
 
 // ----------------------------------------------------------------------------- the kernel
@@ -180,7 +247,7 @@ struct SharedHeader {
 enum : uint32_t { kWhereProducer = 0x100, kWhereMmaFull = 0x200, kWhereMmaTmem = 0x300, kWhereEpilogue = 0x400 };
 
 // One K-block worth of MMAs: nk K-steps of 32 codes, each against every activation tile.
-template <int KIND, int NPOL, int TILE_N>
+template <int KIND, int NPOL, int TILE_N, int CG>
 __device__ __forceinline__ void issue_kblock(uint32_t d0, uint64_t da, uint64_t db, uint32_t idesc, int nk,
                                              uint32_t accumulate)
 {
@@ -191,37 +258,42 @@ __device__ __forceinline__ void issue_kblock(uint32_t d0, uint64_t da, uint64_t 
             const uint64_t koff = uint64_t((kk * MMA_K) >> 4);           // +32 B inside the swizzle row
 #pragma unroll
             for (int pol = 0; pol < NPOL; pol++)
-                tc_mma<KIND>(d0 + pol * TILE_N, da + pol * kATileDesc + koff, db + koff, idesc,
-                             kk == 0 ? accumulate : 1u);
+                tc_mma<KIND, CG>(d0 + pol * TILE_N, da + pol * kATileDesc + koff, db + koff, idesc,
+                                 kk == 0 ? accumulate : 1u);
         }
     } else {
         for (int kk = 0; kk < nk; kk++) {
             const uint64_t koff = uint64_t((kk * MMA_K) >> 4);
 #pragma unroll
             for (int pol = 0; pol < NPOL; pol++)
-                tc_mma<KIND>(d0 + pol * TILE_N, da + pol * kATileDesc + koff, db + koff, idesc,
-                             kk == 0 ? accumulate : 1u);
+                tc_mma<KIND, CG>(d0 + pol * TILE_N, da + pol * kATileDesc + koff, db + koff, idesc,
+                                 kk == 0 ? accumulate : 1u);
         }
     }
 }
 
-template <int KIND, int NPOL, int TILE_N>
+template <int KIND, int NPOL, int TILE_N, int CG>
 __global__ void __launch_bounds__(kThreads, 1)
 segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_constant__ CUtensorMap tm_a_neg,
-                     const __grid_constant__ CUtensorMap tm_b, const KernelParams prm)
+                     const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_y,
+                     const KernelParams prm)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    // layout: [ring: stages x (NPOL A tiles of 16 KiB, B tile of TILE_N*128 B)] [scales] [header]
+    // layout: [ring: stages x (NPOL A tiles of 16 KiB, B part of B_ROWS*128 B)] [output staging] [scales] [header]
+    constexpr int B_ROWS = TILE_N / CG;                  // weight rows this CTA loads per K-block
     constexpr uint32_t a_bytes = TILE_M * BLOCK_K;
-    constexpr uint32_t b_bytes = TILE_N * BLOCK_K;
+    constexpr uint32_t b_bytes = B_ROWS * BLOCK_K;
     constexpr uint32_t stage_bytes = NPOL * a_bytes + b_bytes;
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    float *sh_scale = reinterpret_cast<float *>(smem + size_t(prm.stages) * stage_bytes);   // [nacc][TILE_N]
-    float *sh_bias = sh_scale + prm.nacc * TILE_N;                                           // [TILE_N]
+    uint8_t *sh_out = smem + size_t(prm.stages) * stage_bytes;                             // [warp][out_bufs][2 KiB]
+    float *sh_scale = reinterpret_cast<float *>(sh_out + kEpiWarps * prm.out_bufs * kStageBufBytes);  // [nacc][TILE_N]
+    float *sh_bias = sh_scale + prm.nacc * TILE_N;                                          // [TILE_N]
     SharedHeader *hdr = reinterpret_cast<SharedHeader *>(sh_bias + TILE_N);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    const uint32_t rank = CG == 2 ? cluster_rank() : 0u;       // 0 = leader of the pair
+    const int unit = blockIdx.x / CG, num_units = gridDim.x / CG;
     const int num_tiles = prm.num_m_tiles * prm.num_n_tiles;
     volatile uint32_t *abort_flag = &hdr->abort_flag;
 
@@ -232,19 +304,26 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
         }
         for (int s = 0; s < 2; s++) {
             mbar_init(smem_u32(&hdr->tmem_full[s]), 1);
-            mbar_init(smem_u32(&hdr->tmem_empty[s]), kEpiThreads);
+            mbar_init(smem_u32(&hdr->tmem_empty[s]), CG * kEpiWarps);
         }
         hdr->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(&hdr->tmem_base)), "r"(uint32_t(kTmemCols)) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (CG == 1) {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(&hdr->tmem_base)), "r"(uint32_t(kTmemCols)) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(&hdr->tmem_base)), "r"(uint32_t(kTmemCols)) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (CG == 2) cluster_sync_all();          // the peer's barriers are initialised before anyone signals them
     tc_fence_after();
     const uint32_t tmem_base = hdr->tmem_base;
     const int acc_cols = prm.nacc * TILE_N;     // TMEM columns of one accumulator set
@@ -259,12 +338,14 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_b)) : "memory");
             const uint32_t stages = prm.stages, P = prm.sb.P;
             const uint32_t full0 = smem_u32(&hdr->full[0]), empty0 = smem_u32(&hdr->empty[0]);
+            // completion bytes of both CTAs' loads are counted on the leader's barrier
+            const uint32_t full0_sig = CG == 2 ? map_to_cta(full0, 0) : full0;
             const uint32_t ring0 = smem_u32(smem);
             uint32_t s = 0, ph = 0, issued = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile / prm.num_n_tiles) * TILE_M;
-                const int n0 = (tile % prm.num_n_tiles) * TILE_N;
+            for (int tile = unit; tile < num_tiles && ok; tile += num_units) {
+                const int m0 = (tile / prm.num_n_tiles) * (TILE_M * CG) + int(rank) * TILE_M;
+                const int n0 = (tile % prm.num_n_tiles) * TILE_N + int(rank) * B_ROWS;
                 for (uint32_t p = 0; p < P && ok; p++) {
                     const int k_end = prm.sb.kb[p + 1];
                     for (int k = prm.sb.kb[p]; k < k_end; k += BLOCK_K) {
@@ -272,18 +353,18 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                             ok = false;
                             break;
                         }
-                        const uint32_t bar = full0 + 8 * s;
                         const uint32_t dst = ring0 + s * stage_bytes;
-                        mbar_expect_tx(bar, stage_bytes);
-                        tma_load_2d(dst, &tm_a_pos, bar, k, m0);
-                        if (NPOL == 2) tma_load_2d(dst + a_bytes, &tm_a_neg, bar, k, m0);
-                        tma_load_2d(dst + NPOL * a_bytes, &tm_b, bar, k, n0);
+                        if (rank == 0) mbar_expect_tx(full0 + 8 * s, CG * stage_bytes);
+                        const uint32_t bar = full0_sig + 8 * s;
+                        tma_load_2d<CG>(dst, &tm_a_pos, bar, k, m0);
+                        if (NPOL == 2) tma_load_2d<CG>(dst + a_bytes, &tm_a_neg, bar, k, m0);
+                        tma_load_2d<CG>(dst + NPOL * a_bytes, &tm_b, bar, k, n0);
                         issued++;
                         if (++s == stages) { s = 0; ph ^= 1; }
                     }
                 }
             }
-            if (!ok) {
+            if (!ok && rank == 0) {
                 // let the copies this thread issued land before the CTA's shared memory goes away
                 const uint32_t pending = issued < stages ? issued : stages;
                 for (uint32_t j = 0; j < pending; j++) {
@@ -295,9 +376,9 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(KIND, TILE_N);
+        // ------------------------------------------------------------------ MMA issuer (leader CTA)
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = make_idesc(KIND, TILE_N, TILE_M * CG);
             const uint32_t stages = prm.stages, P = prm.sb.P, acc_stages = prm.acc_stages;
             const uint32_t full0 = smem_u32(&hdr->full[0]), empty0 = smem_u32(&hdr->empty[0]);
             const uint64_t desc0 = make_smem_desc(smem_u32(smem));
@@ -305,7 +386,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
             constexpr uint64_t kBDesc = uint64_t(NPOL * a_bytes) >> 4;
             uint32_t s = 0, ph = 0, as = 0, aph = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            for (int tile = unit; tile < num_tiles && ok; tile += num_units) {
                 if (!mbar_wait(smem_u32(&hdr->tmem_empty[as]), aph ^ 1, abort_flag, prm.status, kWhereMmaTmem)) {
                     ok = false;
                     break;
@@ -324,30 +405,39 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                         const uint64_t da = desc0 + s * kStageDesc;
                         const int rem = k_end - k;
                         const int nk = rem >= BLOCK_K ? BLOCK_K / MMA_K : (rem + MMA_K - 1) / MMA_K;
-                        issue_kblock<KIND, NPOL, TILE_N>(d0, da, da + kBDesc, idesc, nk, accumulate);
+                        issue_kblock<KIND, NPOL, TILE_N, CG>(d0, da, da + kBDesc, idesc, nk, accumulate);
                         accumulate = 1;
-                        tc_commit(empty0 + 8 * s);                 // frees the ring slot when these MMAs retire
+                        tc_commit<CG>(empty0 + 8 * s);             // frees the ring slot when these MMAs retire
                         if (++s == stages) { s = 0; ph ^= 1; }
                     }
                 }
-                if (ok) tc_commit(smem_u32(&hdr->tmem_full[as]));  // accumulators of this tile complete
+                if (ok) tc_commit<CG>(smem_u32(&hdr->tmem_full[as]));  // accumulators of this tile complete
                 if (++as == acc_stages) { as = 0; aph ^= 1; }
             }
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
-        const int et = threadIdx.x - 64;           // 0..127
+        const int et = threadIdx.x - 64;           // 0..255
+        const int ew = warp - 2;                   // 0..7
         const int lane_grp = warp & 3;             // TMEM lanes 32*lane_grp .. +31 are this warp's
-        uint32_t as = 0, aph = 0;
+        const int col_half = ew >> 2;              // which half of the tile's 32-column slabs
+        constexpr int kSlabs = TILE_N / 32;
+        constexpr int kSlabsPerWarp = kSlabs >= 2 ? kSlabs / 2 : 1;
+        const bool has_work = kSlabs >= 2 || col_half == 0;
+        const uint32_t out0 = smem_u32(sh_out) + uint32_t(ew * prm.out_bufs) * kStageBufBytes;
+        const uint32_t tmem_empty_sig0 = CG == 2 ? map_to_cta(smem_u32(&hdr->tmem_empty[0]), 0)
+                                                 : smem_u32(&hdr->tmem_empty[0]);
+        const int cols_per_store = prm.y_is_f32 ? 16 : 32;     // one staged box is 32 rows x 64 bytes
+        uint32_t as = 0, aph = 0, ob = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
-            const int m0 = (tile / prm.num_n_tiles) * TILE_M;
+        for (int tile = unit; tile < num_tiles; tile += num_units) {
+            const int m0 = (tile / prm.num_n_tiles) * (TILE_M * CG) + int(rank) * TILE_M;
             const int n0 = (tile % prm.num_n_tiles) * TILE_N;
             const uint32_t cur_as = as, cur_aph = aph;
             if (++as == uint32_t(prm.acc_stages)) { as = 0; aph ^= 1; }
 
             // per-column dequantization factors of this tile: c[a][j] = s_act[p][pol] * s_w[p][q(n0+j)]
-            asm volatile("bar.sync 1, 128;" ::: "memory");       // previous tile's readers are done
+            asm volatile("bar.sync 1, 256;" ::: "memory");       // previous tile's readers are done
             for (int j = et; j < TILE_N; j += kEpiThreads) {
                 const int n = n0 + j;
                 int q = 0;
@@ -359,74 +449,127 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                 }
                 sh_bias[j] = (prm.bias && n < prm.N) ? prm.bias[n] : 0.0f;
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            asm volatile("bar.sync 1, 256;" ::: "memory");
 
             if (ok) ok = mbar_wait(smem_u32(&hdr->tmem_full[cur_as]), cur_aph, abort_flag, prm.status, kWhereEpilogue);
             if (!ok) continue;                      // keep the named barriers balanced, do no more work
             tc_fence_after();
 
-            const int row = m0 + lane_grp * 32 + lane;
+            const int row0 = m0 + lane_grp * 32;    // first row of this warp
+            const int row = row0 + lane;
             const uint32_t t_row = tmem_base + (uint32_t(lane_grp * 32) << 16) + cur_as * acc_cols;
+            if (has_work) {
 #pragma unroll 1
-            for (int c0 = 0; c0 < TILE_N; c0 += 32) {
-                float y[32];
+                for (int sl = 0; sl < kSlabsPerWarp; sl++) {
+                    const int c0 = (col_half * kSlabsPerWarp + sl) * 32;
+                    float y[32];
 #pragma unroll
-                for (int j = 0; j < 32; j++) y[j] = 0.0f;
+                    for (int j = 0; j < 32; j++) y[j] = 0.0f;
 #pragma unroll 1
-                for (int a = 0; a < prm.nacc; a++) {
-                    uint32_t r[32];
-                    tc_ld32(t_row + uint32_t(a * TILE_N + c0), r);
-                    tc_wait_ld();
-                    const float *sc = sh_scale + a * TILE_N + c0;
+                    for (int a = 0; a < prm.nacc; a++) {
+                        uint32_t r[32];
+                        tc_ld32(t_row + uint32_t(a * TILE_N + c0), r);
+                        tc_wait_ld();
+                        const float4 *sc = reinterpret_cast<const float4 *>(sh_scale + a * TILE_N + c0);
 #pragma unroll
-                    for (int j = 0; j < 32; j++) {
-                        const float v = KIND == 0 ? __int2float_rn(int(r[j])) : __uint_as_float(r[j]);
-                        y[j] = fmaf(sc[j], v, y[j]);
-                    }
-                    if (prm.acc_dump && row < prm.M) {
-                        uint32_t *dump = static_cast<uint32_t *>(prm.acc_dump) +
-                                         (size_t(a) * prm.M + row) * size_t(prm.N) + n0 + c0;
+                        for (int j4 = 0; j4 < 8; j4++) {
+                            const float4 c = sc[j4];
+                            const float cc[4] = {c.x, c.y, c.z, c.w};
 #pragma unroll
-                        for (int j = 0; j < 32; j++)
-                            if (n0 + c0 + j < prm.N) dump[j] = r[j];
-                    }
-                }
-                if (row < prm.M) {
-#pragma unroll
-                    for (int j = 0; j < 32; j++) y[j] += sh_bias[c0 + j];
-                    const int ncol = prm.N - (n0 + c0);          // valid columns in this slab (multiple of 8)
-                    if (prm.y_is_f32) {
-                        float *dst = static_cast<float *>(prm.Y) + size_t(row) * prm.ldy + n0 + c0;
-#pragma unroll
-                        for (int j = 0; j < 32; j += 4)
-                            if (j < ncol) *reinterpret_cast<float4 *>(dst + j) = make_float4(y[j], y[j + 1], y[j + 2], y[j + 3]);
-                    } else {
-                        __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(prm.Y) + size_t(row) * prm.ldy + n0 + c0;
-#pragma unroll
-                        for (int j = 0; j < 32; j += 8) {
-                            if (j < ncol) {
-                                uint32_t w[4];
-#pragma unroll
-                                for (int t = 0; t < 4; t++) {
-                                    __nv_bfloat162 h = __floats2bfloat162_rn(y[j + 2 * t], y[j + 2 * t + 1]);
-                                    w[t] = *reinterpret_cast<uint32_t *>(&h);
-                                }
-                                *reinterpret_cast<uint4 *>(dst + j) = make_uint4(w[0], w[1], w[2], w[3]);
+                            for (int t = 0; t < 4; t++) {
+                                const int j = 4 * j4 + t;
+                                const float v = KIND == 0 ? __int2float_rn(int(r[j])) : __uint_as_float(r[j]);
+                                y[j] = fmaf(cc[t], v, y[j]);
                             }
+                        }
+                        if (prm.acc_dump && row < prm.M) {
+                            uint32_t *dump = static_cast<uint32_t *>(prm.acc_dump) +
+                                             (size_t(a) * prm.M + row) * size_t(prm.N) + n0 + c0;
+#pragma unroll
+                            for (int j = 0; j < 32; j++)
+                                if (n0 + c0 + j < prm.N) dump[j] = r[j];
+                        }
+                    }
+                    {
+                        const float4 *bs = reinterpret_cast<const float4 *>(sh_bias + c0);
+#pragma unroll
+                        for (int j4 = 0; j4 < 8; j4++) {
+                            const float4 b = bs[j4];
+                            y[4 * j4 + 0] += b.x; y[4 * j4 + 1] += b.y; y[4 * j4 + 2] += b.z; y[4 * j4 + 3] += b.w;
+                        }
+                    }
+                    // 16-byte chunks of this thread's 32 outputs: 4 (bf16) or 8 (fp32)
+                    uint4 w[8];
+                    if (prm.y_is_f32) {
+#pragma unroll
+                        for (int c = 0; c < 8; c++)
+                            w[c] = make_uint4(__float_as_uint(y[4 * c]), __float_as_uint(y[4 * c + 1]),
+                                              __float_as_uint(y[4 * c + 2]), __float_as_uint(y[4 * c + 3]));
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 4; c++) {
+                            uint32_t h[4];
+#pragma unroll
+                            for (int t = 0; t < 4; t++) {
+                                __nv_bfloat162 v2 = __floats2bfloat162_rn(y[8 * c + 2 * t], y[8 * c + 2 * t + 1]);
+                                h[t] = *reinterpret_cast<uint32_t *>(&v2);
+                            }
+                            w[c] = make_uint4(h[0], h[1], h[2], h[3]);
+                        }
+#pragma unroll
+                        for (int c = 4; c < 8; c++) w[c] = make_uint4(0, 0, 0, 0);
+                    }
+                    // stage 32 rows x 64 bytes per box (64B swizzle: 16-byte chunk index ^ ((row >> 1) & 3)),
+                    // then one lane hands the box to the TMA store, which clips it at the matrix edge
+                    const int nbox = prm.y_is_f32 ? 2 : 1;
+#pragma unroll
+                    for (int b = 0; b < 2; b++) {
+                        if (b < nbox) {
+                            const uint32_t buf = out0 + ob * kStageBufBytes;
+                            if (lane == 0) {                   // the store that last read this buffer is done with it
+                                if (prm.out_bufs == 2) bulk_wait_read<1>(); else bulk_wait_read<0>();
+                            }
+                            __syncwarp();
+                            const uint32_t rowaddr = buf + uint32_t(lane) * 64u;
+                            const uint32_t sw = (uint32_t(lane) >> 1) & 3u;
+#pragma unroll
+                            for (int c = 0; c < 4; c++) {
+                                const uint4 v = w[4 * b + c];
+                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                                             ::"r"(rowaddr + ((uint32_t(c) ^ sw) << 4)), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                                             : "memory");
+                            }
+                            fence_async_smem();
+                            __syncwarp();
+                            const int x = n0 + c0 + b * cols_per_store;
+                            if (lane == 0 && row0 < prm.M && x < prm.N) {
+                                tma_store_2d(&tm_y, buf, x, row0);
+                                bulk_commit();
+                            }
+                            if (prm.out_bufs == 2) ob ^= 1;
                         }
                     }
                 }
             }
             tc_fence_before();
-            mbar_arrive(smem_u32(&hdr->tmem_empty[cur_as]));
+            __syncwarp();
+            if (lane == 0) {
+                if (CG == 2) mbar_arrive_cluster(tmem_empty_sig0 + 8 * cur_as);
+                else mbar_arrive(tmem_empty_sig0 + 8 * cur_as);
+            }
         }
+        if (lane == 0) bulk_wait_all();             // staged boxes are read before shared memory goes away
     }
 
     tc_fence_before();
     __syncthreads();
+    if (CG == 2) cluster_sync_all();                // neither CTA leaves while the other may still signal it
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(uint32_t(kTmemCols)) : "memory");
+        if (CG == 1)
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(uint32_t(kTmemCols)) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(uint32_t(kTmemCols)) : "memory");
     }
 }
 
@@ -466,75 +609,132 @@ bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, in
     return r == CUDA_SUCCESS;
 }
 
-int g_tune_tile_n = 0, g_tune_stages = 0;
+// 2-D map over the output [M, N] (bf16 or fp32, row pitch ldy elements): box = 64 bytes x 32 rows,
+// 64B swizzle; stores are clipped at the matrix edge.
+bool make_out_map(CUtensorMap *map, void *base, int64_t M, int64_t N, int64_t ldy, bool f32)
+{
+    EncodeFn enc = get_encode_fn();
+    if (!enc) return false;
+    const int elem = f32 ? 4 : 2;
+    cuuint64_t dims[2] = {cuuint64_t(N), cuuint64_t(M)};
+    cuuint64_t strides[1] = {cuuint64_t(ldy) * elem};
+    cuuint32_t box[2] = {cuuint32_t(64 / elem), 32};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims,
+                     strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+                     CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
 
-template <int KIND, int NPOL, int TILE_N>
+int g_tune_tile_n = 0, g_tune_stages = 0, g_tune_cta_group = 0;
+
+template <int KIND, int NPOL, int TILE_N, int CG>
 sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cudaStream_t st)
 {
-    CUtensorMap ta, tn, tb;
+    constexpr int B_ROWS = TILE_N / CG;
+    CUtensorMap ta, tn, tb, ty;
     if (!make_map(&ta, g.a_pos, g.M, g.K, g.lda, TILE_M)) return SQ_ERR_CUDA;
     if (!make_map(&tn, g.a_neg ? g.a_neg : g.a_pos, g.M, g.K, g.lda, TILE_M)) return SQ_ERR_CUDA;
-    if (!make_map(&tb, g.b, g.N, g.K, g.ldb, TILE_N)) return SQ_ERR_CUDA;
+    if (!make_map(&tb, g.b, g.N, g.K, g.ldb, B_ROWS)) return SQ_ERR_CUDA;
+    if (!make_out_map(&ty, g.Y, g.M, g.N, g.ldy, g.y_dtype == SQ_F32)) return SQ_ERR_CUDA;
 
-    const uint32_t stage_bytes = prm.npol * TILE_M * BLOCK_K + TILE_N * BLOCK_K;
+    const uint32_t stage_bytes = NPOL * TILE_M * BLOCK_K + B_ROWS * BLOCK_K;
     const uint32_t tail = uint32_t(prm.nacc + 1) * TILE_N * 4 + sizeof(SharedHeader);
-    int stages = int((kSmemBudget - 1024 - tail) / stage_bytes);
+    // two staging buffers per epilogue warp unless that costs ring depth below four stages
+    int out_bufs = 2;
+    int stages = int((kSmemBudget - 1024 - tail - kEpiWarps * 2 * kStageBufBytes) / stage_bytes);
+    if (stages < 4) {
+        const int s1 = int((kSmemBudget - 1024 - tail - kEpiWarps * kStageBufBytes) / stage_bytes);
+        if (s1 > stages) { stages = s1; out_bufs = 1; }
+    }
     if (stages > kMaxStages) stages = kMaxStages;
     if (g_tune_stages >= 2 && g_tune_stages < stages) stages = g_tune_stages;
     if (stages < 2) return SQ_ERR_UNSUPPORTED;
     prm.stages = stages;
-    prm.num_m_tiles = int((g.M + TILE_M - 1) / TILE_M);
+    prm.out_bufs = out_bufs;
+    prm.num_m_tiles = int((g.M + TILE_M * CG - 1) / (TILE_M * CG));
     prm.num_n_tiles = int((g.N + TILE_N - 1) / TILE_N);
-    const size_t smem = 1024 + size_t(stages) * stage_bytes + tail;
+    const size_t smem = 1024 + size_t(stages) * stage_bytes + size_t(kEpiWarps) * out_bufs * kStageBufBytes + tail;
 
-    auto kern = segquant_gemm_kernel<KIND, NPOL, TILE_N>;
+    auto kern = segquant_gemm_kernel<KIND, NPOL, TILE_N, CG>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
         return SQ_ERR_CUDA;
     const int tiles = prm.num_m_tiles * prm.num_n_tiles;
-    const int grid = tiles < sm_count ? tiles : sm_count;
-    kern<<<grid, kThreads, smem, st>>>(ta, tn, tb, prm);
+
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(unsigned(sm_count / CG * CG));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CG;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = CG == 2 ? 1 : 0;
+
+    // persistent grid: one CTA (pair) per SM (pair) that can be resident at the same time
+    int units = sm_count / CG;
+    if (CG == 2) {
+        static size_t cached_smem = 0;          // per kernel instantiation
+        static int cached_clusters = 0;
+        if (cached_smem != smem) {
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) return SQ_ERR_CUDA;
+            cached_clusters = n;
+            cached_smem = smem;
+        }
+        if (cached_clusters < units) units = cached_clusters;
+    }
+    const int grid = (tiles < units ? tiles : units) * CG;
+    cfg.gridDim = dim3(unsigned(grid));
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ta, tn, tb, ty, prm);
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
+    return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SQ_OK : SQ_ERR_CUDA;
 }
 
-template <int KIND>
-sq_status launch_kind(const GemmArgs &g, KernelParams &prm, int tile_n, int sm_count, cudaStream_t st)
+template <int KIND, int NPOL, int CG>
+sq_status launch_tile(const GemmArgs &g, KernelParams &prm, int tile_n, int sm_count, cudaStream_t st)
 {
-    if (prm.npol == 2) {
-        switch (tile_n) {
-            case 256: return launch_variant<KIND, 2, 256>(g, prm, sm_count, st);
-            case 128: return launch_variant<KIND, 2, 128>(g, prm, sm_count, st);
-            case 64: return launch_variant<KIND, 2, 64>(g, prm, sm_count, st);
-            case 32: return launch_variant<KIND, 2, 32>(g, prm, sm_count, st);
-        }
-    } else {
-        switch (tile_n) {
-            case 256: return launch_variant<KIND, 1, 256>(g, prm, sm_count, st);
-            case 128: return launch_variant<KIND, 1, 128>(g, prm, sm_count, st);
-            case 64: return launch_variant<KIND, 1, 64>(g, prm, sm_count, st);
-            case 32: return launch_variant<KIND, 1, 32>(g, prm, sm_count, st);
-        }
+    switch (tile_n) {
+        case 256: return launch_variant<KIND, NPOL, 256, CG>(g, prm, sm_count, st);
+        case 128: return launch_variant<KIND, NPOL, 128, CG>(g, prm, sm_count, st);
+        case 64: return launch_variant<KIND, NPOL, 64, CG>(g, prm, sm_count, st);
+        case 32: return launch_variant<KIND, NPOL, 32, CG>(g, prm, sm_count, st);
     }
     return SQ_ERR_UNSUPPORTED;
 }
 
+template <int KIND>
+sq_status launch_kind(const GemmArgs &g, KernelParams &prm, int npol, int cg, int tile_n, int sm_count,
+                      cudaStream_t st)
+{
+    if (npol == 2)
+        return cg == 2 ? launch_tile<KIND, 2, 2>(g, prm, tile_n, sm_count, st)
+                       : launch_tile<KIND, 2, 1>(g, prm, tile_n, sm_count, st);
+    return cg == 2 ? launch_tile<KIND, 1, 2>(g, prm, tile_n, sm_count, st)
+                   : launch_tile<KIND, 1, 1>(g, prm, tile_n, sm_count, st);
+}
+
 }  // namespace
 
-void set_gemm_tuning(int tile_n, int stages)
+void set_gemm_tuning(int tile_n, int stages, int cta_group)
 {
     g_tune_tile_n = tile_n;
     g_tune_stages = stages;
+    g_tune_cta_group = cta_group;
 }
 
 sq_status launch_gemm(const GemmArgs &g, cudaStream_t st)
 {
     KernelParams prm{};
     prm.M = int(g.M); prm.N = int(g.N); prm.K = int(g.K);
-    prm.npol = g.a_neg ? 2 : 1;
-    prm.nacc = g.sb.P * prm.npol;
+    const int npol = g.a_neg ? 2 : 1;
+    prm.nacc = g.sb.P * npol;
     prm.sb = g.sb;
     prm.s_pos = g.s_pos; prm.s_neg = g.s_neg; prm.s_w = g.s_w; prm.bias = g.bias;
-    prm.Y = g.Y; prm.ldy = g.ldy; prm.y_is_f32 = g.y_dtype == SQ_F32;
+    prm.y_is_f32 = g.y_dtype == SQ_F32;
     prm.acc_dump = g.acc_dump;
     prm.status = g.status;
 
@@ -551,8 +751,13 @@ sq_status launch_gemm(const GemmArgs &g, cudaStream_t st)
     if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
         return SQ_ERR_CUDA;
 
-    return g.code == SQ_CODE_INT8 ? launch_kind<0>(g, prm, tile_n, sm_count, st)
-                                  : launch_kind<1>(g, prm, tile_n, sm_count, st);
+    // CTA pairs whenever a tile has more than 128 rows to work on
+    int cg = g.M > TILE_M ? 2 : 1;
+    if (g_tune_cta_group == 1 || g_tune_cta_group == 2) cg = g_tune_cta_group;
+    if (sm_count < 2) cg = 1;
+
+    return g.code == SQ_CODE_INT8 ? launch_kind<0>(g, prm, npol, cg, tile_n, sm_count, st)
+                                  : launch_kind<1>(g, prm, npol, cg, tile_n, sm_count, st);
 }
 
 }  // namespace sq

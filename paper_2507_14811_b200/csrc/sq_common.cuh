@@ -66,6 +66,6 @@ struct GemmArgs {
     uint32_t *status;
 };
 sq_status launch_gemm(const GemmArgs &g, cudaStream_t st);
-void set_gemm_tuning(int tile_n, int stages);
+void set_gemm_tuning(int tile_n, int stages, int cta_group);
 
 }  // namespace sq

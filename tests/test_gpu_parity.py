@@ -22,13 +22,13 @@ def custom_spec(name, M, K, N, kb, nb, dual, code, x_dtype="bf16", x_kind="norma
                         x_kind=x_kind, w_kind=w_kind, seed=seed, cal_rows=cal_rows, x_seg_std=x_seg_std or [])
 
 
-def run_parity(spec, rows=None, flags=0, tile_n=0):
+def run_parity(spec, rows=None, flags=0, tile_n=0, cta_group=0):
     """Full element-by-element parity of one layer.  rows: optional subset of rows the oracle computes."""
     data = WL.make_layer(spec)
     qmin_sym = bool(flags & B.SQ_FLAG_QMIN_SYM)
     s_pos, s_neg, s_w, Wq, (qmax, qmin_abs) = oracle_scales(data, qmin_sym)
 
-    B.segquant_set_tuning(tile_n, 0)
+    B.segquant_set_tuning(tile_n, 0, cta_group)
     try:
         layer = SegQuantLinear(data.W, data.bias, spec.kb, spec.nb, spec.dual, spec.code, DEV, flags)
         g_pos, g_neg = layer.calibrate(data.X_cal)
@@ -46,7 +46,7 @@ def run_parity(spec, rows=None, flags=0, tile_n=0):
         layer.check_status()
         torch.cuda.synchronize()
     finally:
-        B.segquant_set_tuning(0, 0)
+        B.segquant_set_tuning(0, 0, 0)
 
     sel = np.arange(spec.M) if rows is None else np.asarray(rows)
     Xs = to_f32_np(data.X)[sel]
@@ -110,14 +110,54 @@ def test_small_shapes_full_parity(case):
     run_parity(custom_spec(name, M, K, N, kb, nb, dual, code, x_seg_std=[1.0 + 2 * i for i in range(len(kb) - 1)]))
 
 
+@pytest.mark.parametrize("cta_group", [1, 2])
 @pytest.mark.parametrize("tile_n", [32, 64, 128, 256])
-def test_every_tile_width(tile_n):
-    run_parity(custom_spec("tile", 200, 384, 520, [0, 384], [0, 256, 520], False, "int8"), tile_n=tile_n)
+def test_every_tile_width(tile_n, cta_group):
+    run_parity(custom_spec("tile", 200, 384, 520, [0, 384], [0, 256, 520], False, "int8"), tile_n=tile_n,
+               cta_group=cta_group)
 
 
+@pytest.mark.parametrize("cta_group", [1, 2])
 @pytest.mark.parametrize("tile_n", [64, 128, 256])
-def test_every_tile_width_dual(tile_n):
-    run_parity(custom_spec("tile_dual", 300, 640, 776, [0, 640], [0, 776], True, "int8"), tile_n=tile_n)
+def test_every_tile_width_dual(tile_n, cta_group):
+    run_parity(custom_spec("tile_dual", 300, 640, 776, [0, 640], [0, 776], True, "int8"), tile_n=tile_n,
+               cta_group=cta_group)
+
+
+@pytest.mark.parametrize("cta_group", [1, 2])
+@pytest.mark.parametrize("case", [
+    # the CTA-pair tile is 256 rows: M at, just below and just above its multiples; a second CTA with no rows
+    ("pair_exact", 512, 256, 256, [0, 256], [0, 256], True, "int8"),
+    ("pair_plus_one", 257, 256, 264, [0, 128, 256], [0, 264], True, "int8"),
+    ("pair_second_cta_empty", 120, 256, 136, [0, 256], [0, 136], False, "int8"),
+    ("pair_many_tiles", 1100, 384, 1032, [0, 384], [0, 512, 1032], False, "int8"),
+    ("pair_e4m3", 640, 512, 520, [0, 256, 512], [0, 520], True, "e4m3"),
+])
+def test_cta_pair_edges(case, cta_group):
+    name, M, K, N, kb, nb, dual, code = case
+    run_parity(custom_spec(name, M, K, N, kb, nb, dual, code), cta_group=cta_group)
+
+
+def test_strided_output_and_code_matrices():
+    """Y with a row pitch larger than N (a column slice of a wider buffer) is written only inside its
+    N columns, and code matrices with a padded pitch are read correctly."""
+    spec = custom_spec("strided", 300, 256, 200, [0, 256], [0, 200], True, "int8")
+    data = WL.make_layer(spec)
+    s_pos, s_neg, s_w, Wq, (qmax, qmin_abs) = oracle_scales(data)
+    layer = SegQuantLinear(data.W, data.bias, spec.kb, spec.nb, True, "int8", DEV)
+    layer.calibrate(data.X_cal)
+    Xd = data.X.to(DEV)
+    wide = torch.full((spec.M, 256), 7.0, dtype=torch.bfloat16, device=DEV)
+    Y = wide[:, 8:208]
+    c_pos, c_neg = B.segquant_quantize_act(Xd, layer.seg, layer.s_pos, layer.s_neg, "int8")
+    B.segquant_dualscale_gemm(c_pos, c_neg, layer.Wq, layer.seg, "int8", layer.s_pos, layer.s_neg, layer.s_w,
+                              layer.bias, layer.workspace, Y=Y)
+    layer.check_status()
+    torch.cuda.synchronize()
+    assert torch.all(wide[:, :8] == 7.0) and torch.all(wide[:, 208:] == 7.0)
+    res = O.layer_forward(to_f32_np(data.X), Wq, O.SegTable(spec.kb, spec.nb), s_pos, s_neg, s_w,
+                          to_f32_np(data.bias))
+    check_bf16_output(Y.contiguous(), res.y64, res.y_abs, 2)
 
 
 def test_fp32_input_and_student_t():
