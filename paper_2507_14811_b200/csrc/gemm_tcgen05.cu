@@ -12,8 +12,8 @@
 //               polarity against the same weight tile; every (K-segment, polarity) has its own
 //               accumulator in TMEM
 //   warps 2..9  epilogue: tcgen05.ld of all accumulators of a 32-column slab, fp32 FMA with the
-//               per-(segment, polarity, column) scale, + bias, -> bf16 / fp32, staged in shared
-//               memory and written by TMA stores (whole sectors, clipped at the matrix edge)
+//               per-(segment, polarity, column) scale, + bias, -> bf16 / fp32, written from
+//               registers with 32-byte stores (every store covers whole 32-byte sectors of Y)
 // Accumulators: NACC = P * npol, each 128 lanes x TILE_N columns; NACC * TILE_N <= 512 columns.
 // If they use at most half of TMEM the accumulator set is double-buffered so that the epilogue of
 // one tile overlaps the main loop of the next.
@@ -36,7 +36,6 @@ constexpr int kThreads = 64 + kEpiThreads;
 constexpr int kMaxStages = 8;
 constexpr int kTmemCols = 512;
 constexpr uint32_t kSmemBudget = 227 * 1024;
-constexpr uint32_t kStageBufBytes = 32 * 64;            // output staging: 32 rows x 64 bytes
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s
 
 struct KernelParams {
@@ -44,11 +43,13 @@ struct KernelParams {
     int nacc;          // P * npol
     int acc_stages;    // 1 or 2 accumulator sets in TMEM
     int stages;        // shared-memory ring depth
-    int out_bufs;      // 1 or 2 output staging buffers per epilogue warp
     int num_m_tiles, num_n_tiles;
     SegBounds sb;
     const float *s_pos, *s_neg, *s_w, *bias;
+    void *Y;
+    long long ldy;     // elements
     int y_is_f32;
+    int y_wide;        // rows of Y are 32-byte aligned: 256-bit stores allowed
     void *acc_dump;
     uint32_t *status;
 };
@@ -91,7 +92,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 // arrive on a barrier given by a shared::cluster address (possibly in the peer CTA)
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr)
 {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 {
@@ -141,17 +142,23 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
             ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y) : "memory");
 }
 
-// 2-D tiled TMA store of a staged box from this CTA's shared memory (bulk async-group completion).
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y)
+__device__ __forceinline__ float4 ld_shared_f4(uint32_t addr)
 {
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y) : "memory");
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
 }
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// 16- and 32-byte global stores
+__device__ __forceinline__ void st_global_16(void *p, uint4 v)
+{
+    asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void st_global_32(void *p, uint4 a, uint4 b)
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(p), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w) : "memory");
+}
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -275,18 +282,16 @@ __device__ __forceinline__ void issue_kblock(uint32_t d0, uint64_t da, uint64_t 
 template <int KIND, int NPOL, int TILE_N, int CG>
 __global__ void __launch_bounds__(kThreads, 1)
 segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_constant__ CUtensorMap tm_a_neg,
-                     const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_y,
-                     const KernelParams prm)
+                     const __grid_constant__ CUtensorMap tm_b, const KernelParams prm)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    // layout: [ring: stages x (NPOL A tiles of 16 KiB, B part of B_ROWS*128 B)] [output staging] [scales] [header]
+    // layout: [ring: stages x (NPOL A tiles of 16 KiB, B part of B_ROWS*128 B)] [scales] [header]
     constexpr int B_ROWS = TILE_N / CG;                  // weight rows this CTA loads per K-block
     constexpr uint32_t a_bytes = TILE_M * BLOCK_K;
     constexpr uint32_t b_bytes = B_ROWS * BLOCK_K;
     constexpr uint32_t stage_bytes = NPOL * a_bytes + b_bytes;
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t *sh_out = smem + size_t(prm.stages) * stage_bytes;                             // [warp][out_bufs][2 KiB]
-    float *sh_scale = reinterpret_cast<float *>(sh_out + kEpiWarps * prm.out_bufs * kStageBufBytes);  // [nacc][TILE_N]
+    float *sh_scale = reinterpret_cast<float *>(smem + size_t(prm.stages) * stage_bytes);   // [nacc][TILE_N]
     float *sh_bias = sh_scale + prm.nacc * TILE_N;                                          // [TILE_N]
     SharedHeader *hdr = reinterpret_cast<SharedHeader *>(sh_bias + TILE_N);
 
@@ -424,11 +429,13 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
         constexpr int kSlabs = TILE_N / 32;
         constexpr int kSlabsPerWarp = kSlabs >= 2 ? kSlabs / 2 : 1;
         const bool has_work = kSlabs >= 2 || col_half == 0;
-        const uint32_t out0 = smem_u32(sh_out) + uint32_t(ew * prm.out_bufs) * kStageBufBytes;
+        const int nacc = prm.nacc;
+        const int units = has_work ? kSlabsPerWarp * nacc : 0;      // (slab, accumulator) pairs of this warp
+        const int col_base = col_half * kSlabsPerWarp * 32;
         const uint32_t tmem_empty_sig0 = CG == 2 ? map_to_cta(smem_u32(&hdr->tmem_empty[0]), 0)
                                                  : smem_u32(&hdr->tmem_empty[0]);
-        const int cols_per_store = prm.y_is_f32 ? 16 : 32;     // one staged box is 32 rows x 64 bytes
-        uint32_t as = 0, aph = 0, ob = 0;
+        const uint32_t sc_base = smem_u32(sh_scale), bias_base = smem_u32(sh_bias);
+        uint32_t as = 0, aph = 0;
         bool ok = true;
         for (int tile = unit; tile < num_tiles; tile += num_units) {
             const int m0 = (tile / prm.num_n_tiles) * (TILE_M * CG) + int(rank) * TILE_M;
@@ -455,57 +462,81 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
             if (!ok) continue;                      // keep the named barriers balanced, do no more work
             tc_fence_after();
 
-            const int row0 = m0 + lane_grp * 32;    // first row of this warp
-            const int row = row0 + lane;
+            const int row = m0 + lane_grp * 32 + lane;
             const uint32_t t_row = tmem_base + (uint32_t(lane_grp * 32) << 16) + cur_as * acc_cols;
-            if (has_work) {
-#pragma unroll 1
-                for (int sl = 0; sl < kSlabsPerWarp; sl++) {
-                    const int c0 = (col_half * kSlabsPerWarp + sl) * 32;
-                    float y[32];
+            const uint32_t release_bar = tmem_empty_sig0 + 8 * cur_as;
+
+            // The (slab, accumulator) units of this warp are read from TMEM one ahead of the arithmetic:
+            // while unit u is scaled and summed, the load of unit u + 1 is in flight.  The accumulator set
+            // is handed back to the MMA issuer as soon as the last load has landed in registers.
+            float y[32];
 #pragma unroll
-                    for (int j = 0; j < 32; j++) y[j] = 0.0f;
-#pragma unroll 1
-                    for (int a = 0; a < prm.nacc; a++) {
-                        uint32_t r[32];
-                        tc_ld32(t_row + uint32_t(a * TILE_N + c0), r);
-                        tc_wait_ld();
-                        const float4 *sc = reinterpret_cast<const float4 *>(sh_scale + a * TILE_N + c0);
+            for (int j = 0; j < 32; j++) y[j] = 0.0f;
+            uint32_t ra[32], rb[32];
+            int i_sl = 0, i_a = 0;                  // next unit to load
+            int c_sl = 0, c_a = 0;                  // next unit to consume
+            auto issue = [&](uint32_t (&r)[32]) {
+                tc_ld32(t_row + uint32_t(i_a * TILE_N + col_base + i_sl * 32), r);
+                if (++i_a == nacc) { i_a = 0; i_sl++; }
+            };
+            auto release = [&]() {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if (CG == 2) mbar_arrive_cluster(release_bar);
+                    else mbar_arrive(release_bar);
+                }
+            };
+            auto consume = [&](const uint32_t (&r)[32]) {
+                const int c0 = col_base + c_sl * 32;
+                const uint32_t sc = sc_base + uint32_t(c_a * TILE_N + c0) * 4u;
 #pragma unroll
-                        for (int j4 = 0; j4 < 8; j4++) {
-                            const float4 c = sc[j4];
-                            const float cc[4] = {c.x, c.y, c.z, c.w};
+                for (int j4 = 0; j4 < 8; j4++) {
+                    const float4 c = ld_shared_f4(sc + 16u * j4);
+                    const float cc[4] = {c.x, c.y, c.z, c.w};
 #pragma unroll
-                            for (int t = 0; t < 4; t++) {
-                                const int j = 4 * j4 + t;
-                                const float v = KIND == 0 ? __int2float_rn(int(r[j])) : __uint_as_float(r[j]);
-                                y[j] = fmaf(cc[t], v, y[j]);
+                    for (int t = 0; t < 4; t++) {
+                        const int j = 4 * j4 + t;
+                        const float v = KIND == 0 ? __int2float_rn(int(r[j])) : __uint_as_float(r[j]);
+                        y[j] = fmaf(cc[t], v, y[j]);
+                    }
+                }
+                if (prm.acc_dump && row < prm.M) {
+                    uint32_t *dump = static_cast<uint32_t *>(prm.acc_dump) +
+                                     (size_t(c_a) * prm.M + row) * size_t(prm.N) + n0 + c0;
+#pragma unroll
+                    for (int j = 0; j < 32; j++)
+                        if (n0 + c0 + j < prm.N) dump[j] = r[j];
+                }
+                if (++c_a < nacc) return;
+                c_a = 0;
+                c_sl++;
+                // last accumulator of the slab: + bias, convert, store this thread's 32 outputs of row `row`
+#pragma unroll
+                for (int j4 = 0; j4 < 8; j4++) {
+                    const float4 b = ld_shared_f4(bias_base + uint32_t(c0) * 4u + 16u * j4);
+                    y[4 * j4 + 0] += b.x; y[4 * j4 + 1] += b.y; y[4 * j4 + 2] += b.z; y[4 * j4 + 3] += b.w;
+                }
+                // 16-byte chunks (8 bf16 or 4 fp32); N is a multiple of 8, so a chunk is entirely inside or
+                // outside the matrix
+                if (row < prm.M) {
+                    const int nvalid = prm.N - (n0 + c0);            // valid columns of this slab, may exceed 32
+                    if (prm.y_is_f32) {
+                        float *dst = static_cast<float *>(prm.Y) + size_t(row) * prm.ldy + n0 + c0;
+#pragma unroll
+                        for (int c = 0; c < 4; c++) {                // 8 columns = 32 bytes
+                            if (8 * c < nvalid) {
+                                const uint4 lo = make_uint4(__float_as_uint(y[8 * c]), __float_as_uint(y[8 * c + 1]),
+                                                            __float_as_uint(y[8 * c + 2]), __float_as_uint(y[8 * c + 3]));
+                                const uint4 hi = make_uint4(__float_as_uint(y[8 * c + 4]), __float_as_uint(y[8 * c + 5]),
+                                                            __float_as_uint(y[8 * c + 6]), __float_as_uint(y[8 * c + 7]));
+                                if (prm.y_wide) st_global_32(dst + 8 * c, lo, hi);
+                                else { st_global_16(dst + 8 * c, lo); st_global_16(dst + 8 * c + 4, hi); }
                             }
                         }
-                        if (prm.acc_dump && row < prm.M) {
-                            uint32_t *dump = static_cast<uint32_t *>(prm.acc_dump) +
-                                             (size_t(a) * prm.M + row) * size_t(prm.N) + n0 + c0;
-#pragma unroll
-                            for (int j = 0; j < 32; j++)
-                                if (n0 + c0 + j < prm.N) dump[j] = r[j];
-                        }
-                    }
-                    {
-                        const float4 *bs = reinterpret_cast<const float4 *>(sh_bias + c0);
-#pragma unroll
-                        for (int j4 = 0; j4 < 8; j4++) {
-                            const float4 b = bs[j4];
-                            y[4 * j4 + 0] += b.x; y[4 * j4 + 1] += b.y; y[4 * j4 + 2] += b.z; y[4 * j4 + 3] += b.w;
-                        }
-                    }
-                    // 16-byte chunks of this thread's 32 outputs: 4 (bf16) or 8 (fp32)
-                    uint4 w[8];
-                    if (prm.y_is_f32) {
-#pragma unroll
-                        for (int c = 0; c < 8; c++)
-                            w[c] = make_uint4(__float_as_uint(y[4 * c]), __float_as_uint(y[4 * c + 1]),
-                                              __float_as_uint(y[4 * c + 2]), __float_as_uint(y[4 * c + 3]));
                     } else {
+                        __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(prm.Y) + size_t(row) * prm.ldy + n0 + c0;
+                        uint4 w[4];
 #pragma unroll
                         for (int c = 0; c < 4; c++) {
                             uint32_t h[4];
@@ -517,48 +548,37 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                             w[c] = make_uint4(h[0], h[1], h[2], h[3]);
                         }
 #pragma unroll
-                        for (int c = 4; c < 8; c++) w[c] = make_uint4(0, 0, 0, 0);
-                    }
-                    // stage 32 rows x 64 bytes per box (64B swizzle: 16-byte chunk index ^ ((row >> 1) & 3)),
-                    // then one lane hands the box to the TMA store, which clips it at the matrix edge
-                    const int nbox = prm.y_is_f32 ? 2 : 1;
-#pragma unroll
-                    for (int b = 0; b < 2; b++) {
-                        if (b < nbox) {
-                            const uint32_t buf = out0 + ob * kStageBufBytes;
-                            if (lane == 0) {                   // the store that last read this buffer is done with it
-                                if (prm.out_bufs == 2) bulk_wait_read<1>(); else bulk_wait_read<0>();
+                        for (int c = 0; c < 2; c++) {                // 16 columns = 32 bytes
+                            if (16 * c + 8 < nvalid && prm.y_wide) {
+                                st_global_32(dst + 16 * c, w[2 * c], w[2 * c + 1]);
+                            } else {
+                                if (16 * c < nvalid) st_global_16(dst + 16 * c, w[2 * c]);
+                                if (16 * c + 8 < nvalid) st_global_16(dst + 16 * c + 8, w[2 * c + 1]);
                             }
-                            __syncwarp();
-                            const uint32_t rowaddr = buf + uint32_t(lane) * 64u;
-                            const uint32_t sw = (uint32_t(lane) >> 1) & 3u;
-#pragma unroll
-                            for (int c = 0; c < 4; c++) {
-                                const uint4 v = w[4 * b + c];
-                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                                             ::"r"(rowaddr + ((uint32_t(c) ^ sw) << 4)), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
-                                             : "memory");
-                            }
-                            fence_async_smem();
-                            __syncwarp();
-                            const int x = n0 + c0 + b * cols_per_store;
-                            if (lane == 0 && row0 < prm.M && x < prm.N) {
-                                tma_store_2d(&tm_y, buf, x, row0);
-                                bulk_commit();
-                            }
-                            if (prm.out_bufs == 2) ob ^= 1;
                         }
                     }
                 }
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-                if (CG == 2) mbar_arrive_cluster(tmem_empty_sig0 + 8 * cur_as);
-                else mbar_arrive(tmem_empty_sig0 + 8 * cur_as);
+#pragma unroll
+                for (int j = 0; j < 32; j++) y[j] = 0.0f;
+            };
+
+            if (units == 0) {
+                release();
+            } else {
+                issue(ra);
+#pragma unroll 1
+                for (int u = 0; u < units; u += 2) {
+                    tc_wait_ld();
+                    if (u + 1 < units) issue(rb); else release();
+                    consume(ra);
+                    if (u + 1 < units) {
+                        tc_wait_ld();
+                        if (u + 2 < units) issue(ra); else release();
+                        consume(rb);
+                    }
+                }
             }
         }
-        if (lane == 0) bulk_wait_all();             // staged boxes are read before shared memory goes away
     }
 
     tc_fence_before();
@@ -609,52 +629,27 @@ bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, in
     return r == CUDA_SUCCESS;
 }
 
-// 2-D map over the output [M, N] (bf16 or fp32, row pitch ldy elements): box = 64 bytes x 32 rows,
-// 64B swizzle; stores are clipped at the matrix edge.
-bool make_out_map(CUtensorMap *map, void *base, int64_t M, int64_t N, int64_t ldy, bool f32)
-{
-    EncodeFn enc = get_encode_fn();
-    if (!enc) return false;
-    const int elem = f32 ? 4 : 2;
-    cuuint64_t dims[2] = {cuuint64_t(N), cuuint64_t(M)};
-    cuuint64_t strides[1] = {cuuint64_t(ldy) * elem};
-    cuuint32_t box[2] = {cuuint32_t(64 / elem), 32};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = enc(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims,
-                     strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
-                     CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
-}
-
 int g_tune_tile_n = 0, g_tune_stages = 0, g_tune_cta_group = 0;
 
 template <int KIND, int NPOL, int TILE_N, int CG>
 sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cudaStream_t st)
 {
     constexpr int B_ROWS = TILE_N / CG;
-    CUtensorMap ta, tn, tb, ty;
+    CUtensorMap ta, tn, tb;
     if (!make_map(&ta, g.a_pos, g.M, g.K, g.lda, TILE_M)) return SQ_ERR_CUDA;
     if (!make_map(&tn, g.a_neg ? g.a_neg : g.a_pos, g.M, g.K, g.lda, TILE_M)) return SQ_ERR_CUDA;
     if (!make_map(&tb, g.b, g.N, g.K, g.ldb, B_ROWS)) return SQ_ERR_CUDA;
-    if (!make_out_map(&ty, g.Y, g.M, g.N, g.ldy, g.y_dtype == SQ_F32)) return SQ_ERR_CUDA;
 
     const uint32_t stage_bytes = NPOL * TILE_M * BLOCK_K + B_ROWS * BLOCK_K;
     const uint32_t tail = uint32_t(prm.nacc + 1) * TILE_N * 4 + sizeof(SharedHeader);
-    // two staging buffers per epilogue warp unless that costs ring depth below four stages
-    int out_bufs = 2;
-    int stages = int((kSmemBudget - 1024 - tail - kEpiWarps * 2 * kStageBufBytes) / stage_bytes);
-    if (stages < 4) {
-        const int s1 = int((kSmemBudget - 1024 - tail - kEpiWarps * kStageBufBytes) / stage_bytes);
-        if (s1 > stages) { stages = s1; out_bufs = 1; }
-    }
+    int stages = int((kSmemBudget - 1024 - tail) / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (g_tune_stages >= 2 && g_tune_stages < stages) stages = g_tune_stages;
     if (stages < 2) return SQ_ERR_UNSUPPORTED;
     prm.stages = stages;
-    prm.out_bufs = out_bufs;
     prm.num_m_tiles = int((g.M + TILE_M * CG - 1) / (TILE_M * CG));
     prm.num_n_tiles = int((g.N + TILE_N - 1) / TILE_N);
-    const size_t smem = 1024 + size_t(stages) * stage_bytes + size_t(kEpiWarps) * out_bufs * kStageBufBytes + tail;
+    const size_t smem = 1024 + size_t(stages) * stage_bytes + tail;
 
     auto kern = segquant_gemm_kernel<KIND, NPOL, TILE_N, CG>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
@@ -689,7 +684,7 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
     }
     const int grid = (tiles < units ? tiles : units) * CG;
     cfg.gridDim = dim3(unsigned(grid));
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ta, tn, tb, ty, prm);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ta, tn, tb, prm);
     count_launch();
     return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SQ_OK : SQ_ERR_CUDA;
 }
@@ -734,7 +729,9 @@ sq_status launch_gemm(const GemmArgs &g, cudaStream_t st)
     prm.nacc = g.sb.P * npol;
     prm.sb = g.sb;
     prm.s_pos = g.s_pos; prm.s_neg = g.s_neg; prm.s_w = g.s_w; prm.bias = g.bias;
+    prm.Y = g.Y; prm.ldy = g.ldy;
     prm.y_is_f32 = g.y_dtype == SQ_F32;
+    prm.y_wide = (reinterpret_cast<uintptr_t>(g.Y) % 32 == 0) && ((size_t(g.ldy) * (prm.y_is_f32 ? 4 : 2)) % 32 == 0);
     prm.acc_dump = g.acc_dump;
     prm.status = g.status;
 
