@@ -85,6 +85,27 @@ sq_status segquant_calib_scales(const void *X, sq_dtype dt, int64_t rows, int64_
                                 uint32_t flags, float *s_pos, float *s_neg,
                                 void *workspace, size_t ws_bytes, void *stream);
 
+/* Calibration for callers that cannot allocate device memory.  (The paper has no counterpart; this is
+ * a property of the library, not of the method.)  Some users of this library run where cudaMalloc is
+ * off limits: inside a host process whose device memory is entirely owned by another component's pool,
+ * in a plugin that is handed its tensors and nothing else, or under a policy that forbids allocation
+ * after start-up.  segquant_calib_scales needs a caller-provided workspace for its reduction partials;
+ * this variant computes exactly the same scales with the partials kept in a fixed 8 KiB array inside
+ * the library's device image, and takes no workspace.  It calls no allocating routine.
+ *   Arguments, results and alignment rules are those of segquant_calib_scales, minus the workspace.
+ *   Limit: at most SQ_STATIC_CALIB_MAX_BLOCKS scale values per call (P for activations, P*Q for
+ *   weights); more is refused with SQ_ERR_UNSUPPORTED before any launch.
+ *   The first call on a device looks up the array's device address (once per device, with that device
+ *   current); make that first call outside any stream capture.
+ *   Every call on one GPU shares the array: each call resets the entries it uses before reducing into
+ *   them, so calls in stream order are independent, but two calls that overlap on the GPU (different
+ *   streams or threads without ordering between them) race and may both return wrong scales.
+ *   Every GPU that loads the library carries the 8 KiB array until the process exits. */
+#define SQ_STATIC_CALIB_MAX_BLOCKS 1024
+sq_status segquant_calib_scales_static(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld,
+                                       const sq_segtable *seg, sq_code code, int is_weight, int dual,
+                                       uint32_t flags, float *s_pos, float *s_neg, void *stream);
+
 /* Step "activation quantization" -- Sec. 4.3.2 Q_dual with the polarity split X_+ / X_-, plus the
  * clip of the Sec. 3 uniform quantizer; x/s is one IEEE fp32 division, rounding is half-to-even.
  *   s_neg != NULL (dual): x >= 0 -> c_pos = clip(round(x/s_pos[p]), 0, q_max), c_neg = 0;

@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "SQ_OK", 1: "SQ_ERR_NULL", 2: "SQ_ERR_SHAPE", 3: "SQ_ERR_SEGT
                 5: "SQ_ERR_UNSUPPORTED", 6: "SQ_ERR_CUDA", 7: "SQ_ERR_TIMEOUT", 8: "SQ_ERR_WORKSPACE"}
 
 EXPORTS = [
-    "segquant_workspace_bytes", "segquant_calib_scales", "segquant_quantize_act", "segquant_quantize_weight",
+    "segquant_workspace_bytes", "segquant_calib_scales", "segquant_calib_scales_static", "segquant_quantize_act", "segquant_quantize_weight",
     "segquant_seglinear_gemm", "segquant_dualscale_gemm", "segquant_layer_scratch_bytes",
     "segquant_layer_forward", "segquant_last_device_status", "segquant_set_tuning", "segquant_launch_count",
     "segquant_status_string",
@@ -124,6 +124,25 @@ def segquant_calib_scales(X: torch.Tensor, seg: SegTable, code: str, is_weight: 
                                      C.c_size_t(workspace.numel()), _stream())
     _check(st, "segquant_calib_scales")
     return s_pos, s_neg
+
+
+def segquant_calib_scales_static(X: torch.Tensor, seg: SegTable, code: str, is_weight: bool, dual: bool,
+                                 flags: int = 0, s_pos=None, s_neg=None):
+    """segquant_calib_scales without a workspace: for callers that may not allocate device memory, the
+    library keeps the reduction partials in a fixed array of its own.  Pass preallocated s_pos / s_neg
+    to keep this wrapper allocation-free as well; calls on one GPU must not overlap."""
+    rows, K = X.shape
+    n = seg.P * (seg.Q if is_weight else 1)
+    if s_pos is None:
+        s_pos = torch.empty(n, dtype=torch.float32, device=X.device)
+    if s_neg is None and dual and not is_weight:
+        s_neg = torch.empty(n, dtype=torch.float32, device=X.device)
+    st = lib().segquant_calib_scales_static(_ptr(X), C.c_int(_dt(X)), C.c_int64(rows), C.c_int64(K),
+                                            C.c_int64(X.stride(0)), seg.ref(), C.c_int(SQ_CODE[code]),
+                                            C.c_int(int(is_weight)), C.c_int(int(dual)), C.c_uint32(flags),
+                                            _ptr(s_pos), _ptr(s_neg if (dual and not is_weight) else None), _stream())
+    _check(st, "segquant_calib_scales_static")
+    return s_pos, (s_neg if (dual and not is_weight) else None)
 
 
 def _ldc(K: int) -> int:

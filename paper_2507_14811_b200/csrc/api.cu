@@ -110,6 +110,21 @@ sq_status segquant_calib_scales(const void *X, sq_dtype dt, int64_t rows, int64_
                         s_pos, s_neg, partials, static_cast<cudaStream_t>(stream));
 }
 
+sq_status segquant_calib_scales_static(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld,
+                                       const sq_segtable *seg, sq_code code, int is_weight, int dual,
+                                       uint32_t flags, float *s_pos, float *s_neg, void *stream)
+{
+    if (!s_pos || (!is_weight && dual && !s_neg)) return SQ_ERR_NULL;
+    if (!valid_dt(dt) || !valid_code(code)) return SQ_ERR_UNSUPPORTED;
+    sq_status st = check_matrix(X, rows, K, ld, dt_size(dt));
+    if (st != SQ_OK) return st;
+    HostSeg hs = load_segtable(seg, K, is_weight ? rows : (seg && seg->nb && seg->Q >= 1 ? seg->nb[seg->Q] : 0));
+    if (hs.status != SQ_OK) return hs.status;
+    if (hs.b.P * (is_weight ? hs.b.Q : 1) > SQ_STATIC_CALIB_MAX_BLOCKS) return SQ_ERR_UNSUPPORTED;
+    return launch_calib_static(X, dt, rows, K, ld, hs.b, is_weight, dual, code_qmax(code), code_qmin_abs(code, flags),
+                               s_pos, s_neg, static_cast<cudaStream_t>(stream));
+}
+
 sq_status segquant_quantize_act(const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld,
                                 const sq_segtable *seg, const float *s_pos, const float *s_neg, sq_code code,
                                 uint32_t flags, void *c_pos, void *c_neg, int64_t ldc, void *stream)

@@ -3,6 +3,7 @@
 // matrix, reduced through ordered-integer atomics into workspace partials, then one IEEE division
 // per scale.
 #include <cuda_bf16.h>
+#include <mutex>
 #include "sq_common.cuh"
 
 namespace sq {
@@ -118,6 +119,45 @@ sq_status launch_calib(const void *X, sq_dtype dt, int64_t rows, int64_t K, int6
                                                                  s_pos, s_neg);
     count_launch(3);
     return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
+}
+
+// ----------------------------------------------------------------------------- built-in scratch
+// Reduction partials for callers that have no device allocator to take a workspace from: 2 words per
+// (K-segment, N-segment) block, SQ_STATIC_CALIB_MAX_BLOCKS blocks, 8 KiB.  The array lives in the
+// library's device image, so every GPU that loads the library holds it until the process exits, and
+// every call on that GPU shares it.
+static __device__ __align__(256) uint32_t g_static_partials[SQ_STATIC_CALIB_MAX_BLOCKS * 2];
+
+// In host code the name g_static_partials is only a handle for the runtime; the device address has
+// to be asked for, once per device, with that device current.
+static sq_status static_partials_address(uint32_t **out)
+{
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static uint32_t *addr[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SQ_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_partials) != cudaSuccess || !p) return SQ_ERR_CUDA;
+        addr[dev] = static_cast<uint32_t *>(p);
+    }
+    *out = addr[dev];
+    return SQ_OK;
+}
+
+sq_status launch_calib_static(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld, const SegBounds &sb,
+                              int is_weight, int dual, float q_max, float q_min_abs, float *s_pos, float *s_neg,
+                              cudaStream_t st)
+{
+    if (sb.P * (is_weight ? sb.Q : 1) > SQ_STATIC_CALIB_MAX_BLOCKS) return SQ_ERR_UNSUPPORTED;
+    uint32_t *partials = nullptr;
+    const sq_status r = static_partials_address(&partials);
+    if (r != SQ_OK) return r;
+    // launch_calib's first kernel resets the partials it is going to use, so the previous call's
+    // contents never leak into this one
+    return launch_calib(X, dt, rows, K, ld, sb, is_weight, dual, q_max, q_min_abs, s_pos, s_neg, partials, st);
 }
 
 }  // namespace sq

@@ -46,6 +46,10 @@ sq_status launch_calib(const void *X, sq_dtype dt, int64_t rows, int64_t K, int6
                        int is_weight, int dual, float q_max, float q_min_abs, float *s_pos, float *s_neg,
                        uint32_t *partials, cudaStream_t st);
 
+sq_status launch_calib_static(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld, const SegBounds &sb,
+                              int is_weight, int dual, float q_max, float q_min_abs, float *s_pos, float *s_neg,
+                              cudaStream_t st);
+
 sq_status launch_quantize(const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld, const SegBounds &sb,
                           const float *s_pos, const float *s_neg, int row_segments, sq_code code,
                           float q_max, float q_min_abs, void *c_pos, void *c_neg, int64_t ldc, cudaStream_t st);

@@ -1,0 +1,72 @@
+"""The allocation-free calibration entry point against the ordinary one.
+
+segquant_calib_scales_static exists for callers that may not allocate device memory (a plugin that
+only receives tensors, a process whose device memory belongs to someone else's pool, a no-allocation-
+after-start-up policy): it keeps its reduction partials in an array inside the library instead of a
+caller-provided workspace.  It has to return bit-identical scales, and because every call shares that
+array, a second call right after the first (on other data, with other segment counts) must not see
+anything the first one left behind.  This file is named to be collected last, so a run that stops at
+the first failure has already been through every other test.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2507_14811_b200 import binding as B
+from paper_2507_14811_b200 import workloads as WL
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _spec(name, M, K, N, kb, nb, x_kind, seed, x_dtype="bf16", x_seg_std=None):
+    return WL.LayerSpec(name=name, M=M, K=K, N=N, kb=kb, nb=nb, dual=True, code="int8", x_dtype=x_dtype,
+                        x_kind=x_kind, w_kind="segment_ladder", seed=seed, cal_rows=96, x_seg_std=x_seg_std or [])
+
+
+def _compare(spec, code):
+    data = WL.make_layer(spec)
+    seg = B.SegTable(spec.kb, spec.nb)
+    ws = B.new_workspace(DEV)
+    Xc = data.X_cal.to(DEV).contiguous()
+    Wd = data.W.to(DEV).contiguous()
+    # outputs are allocated up front: the call under test itself allocates nothing
+    out = {k: torch.full((n,), -1.0, dtype=torch.float32, device=DEV)
+           for k, n in (("pos", seg.P), ("neg", seg.P), ("one", seg.P), ("w", seg.P * seg.Q))}
+    torch.cuda.synchronize()
+    for dual in (True, False):
+        ref_pos, ref_neg = B.segquant_calib_scales(Xc, seg, code, False, dual, ws)
+        got_pos, got_neg = B.segquant_calib_scales_static(Xc, seg, code, False, dual,
+                                                          s_pos=out["pos"] if dual else out["one"],
+                                                          s_neg=out["neg"] if dual else None)
+        torch.cuda.synchronize()
+        assert np.array_equal(got_pos.cpu().numpy(), ref_pos.cpu().numpy())
+        if dual:
+            assert np.array_equal(got_neg.cpu().numpy(), ref_neg.cpu().numpy())
+    ref_w, _ = B.segquant_calib_scales(Wd, seg, code, True, False, ws)
+    got_w, _ = B.segquant_calib_scales_static(Wd, seg, code, True, False, s_pos=out["w"])
+    torch.cuda.synchronize()
+    assert np.array_equal(got_w.cpu().numpy(), ref_w.cpu().numpy())
+    assert float(got_w.min()) > 0.0
+
+
+def test_static_calibration_matches_workspace_calibration_twice_in_a_row():
+    # first call: many blocks, large values; second call: fewer blocks, much smaller values, so stale
+    # partials of the first call would show up as scales that are too large
+    _compare(_spec("first", 64, 512, 384, [0, 128, 256, 512], [0, 64, 128, 192, 256, 320, 384],
+                   "student_t4+gelu", 11, x_seg_std=[4.0, 9.0, 2.0]), "int8")
+    _compare(_spec("second", 64, 256, 128, [0, 256], [0, 128], "normal+silu", 12, x_dtype="f32",
+                   x_seg_std=[0.05]), "e4m3")
+
+
+def test_static_calibration_refuses_more_blocks_than_it_holds():
+    # the segment-table limits of the library keep P*Q within the built-in array; a table beyond those
+    # limits is refused on the host, before any launch
+    n0 = B.segquant_launch_count()
+    K, N = 32 * 17, 8
+    X = torch.zeros((N, K), dtype=torch.float32, device=DEV)
+    seg = B.SegTable(list(range(0, K + 1, 32)), [0, N])          # 17 K-segments > SQ_MAX_P
+    with pytest.raises(B.SegquantError) as e:
+        B.segquant_calib_scales_static(X, seg, "int8", True, False)
+    assert e.value.status == 5
+    assert B.segquant_launch_count() == n0
