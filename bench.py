@@ -154,6 +154,12 @@ class BenchLayer:
             self.B.segquant_seglinear_gemm(self.c_pos, L.Wq, L.seg, L.code, L.s_pos, L.s_w, L.bias, L.workspace,
                                            Y=self.Y)
 
+    def gemm_plain(self):
+        """The same shape as a plain single-scale W8A8 layer (one code matrix): the denominator of the
+        DualScale overhead.  Timing only; its output is not checked."""
+        L = self.layer
+        self.B.segquant_seglinear_gemm(self.c_pos, L.Wq, L.seg, L.code, L.s_pos, L.s_w, L.bias, L.workspace, Y=self.Y)
+
     def forward_e2e(self):
         self.layer.forward(self.X_host, Y=self.Y_host, x_stage=self.x_stage, y_stage=self.y_stage)
 
@@ -165,7 +171,7 @@ def time_workload(layers, steps, warmup, flush, sampler=None):
     ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(nl)] for _ in range(steps)]
     for _ in range(warmup):
         for bl in layers:
-            flush.zero_()
+            flush()
             bl.quantize()
             bl.gemm()
     torch.cuda.synchronize()
@@ -173,7 +179,7 @@ def time_workload(layers, steps, warmup, flush, sampler=None):
         sampler.start()
     for s in range(steps):
         for i, bl in enumerate(layers):
-            flush.zero_()
+            flush()
             ev[s][i][0].record()
             bl.quantize()
             ev[s][i][1].record()
@@ -186,6 +192,27 @@ def time_workload(layers, steps, warmup, flush, sampler=None):
     return q_ms.mean(axis=0), g_ms.mean(axis=0), clocks
 
 
+def time_plain(layers, steps, flush):
+    """Mean time of the plain single-scale GEMM on every dual layer's shape (None for single-scale layers)."""
+    out = []
+    for bl in layers:
+        if not bl.spec.dual:
+            out.append(None)
+            continue
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
+        for _ in range(3):
+            bl.gemm_plain()
+        for s in range(steps):
+            flush()
+            bl.quantize()
+            ev[s][0].record()
+            bl.gemm_plain()
+            ev[s][1].record()
+        torch.cuda.synchronize()
+        out.append(float(np.mean([a.elapsed_time(b) for a, b in ev])))
+    return out
+
+
 def time_e2e(layers, steps, warmup, flush):
     nl = len(layers)
     ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(nl)] for _ in range(steps)]
@@ -195,7 +222,7 @@ def time_e2e(layers, steps, warmup, flush):
     torch.cuda.synchronize()
     for s in range(steps):
         for i, bl in enumerate(layers):
-            flush.zero_()
+            flush()
             ev[s][i][0].record()
             bl.forward_e2e()
             ev[s][i][1].record()
@@ -254,7 +281,15 @@ def run_ours(args):
 
     specs = WL.WORKLOADS[args.workload]
     layers = [BenchLayer(s, dev) for s in specs]
-    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    flush_w = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    flush_r = torch.zeros(L2_FLUSH_BYTES // 4, dtype=torch.int32, device=dev)
+
+    def flush():
+        """Evicts the layer's inputs from L2: a write larger than L2, then a read larger than L2 so that
+        the cache is left holding clean lines (dirty lines of the write would otherwise be written back
+        during the timed kernel and be charged to it)."""
+        flush_w.zero_()
+        flush_r.sum()
     sampler = ClockSampler(local)
 
     def barrier():
@@ -270,6 +305,7 @@ def run_ours(args):
     barrier()
     for bl in layers:
         bl.layer.check_status()
+    plain_ms = time_plain(layers, max(3, min(args.steps, 20)), flush)
     e2e_ms = time_e2e(layers, max(3, args.steps // 4), args.warmup, flush)
     barrier()
 
@@ -291,7 +327,7 @@ def run_ours(args):
     achieved = gemm_ops / (gemm_ms * 1e-3) / 1e12
 
     per_layer = []
-    for s, q, g in zip(specs, q_ms, g_ms):
+    for s, q, g, pl in zip(specs, q_ms, g_ms, plain_ms):
         eo, uo = layer_ops(s)
         t_tensor = eo / (peak8 * 1e12)
         t_hbm = gemm_bytes(s) / (peaks["hbm_gbs"] * 1e9)
@@ -304,6 +340,8 @@ def run_ours(args):
             "gemm_roofline_frac": round(max(t_tensor, t_hbm) / (g * 1e-3), 4),
             "quant_gbs": round(quant_bytes(s) / (q * 1e-3) / 1e9, 1),
             "quant_frac_of_measured_hbm": round(quant_bytes(s) / (q * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+            "plain_w8a8_gemm_us": None if pl is None else round(pl * 1e3, 2),
+            "dual_gemm_time_over_plain": None if pl is None else round(float(g) / pl, 3),
         })
 
     out = None
@@ -323,7 +361,7 @@ def run_ours(args):
                                   for s in specs],
                        "step": "per layer: quantize_act -> dual/seg GEMM + dequant epilogue (bf16 out)",
                        "ops": "executed tensor ops: 4MNK for dual layers, 2MNK for single-scale layers",
-                       "l2": f"flushed before every layer ({L2_FLUSH_BYTES >> 20} MiB write), flush outside the timed intervals",
+                       "l2": f"flushed before every layer ({L2_FLUSH_BYTES >> 20} MiB write, then {L2_FLUSH_BYTES >> 20} MiB read), flush outside the timed intervals",
                        "parallelism": f"{world} independent row-sharded replicas, no collective" if world > 1 else "1 GPU"},
             "useful_tops": round(world * useful_ops / (step_ms * 1e-3) / 1e12, 2),
             "frac_of_nominal_4500_tops": round(exec_ops / (step_ms * 1e-3) / 1e12 / NOMINAL_8BIT_TOPS, 4),

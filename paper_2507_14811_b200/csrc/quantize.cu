@@ -1,6 +1,8 @@
 // Activation / weight quantization kernels (Sec. 3 uniform quantizer, Sec. 4.3.2 Q_dual and polarity
 // split, Sec. 4.2.2 one scale per segment).  HBM-streaming: every thread converts 16 consecutive
-// elements of one row (128-bit loads, one 128-bit store per code matrix).
+// elements of one row (128-bit loads, one 128-bit store per code matrix).  The codes are those of
+// "one IEEE fp32 division, round half to even, clip"; the common case computes them with a handful of
+// full-rate fp32 instructions per element (see SegConst) so that the pass stays memory bound.
 #include <cuda_bf16.h>
 #include "sq_common.cuh"
 
@@ -50,6 +52,8 @@ __device__ __forceinline__ uint32_t cvt_e4m3x2(float a, float b)
 }
 
 // One element -> (code for the positive / only matrix, code for the negative matrix), as bytes.
+// Reference form: one IEEE division, round half to even, clip.  Used where a vector straddles a
+// segment bound or the end of a row, and for scales outside the range of the fast form below.
 template <int CODE, bool DUAL>
 __device__ __forceinline__ void quant1(float x, float sp, float sn, int lo, int hi, uint32_t &cp, uint32_t &cn)
 {
@@ -69,59 +73,164 @@ __device__ __forceinline__ void quant1(float x, float sp, float sn, int lo, int 
     }
 }
 
+// Per-segment constants of the fast form.  The quotient x / s is obtained, correctly rounded, from the
+// correctly rounded reciprocal r = RN(1/s) by one multiply and two FMAs:
+//   q0 = RN(x r),  e = x - q0 s (exact in one FMA),  q = RN(q0 + e r)
+// which equals RN(x / s) when nothing over- or underflows on the way.  That is guaranteed by taking the
+// fast form only for 2^-100 <= s <= 2^100 and by first limiting |x| to 1024 s: such an input is clipped
+// to the end of the code range whether limited or not, and a quotient too small to be normal rounds
+// to code 0 whatever its last bits are.
+struct SegConst {
+    float s, r, lim;   // scale, RN(1/s), 1024 s
+    int fast;
+};
+__device__ __forceinline__ SegConst seg_const(float s)
+{
+    SegConst c;
+    c.s = s;
+    c.r = __frcp_rn(s);
+    c.lim = s * 1024.0f;
+    c.fast = (s >= 7.8886090522101181e-31f && s <= 1.2676506002282294e+30f) ? 1 : 0;
+    return c;
+}
+// packed fp32 pairs: sm_100 executes mul / fma / add on two fp32 values per instruction
+__device__ __forceinline__ uint64_t pack2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// two correctly rounded quotients x / s from r = RN(1/s): q0 = RN(x r), e = x - q0 s, q = RN(q0 + e r)
+__device__ __forceinline__ uint64_t div2_rn_fast(uint64_t x2, uint64_t neg_s2, uint64_t r2)
+{
+    const uint64_t q0 = mul2(x2, r2);
+    const uint64_t e = fma2(q0, neg_s2, x2);
+    return fma2(e, r2, q0);
+}
+
+constexpr float kRoundMagic = 12582912.0f;   // 1.5 * 2^23: v + magic rounds v to an integer, half to even
+
+// 16 elements of one K-segment -> packed codes.  int8: clip in fp32 (the bounds are integers, so
+// clip-then-round equals round-then-clip), add the magic constant, and the low byte of the sum's bit
+// pattern is the two's-complement code.  Dual: the positive matrix quantizes max(x, 0), the negative
+// one min(x, 0), each with its own constants, which reproduces the per-element polarity select.
+template <int CODE, bool DUAL>
+__device__ __forceinline__ void quant16(const float (&x)[kVec], const SegConst &cp, const SegConst &cn, float lo,
+                                        float hi, uint32_t (&wp)[4], uint32_t (&wn)[4])
+{
+    uint32_t bp[kVec], bn[kVec];
+    const uint64_t rp2 = pack2(cp.r, cp.r), nsp2 = pack2(-cp.s, -cp.s);
+    const uint64_t rn2 = pack2(cn.r, cn.r), nsn2 = pack2(-cn.s, -cn.s);
+    const uint64_t magic2 = pack2(kRoundMagic, kRoundMagic);
+#pragma unroll
+    for (int i = 0; i < kVec; i += 2) {
+        float a0, a1;
+        if (DUAL) {
+            const uint64_t qp2 = div2_rn_fast(pack2(fminf(fmaxf(x[i], 0.0f), cp.lim), fminf(fmaxf(x[i + 1], 0.0f), cp.lim)), nsp2, rp2);
+            const uint64_t qn2 = div2_rn_fast(pack2(fmaxf(fminf(x[i], 0.0f), -cn.lim), fmaxf(fminf(x[i + 1], 0.0f), -cn.lim)), nsn2, rn2);
+            if (CODE == SQ_CODE_INT8) {
+                unpack2(qp2, a0, a1);
+                unpack2(add2(pack2(fminf(a0, hi), fminf(a1, hi)), magic2), a0, a1);
+                bp[i] = __float_as_uint(a0); bp[i + 1] = __float_as_uint(a1);
+                unpack2(qn2, a0, a1);
+                unpack2(add2(pack2(fmaxf(a0, lo), fmaxf(a1, lo)), magic2), a0, a1);
+                bn[i] = __float_as_uint(a0); bn[i + 1] = __float_as_uint(a1);
+            } else {
+                unpack2(qp2, a0, a1);
+                bp[i] = __float_as_uint(a0); bp[i + 1] = __float_as_uint(a1);
+                unpack2(qn2, a0, a1);
+                bn[i] = __float_as_uint(a0); bn[i + 1] = __float_as_uint(a1);
+            }
+        } else {
+            const uint64_t q2 = div2_rn_fast(pack2(fminf(fmaxf(x[i], -cp.lim), cp.lim), fminf(fmaxf(x[i + 1], -cp.lim), cp.lim)), nsp2, rp2);
+            unpack2(q2, a0, a1);
+            if (CODE == SQ_CODE_INT8)
+                unpack2(add2(pack2(fminf(fmaxf(a0, lo), hi), fminf(fmaxf(a1, lo), hi)), magic2), a0, a1);
+            bp[i] = __float_as_uint(a0); bp[i + 1] = __float_as_uint(a1);
+        }
+    }
+#pragma unroll
+    for (int g = 0; g < 4; g++) {
+        if (CODE == SQ_CODE_INT8) {
+            wp[g] = __byte_perm(__byte_perm(bp[4 * g], bp[4 * g + 1], 0x0040), __byte_perm(bp[4 * g + 2], bp[4 * g + 3], 0x0040), 0x5410);
+            if (DUAL)
+                wn[g] = __byte_perm(__byte_perm(bn[4 * g], bn[4 * g + 1], 0x0040), __byte_perm(bn[4 * g + 2], bn[4 * g + 3], 0x0040), 0x5410);
+        } else {
+            uint32_t w = cvt_e4m3x2(__uint_as_float(bp[4 * g]), __uint_as_float(bp[4 * g + 1])) |
+                         (cvt_e4m3x2(__uint_as_float(bp[4 * g + 2]), __uint_as_float(bp[4 * g + 3])) << 16);
+            wp[g] = w & ~(__vcmpeq4(w & 0x7F7F7F7Fu, 0u) & 0x80808080u);      // -0 is stored as +0
+            if (DUAL) {
+                w = cvt_e4m3x2(__uint_as_float(bn[4 * g]), __uint_as_float(bn[4 * g + 1])) |
+                    (cvt_e4m3x2(__uint_as_float(bn[4 * g + 2]), __uint_as_float(bn[4 * g + 3])) << 16);
+                wn[g] = w & ~(__vcmpeq4(w & 0x7F7F7F7Fu, 0u) & 0x80808080u);
+            }
+        }
+    }
+}
+
 template <typename Tin, int CODE, bool DUAL>
 __global__ void __launch_bounds__(kThreads)
-quantize_kernel(const Tin *__restrict__ X, int64_t M, int K, int64_t ld, SegBounds sb,
+quantize_kernel(const Tin *__restrict__ X, int64_t M, int K, int64_t ld, const SegBounds sb,
                 const float *__restrict__ s_pos, const float *__restrict__ s_neg, int row_segments,
                 int lo, int hi, uint8_t *__restrict__ c_pos, uint8_t *__restrict__ c_neg, int64_t ldc)
 {
-    __shared__ float sh_sp[kMaxBlocks];
-    __shared__ float sh_sn[DUAL ? kMaxBlocks : 1];
-    __shared__ int sh_kb[SQ_MAX_P + 1];
-    const int Qs = row_segments ? sb.Q : 1;
-    for (int i = threadIdx.x; i < sb.P * Qs; i += kThreads) {
-        sh_sp[i] = s_pos[i];
-        if (DUAL) sh_sn[i] = s_neg[i];
-    }
-    for (int i = threadIdx.x; i <= sb.P; i += kThreads) sh_kb[i] = sb.kb[i];
-    __syncthreads();
-
     const int V = (K + kVec - 1) / kVec;
     const int64_t idx = int64_t(blockIdx.x) * kThreads + threadIdx.x;
     if (idx >= M * int64_t(V)) return;
     const int64_t row = idx / V;
     const int k0 = int(idx - row * V) * kVec;
 
+    // segment of this vector (bounds come with the kernel parameters); the scale loads below do not
+    // depend on the data loads, so both are in flight together
+    const int Qs = row_segments ? sb.Q : 1;
     int q = 0;
     if (row_segments) while (q + 1 < sb.Q && row >= sb.nb[q + 1]) q++;
     int p = 0;
-    while (p + 1 < sb.P && k0 >= sh_kb[p + 1]) p++;
+    while (p + 1 < sb.P && k0 >= sb.kb[p + 1]) p++;
+    const bool whole = k0 + kVec <= sb.kb[p + 1];            // vector inside one K-segment (and inside K)
 
     const Tin *src = X + row * ld + k0;
     uint8_t *dp = c_pos + row * ldc + k0;
     uint8_t *dn = DUAL ? c_neg + row * ldc + k0 : nullptr;
 
-    if (k0 + kVec <= sh_kb[p + 1]) {            // whole vector inside one K-segment (and inside K)
-        const float sp = sh_sp[p * Qs + q];
-        const float sn = DUAL ? sh_sn[p * Qs + q] : 0.0f;
-        float x[kVec];
-        load16(src, x);
-        uint32_t wp[4] = {0, 0, 0, 0}, wn[4] = {0, 0, 0, 0};
-#pragma unroll
-        for (int i = 0; i < kVec; i++) {
-            uint32_t a, b;
-            quant1<CODE, DUAL>(x[i], sp, sn, lo, hi, a, b);
-            wp[i >> 2] |= a << (8 * (i & 3));
-            if (DUAL) wn[i >> 2] |= b << (8 * (i & 3));
-        }
+    float x[kVec];
+    if (whole) load16(src, x);
+    const SegConst cp = seg_const(__ldg(s_pos + p * Qs + q));
+    const SegConst cn = seg_const(DUAL ? __ldg(s_neg + p * Qs + q) : 1.0f);
+    if (whole && cp.fast && cn.fast) {
+        uint32_t wp[4], wn[4];
+        quant16<CODE, DUAL>(x, cp, cn, float(lo), float(hi), wp, wn);
         *reinterpret_cast<uint4 *>(dp) = make_uint4(wp[0], wp[1], wp[2], wp[3]);
         if (DUAL) *reinterpret_cast<uint4 *>(dn) = make_uint4(wn[0], wn[1], wn[2], wn[3]);
-    } else {                                    // vector crosses a segment bound or the end of the row
+    } else {                                    // segment bound or end of row inside the vector, or an extreme scale
         const int n = min(kVec, K - k0);
         for (int i = 0; i < n; i++) {
-            while (p + 1 < sb.P && k0 + i >= sh_kb[p + 1]) p++;
+            while (p + 1 < sb.P && k0 + i >= sb.kb[p + 1]) p++;
             uint32_t a, b;
-            quant1<CODE, DUAL>(load1(src + i), sh_sp[p * Qs + q], DUAL ? sh_sn[p * Qs + q] : 0.0f, lo, hi, a, b);
+            quant1<CODE, DUAL>(load1(src + i), __ldg(s_pos + p * Qs + q), DUAL ? __ldg(s_neg + p * Qs + q) : 0.0f, lo, hi,
+                               a, b);
             dp[i] = uint8_t(a);
             if (DUAL) dn[i] = uint8_t(b);
         }

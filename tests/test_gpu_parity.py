@@ -160,6 +160,42 @@ def test_strided_output_and_code_matrices():
     check_bf16_output(Y.contiguous(), res.y64, res.y_abs, 2)
 
 
+@pytest.mark.parametrize("code", ["int8", "e4m3"])
+@pytest.mark.parametrize("dual", [True, False])
+def test_quantizer_codes_equal_the_division_definition_on_adversarial_values(code, dual):
+    """Codes are defined by one IEEE fp32 division, round half to even, clip.  Random mantissas for scale
+    and input, quotients spread over and beyond the code range, exact ties, tiny quotients, and scales
+    at the extremes of the fp32 range (which take the kernel's division path)."""
+    rs = np.random.default_rng(5)
+    M, P, seg_len = 1024, 8, 512
+    K = P * seg_len
+    kb = [i * seg_len for i in range(P + 1)]
+    exps = [0, -7, 13, -30, 40, -110, 105, 3]
+    sp = (rs.uniform(1.0, 2.0, P) * np.exp2(exps)).astype(np.float32)
+    sn = (rs.uniform(1.0, 2.0, P) * np.exp2(exps[::-1])).astype(np.float32)
+    qmax, qmin_abs = QRANGE[code]
+    X = np.empty((M, K), np.float32)
+    for p in range(P):
+        blk = rs.uniform(-1.3 * qmax, 1.3 * qmax, (M, seg_len))
+        blk[:, :64] = np.round(blk[:, :64]) + 0.5                      # exact ties
+        blk[:, 64:96] *= 1e-3                                          # near zero
+        blk[:, 96:100] *= 1e6                                          # far outside the range
+        s_elem = np.where(blk >= 0, sp[p], sn[p] if dual else sp[p]).astype(np.float64)
+        with np.errstate(over="ignore"):
+            X[:, kb[p]:kb[p + 1]] = (blk * s_elem).astype(np.float32)
+    X[~np.isfinite(X)] = 0.0
+    seg = B.SegTable(kb, [0, 8])
+    Xd = torch.from_numpy(X).to(DEV)
+    c_pos, c_neg = B.segquant_quantize_act(Xd, seg, torch.from_numpy(sp).to(DEV),
+                                           torch.from_numpy(sn).to(DEV) if dual else None, code)
+    torch.cuda.synchronize()
+    r_pos, r_neg = O.quantize_act(X, kb, sp, sn if dual else None, code=code, q_max=qmax, q_min_abs=qmin_abs)
+    dt = np.int8 if code == "int8" else np.uint8
+    assert np.array_equal(c_pos.cpu().numpy().view(dt), r_pos)
+    if dual:
+        assert np.array_equal(c_neg.cpu().numpy().view(dt), r_neg)
+
+
 def test_fp32_input_and_student_t():
     run_parity(custom_spec("f32_in", 160, 256, 128, [0, 128, 256], [0, 128], True, "int8", x_dtype="f32",
                            x_kind="student_t4+silu"))
