@@ -279,7 +279,10 @@ __device__ __forceinline__ void issue_kblock(uint32_t d0, uint64_t da, uint64_t 
     }
 }
 
-template <int KIND, int NPOL, int TILE_N, int CG>
+// DEBUG_OUT = false is the production variant: bf16 output and no accumulator dump, which keeps the
+// epilogue loop small enough for the instruction cache (the two rarely used branches made every
+// tile's epilogue about a quarter slower).  DEBUG_OUT = true adds the fp32 output and the dump.
+template <int KIND, int NPOL, int TILE_N, int CG, bool DEBUG_OUT>
 __global__ void __launch_bounds__(kThreads, 1)
 segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_constant__ CUtensorMap tm_a_neg,
                      const __grid_constant__ CUtensorMap tm_b, const KernelParams prm)
@@ -501,7 +504,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                         y[j] = fmaf(cc[t], v, y[j]);
                     }
                 }
-                if (prm.acc_dump && row < prm.M) {
+                if (DEBUG_OUT && prm.acc_dump && row < prm.M) {
                     uint32_t *dump = static_cast<uint32_t *>(prm.acc_dump) +
                                      (size_t(c_a) * prm.M + row) * size_t(prm.N) + n0 + c0;
 #pragma unroll
@@ -521,7 +524,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                 // outside the matrix
                 if (row < prm.M) {
                     const int nvalid = prm.N - (n0 + c0);            // valid columns of this slab, may exceed 32
-                    if (prm.y_is_f32) {
+                    if (DEBUG_OUT && prm.y_is_f32) {
                         float *dst = static_cast<float *>(prm.Y) + size_t(row) * prm.ldy + n0 + c0;
 #pragma unroll
                         for (int c = 0; c < 4; c++) {                // 8 columns = 32 bytes
@@ -631,7 +634,7 @@ bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, in
 
 int g_tune_tile_n = 0, g_tune_stages = 0, g_tune_cta_group = 0;
 
-template <int KIND, int NPOL, int TILE_N, int CG>
+template <int KIND, int NPOL, int TILE_N, int CG, bool DEBUG_OUT>
 sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cudaStream_t st)
 {
     constexpr int B_ROWS = TILE_N / CG;
@@ -651,7 +654,7 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
     prm.num_n_tiles = int((g.N + TILE_N - 1) / TILE_N);
     const size_t smem = 1024 + size_t(stages) * stage_bytes + tail;
 
-    auto kern = segquant_gemm_kernel<KIND, NPOL, TILE_N, CG>;
+    auto kern = segquant_gemm_kernel<KIND, NPOL, TILE_N, CG, DEBUG_OUT>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
         return SQ_ERR_CUDA;
     const int tiles = prm.num_m_tiles * prm.num_n_tiles;
@@ -692,11 +695,16 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
 template <int KIND, int NPOL, int CG>
 sq_status launch_tile(const GemmArgs &g, KernelParams &prm, int tile_n, int sm_count, cudaStream_t st)
 {
+    const bool dbg = prm.y_is_f32 || prm.acc_dump != nullptr;
     switch (tile_n) {
-        case 256: return launch_variant<KIND, NPOL, 256, CG>(g, prm, sm_count, st);
-        case 128: return launch_variant<KIND, NPOL, 128, CG>(g, prm, sm_count, st);
-        case 64: return launch_variant<KIND, NPOL, 64, CG>(g, prm, sm_count, st);
-        case 32: return launch_variant<KIND, NPOL, 32, CG>(g, prm, sm_count, st);
+        case 256: return dbg ? launch_variant<KIND, NPOL, 256, CG, true>(g, prm, sm_count, st)
+                             : launch_variant<KIND, NPOL, 256, CG, false>(g, prm, sm_count, st);
+        case 128: return dbg ? launch_variant<KIND, NPOL, 128, CG, true>(g, prm, sm_count, st)
+                             : launch_variant<KIND, NPOL, 128, CG, false>(g, prm, sm_count, st);
+        case 64: return dbg ? launch_variant<KIND, NPOL, 64, CG, true>(g, prm, sm_count, st)
+                            : launch_variant<KIND, NPOL, 64, CG, false>(g, prm, sm_count, st);
+        case 32: return dbg ? launch_variant<KIND, NPOL, 32, CG, true>(g, prm, sm_count, st)
+                            : launch_variant<KIND, NPOL, 32, CG, false>(g, prm, sm_count, st);
     }
     return SQ_ERR_UNSUPPORTED;
 }
