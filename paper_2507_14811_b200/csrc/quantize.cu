@@ -76,23 +76,35 @@ __device__ __forceinline__ void quant1(float x, float sp, float sn, int lo, int 
 // Per-segment constants of the fast form.  The quotient x / s is obtained, correctly rounded, from the
 // correctly rounded reciprocal r = RN(1/s) by one multiply and two FMAs:
 //   q0 = RN(x r),  e = x - q0 s (exact in one FMA),  q = RN(q0 + e r)
-// which equals RN(x / s) when nothing over- or underflows on the way.  That is guaranteed by taking the
-// fast form only for 2^-100 <= s <= 2^100 and by first limiting |x| to 1024 s: such an input is clipped
-// to the end of the code range whether limited or not, and a quotient too small to be normal rounds
-// to code 0 whatever its last bits are.
+// which equals RN(x / s) when nothing over- or underflows on the way.  To rule that out, and to get the
+// polarity split for free, the input is first mapped to u = sat(x / L) in [0, 1] by one saturating FMA,
+// L = 2^(exponent(s) + 11) >= 1024 s.  L is a power of two, so x / L is exact and u / (s / L) has the
+// bits of x / s; negative x give u = 0 (the other polarity's zero code) and x > L, which is clipped to
+// the end of the code range anyway, gives u = 1.  A quotient too small to be normal rounds to code 0
+// whatever its last bits are.  The fast form is taken for 2^-100 <= s <= 2^100.
 struct SegConst {
-    float s, r, lim;   // scale, RN(1/s), 1024 s
+    float inv_l;       // 1 / L
+    float s_l, r_l;    // s / L and RN(L / s) = RN(1 / s) L
     int fast;
 };
 __device__ __forceinline__ SegConst seg_const(float s)
 {
     SegConst c;
-    c.s = s;
-    c.r = __frcp_rn(s);
-    c.lim = s * 1024.0f;
     c.fast = (s >= 7.8886090522101181e-31f && s <= 1.2676506002282294e+30f) ? 1 : 0;
+    const uint32_t l_bits = (__float_as_uint(s) & 0x7F800000u) + (11u << 23);
+    const float l = __uint_as_float(l_bits);
+    c.inv_l = __uint_as_float((254u << 23) - l_bits);
+    c.s_l = s * c.inv_l;
+    c.r_l = __frcp_rn(s) * l;
     return c;
 }
+__device__ __forceinline__ float fma_sat(float a, float b, float c)
+{
+    float d;
+    asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 // packed fp32 pairs: sm_100 executes mul / fma / add on two fp32 values per instruction
 __device__ __forceinline__ uint64_t pack2(float lo, float hi)
 {
@@ -134,22 +146,23 @@ constexpr float kRoundMagic = 12582912.0f;   // 1.5 * 2^23: v + magic rounds v t
 
 // 16 elements of one K-segment -> packed codes.  int8: clip in fp32 (the bounds are integers, so
 // clip-then-round equals round-then-clip), add the magic constant, and the low byte of the sum's bit
-// pattern is the two's-complement code.  Dual: the positive matrix quantizes max(x, 0), the negative
-// one min(x, 0), each with its own constants, which reproduces the per-element polarity select.
+// pattern is the two's-complement code.  Dual: the positive matrix quantizes max(x, 0) = L sat(x / L),
+// the negative one min(x, 0) = -L sat(-x / L), each with its own constants, which reproduces the
+// per-element polarity select.  Single scale: |x| is quantized and the sign put back when rounding.
 template <int CODE, bool DUAL>
 __device__ __forceinline__ void quant16(const float (&x)[kVec], const SegConst &cp, const SegConst &cn, float lo,
                                         float hi, uint32_t (&wp)[4], uint32_t (&wn)[4])
 {
     uint32_t bp[kVec], bn[kVec];
-    const uint64_t rp2 = pack2(cp.r, cp.r), nsp2 = pack2(-cp.s, -cp.s);
-    const uint64_t rn2 = pack2(cn.r, cn.r), nsn2 = pack2(-cn.s, -cn.s);
+    const uint64_t rp2 = pack2(cp.r_l, cp.r_l), nsp2 = pack2(-cp.s_l, -cp.s_l);
+    const uint64_t rn2 = pack2(-cn.r_l, -cn.r_l), nsn2 = pack2(cn.s_l, cn.s_l);   // negated: quotients <= 0
     const uint64_t magic2 = pack2(kRoundMagic, kRoundMagic);
 #pragma unroll
     for (int i = 0; i < kVec; i += 2) {
         float a0, a1;
         if (DUAL) {
-            const uint64_t qp2 = div2_rn_fast(pack2(fminf(fmaxf(x[i], 0.0f), cp.lim), fminf(fmaxf(x[i + 1], 0.0f), cp.lim)), nsp2, rp2);
-            const uint64_t qn2 = div2_rn_fast(pack2(fmaxf(fminf(x[i], 0.0f), -cn.lim), fmaxf(fminf(x[i + 1], 0.0f), -cn.lim)), nsn2, rn2);
+            const uint64_t qp2 = div2_rn_fast(pack2(fma_sat(x[i], cp.inv_l, 0.0f), fma_sat(x[i + 1], cp.inv_l, 0.0f)), nsp2, rp2);
+            const uint64_t qn2 = div2_rn_fast(pack2(fma_sat(x[i], -cn.inv_l, 0.0f), fma_sat(x[i + 1], -cn.inv_l, 0.0f)), nsn2, rn2);
             if (CODE == SQ_CODE_INT8) {
                 unpack2(qp2, a0, a1);
                 unpack2(add2(pack2(fminf(a0, hi), fminf(a1, hi)), magic2), a0, a1);
@@ -164,10 +177,15 @@ __device__ __forceinline__ void quant16(const float (&x)[kVec], const SegConst &
                 bn[i] = __float_as_uint(a0); bn[i + 1] = __float_as_uint(a1);
             }
         } else {
-            const uint64_t q2 = div2_rn_fast(pack2(fminf(fmaxf(x[i], -cp.lim), cp.lim), fminf(fmaxf(x[i + 1], -cp.lim), cp.lim)), nsp2, rp2);
+            const uint64_t q2 = div2_rn_fast(pack2(fma_sat(fabsf(x[i]), cp.inv_l, 0.0f), fma_sat(fabsf(x[i + 1]), cp.inv_l, 0.0f)), nsp2, rp2);
             unpack2(q2, a0, a1);
-            if (CODE == SQ_CODE_INT8)
-                unpack2(add2(pack2(fminf(fmaxf(a0, lo), hi), fminf(fmaxf(a1, lo), hi)), magic2), a0, a1);
+            if (CODE == SQ_CODE_INT8) {                  // the range is symmetric: clip |q|, round with the sign of x
+                a0 = fmaf(fminf(a0, hi), copysignf(1.0f, x[i]), kRoundMagic);
+                a1 = fmaf(fminf(a1, hi), copysignf(1.0f, x[i + 1]), kRoundMagic);
+            } else {
+                a0 = copysignf(a0, x[i]);
+                a1 = copysignf(a1, x[i + 1]);
+            }
             bp[i] = __float_as_uint(a0); bp[i + 1] = __float_as_uint(a1);
         }
     }
