@@ -149,6 +149,46 @@ __device__ __forceinline__ float4 ld_shared_f4(uint32_t addr)
     return v;
 }
 
+__device__ __forceinline__ void ld_shared_2x64(uint32_t addr, uint64_t &a, uint64_t &b)
+{
+    asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "r"(addr));
+}
+__device__ __forceinline__ float ld_shared_f32(uint32_t addr)
+{
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t ld_shared_u32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+// packed fp32 pairs (two outputs per instruction)
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ uint64_t pack_b32x2(uint32_t lo, uint32_t hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
 // 16- and 32-byte global stores
 __device__ __forceinline__ void st_global_16(void *p, uint4 v)
 {
@@ -241,6 +281,14 @@ __host__ __device__ constexpr uint32_t make_idesc(int kind, int tile_n, int mma_
 
 // ----------------------------------------------------------------------------- the kernel
 
+// bytes of the epilogue's tables between the ring and the header (multiple of 16)
+template <bool GENERIC>
+__host__ __device__ constexpr uint32_t epi_table_bytes(int nacc, int Q, int tile_n)
+{
+    return GENERIC ? uint32_t(nacc + 1) * tile_n * 4u
+                   : ((uint32_t(tile_n) + uint32_t(nacc) * Q + uint32_t(Q) + 1u) * 4u + 15u) & ~15u;
+}
+
 struct SharedHeader {
     uint64_t full[kMaxStages];
     uint64_t empty[kMaxStages];
@@ -279,10 +327,12 @@ __device__ __forceinline__ void issue_kblock(uint32_t d0, uint64_t da, uint64_t 
     }
 }
 
-// DEBUG_OUT = false is the production variant: bf16 output and no accumulator dump, which keeps the
-// epilogue loop small enough for the instruction cache (the two rarely used branches made every
-// tile's epilogue about a quarter slower).  DEBUG_OUT = true adds the fp32 output and the dump.
-template <int KIND, int NPOL, int TILE_N, int CG, bool DEBUG_OUT>
+// GENERIC = false is the production variant: bf16 output, no accumulator dump, every interior N-bound
+// a multiple of 32 (so that each 32-column slab of the output lies in one N-segment and takes ONE
+// dequantization factor per accumulator).  Its epilogue loop is small enough for the instruction
+// cache and runs its FMAs on packed fp32 pairs.  GENERIC = true handles everything else (fp32 output,
+// accumulator dump, arbitrary N-bounds) with a per-column factor table rebuilt for every tile.
+template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC>
 __global__ void __launch_bounds__(kThreads, 1)
 segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_constant__ CUtensorMap tm_a_neg,
                      const __grid_constant__ CUtensorMap tm_b, const KernelParams prm)
@@ -294,9 +344,12 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     constexpr uint32_t b_bytes = B_ROWS * BLOCK_K;
     constexpr uint32_t stage_bytes = NPOL * a_bytes + b_bytes;
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    float *sh_scale = reinterpret_cast<float *>(smem + size_t(prm.stages) * stage_bytes);   // [nacc][TILE_N]
-    float *sh_bias = sh_scale + prm.nacc * TILE_N;                                          // [TILE_N]
-    SharedHeader *hdr = reinterpret_cast<SharedHeader *>(sh_bias + TILE_N);
+    float *sh_scale = reinterpret_cast<float *>(smem + size_t(prm.stages) * stage_bytes);   // GENERIC: [nacc][TILE_N]
+    float *sh_bias = sh_scale + (GENERIC ? prm.nacc * TILE_N : 0);                          // [TILE_N], per tile
+    float *sh_tab = sh_bias + TILE_N;                                                       // !GENERIC: [nacc][Q]
+    int *sh_nb = reinterpret_cast<int *>(sh_tab + (GENERIC ? 0 : prm.nacc * prm.sb.Q));     // !GENERIC: [Q + 1]
+    SharedHeader *hdr = reinterpret_cast<SharedHeader *>(
+        reinterpret_cast<uint8_t *>(smem + size_t(prm.stages) * stage_bytes) + epi_table_bytes<GENERIC>(prm.nacc, prm.sb.Q, TILE_N));
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -317,6 +370,15 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
         hdr->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (!GENERIC) {
+        // dequantization factors c[a][q] = s_act[p][pol] * s_w[p][q], a = p * NPOL + pol (one fp32 multiply)
+        for (int i = threadIdx.x; i < prm.nacc * prm.sb.Q; i += kThreads) {
+            const int a = i / prm.sb.Q, q = i - a * prm.sb.Q, p = a / NPOL;
+            const float s_act = (NPOL == 2 && (a & 1)) ? prm.s_neg[p] : prm.s_pos[p];
+            sh_tab[i] = s_act * prm.s_w[p * prm.sb.Q + q];
+        }
+        for (int i = threadIdx.x; i <= prm.sb.Q; i += kThreads) sh_nb[i] = prm.sb.nb[i];
     }
     if (warp == 1) {
         if (CG == 1) {
@@ -425,6 +487,143 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
+        // Warp w may read TMEM lanes 32 * (w % 4) .. + 31; the two warps of one lane group take one half
+        // of the tile's 32-column slabs each.
+        if constexpr (!GENERIC) {
+            const int et = threadIdx.x - 64;
+            const int ew = warp - 2;
+            const int lane_grp = warp & 3;
+            constexpr int kColGroups = kEpiWarps / 4;
+            constexpr int kSlabs = TILE_N / 32;
+            constexpr int kSlabsPerWarp = (kSlabs + kColGroups - 1) / kColGroups;
+            const int slab0 = (ew >> 2) * kSlabsPerWarp;
+            const int my_slabs = max(0, min(kSlabsPerWarp, kSlabs - slab0));
+            const int nacc = prm.nacc;
+            const int units = my_slabs * nacc;                              // (slab, accumulator) pairs of this warp
+            const int Q = prm.sb.Q;
+            const uint32_t tmem_empty_sig0 = CG == 2 ? map_to_cta(smem_u32(&hdr->tmem_empty[0]), 0)
+                                                     : smem_u32(&hdr->tmem_empty[0]);
+            const uint32_t tab_addr = smem_u32(sh_tab), nb_addr = smem_u32(sh_nb), bias_addr = smem_u32(sh_bias);
+            // bias slice of a tile, one column per thread, fetched one tile ahead into a register
+            auto fetch_bias = [&](int tile) -> float {
+                if (tile >= num_tiles || et >= TILE_N || !prm.bias) return 0.0f;
+                const int n = (tile % prm.num_n_tiles) * TILE_N + et;
+                return n < prm.N ? __ldg(prm.bias + n) : 0.0f;
+            };
+            float bias_next = fetch_bias(unit);
+            uint32_t as = 0, aph = 0;
+            bool ok = true;
+            for (int tile = unit; tile < num_tiles; tile += num_units) {
+                const int m0 = (tile / prm.num_n_tiles) * (TILE_M * CG) + int(rank) * TILE_M;
+                const int n0 = (tile % prm.num_n_tiles) * TILE_N;
+                const uint32_t cur_as = as, cur_aph = aph;
+                if (++as == uint32_t(prm.acc_stages)) { as = 0; aph ^= 1; }
+
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // previous tile's readers are done
+                if (et < TILE_N) sh_bias[et] = bias_next;
+                bias_next = fetch_bias(tile + num_units);                        // lands during this tile's work
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+
+                if (ok) ok = mbar_wait(smem_u32(&hdr->tmem_full[cur_as]), cur_aph, abort_flag, prm.status, kWhereEpilogue);
+                if (!ok) continue;                  // keep the named barriers balanced, do no more work
+                tc_fence_after();
+
+                const int row = m0 + lane_grp * 32 + lane;
+                const uint32_t t_row = tmem_base + (uint32_t(lane_grp * 32) << 16) + cur_as * acc_cols;
+                const uint32_t release_bar = tmem_empty_sig0 + 8 * cur_as;
+
+                // The (slab, accumulator) units of this warp are read from TMEM one ahead of the arithmetic;
+                // the accumulator set goes back to the MMA issuer as soon as the last load has landed.
+                // Per output: y = bias, then y = fma(c[a][q], acc[a], y) over a = (p, polarity) ascending,
+                // two outputs per instruction on packed fp32 pairs.
+                uint64_t y2[16];
+                uint32_t ra[32], rb[32];
+                int i_sl = 0, i_a = 0;              // next unit to load
+                int c_sl = 0, c_a = 0;              // next unit to consume
+                int q_seg = 0;                      // N-segment of the slab being consumed
+                auto issue = [&](uint32_t (&r)[32]) {
+                    tc_ld32(t_row + uint32_t(i_a * TILE_N + (slab0 + i_sl) * 32), r);
+                    if (++i_a == nacc) { i_a = 0; i_sl++; }
+                };
+                auto release = [&]() {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (CG == 2) mbar_arrive_cluster(release_bar);
+                        else mbar_arrive(release_bar);
+                    }
+                };
+                auto consume = [&](const uint32_t (&r)[32]) {
+                    const int c0 = (slab0 + c_sl) * 32;
+                    const int nf = n0 + c0;                          // first column of the slab
+                    if (c_a == 0) {
+                        // segment of the slab: the number of interior bounds nb[1..Q-1] that are <= nf
+                        q_seg = 0;
+                        for (int base = 1; base < Q; base += 32) {
+                            const int i = base + lane;
+                            const bool le = i < Q && nf >= int(ld_shared_u32(nb_addr + 4u * uint32_t(i < Q ? i : 0)));
+                            q_seg += __popc(__ballot_sync(0xFFFFFFFFu, le));
+                        }
+#pragma unroll
+                        for (int j4 = 0; j4 < 8; j4++)
+                            ld_shared_2x64(bias_addr + uint32_t(c0 + 4 * j4) * 4u, y2[2 * j4], y2[2 * j4 + 1]);
+                    }
+                    const float c = ld_shared_f32(tab_addr + uint32_t(c_a * Q + q_seg) * 4u);
+                    const uint64_t c2 = pack_f32x2(c, c);
+#pragma unroll
+                    for (int j = 0; j < 16; j++) {
+                        const uint64_t v2 = KIND == 0 ? pack_f32x2(__int2float_rn(int(r[2 * j])), __int2float_rn(int(r[2 * j + 1])))
+                                                      : pack_b32x2(r[2 * j], r[2 * j + 1]);
+                        y2[j] = fma_f32x2(c2, v2, y2[j]);
+                    }
+                    if (++c_a < nacc) return;
+                    c_a = 0;
+                    c_sl++;
+                    // last accumulator of the slab: convert and store this thread's 32 outputs of row `row` in
+                    // 16-byte chunks of 8 bf16; N is a multiple of 8, so a chunk is entirely inside or outside
+                    if (row < prm.M) {
+                        const int nvalid = prm.N - nf;               // valid columns of this slab, may exceed 32
+                        __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(prm.Y) + size_t(row) * prm.ldy + nf;
+                        uint32_t h[16];
+#pragma unroll
+                        for (int j = 0; j < 16; j++) {
+                            float lo, hi;
+                            unpack_f32x2(y2[j], lo, hi);
+                            __nv_bfloat162 v2 = __floats2bfloat162_rn(lo, hi);
+                            h[j] = *reinterpret_cast<uint32_t *>(&v2);
+                        }
+#pragma unroll
+                        for (int cidx = 0; cidx < 2; cidx++) {       // 16 columns = 32 bytes
+                            const uint4 w0 = make_uint4(h[8 * cidx], h[8 * cidx + 1], h[8 * cidx + 2], h[8 * cidx + 3]);
+                            const uint4 w1 = make_uint4(h[8 * cidx + 4], h[8 * cidx + 5], h[8 * cidx + 6], h[8 * cidx + 7]);
+                            if (16 * cidx + 8 < nvalid && prm.y_wide) {
+                                st_global_32(dst + 16 * cidx, w0, w1);
+                            } else {
+                                if (16 * cidx < nvalid) st_global_16(dst + 16 * cidx, w0);
+                                if (16 * cidx + 8 < nvalid) st_global_16(dst + 16 * cidx + 8, w1);
+                            }
+                        }
+                    }
+                };
+
+                if (units == 0) {
+                    release();
+                } else {
+                    issue(ra);
+#pragma unroll 1
+                    for (int u = 0; u < units; u += 2) {
+                        tc_wait_ld();
+                        if (u + 1 < units) issue(rb); else release();
+                        consume(ra);
+                        if (u + 1 < units) {
+                            tc_wait_ld();
+                            if (u + 2 < units) issue(ra); else release();
+                            consume(rb);
+                        }
+                    }
+                }
+            }
+        } else {
         const int et = threadIdx.x - 64;           // 0..255
         const int ew = warp - 2;                   // 0..7
         const int lane_grp = warp & 3;             // TMEM lanes 32*lane_grp .. +31 are this warp's
@@ -504,7 +703,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                         y[j] = fmaf(cc[t], v, y[j]);
                     }
                 }
-                if (DEBUG_OUT && prm.acc_dump && row < prm.M) {
+                if (GENERIC && prm.acc_dump && row < prm.M) {
                     uint32_t *dump = static_cast<uint32_t *>(prm.acc_dump) +
                                      (size_t(c_a) * prm.M + row) * size_t(prm.N) + n0 + c0;
 #pragma unroll
@@ -524,7 +723,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                 // outside the matrix
                 if (row < prm.M) {
                     const int nvalid = prm.N - (n0 + c0);            // valid columns of this slab, may exceed 32
-                    if (DEBUG_OUT && prm.y_is_f32) {
+                    if (GENERIC && prm.y_is_f32) {
                         float *dst = static_cast<float *>(prm.Y) + size_t(row) * prm.ldy + n0 + c0;
 #pragma unroll
                         for (int c = 0; c < 4; c++) {                // 8 columns = 32 bytes
@@ -582,6 +781,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                 }
             }
         }
+        }
     }
 
     tc_fence_before();
@@ -634,7 +834,7 @@ bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, in
 
 int g_tune_tile_n = 0, g_tune_stages = 0, g_tune_cta_group = 0;
 
-template <int KIND, int NPOL, int TILE_N, int CG, bool DEBUG_OUT>
+template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC>
 sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cudaStream_t st)
 {
     constexpr int B_ROWS = TILE_N / CG;
@@ -644,7 +844,7 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
     if (!make_map(&tb, g.b, g.N, g.K, g.ldb, B_ROWS)) return SQ_ERR_CUDA;
 
     const uint32_t stage_bytes = NPOL * TILE_M * BLOCK_K + B_ROWS * BLOCK_K;
-    const uint32_t tail = uint32_t(prm.nacc + 1) * TILE_N * 4 + sizeof(SharedHeader);
+    const uint32_t tail = epi_table_bytes<GENERIC>(prm.nacc, prm.sb.Q, TILE_N) + sizeof(SharedHeader);
     int stages = int((kSmemBudget - 1024 - tail) / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (g_tune_stages >= 2 && g_tune_stages < stages) stages = g_tune_stages;
@@ -654,7 +854,7 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
     prm.num_n_tiles = int((g.N + TILE_N - 1) / TILE_N);
     const size_t smem = 1024 + size_t(stages) * stage_bytes + tail;
 
-    auto kern = segquant_gemm_kernel<KIND, NPOL, TILE_N, CG, DEBUG_OUT>;
+    auto kern = segquant_gemm_kernel<KIND, NPOL, TILE_N, CG, GENERIC>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
         return SQ_ERR_CUDA;
     const int tiles = prm.num_m_tiles * prm.num_n_tiles;
@@ -695,7 +895,8 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
 template <int KIND, int NPOL, int CG>
 sq_status launch_tile(const GemmArgs &g, KernelParams &prm, int tile_n, int sm_count, cudaStream_t st)
 {
-    const bool dbg = prm.y_is_f32 || prm.acc_dump != nullptr;
+    bool dbg = prm.y_is_f32 || prm.acc_dump != nullptr;
+    for (int q = 1; q < prm.sb.Q; q++) dbg = dbg || (prm.sb.nb[q] % 32 != 0);
     switch (tile_n) {
         case 256: return dbg ? launch_variant<KIND, NPOL, 256, CG, true>(g, prm, sm_count, st)
                              : launch_variant<KIND, NPOL, 256, CG, false>(g, prm, sm_count, st);
