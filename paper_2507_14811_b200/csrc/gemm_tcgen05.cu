@@ -944,14 +944,6 @@ sq_status launch_gemm(const GemmArgs &g, cudaStream_t st)
     prm.acc_dump = g.acc_dump;
     prm.status = g.status;
 
-    // widest tile whose accumulators fit the 512 TMEM columns
-    int tile_n = 256;
-    while (tile_n * prm.nacc > kTmemCols) tile_n >>= 1;
-    if (tile_n < 32) return SQ_ERR_UNSUPPORTED;
-    if (g_tune_tile_n >= 32 && g_tune_tile_n <= tile_n && (g_tune_tile_n & (g_tune_tile_n - 1)) == 0)
-        tile_n = g_tune_tile_n;
-    prm.acc_stages = (2 * tile_n * prm.nacc <= kTmemCols) ? 2 : 1;
-
     int dev = 0, sm_count = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return SQ_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
@@ -961,6 +953,27 @@ sq_status launch_gemm(const GemmArgs &g, cudaStream_t st)
     int cg = g.M > TILE_M ? 2 : 1;
     if (g_tune_cta_group == 1 || g_tune_cta_group == 2) cg = g_tune_cta_group;
     if (sm_count < 2) cg = 1;
+
+    // Tile width: the widest tile whose accumulators fit the 512 TMEM columns, unless half that width
+    // fills the machine so much better that it outweighs the narrower tile's higher operand traffic
+    // per MMA (weights 1 : 0.75; a double-buffered accumulator set counts 10 % extra).
+    int tile_max = 256;
+    while (tile_max * prm.nacc > kTmemCols) tile_max >>= 1;
+    if (tile_max < 32) return SQ_ERR_UNSUPPORTED;
+    int tile_n = tile_max;
+    if (tile_max >= 128) {
+        const int64_t units = sm_count / cg;
+        auto score = [&](int tn, double weight) {
+            const int64_t tiles = ((g.M + TILE_M * cg - 1) / (TILE_M * cg)) * ((g.N + tn - 1) / tn);
+            const int64_t waves = (tiles + units - 1) / units;
+            const double dbuf = (2 * tn * prm.nacc <= kTmemCols) ? 1.1 : 1.0;
+            return weight * dbuf * double(tiles) / double(waves * units);
+        };
+        if (score(tile_max / 2, 0.75) > score(tile_max, 1.0)) tile_n = tile_max / 2;
+    }
+    if (g_tune_tile_n >= 32 && g_tune_tile_n <= tile_max && (g_tune_tile_n & (g_tune_tile_n - 1)) == 0)
+        tile_n = g_tune_tile_n;
+    prm.acc_stages = (2 * tile_n * prm.nacc <= kTmemCols) ? 2 : 1;
 
     return g.code == SQ_CODE_INT8 ? launch_kind<0>(g, prm, npol, cg, tile_n, sm_count, st)
                                   : launch_kind<1>(g, prm, npol, cg, tile_n, sm_count, st);
