@@ -371,6 +371,7 @@ def run_ours(args):
             "roofline": {"bound": "tensor", "achieved": round(achieved, 1), "peak": round(peak8, 1),
                          "unit": "TFLOP/s", "frac": round(achieved / peak8, 4),
                          "traffic": GEMM_DRAM_TRAFFIC.get(args.workload),
+                         "traffic_unit": "bytes per step (all GEMM launches of the step, like achieved)",
                          "kernel": "segquant_gemm_kernel", "launches_per_step": len(specs),
                          "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TFLOP/s x 2 (nominal 8-bit : bf16 ratio)",
                          "algorithmic_ops_per_step": gemm_ops, "avg_launch_us": round(gemm_ms * 1e3 / len(specs), 2),
@@ -386,8 +387,9 @@ def run_ours(args):
     return out
 
 
-# DRAM bytes (read + write) per step of the GEMM launches, from ncu captures (see profiles/); None = not captured.
-GEMM_DRAM_TRAFFIC = {}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the GEMM launches of one step, from the ncu
+# capture summarised in profiles/gemm_pair_and_quantize_dit_xl2_sd3_mmdit.md; None = not captured for that workload.
+GEMM_DRAM_TRAFFIC = {"dit_xl2": 12747008 + 18176 + 24225536, "sd3_mmdit": 41480448 + 38845696 + 23170560 + 56780032 + 123167744 + 13605632}
 
 
 # ------------------------------------------------------------------------------------ reference arm
