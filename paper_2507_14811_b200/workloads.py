@@ -173,6 +173,13 @@ WORKLOADS: dict[str, list[LayerSpec]] = {
 
 SDXL_SWEEP_M = [512, 1024, 2048, 4096, 8192, 16384, 32768, 65536]
 
+# the skip-concat layer at every row count of the sweep (the points of its roofline curve)
+WORKLOADS["sdxl_sweep"] = [
+    _spec(f"skip_conv1x1_M{m}", m, 1280, 640, P=2, dual=True, code="int8", x_dtype="bf16",
+          x_kind="normal+silu", w_kind="plain", seed=4000, x_seg_std=[1.0, 8.0])
+    for m in SDXL_SWEEP_M
+]
+
 
 def small_variant(spec: LayerSpec, M: int, K: int | None = None, N: int | None = None) -> LayerSpec:
     """A reduced copy of a layer (same recipe, segment counts and seed) that the CPU oracle
