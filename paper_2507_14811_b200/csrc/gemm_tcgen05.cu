@@ -301,6 +301,57 @@ struct SharedHeader {
 // where-codes written to the status word when a wait expires
 enum : uint32_t { kWhereProducer = 0x100, kWhereMmaFull = 0x200, kWhereMmaTmem = 0x300, kWhereEpilogue = 0x400 };
 
+// A whole K-block (four K-steps of 32 codes, each against every activation tile) issued from one block
+// of PTX.  The issuing thread is the only one feeding the tensor pipe, so its instruction count per
+// MMA matters when MMAs are short (narrow tiles): descriptors differ only in the 14-bit address field
+// of their low word, so each one costs a 32-bit add with an immediate; the accumulate predicate is set
+// once.  %0 TMEM address, %1 / %2 low words of the A / B descriptors of the stage, %3 their common high
+// word, %4 instruction descriptor, %5 accumulate flag of the first K-step, %6 TILE_N (second
+// polarity's accumulator).  Offsets: +2 per K-step (32 bytes >> 4), +1024 to the second activation tile.
+#define SQ_KBLOCK_1(OP)                                                                                   \
+    "{\n\t.reg .pred pf, pt;\n\t.reg .b64 da, db;\n\t.reg .b32 la, lb;\n\t"                              \
+    "setp.ne.b32 pf, %5, 0;\n\tsetp.eq.b32 pt, %5, %5;\n\t"                                               \
+    "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t" OP " [%0], da, db, %4, pf;\n\t"                  \
+    "add.u32 la, %1, 2;\n\tadd.u32 lb, %2, 2;\n\tmov.b64 da, {la, %3};\n\tmov.b64 db, {lb, %3};\n\t"      \
+    OP " [%0], da, db, %4, pt;\n\t"                                                                       \
+    "add.u32 la, %1, 4;\n\tadd.u32 lb, %2, 4;\n\tmov.b64 da, {la, %3};\n\tmov.b64 db, {lb, %3};\n\t"      \
+    OP " [%0], da, db, %4, pt;\n\t"                                                                       \
+    "add.u32 la, %1, 6;\n\tadd.u32 lb, %2, 6;\n\tmov.b64 da, {la, %3};\n\tmov.b64 db, {lb, %3};\n\t"      \
+    OP " [%0], da, db, %4, pt;\n\t}"
+#define SQ_KBLOCK_2(OP)                                                                                   \
+    "{\n\t.reg .pred pf, pt;\n\t.reg .b64 da, db;\n\t.reg .b32 la, lb, td;\n\t"                          \
+    "setp.ne.b32 pf, %5, 0;\n\tsetp.eq.b32 pt, %5, %5;\n\tadd.u32 td, %0, %6;\n\t"                        \
+    "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t" OP " [%0], da, db, %4, pf;\n\t"                  \
+    "add.u32 la, %1, 1024;\n\tmov.b64 da, {la, %3};\n\t" OP " [td], da, db, %4, pf;\n\t"                  \
+    "add.u32 la, %1, 2;\n\tadd.u32 lb, %2, 2;\n\tmov.b64 da, {la, %3};\n\tmov.b64 db, {lb, %3};\n\t"      \
+    OP " [%0], da, db, %4, pt;\n\t"                                                                       \
+    "add.u32 la, %1, 1026;\n\tmov.b64 da, {la, %3};\n\t" OP " [td], da, db, %4, pt;\n\t"                  \
+    "add.u32 la, %1, 4;\n\tadd.u32 lb, %2, 4;\n\tmov.b64 da, {la, %3};\n\tmov.b64 db, {lb, %3};\n\t"      \
+    OP " [%0], da, db, %4, pt;\n\t"                                                                       \
+    "add.u32 la, %1, 1028;\n\tmov.b64 da, {la, %3};\n\t" OP " [td], da, db, %4, pt;\n\t"                  \
+    "add.u32 la, %1, 6;\n\tadd.u32 lb, %2, 6;\n\tmov.b64 da, {la, %3};\n\tmov.b64 db, {lb, %3};\n\t"      \
+    OP " [%0], da, db, %4, pt;\n\t"                                                                       \
+    "add.u32 la, %1, 1030;\n\tmov.b64 da, {la, %3};\n\t" OP " [td], da, db, %4, pt;\n\t}"
+#define SQ_KBLOCK_ARGS ::"r"(d0), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate), "n"(TILE_N) : "memory"
+
+template <int KIND, int NPOL, int TILE_N, int CG>
+__device__ __forceinline__ void issue_full_kblock(uint32_t d0, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                                  uint32_t accumulate)
+{
+    static_assert(BLOCK_K / MMA_K == 4 && ((TILE_M * BLOCK_K) >> 4) == 1024, "offsets are written into the PTX");
+    if (NPOL == 1) {
+        if (KIND == 0 && CG == 1) asm volatile(SQ_KBLOCK_1("tcgen05.mma.cta_group::1.kind::i8") SQ_KBLOCK_ARGS);
+        else if (KIND == 0) asm volatile(SQ_KBLOCK_1("tcgen05.mma.cta_group::2.kind::i8") SQ_KBLOCK_ARGS);
+        else if (CG == 1) asm volatile(SQ_KBLOCK_1("tcgen05.mma.cta_group::1.kind::f8f6f4") SQ_KBLOCK_ARGS);
+        else asm volatile(SQ_KBLOCK_1("tcgen05.mma.cta_group::2.kind::f8f6f4") SQ_KBLOCK_ARGS);
+    } else {
+        if (KIND == 0 && CG == 1) asm volatile(SQ_KBLOCK_2("tcgen05.mma.cta_group::1.kind::i8") SQ_KBLOCK_ARGS);
+        else if (KIND == 0) asm volatile(SQ_KBLOCK_2("tcgen05.mma.cta_group::2.kind::i8") SQ_KBLOCK_ARGS);
+        else if (CG == 1) asm volatile(SQ_KBLOCK_2("tcgen05.mma.cta_group::1.kind::f8f6f4") SQ_KBLOCK_ARGS);
+        else asm volatile(SQ_KBLOCK_2("tcgen05.mma.cta_group::2.kind::f8f6f4") SQ_KBLOCK_ARGS);
+    }
+}
+
 // One K-block worth of MMAs: nk K-steps of 32 codes, each against every activation tile.
 template <int KIND, int NPOL, int TILE_N, int CG>
 __device__ __forceinline__ void issue_kblock(uint32_t d0, uint64_t da, uint64_t db, uint32_t idesc, int nk,
@@ -308,14 +359,7 @@ __device__ __forceinline__ void issue_kblock(uint32_t d0, uint64_t da, uint64_t 
 {
     constexpr uint64_t kATileDesc = uint64_t(TILE_M * BLOCK_K) >> 4;   // next activation tile in the stage
     if (nk == BLOCK_K / MMA_K) {
-#pragma unroll
-        for (int kk = 0; kk < BLOCK_K / MMA_K; kk++) {
-            const uint64_t koff = uint64_t((kk * MMA_K) >> 4);           // +32 B inside the swizzle row
-#pragma unroll
-            for (int pol = 0; pol < NPOL; pol++)
-                tc_mma<KIND, CG>(d0 + pol * TILE_N, da + pol * kATileDesc + koff, db + koff, idesc,
-                                 kk == 0 ? accumulate : 1u);
-        }
+        issue_full_kblock<KIND, NPOL, TILE_N, CG>(d0, uint32_t(da), uint32_t(db), uint32_t(da >> 32), idesc, accumulate);
     } else {
         for (int kk = 0; kk < nk; kk++) {
             const uint64_t koff = uint64_t((kk * MMA_K) >> 4);
