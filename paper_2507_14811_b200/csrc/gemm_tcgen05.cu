@@ -402,6 +402,11 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     const int num_tiles = prm.num_m_tiles * prm.num_n_tiles;
     volatile uint32_t *abort_flag = &hdr->abort_flag;
 
+    if (threadIdx.x == 32 * 0 + 1) {     // descriptor fetches overlap the set-up below
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_a_pos)) : "memory");
+        if (NPOL == 2) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_a_neg)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_b)) : "memory");
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < prm.stages; s++) {
             mbar_init(smem_u32(&hdr->full[s]), 1);
@@ -414,15 +419,6 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
         hdr->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    if (!GENERIC) {
-        // dequantization factors c[a][q] = s_act[p][pol] * s_w[p][q], a = p * NPOL + pol (one fp32 multiply)
-        for (int i = threadIdx.x; i < prm.nacc * prm.sb.Q; i += kThreads) {
-            const int a = i / prm.sb.Q, q = i - a * prm.sb.Q, p = a / NPOL;
-            const float s_act = (NPOL == 2 && (a & 1)) ? prm.s_neg[p] : prm.s_pos[p];
-            sh_tab[i] = s_act * prm.s_w[p * prm.sb.Q + q];
-        }
-        for (int i = threadIdx.x; i <= prm.sb.Q; i += kThreads) sh_nb[i] = prm.sb.nb[i];
     }
     if (warp == 1) {
         if (CG == 1) {
@@ -447,9 +443,6 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_a_pos)) : "memory");
-            if (NPOL == 2) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_a_neg)) : "memory");
-            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_b)) : "memory");
             const uint32_t stages = prm.stages, P = prm.sb.P;
             const uint32_t full0 = smem_u32(&hdr->full[0]), empty0 = smem_u32(&hdr->empty[0]);
             // completion bytes of both CTAs' loads are counted on the leader's barrier
@@ -555,6 +548,14 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                 return n < prm.N ? __ldg(prm.bias + n) : 0.0f;
             };
             float bias_next = fetch_bias(unit);
+            // dequantization factors c[a][q] = s_act[p][pol] * s_w[p][q], a = p * NPOL + pol (one fp32 multiply);
+            // built here, off the producer's and the MMA issuer's path, and published by the first tile's barrier
+            for (int i = et; i < nacc * Q; i += kEpiThreads) {
+                const int a = i / Q, q = i - a * Q, p = a / NPOL;
+                const float s_act = (NPOL == 2 && (a & 1)) ? prm.s_neg[p] : prm.s_pos[p];
+                sh_tab[i] = s_act * prm.s_w[p * Q + q];
+            }
+            for (int i = et; i <= Q; i += kEpiThreads) sh_nb[i] = prm.sb.nb[i];
             uint32_t as = 0, aph = 0;
             bool ok = true;
             for (int tile = unit; tile < num_tiles; tile += num_units) {
