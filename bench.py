@@ -449,14 +449,15 @@ def main():
     ap.add_argument("--tile-n", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--cta-group", type=int, default=0)
+    ap.add_argument("--segment-mode", type=int, default=0)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         out = run_reference(args)
     else:
-        if args.tile_n or args.stages or args.cta_group:
+        if args.tile_n or args.stages or args.cta_group or args.segment_mode:
             from paper_2507_14811_b200 import binding as B
-            B.segquant_set_tuning(args.tile_n, args.stages, args.cta_group)
+            B.segquant_set_tuning(args.tile_n, args.stages, args.cta_group, args.segment_mode)
         out = run_ours(args)
     if out is not None:
         print(json.dumps(out))

@@ -51,7 +51,7 @@ typedef enum { SQ_F32 = 0, SQ_BF16 = 1 } sq_dtype;             /* real-valued el
 #define SQ_FLAG_QMIN_SYM 1u  /* int8 DualScale: clamp the negative path to -127 instead of -128 */
 
 /* limits */
-#define SQ_MAX_P 16   /* K-segments per layer */
+#define SQ_MAX_P 64   /* K-segments per layer */
 #define SQ_MAX_Q 64   /* N-segments per layer */
 
 /* Segment table (the output of the paper's graph pattern detection, App. B Alg. 1):
@@ -139,7 +139,8 @@ sq_status segquant_quantize_weight(const void *W, sq_dtype dt, int64_t N, int64_
  *   accumulators (used by parity tests).
  *   Alignment: Xq, Wq, Y 16 bytes; ldx, ldw multiples of 16; ldy*sizeof(y_dtype) a multiple of 16;
  *   N a multiple of 8; interior K-segment bounds multiples of 32, K a multiple of 16.
- *   Limits: P <= SQ_MAX_P, Q <= SQ_MAX_Q, K <= 131072 (int8: |acc| stays below 2^31).
+ *   Limits: P <= SQ_MAX_P, Q <= SQ_MAX_Q, P * Q <= 2048 (1024 for the dual entry point), K <= 131072
+ *   (int8: |acc| stays below 2^31).
  *   The epilogue multiplies c = s_x*s_w in fp32 and accumulates with fp32 FMAs in ascending p. */
 sq_status segquant_seglinear_gemm(const void *Xq, int64_t ldx, const void *Wq, int64_t ldw,
                                   int64_t M, int64_t N, int64_t K, const sq_segtable *seg, sq_code code,
@@ -151,7 +152,8 @@ sq_status segquant_seglinear_gemm(const void *Xq, int64_t ldx, const void *Wq, i
  *   y[m][n] = sum_p ( s_pos[p]*s_w[p*Q+q(n)]*acc_pos[p][m][n] + s_neg[p]*s_w[p*Q+q(n)]*acc_neg[p][m][n] ) + bias[n]
  *   where acc_pos / acc_neg are the contractions of Xq_pos / Xq_neg with the SAME weight tile.
  *   acc_dump (optional): [P][2][M][N], polarity 0 = positive path.
- *   A layer needs P*2 accumulators of the tile width in tensor memory: P <= 8 here. */
+ *   Layers with several K-segments pass them through tensor memory one after the other and keep fp32
+ *   running sums in registers, so P is only bounded by SQ_MAX_P. */
 sq_status segquant_dualscale_gemm(const void *Xq_pos, const void *Xq_neg, int64_t ldx,
                                   const void *Wq, int64_t ldw, int64_t M, int64_t N, int64_t K,
                                   const sq_segtable *seg, sq_code code,
@@ -183,9 +185,12 @@ sq_status segquant_last_device_status(void *workspace, void *stream, uint32_t *d
 
 /* Tile plan of the GEMM kernel: tile_n in {0 (automatic), 32, 64, 128, 256}; stages 0 (automatic) or
  * 2..8 (shared-memory ring depth); cta_group 0 (automatic: CTA pairs on 256-row tiles when M > 128),
- * 1 (one CTA per 128-row tile) or 2.  Process-wide; meant for benchmarking sweeps and tests.  Values
- * the layer cannot use are replaced by the automatic choice. */
-sq_status segquant_set_tuning(int tile_n, int stages, int cta_group);
+ * 1 (one CTA per 128-row tile) or 2; segment_mode for layers with several K-segments: 0 (automatic:
+ * segments pass through tensor memory one after the other, running sums in registers), 1 (all
+ * accumulators of a tile resident in tensor memory; at most 16 of them) or 2 (sequential).
+ * Process-wide; meant for benchmarking sweeps and tests.  Values the layer cannot use are replaced by
+ * the automatic choice. */
+sq_status segquant_set_tuning(int tile_n, int stages, int cta_group, int segment_mode);
 
 /* Number of kernels the library has launched in this process (all entry points). */
 uint64_t segquant_launch_count(void);

@@ -253,8 +253,9 @@ def check_device_status(workspace):
         raise SegquantError(st, f"device status (detail 0x{detail:x})")
 
 
-def segquant_set_tuning(tile_n: int = 0, stages: int = 0, cta_group: int = 0):
-    _check(lib().segquant_set_tuning(C.c_int(tile_n), C.c_int(stages), C.c_int(cta_group)), "segquant_set_tuning")
+def segquant_set_tuning(tile_n: int = 0, stages: int = 0, cta_group: int = 0, segment_mode: int = 0):
+    _check(lib().segquant_set_tuning(C.c_int(tile_n), C.c_int(stages), C.c_int(cta_group), C.c_int(segment_mode)),
+           "segquant_set_tuning")
 
 
 def segquant_launch_count() -> int:

@@ -70,7 +70,7 @@ static sq_status gemm_common(const void *a_pos, const void *a_neg, int dual, int
     if (hs.status != SQ_OK) return hs.status;
     for (int p = 1; p < hs.b.P; p++)
         if (hs.b.kb[p] % 32 != 0) return SQ_ERR_ALIGN;
-    if (hs.b.P * (dual ? 2 : 1) > 16) return SQ_ERR_UNSUPPORTED;   // accumulators of >= 32 columns in 512
+    if (hs.b.P * (dual ? 2 : 1) * hs.b.Q > 2048) return SQ_ERR_UNSUPPORTED;   // dequantization factors kept in shared memory
     if ((st = check_ws(workspace, ws_bytes)) != SQ_OK) return st;
 
     GemmArgs g{};
@@ -235,9 +235,9 @@ sq_status segquant_last_device_status(void *workspace, void *stream, uint32_t *d
     return SQ_ERR_TIMEOUT;
 }
 
-sq_status segquant_set_tuning(int tile_n, int stages, int cta_group)
+sq_status segquant_set_tuning(int tile_n, int stages, int cta_group, int segment_mode)
 {
-    set_gemm_tuning(tile_n, stages, cta_group);
+    set_gemm_tuning(tile_n, stages, cta_group, segment_mode);
     return SQ_OK;
 }
 

@@ -37,6 +37,7 @@ constexpr int kMaxStages = 8;
 constexpr int kTmemCols = 512;
 constexpr uint32_t kSmemBudget = 227 * 1024;
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s
+constexpr int kMaxFactorTable = 2048;                  // (K-segments x polarities) x N-segments factors in shared memory
 
 struct KernelParams {
     int M, N, K;
@@ -376,7 +377,13 @@ __device__ __forceinline__ void issue_kblock(uint32_t d0, uint64_t da, uint64_t 
 // dequantization factor per accumulator).  Its epilogue loop is small enough for the instruction
 // cache and runs its FMAs on packed fp32 pairs.  GENERIC = true handles everything else (fp32 output,
 // accumulator dump, arbitrary N-bounds) with a per-column factor table rebuilt for every tile.
-template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC>
+// SEQ = true (layers with more than one K-segment): TMEM holds the accumulators of ONE K-segment at a time,
+// in two alternating sets.  The MMA issuer fills a set with segment p while the epilogue warps drain the set
+// of segment p - 1, scale it and add it to fp32 running sums kept in registers for the whole tile; the sums
+// are converted and stored after the last segment.  Any number of K-segments fits, tiles stay wide, and the
+// drain of every segment but the last overlaps tensor work.  SEQ = false keeps every (segment, polarity)
+// accumulator of a tile resident in TMEM and drains once per tile.
+template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ>
 __global__ void __launch_bounds__(kThreads, 1)
 segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_constant__ CUtensorMap tm_a_neg,
                      const __grid_constant__ CUtensorMap tm_b, const KernelParams prm)
@@ -388,12 +395,13 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     constexpr uint32_t b_bytes = B_ROWS * BLOCK_K;
     constexpr uint32_t stage_bytes = NPOL * a_bytes + b_bytes;
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    float *sh_scale = reinterpret_cast<float *>(smem + size_t(prm.stages) * stage_bytes);   // GENERIC: [nacc][TILE_N]
-    float *sh_bias = sh_scale + (GENERIC ? prm.nacc * TILE_N : 0);                          // [TILE_N], per tile
-    float *sh_tab = sh_bias + TILE_N;                                                       // !GENERIC: [nacc][Q]
-    int *sh_nb = reinterpret_cast<int *>(sh_tab + (GENERIC ? 0 : prm.nacc * prm.sb.Q));     // !GENERIC: [Q + 1]
+    constexpr bool kColTable = GENERIC && !SEQ;          // per-column factor table rebuilt per tile
+    float *sh_scale = reinterpret_cast<float *>(smem + size_t(prm.stages) * stage_bytes);   // kColTable: [nacc][TILE_N]
+    float *sh_bias = sh_scale + (kColTable ? prm.nacc * TILE_N : 0);                        // [TILE_N], per tile
+    float *sh_tab = sh_bias + TILE_N;                                                       // !kColTable: [nacc][Q]
+    int *sh_nb = reinterpret_cast<int *>(sh_tab + (kColTable ? 0 : prm.nacc * prm.sb.Q));   // !kColTable: [Q + 1]
     SharedHeader *hdr = reinterpret_cast<SharedHeader *>(
-        reinterpret_cast<uint8_t *>(smem + size_t(prm.stages) * stage_bytes) + epi_table_bytes<GENERIC>(prm.nacc, prm.sb.Q, TILE_N));
+        reinterpret_cast<uint8_t *>(smem + size_t(prm.stages) * stage_bytes) + epi_table_bytes<kColTable>(prm.nacc, prm.sb.Q, TILE_N));
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -436,7 +444,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     if (CG == 2) cluster_sync_all();          // the peer's barriers are initialised before anyone signals them
     tc_fence_after();
     const uint32_t tmem_base = hdr->tmem_base;
-    const int acc_cols = prm.nacc * TILE_N;     // TMEM columns of one accumulator set
+    const int acc_cols = (SEQ ? NPOL : prm.nacc) * TILE_N;     // TMEM columns of one accumulator set
 
     // The producer and the MMA issuer are single threads: their loops are kept to a few dozen
     // instructions per K-block (ring slot and phase advance incrementally, descriptors by addition).
@@ -494,13 +502,22 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
             uint32_t s = 0, ph = 0, as = 0, aph = 0;
             bool ok = true;
             for (int tile = unit; tile < num_tiles && ok; tile += num_units) {
-                if (!mbar_wait(smem_u32(&hdr->tmem_empty[as]), aph ^ 1, abort_flag, prm.status, kWhereMmaTmem)) {
-                    ok = false;
-                    break;
+                if (!SEQ) {
+                    if (!mbar_wait(smem_u32(&hdr->tmem_empty[as]), aph ^ 1, abort_flag, prm.status, kWhereMmaTmem)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
                 }
-                tc_fence_after();
                 for (uint32_t p = 0; p < P && ok; p++) {
-                    const uint32_t d0 = tmem_base + as * acc_cols + p * (NPOL * TILE_N);
+                    if (SEQ) {                                     // one accumulator set per K-segment
+                        if (!mbar_wait(smem_u32(&hdr->tmem_empty[as]), aph ^ 1, abort_flag, prm.status, kWhereMmaTmem)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                    }
+                    const uint32_t d0 = tmem_base + as * acc_cols + (SEQ ? 0u : p * (NPOL * TILE_N));
                     const int k_end = prm.sb.kb[p + 1];
                     uint32_t accumulate = 0;
                     for (int k = prm.sb.kb[p]; k < k_end; k += BLOCK_K) {
@@ -517,16 +534,189 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                         tc_commit<CG>(empty0 + 8 * s);             // frees the ring slot when these MMAs retire
                         if (++s == stages) { s = 0; ph ^= 1; }
                     }
+                    if (SEQ) {
+                        if (ok) tc_commit<CG>(smem_u32(&hdr->tmem_full[as]));  // accumulators of this segment complete
+                        if (++as == acc_stages) { as = 0; aph ^= 1; }
+                    }
                 }
-                if (ok) tc_commit<CG>(smem_u32(&hdr->tmem_full[as]));  // accumulators of this tile complete
-                if (++as == acc_stages) { as = 0; aph ^= 1; }
+                if (!SEQ) {
+                    if (ok) tc_commit<CG>(smem_u32(&hdr->tmem_full[as]));  // accumulators of this tile complete
+                    if (++as == acc_stages) { as = 0; aph ^= 1; }
+                }
             }
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
         // Warp w may read TMEM lanes 32 * (w % 4) .. + 31; the two warps of one lane group take one half
         // of the tile's 32-column slabs each.
-        if constexpr (!GENERIC) {
+        if constexpr (SEQ) {
+            const int et = threadIdx.x - 64;
+            const int ew = warp - 2;
+            const int lane_grp = warp & 3;
+            constexpr int kSlabsPerWarp = TILE_N / 32 / (kEpiWarps / 4);
+            static_assert(kSlabsPerWarp >= 1 && kSlabsPerWarp * (kEpiWarps / 4) * 32 == TILE_N, "SEQ needs TILE_N >= 64");
+            constexpr int kUnits = kSlabsPerWarp * NPOL;                // TMEM loads per segment and warp
+            const int slab0 = (ew >> 2) * kSlabsPerWarp;
+            const int P = prm.sb.P, Q = prm.sb.Q;
+            const uint32_t tmem_empty_sig0 = CG == 2 ? map_to_cta(smem_u32(&hdr->tmem_empty[0]), 0)
+                                                     : smem_u32(&hdr->tmem_empty[0]);
+            const uint32_t tab_addr = smem_u32(sh_tab), nb_addr = smem_u32(sh_nb), bias_addr = smem_u32(sh_bias);
+            auto fetch_bias = [&](int tile) -> float {
+                if (tile >= num_tiles || et >= TILE_N || !prm.bias) return 0.0f;
+                const int n = (tile % prm.num_n_tiles) * TILE_N + et;
+                return n < prm.N ? __ldg(prm.bias + n) : 0.0f;
+            };
+            auto seg_of = [&](int n) {                                  // interior N-bounds <= n, counted warp-wide
+                int cnt = 0;
+                for (int base = 1; base < Q; base += 32) {
+                    const int i = base + lane;
+                    const bool le = i < Q && n >= int(ld_shared_u32(nb_addr + 4u * uint32_t(i < Q ? i : 0)));
+                    cnt += __popc(__ballot_sync(0xFFFFFFFFu, le));
+                }
+                return cnt;
+            };
+            float bias_next = fetch_bias(unit);
+            for (int i = et; i < prm.nacc * Q; i += kEpiThreads) {      // factors c[a][q], a = p * NPOL + pol
+                const int a = i / Q, q = i - a * Q, p = a / NPOL;
+                const float s_act = (NPOL == 2 && (a & 1)) ? prm.s_neg[p] : prm.s_pos[p];
+                sh_tab[i] = s_act * prm.s_w[p * Q + q];
+            }
+            for (int i = et; i <= Q; i += kEpiThreads) sh_nb[i] = prm.sb.nb[i];
+            uint32_t as = 0, aph = 0;
+            bool ok = true;
+            for (int tile = unit; tile < num_tiles; tile += num_units) {
+                const int m0 = (tile / prm.num_n_tiles) * (TILE_M * CG) + int(rank) * TILE_M;
+                const int n0 = (tile % prm.num_n_tiles) * TILE_N;
+
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // previous tile's readers are done
+                if (et < TILE_N) sh_bias[et] = bias_next;
+                bias_next = fetch_bias(tile + num_units);
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+
+                const int row = m0 + lane_grp * 32 + lane;
+                // running sums of this thread's outputs (row `row`, kSlabsPerWarp slabs of 32 columns), start = bias
+                uint64_t y2[kSlabsPerWarp][16];
+                int q_lo[kSlabsPerWarp], q_hi[kSlabsPerWarp];
+#pragma unroll
+                for (int sl = 0; sl < kSlabsPerWarp; sl++) {
+                    const int c0 = (slab0 + sl) * 32;
+                    q_lo[sl] = seg_of(n0 + c0);
+                    q_hi[sl] = GENERIC ? seg_of(min(n0 + c0 + 31, prm.N - 1)) : q_lo[sl];
+#pragma unroll
+                    for (int j4 = 0; j4 < 8; j4++)
+                        ld_shared_2x64(bias_addr + uint32_t(c0 + 4 * j4) * 4u, y2[sl][2 * j4], y2[sl][2 * j4 + 1]);
+                }
+
+                for (int p = 0; p < P; p++) {
+                    const uint32_t cur_as = as, cur_aph = aph;
+                    if (++as == 2u) { as = 0; aph ^= 1; }
+                    if (ok) ok = mbar_wait(smem_u32(&hdr->tmem_full[cur_as]), cur_aph, abort_flag, prm.status, kWhereEpilogue);
+                    if (!ok) continue;
+                    tc_fence_after();
+                    const uint32_t t_row = tmem_base + (uint32_t(lane_grp * 32) << 16) + cur_as * acc_cols;
+                    // With two slabs of running sums per thread there are registers for a second load buffer, and
+                    // unit u + 1 is read while unit u is added; with four slabs the loads are taken one at a time.
+                    constexpr bool kAhead = kSlabsPerWarp <= 2;
+                    uint32_t ra[32], rb[kAhead ? 32 : 1];
+                    tc_ld32(t_row + uint32_t(slab0 * 32), ra);                       // unit 0 = (slab 0, polarity 0)
+#pragma unroll
+                    for (int u = 0; u < kUnits; u++) {
+                        const int sl = u / NPOL, pol = u % NPOL;
+                        uint32_t (&r)[32] = (kAhead && (u & 1)) ? reinterpret_cast<uint32_t (&)[32]>(rb) : ra;
+                        tc_wait_ld();
+                        if (kAhead && u + 1 < kUnits) {
+                            tc_ld32(t_row + uint32_t(((u + 1) % NPOL) * TILE_N + (slab0 + (u + 1) / NPOL) * 32),
+                                    (u & 1) ? ra : reinterpret_cast<uint32_t (&)[32]>(rb));
+                        } else if (u + 1 == kUnits) {                                // set read: hand it back
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) {
+                                if (CG == 2) mbar_arrive_cluster(tmem_empty_sig0 + 8 * cur_as);
+                                else mbar_arrive(tmem_empty_sig0 + 8 * cur_as);
+                            }
+                        }
+                        const int a = p * NPOL + pol;
+                        const int nf = n0 + (slab0 + sl) * 32;
+                        if (!GENERIC || q_lo[sl] == q_hi[sl]) {                      // slab inside one N-segment
+                            const float c = ld_shared_f32(tab_addr + uint32_t(a * Q + q_lo[sl]) * 4u);
+                            const uint64_t c2 = pack_f32x2(c, c);
+#pragma unroll
+                            for (int j = 0; j < 16; j++) {
+                                const uint64_t v2 = KIND == 0 ? pack_f32x2(__int2float_rn(int(r[2 * j])), __int2float_rn(int(r[2 * j + 1])))
+                                                              : pack_b32x2(r[2 * j], r[2 * j + 1]);
+                                y2[sl][j] = fma_f32x2(c2, v2, y2[sl][j]);
+                            }
+                        } else {
+                            int q = q_lo[sl];
+#pragma unroll
+                            for (int j = 0; j < 16; j++) {
+                                float cc[2];
+#pragma unroll
+                                for (int t = 0; t < 2; t++) {
+                                    while (q < q_hi[sl] && nf + 2 * j + t >= int(ld_shared_u32(nb_addr + 4u * uint32_t(q + 1)))) q++;
+                                    cc[t] = ld_shared_f32(tab_addr + uint32_t(a * Q + q) * 4u);
+                                }
+                                const uint64_t v2 = KIND == 0 ? pack_f32x2(__int2float_rn(int(r[2 * j])), __int2float_rn(int(r[2 * j + 1])))
+                                                              : pack_b32x2(r[2 * j], r[2 * j + 1]);
+                                y2[sl][j] = fma_f32x2(pack_f32x2(cc[0], cc[1]), v2, y2[sl][j]);
+                            }
+                        }
+                        if (GENERIC && prm.acc_dump && row < prm.M) {
+                            uint32_t *dump = static_cast<uint32_t *>(prm.acc_dump) + (size_t(a) * prm.M + row) * size_t(prm.N) + nf;
+#pragma unroll
+                            for (int j = 0; j < 32; j++)
+                                if (nf + j < prm.N) dump[j] = r[j];
+                        }
+                        if (!kAhead && u + 1 < kUnits)
+                            tc_ld32(t_row + uint32_t(((u + 1) % NPOL) * TILE_N + (slab0 + (u + 1) / NPOL) * 32), ra);
+                    }
+                }
+                if (!ok) continue;
+                // all segments added: convert and store this thread's outputs, 16-byte chunks of 8 bf16 / 4 fp32
+                if (row < prm.M) {
+#pragma unroll
+                    for (int sl = 0; sl < kSlabsPerWarp; sl++) {
+                        const int nf = n0 + (slab0 + sl) * 32;
+                        const int nvalid = prm.N - nf;
+                        if (GENERIC && prm.y_is_f32) {
+                            float *dst = static_cast<float *>(prm.Y) + size_t(row) * prm.ldy + nf;
+#pragma unroll
+                            for (int c = 0; c < 4; c++) {
+                                if (8 * c < nvalid) {
+                                    const uint4 lo = make_uint4(uint32_t(y2[sl][4 * c]), uint32_t(y2[sl][4 * c] >> 32),
+                                                                uint32_t(y2[sl][4 * c + 1]), uint32_t(y2[sl][4 * c + 1] >> 32));
+                                    const uint4 hi = make_uint4(uint32_t(y2[sl][4 * c + 2]), uint32_t(y2[sl][4 * c + 2] >> 32),
+                                                                uint32_t(y2[sl][4 * c + 3]), uint32_t(y2[sl][4 * c + 3] >> 32));
+                                    if (prm.y_wide) st_global_32(dst + 8 * c, lo, hi);
+                                    else { st_global_16(dst + 8 * c, lo); st_global_16(dst + 8 * c + 4, hi); }
+                                }
+                            }
+                        } else {
+                            __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(prm.Y) + size_t(row) * prm.ldy + nf;
+                            uint32_t h[16];
+#pragma unroll
+                            for (int j = 0; j < 16; j++) {
+                                float lo, hi;
+                                unpack_f32x2(y2[sl][j], lo, hi);
+                                __nv_bfloat162 v2 = __floats2bfloat162_rn(lo, hi);
+                                h[j] = *reinterpret_cast<uint32_t *>(&v2);
+                            }
+#pragma unroll
+                            for (int cidx = 0; cidx < 2; cidx++) {
+                                const uint4 w0 = make_uint4(h[8 * cidx], h[8 * cidx + 1], h[8 * cidx + 2], h[8 * cidx + 3]);
+                                const uint4 w1 = make_uint4(h[8 * cidx + 4], h[8 * cidx + 5], h[8 * cidx + 6], h[8 * cidx + 7]);
+                                if (16 * cidx + 8 < nvalid && prm.y_wide) {
+                                    st_global_32(dst + 16 * cidx, w0, w1);
+                                } else {
+                                    if (16 * cidx < nvalid) st_global_16(dst + 16 * cidx, w0);
+                                    if (16 * cidx + 8 < nvalid) st_global_16(dst + 16 * cidx + 8, w1);
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+        } else if constexpr (!GENERIC) {
             const int et = threadIdx.x - 64;
             const int ew = warp - 2;
             const int lane_grp = warp & 3;
@@ -877,9 +1067,9 @@ bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, in
     return r == CUDA_SUCCESS;
 }
 
-int g_tune_tile_n = 0, g_tune_stages = 0, g_tune_cta_group = 0;
+int g_tune_tile_n = 0, g_tune_stages = 0, g_tune_cta_group = 0, g_tune_seq = 0;
 
-template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC>
+template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ>
 sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cudaStream_t st)
 {
     constexpr int B_ROWS = TILE_N / CG;
@@ -889,7 +1079,7 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
     if (!make_map(&tb, g.b, g.N, g.K, g.ldb, B_ROWS)) return SQ_ERR_CUDA;
 
     const uint32_t stage_bytes = NPOL * TILE_M * BLOCK_K + B_ROWS * BLOCK_K;
-    const uint32_t tail = epi_table_bytes<GENERIC>(prm.nacc, prm.sb.Q, TILE_N) + sizeof(SharedHeader);
+    const uint32_t tail = epi_table_bytes<GENERIC && !SEQ>(prm.nacc, prm.sb.Q, TILE_N) + sizeof(SharedHeader);
     int stages = int((kSmemBudget - 1024 - tail) / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (g_tune_stages >= 2 && g_tune_stages < stages) stages = g_tune_stages;
@@ -899,7 +1089,7 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
     prm.num_n_tiles = int((g.N + TILE_N - 1) / TILE_N);
     const size_t smem = 1024 + size_t(stages) * stage_bytes + tail;
 
-    auto kern = segquant_gemm_kernel<KIND, NPOL, TILE_N, CG, GENERIC>;
+    auto kern = segquant_gemm_kernel<KIND, NPOL, TILE_N, CG, GENERIC, SEQ>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
         return SQ_ERR_CUDA;
     const int tiles = prm.num_m_tiles * prm.num_n_tiles;
@@ -938,41 +1128,47 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
 }
 
 template <int KIND, int NPOL, int CG>
-sq_status launch_tile(const GemmArgs &g, KernelParams &prm, int tile_n, int sm_count, cudaStream_t st)
+sq_status launch_tile(const GemmArgs &g, KernelParams &prm, int tile_n, bool seq, int sm_count, cudaStream_t st)
 {
     bool dbg = prm.y_is_f32 || prm.acc_dump != nullptr;
     for (int q = 1; q < prm.sb.Q; q++) dbg = dbg || (prm.sb.nb[q] % 32 != 0);
+    if (seq) {      // sequential K-segments: one tile width per polarity count
+        constexpr int TN = NPOL == 1 ? 256 : 128;
+        return dbg ? launch_variant<KIND, NPOL, TN, CG, true, true>(g, prm, sm_count, st)
+                   : launch_variant<KIND, NPOL, TN, CG, false, true>(g, prm, sm_count, st);
+    }
     switch (tile_n) {
-        case 256: return dbg ? launch_variant<KIND, NPOL, 256, CG, true>(g, prm, sm_count, st)
-                             : launch_variant<KIND, NPOL, 256, CG, false>(g, prm, sm_count, st);
-        case 128: return dbg ? launch_variant<KIND, NPOL, 128, CG, true>(g, prm, sm_count, st)
-                             : launch_variant<KIND, NPOL, 128, CG, false>(g, prm, sm_count, st);
-        case 64: return dbg ? launch_variant<KIND, NPOL, 64, CG, true>(g, prm, sm_count, st)
-                            : launch_variant<KIND, NPOL, 64, CG, false>(g, prm, sm_count, st);
-        case 32: return dbg ? launch_variant<KIND, NPOL, 32, CG, true>(g, prm, sm_count, st)
-                            : launch_variant<KIND, NPOL, 32, CG, false>(g, prm, sm_count, st);
+        case 256: return dbg ? launch_variant<KIND, NPOL, 256, CG, true, false>(g, prm, sm_count, st)
+                             : launch_variant<KIND, NPOL, 256, CG, false, false>(g, prm, sm_count, st);
+        case 128: return dbg ? launch_variant<KIND, NPOL, 128, CG, true, false>(g, prm, sm_count, st)
+                             : launch_variant<KIND, NPOL, 128, CG, false, false>(g, prm, sm_count, st);
+        case 64: return dbg ? launch_variant<KIND, NPOL, 64, CG, true, false>(g, prm, sm_count, st)
+                            : launch_variant<KIND, NPOL, 64, CG, false, false>(g, prm, sm_count, st);
+        case 32: return dbg ? launch_variant<KIND, NPOL, 32, CG, true, false>(g, prm, sm_count, st)
+                            : launch_variant<KIND, NPOL, 32, CG, false, false>(g, prm, sm_count, st);
     }
     return SQ_ERR_UNSUPPORTED;
 }
 
 template <int KIND>
-sq_status launch_kind(const GemmArgs &g, KernelParams &prm, int npol, int cg, int tile_n, int sm_count,
+sq_status launch_kind(const GemmArgs &g, KernelParams &prm, int npol, int cg, int tile_n, bool seq, int sm_count,
                       cudaStream_t st)
 {
     if (npol == 2)
-        return cg == 2 ? launch_tile<KIND, 2, 2>(g, prm, tile_n, sm_count, st)
-                       : launch_tile<KIND, 2, 1>(g, prm, tile_n, sm_count, st);
-    return cg == 2 ? launch_tile<KIND, 1, 2>(g, prm, tile_n, sm_count, st)
-                   : launch_tile<KIND, 1, 1>(g, prm, tile_n, sm_count, st);
+        return cg == 2 ? launch_tile<KIND, 2, 2>(g, prm, tile_n, seq, sm_count, st)
+                       : launch_tile<KIND, 2, 1>(g, prm, tile_n, seq, sm_count, st);
+    return cg == 2 ? launch_tile<KIND, 1, 2>(g, prm, tile_n, seq, sm_count, st)
+                   : launch_tile<KIND, 1, 1>(g, prm, tile_n, seq, sm_count, st);
 }
 
 }  // namespace
 
-void set_gemm_tuning(int tile_n, int stages, int cta_group)
+void set_gemm_tuning(int tile_n, int stages, int cta_group, int segment_mode)
 {
     g_tune_tile_n = tile_n;
     g_tune_stages = stages;
     g_tune_cta_group = cta_group;
+    g_tune_seq = segment_mode;
 }
 
 sq_status launch_gemm(const GemmArgs &g, cudaStream_t st)
@@ -999,6 +1195,18 @@ sq_status launch_gemm(const GemmArgs &g, cudaStream_t st)
     if (g_tune_cta_group == 1 || g_tune_cta_group == 2) cg = g_tune_cta_group;
     if (sm_count < 2) cg = 1;
 
+    // More than one K-segment: segments go through TMEM one after the other (SEQ) unless the caller asks for
+    // all accumulators of a tile to stay resident, which needs 32 columns for each of them.
+    bool seq = g.sb.P > 1;
+    if (g_tune_seq == 1 && prm.nacc * 32 <= kTmemCols) seq = false;
+    if (g_tune_seq == 2) seq = true;
+    if (prm.nacc * g.sb.Q > kMaxFactorTable) return SQ_ERR_UNSUPPORTED;
+    if (seq) {
+        prm.acc_stages = 2;
+        return g.code == SQ_CODE_INT8 ? launch_kind<0>(g, prm, npol, cg, 0, true, sm_count, st)
+                                      : launch_kind<1>(g, prm, npol, cg, 0, true, sm_count, st);
+    }
+
     // Tile width: the widest tile whose accumulators fit the 512 TMEM columns, unless half that width
     // fills the machine so much better that it outweighs the narrower tile's higher operand traffic
     // per MMA (weights 1 : 0.75; a double-buffered accumulator set counts 10 % extra).
@@ -1020,8 +1228,8 @@ sq_status launch_gemm(const GemmArgs &g, cudaStream_t st)
         tile_n = g_tune_tile_n;
     prm.acc_stages = (2 * tile_n * prm.nacc <= kTmemCols) ? 2 : 1;
 
-    return g.code == SQ_CODE_INT8 ? launch_kind<0>(g, prm, npol, cg, tile_n, sm_count, st)
-                                  : launch_kind<1>(g, prm, npol, cg, tile_n, sm_count, st);
+    return g.code == SQ_CODE_INT8 ? launch_kind<0>(g, prm, npol, cg, tile_n, false, sm_count, st)
+                                  : launch_kind<1>(g, prm, npol, cg, tile_n, false, sm_count, st);
 }
 
 }  // namespace sq

@@ -8,10 +8,10 @@ namespace sq {
 
 // Workspace layout (device, 256-byte aligned):
 //   [0,256)        status words: word 0 = first expired wait (0 = none)
-//   [256, 256+32K) calibration partials: 2 ordered-uint words per (p,q) block
+//   [256, 256+32Ki) calibration partials: 2 ordered-uint words per (p,q) block
 constexpr size_t kWsStatusBytes = 256;
-constexpr int kMaxBlocks = SQ_MAX_P * SQ_MAX_Q;               // 1024 (p,q) blocks
-constexpr size_t kWsCalibBytes = size_t(kMaxBlocks) * 2 * 4;  // 8 KiB
+constexpr int kMaxBlocks = SQ_MAX_P * SQ_MAX_Q;               // 4096 (p,q) blocks
+constexpr size_t kWsCalibBytes = size_t(kMaxBlocks) * 2 * 4;  // 32 KiB
 constexpr size_t kWsBytes = kWsStatusBytes + kWsCalibBytes;
 
 // Segment bounds by value in kernel parameters (constant bank).
@@ -70,6 +70,6 @@ struct GemmArgs {
     uint32_t *status;
 };
 sq_status launch_gemm(const GemmArgs &g, cudaStream_t st);
-void set_gemm_tuning(int tile_n, int stages, int cta_group);
+void set_gemm_tuning(int tile_n, int stages, int cta_group, int segment_mode);
 
 }  // namespace sq

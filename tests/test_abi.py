@@ -78,10 +78,11 @@ def test_gemm_argument_validation(L):
     assert gemm(L, K=136, kb=(0, 136), ldx=144, ldw=144) == 4   # K not a multiple of 16
     assert gemm(L, N=68, nb=(0, 68), ldy=72) == 4               # N not a multiple of 8
     assert gemm(L, code=7) == 5                                 # unknown code
-    kb17 = tuple(range(0, 17 * 32 + 1, 32))
-    assert gemm(L, K=17 * 32, kb=kb17, ldx=17 * 32, ldw=17 * 32) == 5      # too many K-segments
-    kb9 = tuple(range(0, 9 * 32 + 1, 32))
-    assert gemm(L, K=9 * 32, kb=kb9, ldx=9 * 32, ldw=9 * 32, dual=True) == 5   # 18 accumulators
+    kb65 = tuple(range(0, 65 * 32 + 1, 32))
+    assert gemm(L, K=65 * 32, kb=kb65, ldx=65 * 32, ldw=65 * 32) == 5      # more K-segments than SQ_MAX_P
+    kb40 = tuple(range(0, 40 * 32 + 1, 32))
+    nb64 = tuple(range(0, 64 * 8 + 1, 8))
+    assert gemm(L, N=512, K=40 * 32, kb=kb40, nb=nb64, ldx=40 * 32, ldw=40 * 32, ldy=512) == 5   # 2560 factors > 2048
     assert gemm(L, ws=0) == 8                                   # workspace
     assert gemm(L, ws_bytes=8) == 8
     assert gemm(L, ws=FAKE + 16) == 4

@@ -22,13 +22,13 @@ def custom_spec(name, M, K, N, kb, nb, dual, code, x_dtype="bf16", x_kind="norma
                         x_kind=x_kind, w_kind=w_kind, seed=seed, cal_rows=cal_rows, x_seg_std=x_seg_std or [])
 
 
-def run_parity(spec, rows=None, flags=0, tile_n=0, cta_group=0):
+def run_parity(spec, rows=None, flags=0, tile_n=0, cta_group=0, segment_mode=0):
     """Full element-by-element parity of one layer.  rows: optional subset of rows the oracle computes."""
     data = WL.make_layer(spec)
     qmin_sym = bool(flags & B.SQ_FLAG_QMIN_SYM)
     s_pos, s_neg, s_w, Wq, (qmax, qmin_abs) = oracle_scales(data, qmin_sym)
 
-    B.segquant_set_tuning(tile_n, 0, cta_group)
+    B.segquant_set_tuning(tile_n, 0, cta_group, segment_mode)
     try:
         layer = SegQuantLinear(data.W, data.bias, spec.kb, spec.nb, spec.dual, spec.code, DEV, flags)
         g_pos, g_neg = layer.calibrate(data.X_cal)
@@ -46,7 +46,7 @@ def run_parity(spec, rows=None, flags=0, tile_n=0, cta_group=0):
         layer.check_status()
         torch.cuda.synchronize()
     finally:
-        B.segquant_set_tuning(0, 0, 0)
+        B.segquant_set_tuning(0, 0, 0, 0)
 
     sel = np.arange(spec.M) if rows is None else np.asarray(rows)
     Xs = to_f32_np(data.X)[sel]
@@ -138,6 +138,31 @@ def test_cta_pair_edges(case, cta_group):
     run_parity(custom_spec(name, M, K, N, kb, nb, dual, code), cta_group=cta_group)
 
 
+@pytest.mark.parametrize("segment_mode", [1, 2])
+@pytest.mark.parametrize("case", [
+    # layers with several K-segments, with all accumulators resident in tensor memory (1) and with the
+    # segments passing through it one after the other (2)
+    ("two_k_dual", 300, 512, 384, [0, 256, 512], [0, 384], True, "int8"),
+    ("three_k_single_uneven", 260, 416, 264, [0, 96, 160, 416], [0, 136, 264], False, "int8"),
+    ("four_k_dual_e4m3", 520, 1024, 256, [0, 256, 512, 768, 1024], [0, 128, 256], True, "e4m3"),
+    ("eight_k_single_one_row_tile", 100, 1024, 520, list(range(0, 1025, 128)), [0, 520], False, "int8"),
+])
+def test_k_segments_resident_and_sequential(case, segment_mode):
+    name, M, K, N, kb, nb, dual, code = case
+    run_parity(custom_spec(name, M, K, N, kb, nb, dual, code, x_seg_std=[1.0 + 3 * i for i in range(len(kb) - 1)]),
+               segment_mode=segment_mode)
+
+
+@pytest.mark.parametrize("dual", [False, True])
+def test_many_small_k_segments(dual):
+    """24 K-segments of 64 codes (the head-merge reshape in front of an attention output projection) and
+    40 segments of 32: more accumulators than tensor memory could hold at once."""
+    run_parity(custom_spec("heads24", 300, 1536, 320, list(range(0, 1537, 64)), [0, 320], dual, "int8",
+                           x_seg_std=[0.5 + 0.4 * i for i in range(24)]))
+    run_parity(custom_spec("seg40", 140, 1280, 136, list(range(0, 1281, 32)), [0, 64, 136], dual, "int8",
+                           x_seg_std=[1.0 + 0.2 * i for i in range(40)]))
+
+
 def test_strided_output_and_code_matrices():
     """Y with a row pitch larger than N (a column slice of a wider buffer) is written only inside its
     N columns, and code matrices with a padded pitch are read correctly."""
@@ -194,6 +219,39 @@ def test_quantizer_codes_equal_the_division_definition_on_adversarial_values(cod
     assert np.array_equal(c_pos.cpu().numpy().view(dt), r_pos)
     if dual:
         assert np.array_equal(c_neg.cpu().numpy().view(dt), r_neg)
+
+
+def test_int32_accumulators_at_the_largest_k_with_extreme_codes():
+    """K = 131072 is the largest K the library accepts for int8 codes: with every activation code at +-127 / -128
+    and every weight code at +-127 the sums reach 2.13e9, just inside int32.  The code matrices are handed to
+    the GEMM directly; rows alternate sign patterns so that both extremes and cancelling sums occur."""
+    M, N, K = 136, 64, 131072
+    rs = np.random.default_rng(3)
+    xq = np.empty((M, K), np.int8)
+    xq[0::4] = 127
+    xq[1::4] = -128
+    xq[2::4] = np.where(np.arange(K) % 2 == 0, 127, -128).astype(np.int8)
+    xq[3::4] = rs.integers(-128, 128, (M // 4, K), dtype=np.int8)
+    wq = np.empty((N, K), np.int8)
+    wq[0::2] = 127
+    wq[1::2] = np.where(np.arange(K) % 3 == 0, -127, 127).astype(np.int8)
+    ref = xq.astype(np.float64) @ wq.astype(np.float64).T                 # exact: |sum| < 2^53
+    assert np.abs(ref).max() > 2.1e9 and np.abs(ref).max() < 2 ** 31
+    seg = B.SegTable([0, K], [0, N])
+    one = torch.ones(1, device=DEV)
+    ws = B.new_workspace(DEV)
+    Xd = torch.from_numpy(xq.view(np.uint8)).to(DEV)
+    Wd = torch.from_numpy(wq.view(np.uint8)).to(DEV)
+    Y, dump = B.segquant_seglinear_gemm(Xd, Wd, seg, "int8", one, one, None, ws, y_dtype=torch.float32, dump_acc=True)
+    B.check_device_status(ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(dump.cpu().numpy()[0].astype(np.float64), ref)
+    # K one block beyond the limit is refused on the host
+    with pytest.raises(B.SegquantError) as e:
+        B.segquant_seglinear_gemm(torch.zeros((8, K + 128), dtype=torch.uint8, device=DEV),
+                                  torch.zeros((8, K + 128), dtype=torch.uint8, device=DEV),
+                                  B.SegTable([0, K + 128], [0, 8]), "int8", one, one, None, ws)
+    assert e.value.status == 2
 
 
 def test_fp32_input_and_student_t():

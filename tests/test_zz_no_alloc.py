@@ -60,13 +60,17 @@ def test_static_calibration_matches_workspace_calibration_twice_in_a_row():
 
 
 def test_static_calibration_refuses_more_blocks_than_it_holds():
-    # the segment-table limits of the library keep P*Q within the built-in array; a table beyond those
-    # limits is refused on the host, before any launch
+    # 33 K-segments x 32 N-segments = 1056 weight blocks: a valid table for the workspace version, one more
+    # row of blocks than the built-in array holds; refused on the host, before any launch
     n0 = B.segquant_launch_count()
-    K, N = 32 * 17, 8
+    P, Q = 33, 32
+    K, N = 32 * P, 8 * Q
     X = torch.zeros((N, K), dtype=torch.float32, device=DEV)
-    seg = B.SegTable(list(range(0, K + 1, 32)), [0, N])          # 17 K-segments > SQ_MAX_P
+    seg = B.SegTable(list(range(0, K + 1, 32)), list(range(0, N + 1, 8)))
     with pytest.raises(B.SegquantError) as e:
         B.segquant_calib_scales_static(X, seg, "int8", True, False)
     assert e.value.status == 5
     assert B.segquant_launch_count() == n0
+    s_w, _ = B.segquant_calib_scales(X, seg, "int8", True, False, B.new_workspace(DEV))
+    torch.cuda.synchronize()
+    assert s_w.numel() == P * Q and bool(torch.all(s_w == 1.0))       # all-zero blocks: unit scale
