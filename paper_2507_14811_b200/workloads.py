@@ -173,6 +173,15 @@ WORKLOADS: dict[str, list[LayerSpec]] = {
 
 SDXL_SWEEP_M = [512, 1024, 2048, 4096, 8192, 16384, 32768, 65536]
 
+# input segmentation by attention heads: the head-merge reshape in front of an attention output projection
+# gives 24 K-segments of 64 channels (SD3.5-medium-like shape), each with its own activation range
+WORKLOADS["sd3_heads"] = [
+    _spec("attn_out_24x64", 8858, 1536, 1536, P=24, dual=False, code="int8", x_dtype="bf16",
+          x_kind="normal", w_kind="plain", seed=5000, x_seg_std=[0.5 + 0.25 * i for i in range(24)]),
+    _spec("attn_out_6x256", 8858, 1536, 1536, P=6, dual=False, code="int8", x_dtype="bf16",
+          x_kind="normal", w_kind="plain", seed=5001, x_seg_std=[0.5 + i for i in range(6)]),
+]
+
 # the skip-concat layer at every row count of the sweep (the points of its roofline curve)
 WORKLOADS["sdxl_sweep"] = [
     _spec(f"skip_conv1x1_M{m}", m, 1280, 640, P=2, dual=True, code="int8", x_dtype="bf16",

@@ -319,7 +319,7 @@ def test_reduced_benchmark_layers(wl, idx, M, K, N):
 
 @pytest.mark.parametrize("wl,idx", [("dit_xl2", 0), ("dit_xl2", 1), ("sd3_mmdit", 0), ("sd3_mmdit", 1),
                                     ("sd3_mmdit", 2), ("flux", 0), ("flux", 1), ("flux", 2), ("sdxl_skip", 0),
-                                    ("sdxl_sweep", 0), ("sdxl_sweep", 7)])
+                                    ("sdxl_sweep", 0), ("sdxl_sweep", 7), ("sd3_heads", 0), ("sd3_heads", 1)])
 def test_full_size_layers_sampled_rows(wl, idx):
     spec = WL.WORKLOADS[wl][idx]
     rs = np.random.default_rng(99)
