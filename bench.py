@@ -257,10 +257,14 @@ def oracle_sample(specs, target_s=12.0, probe_rows=8):
     _, t_probe = run(probe_rows)
     max_rows = min(s.M for s in specs)
     rows = int(max(probe_rows, min(max_rows, probe_rows * target_s / max(t_probe, 1e-6))))
-    ops, t = run(rows)
+    ops, t, reps = 0.0, 0.0, 0
+    while reps < 1 or (t < 0.8 * target_s and reps < 20):      # a whole small workload is repeated up to the target
+        o, dt = run(rows)
+        ops, t, reps = ops + o, t + dt, reps + 1
+    what = "every row" if rows == max_rows else f"the first {rows} rows"
     return {"value": ops / t / 1e12, "unit": "TOPS", "cores": O.num_threads(), "kind": "oracle",
-            "sample": f"first {rows} rows of every layer of the workload (steps quantize+accumulate+dequant), "
-                      f"{t:.1f} s of CPU time"}, rows, t
+            "sample": f"{what} of every layer of the workload (steps quantize+accumulate+dequant), "
+                      f"{reps} pass(es), {t:.1f} s of CPU time"}, rows, t
 
 
 def run_ours(args):
