@@ -11,12 +11,12 @@
 //   warp 1      tcgen05.mma issuer (one lane, leader CTA only): for every 32-byte K-step one MMA per
 //               polarity against the same weight tile; every (K-segment, polarity) has its own
 //               accumulator in TMEM
-//   warps 2..9  epilogue: tcgen05.ld of all accumulators of a 32-column slab, fp32 FMA with the
-//               per-(segment, polarity, column) scale, + bias, -> bf16 / fp32, written from
+//   warps 2..9  epilogue: tcgen05.ld of the accumulators of a 32-column slab, y = bias + sum over
+//               (segment, polarity) of factor * accumulator in fp32, -> bf16 / fp32, written from
 //               registers with 32-byte stores (every store covers whole 32-byte sectors of Y)
-// Accumulators: NACC = P * npol, each 128 lanes x TILE_N columns; NACC * TILE_N <= 512 columns.
-// If they use at most half of TMEM the accumulator set is double-buffered so that the epilogue of
-// one tile overlaps the main loop of the next.
+// One K-segment: the npol accumulators (128 lanes x TILE_N columns each) of a tile stay in TMEM until the
+// tile's epilogue; if they use at most half of TMEM there are two sets, and the epilogue of one tile
+// overlaps the main loop of the next.  Several K-segments: see SEQ below.
 // Every wait on an mbarrier is bounded (SM cycle counter, about 2 s); on expiry the CTA records
 // which wait gave up in the status word, stops issuing work, lets its own copies land and leaves
 // normally.  No load uses cluster multicast.
@@ -141,13 +141,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         asm volatile(
             "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
             ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y) : "memory");
-}
-
-__device__ __forceinline__ float4 ld_shared_f4(uint32_t addr)
-{
-    float4 v;
-    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
-    return v;
 }
 
 __device__ __forceinline__ void ld_shared_2x64(uint32_t addr, uint64_t &a, uint64_t &b)
@@ -283,11 +276,9 @@ __host__ __device__ constexpr uint32_t make_idesc(int kind, int tile_n, int mma_
 // ----------------------------------------------------------------------------- the kernel
 
 // bytes of the epilogue's tables between the ring and the header (multiple of 16)
-template <bool GENERIC>
 __host__ __device__ constexpr uint32_t epi_table_bytes(int nacc, int Q, int tile_n)
 {
-    return GENERIC ? uint32_t(nacc + 1) * tile_n * 4u
-                   : ((uint32_t(tile_n) + uint32_t(nacc) * Q + uint32_t(Q) + 1u) * 4u + 15u) & ~15u;
+    return ((uint32_t(tile_n) + uint32_t(nacc) * Q + uint32_t(Q) + 1u) * 4u + 15u) & ~15u;
 }
 
 struct SharedHeader {
@@ -372,11 +363,112 @@ __device__ __forceinline__ void issue_kblock(uint32_t d0, uint64_t da, uint64_t 
     }
 }
 
+// ----------------------------------------------------------------------------- epilogue pieces
+
+// N-segment of column n: the number of interior bounds nb[1..Q-1] that are <= n, counted warp-wide
+// (all 32 lanes call it together).
+__device__ __forceinline__ int seg_of_column(int n, int Q, uint32_t nb_addr, int lane)
+{
+    int cnt = 0;
+    for (int base = 1; base < Q; base += 32) {
+        const int i = base + lane;
+        const bool le = i < Q && n >= int(ld_shared_u32(nb_addr + 4u * uint32_t(i < Q ? i : 0)));
+        cnt += __popc(__ballot_sync(0xFFFFFFFFu, le));
+    }
+    return cnt;
+}
+
+// y += c[a][q(column)] * acc for the 32 columns nf .. nf + 31 of one row; y holds 16 packed fp32 pairs, r the
+// raw accumulator words of one TMEM load.  A slab that lies in one N-segment (q_lo == q_hi; always so in the
+// production variant) takes one factor; otherwise the factor is looked up per column.
+template <int KIND, bool GENERIC>
+__device__ __forceinline__ void scale_add_unit(uint64_t (&y2)[16], const uint32_t (&r)[32], int a, int Q, int q_lo,
+                                               int q_hi, int nf, uint32_t tab_addr, uint32_t nb_addr)
+{
+    if (!GENERIC || q_lo == q_hi) {
+        const float c = ld_shared_f32(tab_addr + uint32_t(a * Q + q_lo) * 4u);
+        const uint64_t c2 = pack_f32x2(c, c);
+#pragma unroll
+        for (int j = 0; j < 16; j++) {
+            const uint64_t v2 = KIND == 0 ? pack_f32x2(__int2float_rn(int(r[2 * j])), __int2float_rn(int(r[2 * j + 1])))
+                                          : pack_b32x2(r[2 * j], r[2 * j + 1]);
+            y2[j] = fma_f32x2(c2, v2, y2[j]);
+        }
+    } else {
+        int q = q_lo;
+#pragma unroll
+        for (int j = 0; j < 16; j++) {
+            float cc[2];
+#pragma unroll
+            for (int t = 0; t < 2; t++) {
+                while (q < q_hi && nf + 2 * j + t >= int(ld_shared_u32(nb_addr + 4u * uint32_t(q + 1)))) q++;
+                cc[t] = ld_shared_f32(tab_addr + uint32_t(a * Q + q) * 4u);
+            }
+            const uint64_t v2 = KIND == 0 ? pack_f32x2(__int2float_rn(int(r[2 * j])), __int2float_rn(int(r[2 * j + 1])))
+                                          : pack_b32x2(r[2 * j], r[2 * j + 1]);
+            y2[j] = fma_f32x2(pack_f32x2(cc[0], cc[1]), v2, y2[j]);
+        }
+    }
+}
+
+// raw accumulator words of one unit -> dump[a][row][nf .. nf + 31] (parity tests)
+__device__ __forceinline__ void dump_unit(void *acc_dump, const uint32_t (&r)[32], int a, int row, int nf, int M, int N)
+{
+    uint32_t *dump = static_cast<uint32_t *>(acc_dump) + (size_t(a) * M + row) * size_t(N) + nf;
+#pragma unroll
+    for (int j = 0; j < 32; j++)
+        if (nf + j < N) dump[j] = r[j];
+}
+
+// Converts and stores the 32 outputs y of row `row`, columns nf .. nf + 31, in 16-byte chunks (8 bf16 or
+// 4 fp32).  N is a multiple of 8, so a chunk is entirely inside or outside the matrix; two adjacent chunks go
+// out as one 32-byte store when the rows of Y are 32-byte aligned.
+template <bool GENERIC, typename Params>
+__device__ __forceinline__ void store_slab(const uint64_t (&y2)[16], const Params &prm, int row, int nf)
+{
+    const int nvalid = prm.N - nf;                       // valid columns of this slab, may exceed 32
+    if (GENERIC && prm.y_is_f32) {
+        float *dst = static_cast<float *>(prm.Y) + size_t(row) * prm.ldy + nf;
+#pragma unroll
+        for (int c = 0; c < 4; c++) {                    // 8 columns = 32 bytes
+            if (8 * c < nvalid) {
+                const uint4 lo = make_uint4(uint32_t(y2[4 * c]), uint32_t(y2[4 * c] >> 32),
+                                            uint32_t(y2[4 * c + 1]), uint32_t(y2[4 * c + 1] >> 32));
+                const uint4 hi = make_uint4(uint32_t(y2[4 * c + 2]), uint32_t(y2[4 * c + 2] >> 32),
+                                            uint32_t(y2[4 * c + 3]), uint32_t(y2[4 * c + 3] >> 32));
+                if (prm.y_wide) st_global_32(dst + 8 * c, lo, hi);
+                else { st_global_16(dst + 8 * c, lo); st_global_16(dst + 8 * c + 4, hi); }
+            }
+        }
+    } else {
+        __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(prm.Y) + size_t(row) * prm.ldy + nf;
+        uint32_t h[16];
+#pragma unroll
+        for (int j = 0; j < 16; j++) {
+            float lo, hi;
+            unpack_f32x2(y2[j], lo, hi);
+            __nv_bfloat162 v2 = __floats2bfloat162_rn(lo, hi);
+            h[j] = *reinterpret_cast<uint32_t *>(&v2);
+        }
+#pragma unroll
+        for (int c = 0; c < 2; c++) {                    // 16 columns = 32 bytes
+            const uint4 w0 = make_uint4(h[8 * c], h[8 * c + 1], h[8 * c + 2], h[8 * c + 3]);
+            const uint4 w1 = make_uint4(h[8 * c + 4], h[8 * c + 5], h[8 * c + 6], h[8 * c + 7]);
+            if (16 * c + 8 < nvalid && prm.y_wide) {
+                st_global_32(dst + 16 * c, w0, w1);
+            } else {
+                if (16 * c < nvalid) st_global_16(dst + 16 * c, w0);
+                if (16 * c + 8 < nvalid) st_global_16(dst + 16 * c + 8, w1);
+            }
+        }
+    }
+}
+
 // GENERIC = false is the production variant: bf16 output, no accumulator dump, every interior N-bound
 // a multiple of 32 (so that each 32-column slab of the output lies in one N-segment and takes ONE
 // dequantization factor per accumulator).  Its epilogue loop is small enough for the instruction
-// cache and runs its FMAs on packed fp32 pairs.  GENERIC = true handles everything else (fp32 output,
-// accumulator dump, arbitrary N-bounds) with a per-column factor table rebuilt for every tile.
+// cache.  GENERIC = true adds the fp32 output, the accumulator dump for the parity tests and a
+// per-column factor lookup for slabs that straddle an N-bound.
 // SEQ = true (layers with more than one K-segment): TMEM holds the accumulators of ONE K-segment at a time,
 // in two alternating sets.  The MMA issuer fills a set with segment p while the epilogue warps drain the set
 // of segment p - 1, scale it and add it to fp32 running sums kept in registers for the whole tile; the sums
@@ -395,13 +487,11 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     constexpr uint32_t b_bytes = B_ROWS * BLOCK_K;
     constexpr uint32_t stage_bytes = NPOL * a_bytes + b_bytes;
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    constexpr bool kColTable = GENERIC && !SEQ;          // per-column factor table rebuilt per tile
-    float *sh_scale = reinterpret_cast<float *>(smem + size_t(prm.stages) * stage_bytes);   // kColTable: [nacc][TILE_N]
-    float *sh_bias = sh_scale + (kColTable ? prm.nacc * TILE_N : 0);                        // [TILE_N], per tile
-    float *sh_tab = sh_bias + TILE_N;                                                       // !kColTable: [nacc][Q]
-    int *sh_nb = reinterpret_cast<int *>(sh_tab + (kColTable ? 0 : prm.nacc * prm.sb.Q));   // !kColTable: [Q + 1]
-    SharedHeader *hdr = reinterpret_cast<SharedHeader *>(
-        reinterpret_cast<uint8_t *>(smem + size_t(prm.stages) * stage_bytes) + epi_table_bytes<kColTable>(prm.nacc, prm.sb.Q, TILE_N));
+    float *sh_bias = reinterpret_cast<float *>(smem + size_t(prm.stages) * stage_bytes);    // [TILE_N], per tile
+    float *sh_tab = sh_bias + TILE_N;                                                       // [nacc][Q], per launch
+    int *sh_nb = reinterpret_cast<int *>(sh_tab + prm.nacc * prm.sb.Q);                     // [Q + 1]
+    SharedHeader *hdr = reinterpret_cast<SharedHeader *>(reinterpret_cast<uint8_t *>(sh_bias) +
+                                                         epi_table_bytes(prm.nacc, prm.sb.Q, TILE_N));
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -548,65 +638,71 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     } else {
         // ------------------------------------------------------------------ epilogue warps
         // Warp w may read TMEM lanes 32 * (w % 4) .. + 31; the two warps of one lane group take one half
-        // of the tile's 32-column slabs each.
-        if constexpr (SEQ) {
-            const int et = threadIdx.x - 64;
-            const int ew = warp - 2;
-            const int lane_grp = warp & 3;
-            constexpr int kSlabsPerWarp = TILE_N / 32 / (kEpiWarps / 4);
-            static_assert(kSlabsPerWarp >= 1 && kSlabsPerWarp * (kEpiWarps / 4) * 32 == TILE_N, "SEQ needs TILE_N >= 64");
-            constexpr int kUnits = kSlabsPerWarp * NPOL;                // TMEM loads per segment and warp
-            const int slab0 = (ew >> 2) * kSlabsPerWarp;
-            const int P = prm.sb.P, Q = prm.sb.Q;
-            const uint32_t tmem_empty_sig0 = CG == 2 ? map_to_cta(smem_u32(&hdr->tmem_empty[0]), 0)
-                                                     : smem_u32(&hdr->tmem_empty[0]);
-            const uint32_t tab_addr = smem_u32(sh_tab), nb_addr = smem_u32(sh_nb), bias_addr = smem_u32(sh_bias);
-            auto fetch_bias = [&](int tile) -> float {
-                if (tile >= num_tiles || et >= TILE_N || !prm.bias) return 0.0f;
-                const int n = (tile % prm.num_n_tiles) * TILE_N + et;
-                return n < prm.N ? __ldg(prm.bias + n) : 0.0f;
-            };
-            auto seg_of = [&](int n) {                                  // interior N-bounds <= n, counted warp-wide
-                int cnt = 0;
-                for (int base = 1; base < Q; base += 32) {
-                    const int i = base + lane;
-                    const bool le = i < Q && n >= int(ld_shared_u32(nb_addr + 4u * uint32_t(i < Q ? i : 0)));
-                    cnt += __popc(__ballot_sync(0xFFFFFFFFu, le));
-                }
-                return cnt;
-            };
-            float bias_next = fetch_bias(unit);
-            for (int i = et; i < prm.nacc * Q; i += kEpiThreads) {      // factors c[a][q], a = p * NPOL + pol
-                const int a = i / Q, q = i - a * Q, p = a / NPOL;
-                const float s_act = (NPOL == 2 && (a & 1)) ? prm.s_neg[p] : prm.s_pos[p];
-                sh_tab[i] = s_act * prm.s_w[p * Q + q];
+        // of the tile's 32-column slabs each.  Per output: y = bias, then y = fma(c[a][q], acc[a], y) over
+        // a = (p, polarity) ascending, two outputs per instruction on packed fp32 pairs.
+        const int et = threadIdx.x - 64;
+        const int ew = warp - 2;
+        const int lane_grp = warp & 3;
+        constexpr int kColGroups = kEpiWarps / 4;
+        constexpr int kSlabs = TILE_N / 32;
+        constexpr int kSlabsPerWarp = (kSlabs + kColGroups - 1) / kColGroups;
+        const int slab0 = (ew >> 2) * kSlabsPerWarp;
+        const int nacc = prm.nacc;
+        const int P = prm.sb.P, Q = prm.sb.Q;
+        const uint32_t tmem_empty_sig0 = CG == 2 ? map_to_cta(smem_u32(&hdr->tmem_empty[0]), 0)
+                                                 : smem_u32(&hdr->tmem_empty[0]);
+        const uint32_t tab_addr = smem_u32(sh_tab), nb_addr = smem_u32(sh_nb), bias_addr = smem_u32(sh_bias);
+        auto release = [&](uint32_t set) {             // accumulator set `set` is in registers: hand it back
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                if (CG == 2) mbar_arrive_cluster(tmem_empty_sig0 + 8 * set);
+                else mbar_arrive(tmem_empty_sig0 + 8 * set);
             }
-            for (int i = et; i <= Q; i += kEpiThreads) sh_nb[i] = prm.sb.nb[i];
-            uint32_t as = 0, aph = 0;
-            bool ok = true;
-            for (int tile = unit; tile < num_tiles; tile += num_units) {
-                const int m0 = (tile / prm.num_n_tiles) * (TILE_M * CG) + int(rank) * TILE_M;
-                const int n0 = (tile % prm.num_n_tiles) * TILE_N;
+        };
+        // bias slice of a tile, one column per thread, fetched one tile ahead into a register
+        auto fetch_bias = [&](int tile) -> float {
+            if (tile >= num_tiles || et >= TILE_N || !prm.bias) return 0.0f;
+            const int n = (tile % prm.num_n_tiles) * TILE_N + et;
+            return n < prm.N ? __ldg(prm.bias + n) : 0.0f;
+        };
+        float bias_next = fetch_bias(unit);
+        // dequantization factors c[a][q] = s_act[p][pol] * s_w[p][q], a = p * NPOL + pol (one fp32 multiply);
+        // built here, off the producer's and the MMA issuer's path, and published by the first tile's barrier
+        for (int i = et; i < nacc * Q; i += kEpiThreads) {
+            const int a = i / Q, q = i - a * Q, p = a / NPOL;
+            const float s_act = (NPOL == 2 && (a & 1)) ? prm.s_neg[p] : prm.s_pos[p];
+            sh_tab[i] = s_act * prm.s_w[p * Q + q];
+        }
+        for (int i = et; i <= Q; i += kEpiThreads) sh_nb[i] = prm.sb.nb[i];
 
-                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // previous tile's readers are done
-                if (et < TILE_N) sh_bias[et] = bias_next;
-                bias_next = fetch_bias(tile + num_units);
-                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+        uint32_t as = 0, aph = 0;
+        bool ok = true;
+        for (int tile = unit; tile < num_tiles; tile += num_units) {
+            const int m0 = (tile / prm.num_n_tiles) * (TILE_M * CG) + int(rank) * TILE_M;
+            const int n0 = (tile % prm.num_n_tiles) * TILE_N;
+            const int row = m0 + lane_grp * 32 + lane;
 
-                const int row = m0 + lane_grp * 32 + lane;
-                // running sums of this thread's outputs (row `row`, kSlabsPerWarp slabs of 32 columns), start = bias
+            asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // previous tile's readers are done
+            if (et < TILE_N) sh_bias[et] = bias_next;
+            bias_next = fetch_bias(tile + num_units);                        // lands during this tile's work
+            asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+
+            if constexpr (SEQ) {
+                // ---- one accumulator set per K-segment: running sums of the whole tile stay in registers
+                static_assert(!SEQ || kSlabsPerWarp * kColGroups == kSlabs, "SEQ needs TILE_N >= 64");
+                constexpr int kUnits = kSlabsPerWarp * NPOL;                // TMEM loads per segment and warp
                 uint64_t y2[kSlabsPerWarp][16];
                 int q_lo[kSlabsPerWarp], q_hi[kSlabsPerWarp];
 #pragma unroll
                 for (int sl = 0; sl < kSlabsPerWarp; sl++) {
                     const int c0 = (slab0 + sl) * 32;
-                    q_lo[sl] = seg_of(n0 + c0);
-                    q_hi[sl] = GENERIC ? seg_of(min(n0 + c0 + 31, prm.N - 1)) : q_lo[sl];
+                    q_lo[sl] = seg_of_column(n0 + c0, Q, nb_addr, lane);
+                    q_hi[sl] = GENERIC ? seg_of_column(min(n0 + c0 + 31, prm.N - 1), Q, nb_addr, lane) : q_lo[sl];
 #pragma unroll
                     for (int j4 = 0; j4 < 8; j4++)
                         ld_shared_2x64(bias_addr + uint32_t(c0 + 4 * j4) * 4u, y2[sl][2 * j4], y2[sl][2 * j4 + 1]);
                 }
-
                 for (int p = 0; p < P; p++) {
                     const uint32_t cur_as = as, cur_aph = aph;
                     if (++as == 2u) { as = 0; aph ^= 1; }
@@ -624,398 +720,78 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                         const int sl = u / NPOL, pol = u % NPOL;
                         uint32_t (&r)[32] = (kAhead && (u & 1)) ? reinterpret_cast<uint32_t (&)[32]>(rb) : ra;
                         tc_wait_ld();
-                        if (kAhead && u + 1 < kUnits) {
+                        if (kAhead && u + 1 < kUnits)
                             tc_ld32(t_row + uint32_t(((u + 1) % NPOL) * TILE_N + (slab0 + (u + 1) / NPOL) * 32),
                                     (u & 1) ? ra : reinterpret_cast<uint32_t (&)[32]>(rb));
-                        } else if (u + 1 == kUnits) {                                // set read: hand it back
-                            tc_fence_before();
-                            __syncwarp();
-                            if (lane == 0) {
-                                if (CG == 2) mbar_arrive_cluster(tmem_empty_sig0 + 8 * cur_as);
-                                else mbar_arrive(tmem_empty_sig0 + 8 * cur_as);
-                            }
-                        }
+                        else if (u + 1 == kUnits)
+                            release(cur_as);
                         const int a = p * NPOL + pol;
                         const int nf = n0 + (slab0 + sl) * 32;
-                        if (!GENERIC || q_lo[sl] == q_hi[sl]) {                      // slab inside one N-segment
-                            const float c = ld_shared_f32(tab_addr + uint32_t(a * Q + q_lo[sl]) * 4u);
-                            const uint64_t c2 = pack_f32x2(c, c);
-#pragma unroll
-                            for (int j = 0; j < 16; j++) {
-                                const uint64_t v2 = KIND == 0 ? pack_f32x2(__int2float_rn(int(r[2 * j])), __int2float_rn(int(r[2 * j + 1])))
-                                                              : pack_b32x2(r[2 * j], r[2 * j + 1]);
-                                y2[sl][j] = fma_f32x2(c2, v2, y2[sl][j]);
-                            }
-                        } else {
-                            int q = q_lo[sl];
-#pragma unroll
-                            for (int j = 0; j < 16; j++) {
-                                float cc[2];
-#pragma unroll
-                                for (int t = 0; t < 2; t++) {
-                                    while (q < q_hi[sl] && nf + 2 * j + t >= int(ld_shared_u32(nb_addr + 4u * uint32_t(q + 1)))) q++;
-                                    cc[t] = ld_shared_f32(tab_addr + uint32_t(a * Q + q) * 4u);
-                                }
-                                const uint64_t v2 = KIND == 0 ? pack_f32x2(__int2float_rn(int(r[2 * j])), __int2float_rn(int(r[2 * j + 1])))
-                                                              : pack_b32x2(r[2 * j], r[2 * j + 1]);
-                                y2[sl][j] = fma_f32x2(pack_f32x2(cc[0], cc[1]), v2, y2[sl][j]);
-                            }
-                        }
-                        if (GENERIC && prm.acc_dump && row < prm.M) {
-                            uint32_t *dump = static_cast<uint32_t *>(prm.acc_dump) + (size_t(a) * prm.M + row) * size_t(prm.N) + nf;
-#pragma unroll
-                            for (int j = 0; j < 32; j++)
-                                if (nf + j < prm.N) dump[j] = r[j];
-                        }
+                        scale_add_unit<KIND, GENERIC>(y2[sl], r, a, Q, q_lo[sl], q_hi[sl], nf, tab_addr, nb_addr);
+                        if (GENERIC && prm.acc_dump && row < prm.M) dump_unit(prm.acc_dump, r, a, row, nf, prm.M, prm.N);
                         if (!kAhead && u + 1 < kUnits)
                             tc_ld32(t_row + uint32_t(((u + 1) % NPOL) * TILE_N + (slab0 + (u + 1) / NPOL) * 32), ra);
                     }
                 }
-                if (!ok) continue;
-                // all segments added: convert and store this thread's outputs, 16-byte chunks of 8 bf16 / 4 fp32
-                if (row < prm.M) {
+                if (ok && row < prm.M) {
 #pragma unroll
-                    for (int sl = 0; sl < kSlabsPerWarp; sl++) {
-                        const int nf = n0 + (slab0 + sl) * 32;
-                        const int nvalid = prm.N - nf;
-                        if (GENERIC && prm.y_is_f32) {
-                            float *dst = static_cast<float *>(prm.Y) + size_t(row) * prm.ldy + nf;
-#pragma unroll
-                            for (int c = 0; c < 4; c++) {
-                                if (8 * c < nvalid) {
-                                    const uint4 lo = make_uint4(uint32_t(y2[sl][4 * c]), uint32_t(y2[sl][4 * c] >> 32),
-                                                                uint32_t(y2[sl][4 * c + 1]), uint32_t(y2[sl][4 * c + 1] >> 32));
-                                    const uint4 hi = make_uint4(uint32_t(y2[sl][4 * c + 2]), uint32_t(y2[sl][4 * c + 2] >> 32),
-                                                                uint32_t(y2[sl][4 * c + 3]), uint32_t(y2[sl][4 * c + 3] >> 32));
-                                    if (prm.y_wide) st_global_32(dst + 8 * c, lo, hi);
-                                    else { st_global_16(dst + 8 * c, lo); st_global_16(dst + 8 * c + 4, hi); }
-                                }
-                            }
-                        } else {
-                            __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(prm.Y) + size_t(row) * prm.ldy + nf;
-                            uint32_t h[16];
-#pragma unroll
-                            for (int j = 0; j < 16; j++) {
-                                float lo, hi;
-                                unpack_f32x2(y2[sl][j], lo, hi);
-                                __nv_bfloat162 v2 = __floats2bfloat162_rn(lo, hi);
-                                h[j] = *reinterpret_cast<uint32_t *>(&v2);
-                            }
-#pragma unroll
-                            for (int cidx = 0; cidx < 2; cidx++) {
-                                const uint4 w0 = make_uint4(h[8 * cidx], h[8 * cidx + 1], h[8 * cidx + 2], h[8 * cidx + 3]);
-                                const uint4 w1 = make_uint4(h[8 * cidx + 4], h[8 * cidx + 5], h[8 * cidx + 6], h[8 * cidx + 7]);
-                                if (16 * cidx + 8 < nvalid && prm.y_wide) {
-                                    st_global_32(dst + 16 * cidx, w0, w1);
-                                } else {
-                                    if (16 * cidx < nvalid) st_global_16(dst + 16 * cidx, w0);
-                                    if (16 * cidx + 8 < nvalid) st_global_16(dst + 16 * cidx + 8, w1);
-                                }
-                            }
-                        }
-                    }
+                    for (int sl = 0; sl < kSlabsPerWarp; sl++) store_slab<GENERIC>(y2[sl], prm, row, n0 + (slab0 + sl) * 32);
                 }
-            }
-        } else if constexpr (!GENERIC) {
-            const int et = threadIdx.x - 64;
-            const int ew = warp - 2;
-            const int lane_grp = warp & 3;
-            constexpr int kColGroups = kEpiWarps / 4;
-            constexpr int kSlabs = TILE_N / 32;
-            constexpr int kSlabsPerWarp = (kSlabs + kColGroups - 1) / kColGroups;
-            const int slab0 = (ew >> 2) * kSlabsPerWarp;
-            const int my_slabs = max(0, min(kSlabsPerWarp, kSlabs - slab0));
-            const int nacc = prm.nacc;
-            const int units = my_slabs * nacc;                              // (slab, accumulator) pairs of this warp
-            const int Q = prm.sb.Q;
-            const uint32_t tmem_empty_sig0 = CG == 2 ? map_to_cta(smem_u32(&hdr->tmem_empty[0]), 0)
-                                                     : smem_u32(&hdr->tmem_empty[0]);
-            const uint32_t tab_addr = smem_u32(sh_tab), nb_addr = smem_u32(sh_nb), bias_addr = smem_u32(sh_bias);
-            // bias slice of a tile, one column per thread, fetched one tile ahead into a register
-            auto fetch_bias = [&](int tile) -> float {
-                if (tile >= num_tiles || et >= TILE_N || !prm.bias) return 0.0f;
-                const int n = (tile % prm.num_n_tiles) * TILE_N + et;
-                return n < prm.N ? __ldg(prm.bias + n) : 0.0f;
-            };
-            float bias_next = fetch_bias(unit);
-            // dequantization factors c[a][q] = s_act[p][pol] * s_w[p][q], a = p * NPOL + pol (one fp32 multiply);
-            // built here, off the producer's and the MMA issuer's path, and published by the first tile's barrier
-            for (int i = et; i < nacc * Q; i += kEpiThreads) {
-                const int a = i / Q, q = i - a * Q, p = a / NPOL;
-                const float s_act = (NPOL == 2 && (a & 1)) ? prm.s_neg[p] : prm.s_pos[p];
-                sh_tab[i] = s_act * prm.s_w[p * Q + q];
-            }
-            for (int i = et; i <= Q; i += kEpiThreads) sh_nb[i] = prm.sb.nb[i];
-            uint32_t as = 0, aph = 0;
-            bool ok = true;
-            for (int tile = unit; tile < num_tiles; tile += num_units) {
-                const int m0 = (tile / prm.num_n_tiles) * (TILE_M * CG) + int(rank) * TILE_M;
-                const int n0 = (tile % prm.num_n_tiles) * TILE_N;
+            } else {
+                // ---- all accumulators of the tile resident: slab by slab, TMEM loads one unit ahead of the
+                // arithmetic; the set goes back to the MMA issuer as soon as the last load has landed
                 const uint32_t cur_as = as, cur_aph = aph;
                 if (++as == uint32_t(prm.acc_stages)) { as = 0; aph ^= 1; }
-
-                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // previous tile's readers are done
-                if (et < TILE_N) sh_bias[et] = bias_next;
-                bias_next = fetch_bias(tile + num_units);                        // lands during this tile's work
-                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
-
                 if (ok) ok = mbar_wait(smem_u32(&hdr->tmem_full[cur_as]), cur_aph, abort_flag, prm.status, kWhereEpilogue);
                 if (!ok) continue;                  // keep the named barriers balanced, do no more work
                 tc_fence_after();
-
-                const int row = m0 + lane_grp * 32 + lane;
                 const uint32_t t_row = tmem_base + (uint32_t(lane_grp * 32) << 16) + cur_as * acc_cols;
-                const uint32_t release_bar = tmem_empty_sig0 + 8 * cur_as;
+                const int my_slabs = max(0, min(kSlabsPerWarp, kSlabs - slab0));
+                const int units = my_slabs * nacc;                          // (slab, accumulator) pairs of this warp
 
-                // The (slab, accumulator) units of this warp are read from TMEM one ahead of the arithmetic;
-                // the accumulator set goes back to the MMA issuer as soon as the last load has landed.
-                // Per output: y = bias, then y = fma(c[a][q], acc[a], y) over a = (p, polarity) ascending,
-                // two outputs per instruction on packed fp32 pairs.
                 uint64_t y2[16];
                 uint32_t ra[32], rb[32];
                 int i_sl = 0, i_a = 0;              // next unit to load
                 int c_sl = 0, c_a = 0;              // next unit to consume
-                int q_seg = 0;                      // N-segment of the slab being consumed
+                int q_lo = 0, q_hi = 0;             // N-segments of the first and last column of the slab
                 auto issue = [&](uint32_t (&r)[32]) {
                     tc_ld32(t_row + uint32_t(i_a * TILE_N + (slab0 + i_sl) * 32), r);
                     if (++i_a == nacc) { i_a = 0; i_sl++; }
-                };
-                auto release = [&]() {
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) {
-                        if (CG == 2) mbar_arrive_cluster(release_bar);
-                        else mbar_arrive(release_bar);
-                    }
                 };
                 auto consume = [&](const uint32_t (&r)[32]) {
                     const int c0 = (slab0 + c_sl) * 32;
                     const int nf = n0 + c0;                          // first column of the slab
                     if (c_a == 0) {
-                        // segment of the slab: the number of interior bounds nb[1..Q-1] that are <= nf
-                        q_seg = 0;
-                        for (int base = 1; base < Q; base += 32) {
-                            const int i = base + lane;
-                            const bool le = i < Q && nf >= int(ld_shared_u32(nb_addr + 4u * uint32_t(i < Q ? i : 0)));
-                            q_seg += __popc(__ballot_sync(0xFFFFFFFFu, le));
-                        }
+                        q_lo = seg_of_column(nf, Q, nb_addr, lane);
+                        q_hi = GENERIC ? seg_of_column(min(nf + 31, prm.N - 1), Q, nb_addr, lane) : q_lo;
 #pragma unroll
                         for (int j4 = 0; j4 < 8; j4++)
                             ld_shared_2x64(bias_addr + uint32_t(c0 + 4 * j4) * 4u, y2[2 * j4], y2[2 * j4 + 1]);
                     }
-                    const float c = ld_shared_f32(tab_addr + uint32_t(c_a * Q + q_seg) * 4u);
-                    const uint64_t c2 = pack_f32x2(c, c);
-#pragma unroll
-                    for (int j = 0; j < 16; j++) {
-                        const uint64_t v2 = KIND == 0 ? pack_f32x2(__int2float_rn(int(r[2 * j])), __int2float_rn(int(r[2 * j + 1])))
-                                                      : pack_b32x2(r[2 * j], r[2 * j + 1]);
-                        y2[j] = fma_f32x2(c2, v2, y2[j]);
-                    }
+                    scale_add_unit<KIND, GENERIC>(y2, r, c_a, Q, q_lo, q_hi, nf, tab_addr, nb_addr);
+                    if (GENERIC && prm.acc_dump && row < prm.M) dump_unit(prm.acc_dump, r, c_a, row, nf, prm.M, prm.N);
                     if (++c_a < nacc) return;
                     c_a = 0;
                     c_sl++;
-                    // last accumulator of the slab: convert and store this thread's 32 outputs of row `row` in
-                    // 16-byte chunks of 8 bf16; N is a multiple of 8, so a chunk is entirely inside or outside
-                    if (row < prm.M) {
-                        const int nvalid = prm.N - nf;               // valid columns of this slab, may exceed 32
-                        __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(prm.Y) + size_t(row) * prm.ldy + nf;
-                        uint32_t h[16];
-#pragma unroll
-                        for (int j = 0; j < 16; j++) {
-                            float lo, hi;
-                            unpack_f32x2(y2[j], lo, hi);
-                            __nv_bfloat162 v2 = __floats2bfloat162_rn(lo, hi);
-                            h[j] = *reinterpret_cast<uint32_t *>(&v2);
-                        }
-#pragma unroll
-                        for (int cidx = 0; cidx < 2; cidx++) {       // 16 columns = 32 bytes
-                            const uint4 w0 = make_uint4(h[8 * cidx], h[8 * cidx + 1], h[8 * cidx + 2], h[8 * cidx + 3]);
-                            const uint4 w1 = make_uint4(h[8 * cidx + 4], h[8 * cidx + 5], h[8 * cidx + 6], h[8 * cidx + 7]);
-                            if (16 * cidx + 8 < nvalid && prm.y_wide) {
-                                st_global_32(dst + 16 * cidx, w0, w1);
-                            } else {
-                                if (16 * cidx < nvalid) st_global_16(dst + 16 * cidx, w0);
-                                if (16 * cidx + 8 < nvalid) st_global_16(dst + 16 * cidx + 8, w1);
-                            }
-                        }
-                    }
+                    if (row < prm.M) store_slab<GENERIC>(y2, prm, row, nf);      // last accumulator of the slab
                 };
-
                 if (units == 0) {
-                    release();
+                    release(cur_as);
                 } else {
                     issue(ra);
 #pragma unroll 1
                     for (int u = 0; u < units; u += 2) {
                         tc_wait_ld();
-                        if (u + 1 < units) issue(rb); else release();
+                        if (u + 1 < units) issue(rb); else release(cur_as);
                         consume(ra);
                         if (u + 1 < units) {
                             tc_wait_ld();
-                            if (u + 2 < units) issue(ra); else release();
+                            if (u + 2 < units) issue(ra); else release(cur_as);
                             consume(rb);
                         }
                     }
                 }
             }
-        } else {
-        const int et = threadIdx.x - 64;           // 0..255
-        const int ew = warp - 2;                   // 0..7
-        const int lane_grp = warp & 3;             // TMEM lanes 32*lane_grp .. +31 are this warp's
-        const int col_half = ew >> 2;              // which half of the tile's 32-column slabs
-        constexpr int kSlabs = TILE_N / 32;
-        constexpr int kSlabsPerWarp = kSlabs >= 2 ? kSlabs / 2 : 1;
-        const bool has_work = kSlabs >= 2 || col_half == 0;
-        const int nacc = prm.nacc;
-        const int units = has_work ? kSlabsPerWarp * nacc : 0;      // (slab, accumulator) pairs of this warp
-        const int col_base = col_half * kSlabsPerWarp * 32;
-        const uint32_t tmem_empty_sig0 = CG == 2 ? map_to_cta(smem_u32(&hdr->tmem_empty[0]), 0)
-                                                 : smem_u32(&hdr->tmem_empty[0]);
-        const uint32_t sc_base = smem_u32(sh_scale), bias_base = smem_u32(sh_bias);
-        uint32_t as = 0, aph = 0;
-        bool ok = true;
-        for (int tile = unit; tile < num_tiles; tile += num_units) {
-            const int m0 = (tile / prm.num_n_tiles) * (TILE_M * CG) + int(rank) * TILE_M;
-            const int n0 = (tile % prm.num_n_tiles) * TILE_N;
-            const uint32_t cur_as = as, cur_aph = aph;
-            if (++as == uint32_t(prm.acc_stages)) { as = 0; aph ^= 1; }
-
-            // per-column dequantization factors of this tile: c[a][j] = s_act[p][pol] * s_w[p][q(n0+j)]
-            asm volatile("bar.sync 1, 256;" ::: "memory");       // previous tile's readers are done
-            for (int j = et; j < TILE_N; j += kEpiThreads) {
-                const int n = n0 + j;
-                int q = 0;
-                while (q + 1 < prm.sb.Q && n >= prm.sb.nb[q + 1]) q++;
-                for (int p = 0; p < prm.sb.P; p++) {
-                    const float sw = n < prm.N ? prm.s_w[p * prm.sb.Q + q] : 0.0f;
-                    sh_scale[(p * NPOL) * TILE_N + j] = prm.s_pos[p] * sw;
-                    if (NPOL == 2) sh_scale[(p * NPOL + 1) * TILE_N + j] = prm.s_neg[p] * sw;
-                }
-                sh_bias[j] = (prm.bias && n < prm.N) ? prm.bias[n] : 0.0f;
-            }
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-
-            if (ok) ok = mbar_wait(smem_u32(&hdr->tmem_full[cur_as]), cur_aph, abort_flag, prm.status, kWhereEpilogue);
-            if (!ok) continue;                      // keep the named barriers balanced, do no more work
-            tc_fence_after();
-
-            const int row = m0 + lane_grp * 32 + lane;
-            const uint32_t t_row = tmem_base + (uint32_t(lane_grp * 32) << 16) + cur_as * acc_cols;
-            const uint32_t release_bar = tmem_empty_sig0 + 8 * cur_as;
-
-            // The (slab, accumulator) units of this warp are read from TMEM one ahead of the arithmetic:
-            // while unit u is scaled and summed, the load of unit u + 1 is in flight.  The accumulator set
-            // is handed back to the MMA issuer as soon as the last load has landed in registers.
-            float y[32];
-#pragma unroll
-            for (int j = 0; j < 32; j++) y[j] = 0.0f;
-            uint32_t ra[32], rb[32];
-            int i_sl = 0, i_a = 0;                  // next unit to load
-            int c_sl = 0, c_a = 0;                  // next unit to consume
-            auto issue = [&](uint32_t (&r)[32]) {
-                tc_ld32(t_row + uint32_t(i_a * TILE_N + col_base + i_sl * 32), r);
-                if (++i_a == nacc) { i_a = 0; i_sl++; }
-            };
-            auto release = [&]() {
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) {
-                    if (CG == 2) mbar_arrive_cluster(release_bar);
-                    else mbar_arrive(release_bar);
-                }
-            };
-            auto consume = [&](const uint32_t (&r)[32]) {
-                const int c0 = col_base + c_sl * 32;
-                const uint32_t sc = sc_base + uint32_t(c_a * TILE_N + c0) * 4u;
-#pragma unroll
-                for (int j4 = 0; j4 < 8; j4++) {
-                    const float4 c = ld_shared_f4(sc + 16u * j4);
-                    const float cc[4] = {c.x, c.y, c.z, c.w};
-#pragma unroll
-                    for (int t = 0; t < 4; t++) {
-                        const int j = 4 * j4 + t;
-                        const float v = KIND == 0 ? __int2float_rn(int(r[j])) : __uint_as_float(r[j]);
-                        y[j] = fmaf(cc[t], v, y[j]);
-                    }
-                }
-                if (GENERIC && prm.acc_dump && row < prm.M) {
-                    uint32_t *dump = static_cast<uint32_t *>(prm.acc_dump) +
-                                     (size_t(c_a) * prm.M + row) * size_t(prm.N) + n0 + c0;
-#pragma unroll
-                    for (int j = 0; j < 32; j++)
-                        if (n0 + c0 + j < prm.N) dump[j] = r[j];
-                }
-                if (++c_a < nacc) return;
-                c_a = 0;
-                c_sl++;
-                // last accumulator of the slab: + bias, convert, store this thread's 32 outputs of row `row`
-#pragma unroll
-                for (int j4 = 0; j4 < 8; j4++) {
-                    const float4 b = ld_shared_f4(bias_base + uint32_t(c0) * 4u + 16u * j4);
-                    y[4 * j4 + 0] += b.x; y[4 * j4 + 1] += b.y; y[4 * j4 + 2] += b.z; y[4 * j4 + 3] += b.w;
-                }
-                // 16-byte chunks (8 bf16 or 4 fp32); N is a multiple of 8, so a chunk is entirely inside or
-                // outside the matrix
-                if (row < prm.M) {
-                    const int nvalid = prm.N - (n0 + c0);            // valid columns of this slab, may exceed 32
-                    if (GENERIC && prm.y_is_f32) {
-                        float *dst = static_cast<float *>(prm.Y) + size_t(row) * prm.ldy + n0 + c0;
-#pragma unroll
-                        for (int c = 0; c < 4; c++) {                // 8 columns = 32 bytes
-                            if (8 * c < nvalid) {
-                                const uint4 lo = make_uint4(__float_as_uint(y[8 * c]), __float_as_uint(y[8 * c + 1]),
-                                                            __float_as_uint(y[8 * c + 2]), __float_as_uint(y[8 * c + 3]));
-                                const uint4 hi = make_uint4(__float_as_uint(y[8 * c + 4]), __float_as_uint(y[8 * c + 5]),
-                                                            __float_as_uint(y[8 * c + 6]), __float_as_uint(y[8 * c + 7]));
-                                if (prm.y_wide) st_global_32(dst + 8 * c, lo, hi);
-                                else { st_global_16(dst + 8 * c, lo); st_global_16(dst + 8 * c + 4, hi); }
-                            }
-                        }
-                    } else {
-                        __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(prm.Y) + size_t(row) * prm.ldy + n0 + c0;
-                        uint4 w[4];
-#pragma unroll
-                        for (int c = 0; c < 4; c++) {
-                            uint32_t h[4];
-#pragma unroll
-                            for (int t = 0; t < 4; t++) {
-                                __nv_bfloat162 v2 = __floats2bfloat162_rn(y[8 * c + 2 * t], y[8 * c + 2 * t + 1]);
-                                h[t] = *reinterpret_cast<uint32_t *>(&v2);
-                            }
-                            w[c] = make_uint4(h[0], h[1], h[2], h[3]);
-                        }
-#pragma unroll
-                        for (int c = 0; c < 2; c++) {                // 16 columns = 32 bytes
-                            if (16 * c + 8 < nvalid && prm.y_wide) {
-                                st_global_32(dst + 16 * c, w[2 * c], w[2 * c + 1]);
-                            } else {
-                                if (16 * c < nvalid) st_global_16(dst + 16 * c, w[2 * c]);
-                                if (16 * c + 8 < nvalid) st_global_16(dst + 16 * c + 8, w[2 * c + 1]);
-                            }
-                        }
-                    }
-                }
-#pragma unroll
-                for (int j = 0; j < 32; j++) y[j] = 0.0f;
-            };
-
-            if (units == 0) {
-                release();
-            } else {
-                issue(ra);
-#pragma unroll 1
-                for (int u = 0; u < units; u += 2) {
-                    tc_wait_ld();
-                    if (u + 1 < units) issue(rb); else release();
-                    consume(ra);
-                    if (u + 1 < units) {
-                        tc_wait_ld();
-                        if (u + 2 < units) issue(ra); else release();
-                        consume(rb);
-                    }
-                }
-            }
-        }
         }
     }
 
@@ -1079,7 +855,7 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
     if (!make_map(&tb, g.b, g.N, g.K, g.ldb, B_ROWS)) return SQ_ERR_CUDA;
 
     const uint32_t stage_bytes = NPOL * TILE_M * BLOCK_K + B_ROWS * BLOCK_K;
-    const uint32_t tail = epi_table_bytes<GENERIC && !SEQ>(prm.nacc, prm.sb.Q, TILE_N) + sizeof(SharedHeader);
+    const uint32_t tail = epi_table_bytes(prm.nacc, prm.sb.Q, TILE_N) + sizeof(SharedHeader);
     int stages = int((kSmemBudget - 1024 - tail) / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (g_tune_stages >= 2 && g_tune_stages < stages) stages = g_tune_stages;
