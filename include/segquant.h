@@ -178,6 +178,22 @@ sq_status segquant_layer_forward(const void *X, int x_on_host, void *x_stage, sq
                                  void *scratch, size_t scratch_bytes,
                                  void *workspace, size_t ws_bytes, void *stream);
 
+/* segquant_layer_forward for host X and Y with the copies overlapped with the kernels: the rows are cut
+ * into `chunks` pieces of whole 256-row tiles; piece i is copied in on `stream_in`, quantized and
+ * multiplied on `stream`, copied out on `stream_out`, so that piece i+1 arrives and piece i-1 leaves while
+ * piece i is computed.  Results are identical to segquant_layer_forward.  The three streams must differ;
+ * `stream` completes when the last output copy has, so synchronizing `stream` is enough.  X and Y should
+ * be pinned host memory (otherwise the copies do not overlap); x_stage / y_stage / scratch / workspace as
+ * for segquant_layer_forward.  The call creates and releases a few CUDA events; it allocates no device
+ * memory.  1 <= chunks <= 64. */
+sq_status segquant_layer_forward_pipelined(const void *X, void *x_stage, sq_dtype dt, int64_t M, int64_t K, int64_t ld,
+                                           const void *Wq, int64_t ldw, int64_t N, const sq_segtable *seg,
+                                           sq_code code, const float *s_pos, const float *s_neg, const float *s_w,
+                                           const float *bias, uint32_t flags, void *Y, void *y_stage,
+                                           sq_dtype y_dtype, int64_t ldy, void *scratch, size_t scratch_bytes,
+                                           void *workspace, size_t ws_bytes, int chunks, void *stream,
+                                           void *stream_in, void *stream_out);
+
 /* Synchronizes `stream`, reads the device status word of `workspace` and clears it.  Returns SQ_OK,
  * SQ_ERR_TIMEOUT (a bounded wait inside a kernel expired; *detail, if not NULL, receives a code that
  * names the wait) or SQ_ERR_CUDA. */

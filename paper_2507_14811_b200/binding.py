@@ -25,7 +25,7 @@ STATUS_NAMES = {0: "SQ_OK", 1: "SQ_ERR_NULL", 2: "SQ_ERR_SHAPE", 3: "SQ_ERR_SEGT
 EXPORTS = [
     "segquant_workspace_bytes", "segquant_calib_scales", "segquant_calib_scales_static", "segquant_quantize_act", "segquant_quantize_weight",
     "segquant_seglinear_gemm", "segquant_dualscale_gemm", "segquant_layer_scratch_bytes",
-    "segquant_layer_forward", "segquant_last_device_status", "segquant_set_tuning", "segquant_launch_count",
+    "segquant_layer_forward", "segquant_layer_forward_pipelined", "segquant_last_device_status", "segquant_set_tuning", "segquant_launch_count",
     "segquant_status_string",
 ]
 
@@ -238,6 +238,22 @@ def segquant_layer_forward(X, Wq, seg: SegTable, code: str, s_pos, s_neg, s_w, b
         _ptr(y_stage), C.c_int(_dt(Y)), C.c_int64(Y.stride(0)), _ptr(scratch), C.c_size_t(scratch.numel()),
         _ptr(workspace), C.c_size_t(workspace.numel()), _stream())
     _check(st, "segquant_layer_forward")
+    return Y
+
+
+def segquant_layer_forward_pipelined(X, Wq, seg: SegTable, code: str, s_pos, s_neg, s_w, bias, Y, scratch, workspace,
+                                     x_stage, y_stage, chunks: int, stream_in, stream_out, flags: int = 0):
+    """segquant_layer_forward for pinned host X / Y with the copies overlapped with the kernels: chunks of rows
+    go in on stream_in, through the kernels on the current stream, and out on stream_out (torch streams)."""
+    M, K = X.shape
+    N = Wq.shape[0]
+    st = lib().segquant_layer_forward_pipelined(
+        _ptr(X), _ptr(x_stage), C.c_int(_dt(X)), C.c_int64(M), C.c_int64(K), C.c_int64(X.stride(0)), _ptr(Wq),
+        C.c_int64(Wq.stride(0)), C.c_int64(N), seg.ref(), C.c_int(SQ_CODE[code]), _ptr(s_pos), _ptr(s_neg), _ptr(s_w),
+        _ptr(bias), C.c_uint32(flags), _ptr(Y), _ptr(y_stage), C.c_int(_dt(Y)), C.c_int64(Y.stride(0)), _ptr(scratch),
+        C.c_size_t(scratch.numel()), _ptr(workspace), C.c_size_t(workspace.numel()), C.c_int(chunks), _stream(),
+        C.c_void_p(stream_in.cuda_stream), C.c_void_p(stream_out.cuda_stream))
+    _check(st, "segquant_layer_forward_pipelined")
     return Y
 
 

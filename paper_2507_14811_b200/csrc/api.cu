@@ -221,6 +221,82 @@ sq_status segquant_layer_forward(const void *X, int x_on_host, void *x_stage, sq
     return SQ_OK;
 }
 
+sq_status segquant_layer_forward_pipelined(const void *X, void *x_stage, sq_dtype dt, int64_t M, int64_t K, int64_t ld,
+                                           const void *Wq, int64_t ldw, int64_t N, const sq_segtable *seg,
+                                           sq_code code, const float *s_pos, const float *s_neg, const float *s_w,
+                                           const float *bias, uint32_t flags, void *Y, void *y_stage,
+                                           sq_dtype y_dtype, int64_t ldy, void *scratch, size_t scratch_bytes,
+                                           void *workspace, size_t ws_bytes, int chunks, void *stream,
+                                           void *stream_in, void *stream_out)
+{
+    if (!X || !Y || !scratch || !x_stage || !y_stage) return SQ_ERR_NULL;
+    if (!valid_dt(dt) || !valid_dt(y_dtype)) return SQ_ERR_UNSUPPORTED;
+    if (M <= 0 || K <= 0 || N <= 0 || ld < K || ldy < N || chunks < 1 || chunks > 64) return SQ_ERR_SHAPE;
+    if (stream_in == stream || stream_out == stream || stream_in == stream_out) return SQ_ERR_UNSUPPORTED;
+    const int dual = s_neg != nullptr;
+    if (scratch_bytes < segquant_layer_scratch_bytes(M, K, dual)) return SQ_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(scratch) & 255u) return SQ_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream), sin = static_cast<cudaStream_t>(stream_in),
+                 sout = static_cast<cudaStream_t>(stream_out);
+    const int64_t ldc = (K + 127) & ~int64_t(127);
+    uint8_t *c_pos = static_cast<uint8_t *>(scratch);
+    uint8_t *c_neg = dual ? c_pos + ((size_t(M) * ldc + 255) & ~size_t(255)) : nullptr;
+    // rows per chunk: whole 256-row tiles
+    int64_t rows = ((M + chunks - 1) / chunks + 255) & ~int64_t(255);
+
+    // events order the three streams; they are created for this call and released when their work is done
+    cudaEvent_t ev[2 * 64 + 2];
+    int nev = 0;
+    auto new_event = [&]() -> cudaEvent_t {
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        ev[nev++] = e;
+        return e;
+    };
+    sq_status r = SQ_OK;
+    auto fail = [&](sq_status code_) { if (r == SQ_OK) r = code_; };
+    cudaEvent_t e0 = new_event();       // the staging buffers may still be in use by earlier work on `stream`
+    if (!e0 || cudaEventRecord(e0, st) != cudaSuccess || cudaStreamWaitEvent(sin, e0, 0) != cudaSuccess ||
+        cudaStreamWaitEvent(sout, e0, 0) != cudaSuccess)
+        fail(SQ_ERR_CUDA);
+    cudaEvent_t last_out = nullptr;
+    for (int64_t r0 = 0; r0 < M && r == SQ_OK; r0 += rows) {
+        const int64_t m = r0 + rows <= M ? rows : M - r0;
+        const size_t x_off = size_t(r0) * ld * dt_size(dt), y_off = size_t(r0) * ldy * dt_size(y_dtype);
+        cudaEvent_t e_in = new_event(), e_done = new_event();
+        if (!e_in || !e_done) { fail(SQ_ERR_CUDA); break; }
+        if (cudaMemcpyAsync(static_cast<uint8_t *>(x_stage) + x_off, static_cast<const uint8_t *>(X) + x_off,
+                            size_t(m) * ld * dt_size(dt), cudaMemcpyHostToDevice, sin) != cudaSuccess ||
+            cudaEventRecord(e_in, sin) != cudaSuccess || cudaStreamWaitEvent(st, e_in, 0) != cudaSuccess) {
+            fail(SQ_ERR_CUDA);
+            break;
+        }
+        sq_status q = segquant_quantize_act(static_cast<uint8_t *>(x_stage) + x_off, dt, m, K, ld, seg, s_pos, s_neg, code,
+                                            flags, c_pos + size_t(r0) * ldc, dual ? c_neg + size_t(r0) * ldc : nullptr,
+                                            ldc, stream);
+        if (q == SQ_OK)
+            q = dual ? segquant_dualscale_gemm(c_pos + size_t(r0) * ldc, c_neg + size_t(r0) * ldc, ldc, Wq, ldw, m, N, K,
+                                               seg, code, s_pos, s_neg, s_w, bias, static_cast<uint8_t *>(y_stage) + y_off,
+                                               y_dtype, ldy, nullptr, workspace, ws_bytes, stream)
+                     : segquant_seglinear_gemm(c_pos + size_t(r0) * ldc, ldc, Wq, ldw, m, N, K, seg, code, s_pos, s_w, bias,
+                                               static_cast<uint8_t *>(y_stage) + y_off, y_dtype, ldy, nullptr, workspace,
+                                               ws_bytes, stream);
+        if (q != SQ_OK) { fail(q); break; }
+        if (cudaEventRecord(e_done, st) != cudaSuccess || cudaStreamWaitEvent(sout, e_done, 0) != cudaSuccess ||
+            cudaMemcpyAsync(static_cast<uint8_t *>(Y) + y_off, static_cast<uint8_t *>(y_stage) + y_off,
+                            size_t(m) * ldy * dt_size(y_dtype), cudaMemcpyDeviceToHost, sout) != cudaSuccess) {
+            fail(SQ_ERR_CUDA);
+            break;
+        }
+    }
+    // `stream` completes only when the last output copy has: the caller synchronizes one stream
+    last_out = new_event();
+    if (!last_out || cudaEventRecord(last_out, sout) != cudaSuccess || cudaStreamWaitEvent(st, last_out, 0) != cudaSuccess)
+        fail(SQ_ERR_CUDA);
+    for (int i = 0; i < nev; i++) cudaEventDestroy(ev[i]);
+    return r;
+}
+
 sq_status segquant_last_device_status(void *workspace, void *stream, uint32_t *detail)
 {
     if (!workspace) return SQ_ERR_NULL;

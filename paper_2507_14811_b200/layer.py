@@ -48,6 +48,13 @@ class SegQuantLinear:
                                         self.bias, Y, self.scratch_for(M), self.workspace,
                                         x_stage=x_stage, y_stage=y_stage, flags=self.flags)
 
+    def forward_pipelined(self, X_host: torch.Tensor, Y_host: torch.Tensor, x_stage, y_stage, chunks, stream_in, stream_out):
+        """Pinned-host X -> pinned-host Y with the copies overlapped with the kernels (see the C header)."""
+        M = X_host.shape[0]
+        return B.segquant_layer_forward_pipelined(X_host, self.Wq, self.seg, self.code, self.s_pos, self.s_neg, self.s_w,
+                                                  self.bias, Y_host, self.scratch_for(M), self.workspace, x_stage, y_stage,
+                                                  chunks, stream_in, stream_out, flags=self.flags)
+
     def forward_steps(self, X: torch.Tensor, y_dtype=torch.bfloat16, dump_acc=False):
         """The same path as separate calls, returning the intermediate codes (and raw accumulators)."""
         c_pos, c_neg = B.segquant_quantize_act(X, self.seg, self.s_pos, self.s_neg, self.code, self.flags)

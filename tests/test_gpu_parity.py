@@ -163,6 +163,30 @@ def test_many_small_k_segments(dual):
                            x_seg_std=[1.0 + 0.2 * i for i in range(40)]))
 
 
+@pytest.mark.parametrize("chunks", [1, 3, 8])
+def test_pipelined_host_call_equals_the_plain_one(chunks):
+    """Pinned-host input and output with the copies on their own streams: same bytes as the one-stream call."""
+    spec = custom_spec("pipe", 1500, 384, 520, [0, 128, 384], [0, 256, 520], True, "int8")
+    data = WL.make_layer(spec)
+    layer = SegQuantLinear(data.W, data.bias, spec.kb, spec.nb, True, "int8", DEV)
+    layer.calibrate(data.X_cal)
+    Xh = data.X.pin_memory()
+    x_stage = torch.empty_like(data.X, device=DEV)
+    y_stage = torch.empty((spec.M, spec.N), dtype=torch.bfloat16, device=DEV)
+    Y_plain = torch.empty((spec.M, spec.N), dtype=torch.bfloat16).pin_memory()
+    Y_pipe = torch.full((spec.M, spec.N), 3.0, dtype=torch.bfloat16).pin_memory()
+    layer.forward(Xh, Y=Y_plain, x_stage=x_stage, y_stage=y_stage)
+    torch.cuda.synchronize()
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    layer.forward_pipelined(Xh, Y_pipe, x_stage, y_stage, chunks, s_in, s_out)
+    torch.cuda.current_stream().synchronize()          # the compute stream alone is synchronized, as documented
+    layer.check_status()
+    assert torch.equal(Y_plain, Y_pipe)
+    res = O.layer_forward(to_f32_np(data.X), *[oracle_scales(data)[i] for i in (3,)],
+                          O.SegTable(spec.kb, spec.nb), *oracle_scales(data)[:3], to_f32_np(data.bias))
+    check_bf16_output(Y_pipe, res.y64, res.y_abs, 4)
+
+
 def test_strided_output_and_code_matrices():
     """Y with a row pitch larger than N (a column slice of a wider buffer) is written only inside its
     N columns, and code matrices with a padded pitch are read correctly."""
