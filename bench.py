@@ -196,6 +196,27 @@ def time_workload(layers, steps, warmup, flush, sampler=None):
     return q_ms.mean(axis=0), g_ms.mean(axis=0), clocks
 
 
+def time_layers(layers, steps, warmup, flush):
+    """Per-layer mean time of quantize + GEMM issued back to back (one event pair per layer, L2 flushed before)."""
+    nl = len(layers)
+    ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(nl)] for _ in range(steps)]
+    for _ in range(warmup):
+        for bl in layers:
+            flush()
+            bl.quantize()
+            bl.gemm()
+    torch.cuda.synchronize()
+    for s in range(steps):
+        for i, bl in enumerate(layers):
+            flush()
+            ev[s][i][0].record()
+            bl.quantize()
+            bl.gemm()
+            ev[s][i][1].record()
+    torch.cuda.synchronize()
+    return np.array([[ev[s][i][0].elapsed_time(ev[s][i][1]) for i in range(nl)] for s in range(steps)]).mean(axis=0)
+
+
 def time_plain(layers, steps, flush):
     """Mean time of the plain single-scale GEMM on every dual layer's shape (None for single-scale layers)."""
     out = []
@@ -314,11 +335,13 @@ def run_ours(args):
     barrier()
     for bl in layers:
         bl.layer.check_status()
+    layer_ms = time_layers(layers, args.steps, 3, flush)
     plain_ms = time_plain(layers, max(3, min(args.steps, 20)), flush)
     e2e_ms = time_e2e(layers, max(3, args.steps // 4), args.warmup, flush, args.e2e_chunks)
     barrier()
 
-    step_ms = float((q_ms + g_ms).sum())
+    step_ms = float(layer_ms.sum())            # quantize + GEMM of every layer, back to back per layer
+    split_ms = float((q_ms + g_ms).sum())      # the same kernels timed one by one (an event between them)
     e2e_step_ms = float(e2e_ms.sum())
     if world > 1:
         import torch.distributed as dist
@@ -368,11 +391,13 @@ def run_ours(args):
             "config": {"workload": args.workload,
                        "layers": [f"{s.name} M={s.M} K={s.K} N={s.N} P={s.P} Q={s.Q} {'dual' if s.dual else 'single'} {s.code}"
                                   for s in specs],
-                       "step": "per layer: quantize_act -> dual/seg GEMM + dequant epilogue (bf16 out)",
+                       "step": "per layer: quantize_act -> dual/seg GEMM + dequant epilogue (bf16 out), both launches "
+                               "between one pair of CUDA events",
                        "ops": "executed tensor ops: 4MNK for dual layers, 2MNK for single-scale layers",
                        "l2": f"flushed before every layer ({L2_FLUSH_BYTES >> 20} MiB write, then {L2_FLUSH_BYTES >> 20} MiB read), flush outside the timed intervals",
                        "parallelism": f"{world} independent row-sharded replicas, no collective" if world > 1 else "1 GPU"},
             "useful_tops": round(world * useful_ops / (step_ms * 1e-3) / 1e12, 2),
+            "ms_per_step_kernels_timed_one_by_one": round(split_ms, 5),
             "frac_of_nominal_4500_tops": round(exec_ops / (step_ms * 1e-3) / 1e12 / NOMINAL_8BIT_TOPS, 4),
             "e2e": {"value": round(world * exec_ops / (e2e_step_ms * 1e-3) / 1e12, 2), "unit": "TOPS",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_step_ms, 4),
