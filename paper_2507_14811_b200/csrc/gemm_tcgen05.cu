@@ -72,6 +72,13 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
 }
+// Programmatic dependent launch: the kernel may start while the previous kernel of the stream is still
+// finishing.  grid_dependency_wait() returns once that kernel has completed and its writes are visible;
+// every thread calls it before its first access to global memory.  grid_launch_dependents() lets the
+// next kernel of the stream (if launched the same way) be scheduled as this one winds down.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ void cluster_sync_all()
 {
     asm volatile("barrier.cluster.arrive.release;" ::: "memory");
@@ -543,6 +550,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
         if (lane == 0) {
             const uint32_t stages = prm.stages, P = prm.sb.P;
             const uint32_t full0 = smem_u32(&hdr->full[0]), empty0 = smem_u32(&hdr->empty[0]);
+            grid_dependency_wait();                 // the code matrices come from the previous kernel
             // completion bytes of both CTAs' loads are counted on the leader's barrier
             const uint32_t full0_sig = CG == 2 ? map_to_cta(full0, 0) : full0;
             const uint32_t ring0 = smem_u32(smem);
@@ -569,6 +577,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                     }
                 }
             }
+            grid_launch_dependents();               // all of this CTA's loads are issued: the tail begins
             if (!ok && rank == 0) {
                 // let the copies this thread issued land before the CTA's shared memory goes away
                 const uint32_t pending = issued < stages ? issued : stages;
@@ -666,6 +675,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
             const int n = (tile % prm.num_n_tiles) * TILE_N + et;
             return n < prm.N ? __ldg(prm.bias + n) : 0.0f;
         };
+        grid_dependency_wait();                     // scales, bias and Y may belong to the previous kernel
         float bias_next = fetch_bias(unit);
         // dequantization factors c[a][q] = s_act[p][pol] * s_w[p][q], a = p * NPOL + pol (one fp32 multiply);
         // built here, off the producer's and the MMA issuer's path, and published by the first tile's barrier
@@ -875,13 +885,15 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = CG;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = CG == 2 ? 1 : 0;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = CG == 2 ? attr : attr + 1;          // the cluster attribute only for CTA pairs
+    cfg.numAttrs = CG == 2 ? 2 : 1;
 
     // persistent grid: one CTA (pair) per SM (pair) that can be resident at the same time
     int units = sm_count / CG;

@@ -214,6 +214,11 @@ quantize_kernel(const Tin *__restrict__ X, int64_t M, int K, int64_t ld, const S
                 const float *__restrict__ s_pos, const float *__restrict__ s_neg, int row_segments,
                 int lo, int hi, uint8_t *__restrict__ c_pos, uint8_t *__restrict__ c_neg, int64_t ldc)
 {
+    // Programmatic dependent launch: this kernel may be scheduled while the previous kernel of the stream
+    // winds down, and lets the next one be scheduled while its own last blocks run; nothing in global
+    // memory is touched before the previous kernel has completed.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int V = (K + kVec - 1) / kVec;
     const int64_t idx = int64_t(blockIdx.x) * kThreads + threadIdx.x;
     if (idx >= M * int64_t(V)) return;
@@ -263,14 +268,23 @@ sq_status launch_t(const Tin *X, int64_t M, int64_t K, int64_t ld, const SegBoun
     const int64_t V = (K + kVec - 1) / kVec;
     const int64_t blocks = (M * V + kThreads - 1) / kThreads;
     if (blocks > 0x7FFFFFFF) return SQ_ERR_SHAPE;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(unsigned(blocks));
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const int Ki = int(K);
+    uint8_t *cp = static_cast<uint8_t *>(c_pos), *cn = static_cast<uint8_t *>(c_neg);
+    const float *no_neg = nullptr;
     if (s_neg)
-        quantize_kernel<Tin, CODE, true><<<unsigned(blocks), kThreads, 0, st>>>(
-            X, M, int(K), ld, sb, s_pos, s_neg, row_segments, lo, hi, static_cast<uint8_t *>(c_pos),
-            static_cast<uint8_t *>(c_neg), ldc);
+        cudaLaunchKernelEx(&cfg, quantize_kernel<Tin, CODE, true>, X, M, Ki, ld, sb, s_pos, s_neg, row_segments, lo, hi, cp, cn, ldc);
     else
-        quantize_kernel<Tin, CODE, false><<<unsigned(blocks), kThreads, 0, st>>>(
-            X, M, int(K), ld, sb, s_pos, nullptr, row_segments, lo, hi, static_cast<uint8_t *>(c_pos),
-            nullptr, ldc);
+        cudaLaunchKernelEx(&cfg, quantize_kernel<Tin, CODE, false>, X, M, Ki, ld, sb, s_pos, no_neg, row_segments, lo, hi, cp,
+                           static_cast<uint8_t *>(nullptr), ldc);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
 }
