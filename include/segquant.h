@@ -208,6 +208,9 @@ sq_status segquant_last_device_status(void *workspace, void *stream, uint32_t *d
  * the automatic choice. */
 sq_status segquant_set_tuning(int tile_n, int stages, int cta_group, int segment_mode);
 
+/* Text of the CUDA error behind the most recent SQ_ERR_CUDA of a GEMM launch ("no error" if none). */
+const char *segquant_last_cuda_error(void);
+
 /* Number of kernels the library has launched in this process (all entry points). */
 uint64_t segquant_launch_count(void);
 

@@ -25,7 +25,7 @@ STATUS_NAMES = {0: "SQ_OK", 1: "SQ_ERR_NULL", 2: "SQ_ERR_SHAPE", 3: "SQ_ERR_SEGT
 EXPORTS = [
     "segquant_workspace_bytes", "segquant_calib_scales", "segquant_calib_scales_static", "segquant_quantize_act", "segquant_quantize_weight",
     "segquant_seglinear_gemm", "segquant_dualscale_gemm", "segquant_layer_scratch_bytes",
-    "segquant_layer_forward", "segquant_layer_forward_pipelined", "segquant_last_device_status", "segquant_set_tuning", "segquant_launch_count",
+    "segquant_layer_forward", "segquant_layer_forward_pipelined", "segquant_last_device_status", "segquant_set_tuning", "segquant_launch_count", "segquant_last_cuda_error",
     "segquant_status_string",
 ]
 
@@ -54,6 +54,7 @@ def lib():
         L.segquant_layer_scratch_bytes.restype = C.c_size_t
         L.segquant_layer_scratch_bytes.argtypes = [C.c_int64, C.c_int64, C.c_int]
         L.segquant_launch_count.restype = C.c_uint64
+        L.segquant_last_cuda_error.restype = C.c_char_p
         L.segquant_status_string.restype = C.c_char_p
         L.segquant_status_string.argtypes = [C.c_int]
         _lib = L
@@ -99,6 +100,8 @@ def _stream():
 
 def _check(status, where):
     if status != SQ_OK:
+        if status == 6:
+            where = f"{where} ({lib().segquant_last_cuda_error().decode()})"
         raise SegquantError(status, where)
 
 

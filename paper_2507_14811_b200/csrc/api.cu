@@ -7,6 +7,9 @@ namespace sq {
 static std::atomic<uint64_t> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(uint64_t(n), std::memory_order_relaxed); }
 
+static std::atomic<int> g_last_cuda_error{0};
+void note_cuda_error(cudaError_t e) { g_last_cuda_error.store(int(e), std::memory_order_relaxed); }
+
 HostSeg load_segtable(const sq_segtable *seg, int64_t K, int64_t N)
 {
     HostSeg h{};
@@ -315,6 +318,11 @@ sq_status segquant_set_tuning(int tile_n, int stages, int cta_group, int segment
 {
     set_gemm_tuning(tile_n, stages, cta_group, segment_mode);
     return SQ_OK;
+}
+
+const char *segquant_last_cuda_error(void)
+{
+    return cudaGetErrorString(cudaError_t(g_last_cuda_error.load(std::memory_order_relaxed)));
 }
 
 uint64_t segquant_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

@@ -483,6 +483,7 @@ __device__ __forceinline__ void store_slab(const uint64_t (&y2)[16], const Param
 // drain of every segment but the last overlaps tensor work.  SEQ = false keeps every (segment, polarity)
 // accumulator of a tile resident in TMEM and drains once per tile.
 template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ>
+// 320 threads = 10 warps, up to 3 on one SM sub-partition with 16 K registers: at most 168 registers per thread
 __global__ void __launch_bounds__(kThreads, 1)
 segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_constant__ CUtensorMap tm_a_neg,
                      const __grid_constant__ CUtensorMap tm_b, const KernelParams prm)
@@ -876,8 +877,8 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
     const size_t smem = 1024 + size_t(stages) * stage_bytes + tail;
 
     auto kern = segquant_gemm_kernel<KIND, NPOL, TILE_N, CG, GENERIC, SEQ>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
-        return SQ_ERR_CUDA;
+    const cudaError_t ea = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    if (ea != cudaSuccess) { note_cuda_error(ea); return SQ_ERR_CUDA; }
     const int tiles = prm.num_m_tiles * prm.num_n_tiles;
 
     cudaLaunchConfig_t cfg{};
@@ -902,7 +903,8 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
         static int cached_clusters = 0;
         if (cached_smem != smem) {
             int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) return SQ_ERR_CUDA;
+            const cudaError_t eo = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+            if (eo != cudaSuccess || n <= 0) { note_cuda_error(eo != cudaSuccess ? eo : cudaErrorLaunchOutOfResources); return SQ_ERR_CUDA; }
             cached_clusters = n;
             cached_smem = smem;
         }
@@ -912,7 +914,9 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
     cfg.gridDim = dim3(unsigned(grid));
     const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ta, tn, tb, prm);
     count_launch();
-    return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SQ_OK : SQ_ERR_CUDA;
+    const cudaError_t e2 = cudaGetLastError();
+    if (e != cudaSuccess || e2 != cudaSuccess) { note_cuda_error(e != cudaSuccess ? e : e2); return SQ_ERR_CUDA; }
+    return SQ_OK;
 }
 
 template <int KIND, int NPOL, int CG>

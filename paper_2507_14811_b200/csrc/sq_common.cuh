@@ -32,6 +32,7 @@ HostSeg load_segtable(const sq_segtable *seg, int64_t K, int64_t N);
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 void count_launch(int n = 1);
+void note_cuda_error(cudaError_t e);   // remembered for segquant_last_cuda_error()
 
 // per-code ranges
 inline float code_qmax(sq_code c) { return c == SQ_CODE_INT8 ? 127.0f : 448.0f; }
