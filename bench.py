@@ -160,6 +160,19 @@ class BenchLayer:
         L = self.layer
         self.B.segquant_seglinear_gemm(self.c_pos, L.Wq, L.seg, L.code, L.s_pos, L.s_w, L.bias, L.workspace, Y=self.Y)
 
+    def gemm_unsegmented(self):
+        """The same shape and polarity handling with ONE segment (P = Q = 1): the denominator of the SegLinear
+        overhead (the paper reports +37..50 % for its own kernels).  Timing only; its output is not checked."""
+        L = self.layer
+        if not hasattr(self, "_unseg"):
+            self._unseg = self.B.SegTable([0, self.spec.K], [0, self.spec.N])
+        if L.dual:
+            self.B.segquant_dualscale_gemm(self.c_pos, self.c_neg, L.Wq, self._unseg, L.code, L.s_pos[:1], L.s_neg[:1],
+                                           L.s_w[:1], L.bias, L.workspace, Y=self.Y)
+        else:
+            self.B.segquant_seglinear_gemm(self.c_pos, L.Wq, self._unseg, L.code, L.s_pos[:1], L.s_w[:1], L.bias,
+                                           L.workspace, Y=self.Y)
+
     def forward_e2e(self, chunks=0, stream_in=None, stream_out=None):
         """Pinned-host X -> pinned-host Y through the C ABI; chunks > 1 overlaps the copies with the kernels."""
         if chunks > 1:
@@ -217,21 +230,21 @@ def time_layers(layers, steps, warmup, flush):
     return np.array([[ev[s][i][0].elapsed_time(ev[s][i][1]) for i in range(nl)] for s in range(steps)]).mean(axis=0)
 
 
-def time_plain(layers, steps, flush):
-    """Mean time of the plain single-scale GEMM on every dual layer's shape (None for single-scale layers)."""
+def time_variant(layers, steps, flush, pick, call):
+    """Mean GEMM time of a comparison variant (`call`) on the layers selected by `pick`; None for the others."""
     out = []
     for bl in layers:
-        if not bl.spec.dual:
+        if not pick(bl.spec):
             out.append(None)
             continue
         ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
         for _ in range(3):
-            bl.gemm_plain()
+            call(bl)
         for s in range(steps):
             flush()
             bl.quantize()
             ev[s][0].record()
-            bl.gemm_plain()
+            call(bl)
             ev[s][1].record()
         torch.cuda.synchronize()
         out.append(float(np.mean([a.elapsed_time(b) for a, b in ev])))
@@ -336,7 +349,9 @@ def run_ours(args):
     for bl in layers:
         bl.layer.check_status()
     layer_ms = time_layers(layers, args.steps, 3, flush)
-    plain_ms = time_plain(layers, max(3, min(args.steps, 20)), flush)
+    cmp_steps = max(3, min(args.steps, 20))
+    plain_ms = time_variant(layers, cmp_steps, flush, lambda sp: sp.dual, lambda bl: bl.gemm_plain())
+    unseg_ms = time_variant(layers, cmp_steps, flush, lambda sp: sp.P > 1 or sp.Q > 1, lambda bl: bl.gemm_unsegmented())
     e2e_ms = time_e2e(layers, max(3, args.steps // 4), args.warmup, flush, args.e2e_chunks)
     barrier()
 
@@ -359,7 +374,7 @@ def run_ours(args):
     achieved = gemm_ops / (gemm_ms * 1e-3) / 1e12
 
     per_layer = []
-    for s, q, g, pl in zip(specs, q_ms, g_ms, plain_ms):
+    for s, q, g, pl, un in zip(specs, q_ms, g_ms, plain_ms, unseg_ms):
         eo, uo = layer_ops(s)
         t_tensor = eo / (peak8 * 1e12)
         t_hbm = gemm_bytes(s) / (peaks["hbm_gbs"] * 1e9)
@@ -374,6 +389,8 @@ def run_ours(args):
             "quant_frac_of_measured_hbm": round(quant_bytes(s) / (q * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
             "plain_w8a8_gemm_us": None if pl is None else round(pl * 1e3, 2),
             "dual_gemm_time_over_plain": None if pl is None else round(float(g) / pl, 3),
+            "unsegmented_gemm_us": None if un is None else round(un * 1e3, 2),
+            "seglinear_gemm_time_over_unsegmented": None if un is None else round(float(g) / un, 3),
         })
 
     out = None
