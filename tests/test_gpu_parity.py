@@ -187,6 +187,28 @@ def test_pipelined_host_call_equals_the_plain_one(chunks):
     check_bf16_output(Y_pipe, res.y64, res.y_abs, 4)
 
 
+def _random_case(i):
+    rs = np.random.default_rng(1000 + i)
+    P = int(rs.choice([1, 1, 2, 3, 5, 9, 17]))
+    Q = int(rs.choice([1, 1, 2, 4, 7]))
+    kb = np.concatenate([[0], np.cumsum(rs.integers(1, 6, P)) * 32])          # interior bounds multiples of 32
+    if rs.random() < 0.5:
+        kb[-1] -= 16                                                           # K a multiple of 16 only
+    nb = np.concatenate([[0], np.cumsum(rs.integers(1, 12, Q)) * (8 if rs.random() < 0.5 else 32)])
+    M = int(rs.choice([1, 7, 128, 129, 255, 257, 300, 520]))
+    return dict(M=M, K=int(kb[-1]), N=int(nb[-1]), kb=[int(v) for v in kb], nb=[int(v) for v in nb],
+                dual=bool(rs.random() < 0.6), code=str(rs.choice(["int8", "int8", "e4m3"])))
+
+
+@pytest.mark.parametrize("i", range(24))
+def test_random_shapes_and_segment_tables(i):
+    """Seeded random layers: segment counts from 1 to 17 (K) and 1 to 7 (N), bounds at the alignment minima,
+    row counts around the 128- and 256-row tile edges, both code types, dual and single."""
+    c = _random_case(i)
+    run_parity(custom_spec(f"rand{i}", c["M"], c["K"], c["N"], c["kb"], c["nb"], c["dual"], c["code"],
+                           x_seg_std=[0.5 + (j % 5) for j in range(len(c["kb"]) - 1)], seed=100 + i))
+
+
 def test_strided_output_and_code_matrices():
     """Y with a row pitch larger than N (a column slice of a wider buffer) is written only inside its
     N columns, and code matrices with a padded pitch are read correctly."""
