@@ -1,7 +1,7 @@
 // W8A8 GEMM + dequantizing epilogue for sm_100a (Sec. 4.2.2 segment-wise products, Sec. 4.3.2 dual
 // path recombination, App. A symmetric recovery).
 //
-// Persistent kernel, one CTA per SM, 320 threads.  With CG = 2 two neighbouring CTAs (a cluster of
+// Persistent kernel, one CTA per SM, 384 threads.  With CG = 2 two neighbouring CTAs (a cluster of
 // two) work on one 256-row output tile with tcgen05 cta_group::2: each CTA loads its own 128
 // activation rows and HALF of the weight tile, the pair's leader issues every MMA, and each CTA
 // holds the accumulators of its own 128 rows in its tensor memory (TMEM).  CG = 1 is the same
@@ -11,9 +11,14 @@
 //   warp 1      tcgen05.mma issuer (one lane, leader CTA only): for every 32-byte K-step one MMA per
 //               polarity against the same weight tile; every (K-segment, polarity) has its own
 //               accumulator in TMEM
-//   warps 2..9  epilogue: tcgen05.ld of the accumulators of a 32-column slab, y = bias + sum over
+//   warps 2, 3  idle: they fill the first warpgroup, which hands most of its registers to the others
+//   warps 4..11 epilogue: tcgen05.ld of the accumulators of a 32-column slab, y = bias + sum over
 //               (segment, polarity) of factor * accumulator in fp32, -> bf16 / fp32, written from
 //               registers with 32-byte stores (every store covers whole 32-byte sectors of Y)
+// Registers: the kernel starts with 168 per thread; warps 0..3 drop to 72 (setmaxnreg.dec) and the epilogue
+// warps rise to 216 (setmaxnreg.inc): 128 x 72 + 256 x 216 = 384 x 168, the CTA's allocation.  The
+// epilogue uses them to hold up to six 32-column accumulator loads at once, so that a tile's accumulators
+// are back with the MMA issuer early in the epilogue.
 // One K-segment: the npol accumulators (128 lanes x TILE_N columns each) of a tile stay in TMEM until the
 // tile's epilogue; if they use at most half of TMEM there are two sets, and the epilogue of one tile
 // overlaps the main loop of the next.  Several K-segments: see SEQ below.
@@ -32,7 +37,17 @@ constexpr int BLOCK_K = 128;          // bytes (= codes) per K-block: one 128B s
 constexpr int MMA_K = 32;             // codes per tcgen05.mma of an 8-bit kind
 constexpr int kEpiWarps = 8;
 constexpr int kEpiThreads = kEpiWarps * 32;
-constexpr int kThreads = 64 + kEpiThreads;
+constexpr int kFrontThreads = 128;     // warpgroup 0: producer, MMA issuer, two idle warps
+constexpr int kThreads = kFrontThreads + kEpiThreads;
+constexpr int kLaunchRegs = 168;      // per thread at launch: 65536 / 384, rounded down to a multiple of 8
+constexpr int kFrontRegs = 56, kEpiRegs = 224;     // per-thread register counts after the role split
+// setmaxnreg.inc waits, without limit, until the CTA's OWN register allocation (made at launch) has that many
+// registers free, so the new counts must fit in what the launch gave the CTA
+static_assert(kFrontThreads * kFrontRegs + kEpiThreads * kEpiRegs <= kThreads * kLaunchRegs,
+              "register counts after the role split exceed the CTA's allocation");
+static_assert(kFrontRegs % 8 == 0 && kEpiRegs % 8 == 0 && kFrontRegs >= 24 && kEpiRegs <= 256, "setmaxnreg operand");
+constexpr int kEpiBufRegs = 192;      // of kEpiRegs: accumulator load buffers plus running sums (SEQ)
+constexpr int kResidentBufs = 4;      // accumulator load buffers of the resident epilogue
 constexpr int kMaxStages = 8;
 constexpr int kTmemCols = 512;
 constexpr uint32_t kSmemBudget = 227 * 1024;
@@ -114,7 +129,18 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 // Bounded wait.  Returns false if the wait expired or another role already gave up.  The limit is
 // counted on the SM cycle counter; kWaitLimitCycles is about 2 s at the maximum SM clock.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
+__device__ __forceinline__ uint32_t ld_shared_volatile_u32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.volatile.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_shared_volatile_u32(uint32_t addr, uint32_t v)
+{
+    asm volatile("st.volatile.shared::cta.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+// abort_flag: shared-memory address of the CTA's abort word
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t abort_flag,
                                           uint32_t *status, uint32_t where)
 {
     if (mbar_try_wait(bar, parity)) return true;
@@ -122,11 +148,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     uint32_t polls = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++polls & 63u) == 0) {
-            if (*abort_flag) return false;
+            if (ld_shared_volatile_u32(abort_flag)) return false;
             const long long now = clock64();
             if (t0 == 0) t0 = now;
             if (now - t0 > kWaitLimitCycles) {
-                *abort_flag = 1;
+                st_shared_volatile_u32(abort_flag, 1u);
                 atomicCAS(status, 0u, where);
                 return false;
             }
@@ -388,20 +414,32 @@ __device__ __forceinline__ int seg_of_column(int n, int Q, uint32_t nb_addr, int
 // y += c[a][q(column)] * acc for the 32 columns nf .. nf + 31 of one row; y holds 16 packed fp32 pairs, r the
 // raw accumulator words of one TMEM load.  A slab that lies in one N-segment (q_lo == q_hi; always so in the
 // production variant) takes one factor; otherwise the factor is looked up per column.
-template <int KIND, bool GENERIC>
+// INIT: y starts from the bias slice at shared address bias_slab (32 floats) instead of its old value.
+template <int KIND, bool GENERIC, bool INIT = false>
 __device__ __forceinline__ void scale_add_unit(uint64_t (&y2)[16], const uint32_t (&r)[32], int a, int Q, int q_lo,
-                                               int q_hi, int nf, uint32_t tab_addr, uint32_t nb_addr)
+                                               int q_hi, int nf, uint32_t tab_addr, uint32_t nb_addr,
+                                               uint32_t bias_slab = 0)
 {
     if (!GENERIC || q_lo == q_hi) {
         const float c = ld_shared_f32(tab_addr + uint32_t(a * Q + q_lo) * 4u);
         const uint64_t c2 = pack_f32x2(c, c);
 #pragma unroll
-        for (int j = 0; j < 16; j++) {
-            const uint64_t v2 = KIND == 0 ? pack_f32x2(__int2float_rn(int(r[2 * j])), __int2float_rn(int(r[2 * j + 1])))
-                                          : pack_b32x2(r[2 * j], r[2 * j + 1]);
-            y2[j] = fma_f32x2(c2, v2, y2[j]);
+        for (int j4 = 0; j4 < 8; j4++) {
+            uint64_t b0 = y2[2 * j4], b1 = y2[2 * j4 + 1];
+            if (INIT) ld_shared_2x64(bias_slab + uint32_t(16 * j4), b0, b1);
+#pragma unroll
+            for (int t = 0; t < 2; t++) {
+                const int j = 2 * j4 + t;
+                const uint64_t v2 = KIND == 0 ? pack_f32x2(__int2float_rn(int(r[2 * j])), __int2float_rn(int(r[2 * j + 1])))
+                                              : pack_b32x2(r[2 * j], r[2 * j + 1]);
+                y2[j] = fma_f32x2(c2, v2, t == 0 ? b0 : b1);
+            }
         }
     } else {
+        if (INIT) {
+#pragma unroll
+            for (int j4 = 0; j4 < 8; j4++) ld_shared_2x64(bias_slab + uint32_t(16 * j4), y2[2 * j4], y2[2 * j4 + 1]);
+        }
         int q = q_lo;
 #pragma unroll
         for (int j = 0; j < 16; j++) {
@@ -483,7 +521,7 @@ __device__ __forceinline__ void store_slab(const uint64_t (&y2)[16], const Param
 // drain of every segment but the last overlaps tensor work.  SEQ = false keeps every (segment, polarity)
 // accumulator of a tile resident in TMEM and drains once per tile.
 template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ>
-// 320 threads = 10 warps, up to 3 on one SM sub-partition with 16 K registers: at most 168 registers per thread
+// 384 threads = 12 warps, 3 on each SM sub-partition with 16 K registers: 168 registers per thread at launch
 __global__ void __launch_bounds__(kThreads, 1)
 segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_constant__ CUtensorMap tm_a_neg,
                      const __grid_constant__ CUtensorMap tm_b, const KernelParams prm)
@@ -506,7 +544,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     const uint32_t rank = CG == 2 ? cluster_rank() : 0u;       // 0 = leader of the pair
     const int unit = blockIdx.x / CG, num_units = gridDim.x / CG;
     const int num_tiles = prm.num_m_tiles * prm.num_n_tiles;
-    volatile uint32_t *abort_flag = &hdr->abort_flag;
+    const uint32_t abort_flag = smem_u32(&hdr->abort_flag);
 
     if (threadIdx.x == 32 * 0 + 1) {     // descriptor fetches overlap the set-up below
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_a_pos)) : "memory");
@@ -546,7 +584,9 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
 
     // The producer and the MMA issuer are single threads: their loops are kept to a few dozen
     // instructions per K-block (ring slot and phase advance incrementally, descriptors by addition).
-    if (warp == 0) {
+    if (warp < kFrontThreads / 32) {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kFrontRegs));
+      if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             const uint32_t stages = prm.stages, P = prm.sb.P;
@@ -590,7 +630,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                 }
             }
         }
-    } else if (warp == 1) {
+      } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA)
         if (lane == 0 && rank == 0) {
             constexpr uint32_t idesc = make_idesc(KIND, TILE_N, TILE_M * CG);
@@ -645,13 +685,15 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                 }
             }
         }
+      }
     } else {
         // ------------------------------------------------------------------ epilogue warps
         // Warp w may read TMEM lanes 32 * (w % 4) .. + 31; the two warps of one lane group take one half
         // of the tile's 32-column slabs each.  Per output: y = bias, then y = fma(c[a][q], acc[a], y) over
         // a = (p, polarity) ascending, two outputs per instruction on packed fp32 pairs.
-        const int et = threadIdx.x - 64;
-        const int ew = warp - 2;
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kEpiRegs));
+        const int et = threadIdx.x - kFrontThreads;
+        const int ew = warp - kFrontThreads / 32;
         const int lane_grp = warp & 3;
         constexpr int kColGroups = kEpiWarps / 4;
         constexpr int kSlabs = TILE_N / 32;
@@ -699,10 +741,19 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
             bias_next = fetch_bias(tile + num_units);                        // lands during this tile's work
             asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
 
+            // A warp's share of one accumulator set is kUnits TMEM loads (unit u = slab u / NPOL, polarity
+            // u % NPOL).  Up to NB of them are in registers at once: NB loads go out at the start, and the
+            // buffer freed by unit u - 1 takes the load of unit u - 1 + NB while unit u is scaled.  Once the last
+            // load has landed the set goes back to the MMA issuer.  (With one resident set per tile that moment
+            // is on the critical path, so there the last load goes out AHEAD of the wait that precedes unit u.)
             if constexpr (SEQ) {
                 // ---- one accumulator set per K-segment: running sums of the whole tile stay in registers
                 static_assert(!SEQ || kSlabsPerWarp * kColGroups == kSlabs, "SEQ needs TILE_N >= 64");
                 constexpr int kUnits = kSlabsPerWarp * NPOL;                // TMEM loads per segment and warp
+                constexpr int kBufMax = GENERIC ? 2 : (kEpiBufRegs - 32 * kSlabsPerWarp) / 32;
+                constexpr int NB = kUnits < kBufMax ? kUnits : kBufMax;
+                constexpr int kRel = kUnits <= NB ? 0 : kUnits - NB + 1;    // unit before which the set is released
+                static_assert(NB >= 2 || kUnits == 1, "needs two load buffers");
                 uint64_t y2[kSlabsPerWarp][16];
                 int q_lo[kSlabsPerWarp], q_hi[kSlabsPerWarp];
 #pragma unroll
@@ -720,28 +771,24 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                     if (ok) ok = mbar_wait(smem_u32(&hdr->tmem_full[cur_as]), cur_aph, abort_flag, prm.status, kWhereEpilogue);
                     if (!ok) continue;
                     tc_fence_after();
-                    const uint32_t t_row = tmem_base + (uint32_t(lane_grp * 32) << 16) + cur_as * acc_cols;
-                    // With two slabs of running sums per thread there are registers for a second load buffer, and
-                    // unit u + 1 is read while unit u is added; with four slabs the loads are taken one at a time.
-                    constexpr bool kAhead = kSlabsPerWarp <= 2;
-                    uint32_t ra[32], rb[kAhead ? 32 : 1];
-                    tc_ld32(t_row + uint32_t(slab0 * 32), ra);                       // unit 0 = (slab 0, polarity 0)
+                    const uint32_t t_row = tmem_base + (uint32_t(lane_grp * 32) << 16) + cur_as * acc_cols +
+                                           uint32_t(slab0 * 32);
+                    uint32_t buf[NB][32];
+#pragma unroll
+                    for (int u = 0; u < NB; u++) tc_ld32(t_row + uint32_t((u % NPOL) * TILE_N + (u / NPOL) * 32), buf[u]);
 #pragma unroll
                     for (int u = 0; u < kUnits; u++) {
                         const int sl = u / NPOL, pol = u % NPOL;
-                        uint32_t (&r)[32] = (kAhead && (u & 1)) ? reinterpret_cast<uint32_t (&)[32]>(rb) : ra;
                         tc_wait_ld();
-                        if (kAhead && u + 1 < kUnits)
-                            tc_ld32(t_row + uint32_t(((u + 1) % NPOL) * TILE_N + (slab0 + (u + 1) / NPOL) * 32),
-                                    (u & 1) ? ra : reinterpret_cast<uint32_t (&)[32]>(rb));
-                        else if (u + 1 == kUnits)
-                            release(cur_as);
+                        if (u == kRel) release(cur_as);
+                        if (u >= 1 && u - 1 + NB < kUnits)                           // buffer of unit u - 1 is free
+                            tc_ld32(t_row + uint32_t(((u - 1 + NB) % NPOL) * TILE_N + ((u - 1 + NB) / NPOL) * 32),
+                                    buf[(u - 1) % NB]);
                         const int a = p * NPOL + pol;
                         const int nf = n0 + (slab0 + sl) * 32;
-                        scale_add_unit<KIND, GENERIC>(y2[sl], r, a, Q, q_lo[sl], q_hi[sl], nf, tab_addr, nb_addr);
-                        if (GENERIC && prm.acc_dump && row < prm.M) dump_unit(prm.acc_dump, r, a, row, nf, prm.M, prm.N);
-                        if (!kAhead && u + 1 < kUnits)
-                            tc_ld32(t_row + uint32_t(((u + 1) % NPOL) * TILE_N + (slab0 + (u + 1) / NPOL) * 32), ra);
+                        scale_add_unit<KIND, GENERIC>(y2[sl], buf[u % NB], a, Q, q_lo[sl], q_hi[sl], nf, tab_addr, nb_addr);
+                        if (GENERIC && prm.acc_dump && row < prm.M)
+                            dump_unit(prm.acc_dump, buf[u % NB], a, row, nf, prm.M, prm.N);
                     }
                 }
                 if (ok && row < prm.M) {
@@ -749,14 +796,57 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                     for (int sl = 0; sl < kSlabsPerWarp; sl++) store_slab<GENERIC>(y2[sl], prm, row, n0 + (slab0 + sl) * 32);
                 }
             } else {
-                // ---- all accumulators of the tile resident: slab by slab, TMEM loads one unit ahead of the
-                // arithmetic; the set goes back to the MMA issuer as soon as the last load has landed
+                // ---- all accumulators of the tile resident
                 const uint32_t cur_as = as, cur_aph = aph;
                 if (++as == uint32_t(prm.acc_stages)) { as = 0; aph ^= 1; }
                 if (ok) ok = mbar_wait(smem_u32(&hdr->tmem_full[cur_as]), cur_aph, abort_flag, prm.status, kWhereEpilogue);
                 if (!ok) continue;                  // keep the named barriers balanced, do no more work
                 tc_fence_after();
                 const uint32_t t_row = tmem_base + (uint32_t(lane_grp * 32) << 16) + cur_as * acc_cols;
+                constexpr bool kEvenSplit = kSlabsPerWarp * kColGroups == kSlabs;
+                if (kEvenSplit && nacc == NPOL) {
+                    // one K-segment (the usual case): the unit count is a compile-time constant, outputs slab by slab
+                    constexpr int kUnits = kSlabsPerWarp * NPOL;
+                    constexpr int kBufMax = GENERIC ? 2 : kResidentBufs;
+                    constexpr int NB = kUnits < kBufMax ? kUnits : kBufMax;
+                    constexpr int kRel = kUnits <= NB ? 0 : kUnits - NB;
+                    static_assert(NB >= 2 || kUnits == 1, "needs two load buffers");
+                    const uint32_t t_warp = t_row + uint32_t(slab0 * 32);
+                    uint32_t buf[NB][32];
+#pragma unroll
+                    for (int u = 0; u < NB; u++) tc_ld32(t_warp + uint32_t((u % NPOL) * TILE_N + (u / NPOL) * 32), buf[u]);
+                    uint64_t y2[16];
+                    int q_lo = 0, q_hi = 0;
+#pragma unroll
+                    for (int u = 0; u < kUnits; u++) {
+                        const int sl = u / NPOL, pol = u % NPOL;
+                        const int c0 = (slab0 + sl) * 32, nf = n0 + c0;
+                        const bool refill = u >= 1 && u - 1 + NB < kUnits;
+                        const bool last_load = u - 1 + NB == kUnits - 1;
+                        if (refill && last_load)
+                            tc_ld32(t_warp + uint32_t(((u - 1 + NB) % NPOL) * TILE_N + ((u - 1 + NB) / NPOL) * 32),
+                                    buf[(u - 1) % NB]);
+                        tc_wait_ld();
+                        if (u == kRel) release(cur_as);
+                        if (refill && !last_load)
+                            tc_ld32(t_warp + uint32_t(((u - 1 + NB) % NPOL) * TILE_N + ((u - 1 + NB) / NPOL) * 32),
+                                    buf[(u - 1) % NB]);
+                        if (pol == 0) {
+                            q_lo = seg_of_column(nf, Q, nb_addr, lane);
+                            q_hi = GENERIC ? seg_of_column(min(nf + 31, prm.N - 1), Q, nb_addr, lane) : q_lo;
+                            scale_add_unit<KIND, GENERIC, true>(y2, buf[u % NB], pol, Q, q_lo, q_hi, nf, tab_addr, nb_addr,
+                                                                bias_addr + uint32_t(c0) * 4u);
+                        } else {
+                            scale_add_unit<KIND, GENERIC>(y2, buf[u % NB], pol, Q, q_lo, q_hi, nf, tab_addr, nb_addr);
+                        }
+                        if (GENERIC && prm.acc_dump && row < prm.M)
+                            dump_unit(prm.acc_dump, buf[u % NB], pol, row, nf, prm.M, prm.N);
+                        if (pol == NPOL - 1 && row < prm.M) store_slab<GENERIC>(y2, prm, row, nf);
+                    }
+                    continue;
+                }
+                // several K-segments kept resident, or a tile narrower than the warps' column split: the unit
+                // count is a run-time value; loads run one unit ahead of the arithmetic
                 const int my_slabs = max(0, min(kSlabsPerWarp, kSlabs - slab0));
                 const int units = my_slabs * nacc;                          // (slab, accumulator) pairs of this warp
 
