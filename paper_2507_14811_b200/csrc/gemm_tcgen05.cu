@@ -52,6 +52,8 @@ constexpr int kMaxStages = 8;
 constexpr int kTmemCols = 512;
 constexpr uint32_t kSmemBudget = 227 * 1024;
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s
+constexpr uint32_t kStageBytesPerWarp = 32 * 64;       // one 32 x 32 bf16 output block per epilogue warp
+constexpr uint32_t kStageBytes = kEpiWarps * kStageBytesPerWarp;
 constexpr int kMaxFactorTable = 2048;                  // (K-segments x polarities) x N-segments factors in shared memory
 
 struct KernelParams {
@@ -465,14 +467,71 @@ __device__ __forceinline__ void dump_unit(void *acc_dump, const uint32_t (&r)[32
         if (nf + j < N) dump[j] = r[j];
 }
 
+// 32 fp32 outputs (16 packed pairs) -> 32 bf16 (16 words), round to nearest even
+__device__ __forceinline__ void pack_bf16(const uint64_t (&y2)[16], uint32_t (&h)[16])
+{
+#pragma unroll
+    for (int j = 0; j < 16; j++) {
+        float lo, hi;
+        unpack_f32x2(y2[j], lo, hi);
+        __nv_bfloat162 v2 = __floats2bfloat162_rn(lo, hi);
+        h[j] = *reinterpret_cast<uint32_t *>(&v2);
+    }
+}
+
+// Where the production variant's output goes: the warp's 32 x 32 bf16 block is staged in shared memory and
+// written by one TMA store (whole 64-byte row pieces per request instead of one request per lane and piece).
+struct YOut {
+    const CUtensorMap *tm;   // Y as [M, N] bf16, box 32 x 32, 64-byte swizzle
+    uint32_t stage;          // this warp's 2 KiB staging buffer (shared address, 1 KiB aligned)
+    int lane;
+    int row0;                // first row of the warp's 32-row block
+};
+
+// Lane l holds row row0 + l of the block as 16 words h (32 bf16, columns col .. col + 31).  Rows beyond M and
+// columns beyond N are clipped by the tensor map; a block entirely outside is skipped.  The previous store of
+// this warp must have finished READING the staging buffer before it is overwritten; lane 0 issued it, so lane 0
+// waits for it.
+__device__ __forceinline__ void tma_store_block(const uint32_t (&h)[16], const YOut &yo, int col, int M, int N)
+{
+    if (yo.row0 >= M || col >= N) return;               // warp-uniform
+    if (yo.lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+    __syncwarp();
+    const uint32_t row_addr = yo.stage + uint32_t(yo.lane) * 64u;
+    const uint32_t sw = (uint32_t(yo.lane) >> 1) & 3u;  // 64-byte swizzle: 16-byte piece index ^ bits 7-8 of the address
+#pragma unroll
+    for (int c = 0; c < 4; c++)
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + ((uint32_t(c) ^ sw) << 4)),
+                     "r"(h[4 * c]), "r"(h[4 * c + 1]), "r"(h[4 * c + 2]), "r"(h[4 * c + 3]) : "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+    if (yo.lane == 0) {
+        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                     ::"l"(reinterpret_cast<uint64_t>(yo.tm)), "r"(col), "r"(yo.row0), "r"(yo.stage) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    }
+}
+// before the CTA's shared memory goes away (all lanes may call; lane 0 issued the stores)
+__device__ __forceinline__ void tma_store_drain(const YOut &yo)
+{
+    if (yo.lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+    __syncwarp();
+}
+
 // Converts and stores the 32 outputs y of row `row`, columns nf .. nf + 31, in 16-byte chunks (8 bf16 or
 // 4 fp32).  N is a multiple of 8, so a chunk is entirely inside or outside the matrix; two adjacent chunks go
 // out as one 32-byte store when the rows of Y are 32-byte aligned.
+// The production variant (GENERIC = false) is called by all 32 lanes of the warp together and writes through
+// yo; the generic one writes row `row` (< M) from registers.
 template <bool GENERIC, typename Params>
-__device__ __forceinline__ void store_slab(const uint64_t (&y2)[16], const Params &prm, int row, int nf)
+__device__ __forceinline__ void store_slab(const uint64_t (&y2)[16], const Params &prm, int row, int nf, const YOut &yo)
 {
     const int nvalid = prm.N - nf;                       // valid columns of this slab, may exceed 32
-    if (GENERIC && prm.y_is_f32) {
+    if (!GENERIC) {
+        uint32_t h[16];
+        pack_bf16(y2, h);
+        tma_store_block(h, yo, nf, prm.M, prm.N);
+    } else if (prm.y_is_f32) {
         float *dst = static_cast<float *>(prm.Y) + size_t(row) * prm.ldy + nf;
 #pragma unroll
         for (int c = 0; c < 4; c++) {                    // 8 columns = 32 bytes
@@ -524,16 +583,18 @@ template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ>
 // 384 threads = 12 warps, 3 on each SM sub-partition with 16 K registers: 168 registers per thread at launch
 __global__ void __launch_bounds__(kThreads, 1)
 segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_constant__ CUtensorMap tm_a_neg,
-                     const __grid_constant__ CUtensorMap tm_b, const KernelParams prm)
+                     const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_y,
+                     const KernelParams prm)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    // layout: [ring: stages x (NPOL A tiles of 16 KiB, B part of B_ROWS*128 B)] [scales] [header]
+    // layout: [ring: stages x (NPOL A tiles of 16 KiB, B part of B_ROWS*128 B)] [output staging] [scales] [header]
     constexpr int B_ROWS = TILE_N / CG;                  // weight rows this CTA loads per K-block
     constexpr uint32_t a_bytes = TILE_M * BLOCK_K;
     constexpr uint32_t b_bytes = B_ROWS * BLOCK_K;
     constexpr uint32_t stage_bytes = NPOL * a_bytes + b_bytes;
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    float *sh_bias = reinterpret_cast<float *>(smem + size_t(prm.stages) * stage_bytes);    // [TILE_N], per tile
+    uint8_t *sh_stage = smem + size_t(prm.stages) * stage_bytes;      // 1 KiB aligned: stages are multiples of 1 KiB
+    float *sh_bias = reinterpret_cast<float *>(sh_stage + (GENERIC ? 0 : kStageBytes));     // [TILE_N], per tile
     float *sh_tab = sh_bias + TILE_N;                                                       // [nacc][Q], per launch
     int *sh_nb = reinterpret_cast<int *>(sh_tab + prm.nacc * prm.sb.Q);                     // [Q + 1]
     SharedHeader *hdr = reinterpret_cast<SharedHeader *>(reinterpret_cast<uint8_t *>(sh_bias) +
@@ -550,6 +611,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_a_pos)) : "memory");
         if (NPOL == 2) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_a_neg)) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_b)) : "memory");
+        if (!GENERIC) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_y)) : "memory");
     }
     if (threadIdx.x == 0) {
         for (int s = 0; s < prm.stages; s++) {
@@ -729,12 +791,14 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
         }
         for (int i = et; i <= Q; i += kEpiThreads) sh_nb[i] = prm.sb.nb[i];
 
+        YOut yo{&tm_y, smem_u32(sh_stage) + uint32_t(ew) * kStageBytesPerWarp, lane, 0};
         uint32_t as = 0, aph = 0;
         bool ok = true;
         for (int tile = unit; tile < num_tiles; tile += num_units) {
             const int m0 = (tile / prm.num_n_tiles) * (TILE_M * CG) + int(rank) * TILE_M;
             const int n0 = (tile % prm.num_n_tiles) * TILE_N;
             const int row = m0 + lane_grp * 32 + lane;
+            yo.row0 = m0 + lane_grp * 32;
 
             asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // previous tile's readers are done
             if (et < TILE_N) sh_bias[et] = bias_next;
@@ -791,9 +855,10 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                             dump_unit(prm.acc_dump, buf[u % NB], a, row, nf, prm.M, prm.N);
                     }
                 }
-                if (ok && row < prm.M) {
+                if (ok && (!GENERIC || row < prm.M)) {
 #pragma unroll
-                    for (int sl = 0; sl < kSlabsPerWarp; sl++) store_slab<GENERIC>(y2[sl], prm, row, n0 + (slab0 + sl) * 32);
+                    for (int sl = 0; sl < kSlabsPerWarp; sl++)
+                        store_slab<GENERIC>(y2[sl], prm, row, n0 + (slab0 + sl) * 32, yo);
                 }
             } else {
                 // ---- all accumulators of the tile resident
@@ -841,7 +906,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                         }
                         if (GENERIC && prm.acc_dump && row < prm.M)
                             dump_unit(prm.acc_dump, buf[u % NB], pol, row, nf, prm.M, prm.N);
-                        if (pol == NPOL - 1 && row < prm.M) store_slab<GENERIC>(y2, prm, row, nf);
+                        if (pol == NPOL - 1 && (!GENERIC || row < prm.M)) store_slab<GENERIC>(y2, prm, row, nf, yo);
                     }
                     continue;
                 }
@@ -874,7 +939,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                     if (++c_a < nacc) return;
                     c_a = 0;
                     c_sl++;
-                    if (row < prm.M) store_slab<GENERIC>(y2, prm, row, nf);      // last accumulator of the slab
+                    if (!GENERIC || row < prm.M) store_slab<GENERIC>(y2, prm, row, nf, yo);   // last accumulator of the slab
                 };
                 if (units == 0) {
                     release(cur_as);
@@ -894,6 +959,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                 }
             }
         }
+        if (!GENERIC) tma_store_drain(yo);          // the staging buffers are read before the CTA may exit
     }
 
     tc_fence_before();
@@ -944,19 +1010,37 @@ bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, in
     return r == CUDA_SUCCESS;
 }
 
+// 2-D map over the bf16 output [M, N] with row pitch ldy (elements): box = 32 columns x 32 rows, 64-byte
+// swizzle (the layout tma_store_block writes).  Needs a 16-byte aligned base and pitch.
+bool make_map_y(CUtensorMap *map, void *base, int64_t M, int64_t N, int64_t ldy)
+{
+    EncodeFn enc = get_encode_fn();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {cuuint64_t(N), cuuint64_t(M)};
+    cuuint64_t strides[1] = {cuuint64_t(ldy) * 2};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 int g_tune_tile_n = 0, g_tune_stages = 0, g_tune_cta_group = 0, g_tune_seq = 0;
 
 template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ>
 sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cudaStream_t st)
 {
     constexpr int B_ROWS = TILE_N / CG;
-    CUtensorMap ta, tn, tb;
+    CUtensorMap ta, tn, tb, ty;
+    if (GENERIC) ty = CUtensorMap{};                // unused by the generic variant
+    else if (!make_map_y(&ty, g.Y, g.M, g.N, g.ldy)) return SQ_ERR_CUDA;
     if (!make_map(&ta, g.a_pos, g.M, g.K, g.lda, TILE_M)) return SQ_ERR_CUDA;
     if (!make_map(&tn, g.a_neg ? g.a_neg : g.a_pos, g.M, g.K, g.lda, TILE_M)) return SQ_ERR_CUDA;
     if (!make_map(&tb, g.b, g.N, g.K, g.ldb, B_ROWS)) return SQ_ERR_CUDA;
 
     const uint32_t stage_bytes = NPOL * TILE_M * BLOCK_K + B_ROWS * BLOCK_K;
-    const uint32_t tail = epi_table_bytes(prm.nacc, prm.sb.Q, TILE_N) + sizeof(SharedHeader);
+    const uint32_t tail = (GENERIC ? 0u : kStageBytes) + epi_table_bytes(prm.nacc, prm.sb.Q, TILE_N) + sizeof(SharedHeader);
     int stages = int((kSmemBudget - 1024 - tail) / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (g_tune_stages >= 2 && g_tune_stages < stages) stages = g_tune_stages;
@@ -1002,7 +1086,7 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
     }
     const int grid = (tiles < units ? tiles : units) * CG;
     cfg.gridDim = dim3(unsigned(grid));
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ta, tn, tb, prm);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ta, tn, tb, ty, prm);
     count_launch();
     const cudaError_t e2 = cudaGetLastError();
     if (e != cudaSuccess || e2 != cudaSuccess) { note_cuda_error(e != cudaSuccess ? e : e2); return SQ_ERR_CUDA; }
@@ -1013,6 +1097,8 @@ template <int KIND, int NPOL, int CG>
 sq_status launch_tile(const GemmArgs &g, KernelParams &prm, int tile_n, bool seq, int sm_count, cudaStream_t st)
 {
     bool dbg = prm.y_is_f32 || prm.acc_dump != nullptr;
+    // the production variant writes Y with TMA stores: 16-byte aligned base and row pitch
+    dbg = dbg || reinterpret_cast<uintptr_t>(g.Y) % 16 != 0 || (size_t(g.ldy) * 2) % 16 != 0;
     for (int q = 1; q < prm.sb.Q; q++) dbg = dbg || (prm.sb.nb[q] % 32 != 0);
     if (seq) {      // sequential K-segments: one tile width per polarity count
         constexpr int TN = NPOL == 1 ? 256 : 128;
