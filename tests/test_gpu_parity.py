@@ -231,6 +231,46 @@ def test_strided_output_and_code_matrices():
     check_bf16_output(Y.contiguous(), res.y64, res.y_abs, 2)
 
 
+@pytest.mark.parametrize("col0,pitch", [(0, 328), (8, 328), (16, 328), (4, 328), (0, 324), (24, 1024)])
+@pytest.mark.parametrize("dual", [True, False])
+def test_output_alignment_and_pitch_variants(col0, pitch, dual):
+    """The bf16 output goes out through TMA stores, which need Y and its pitch 16-byte aligned: the interface
+    demands exactly that, so a column offset of 4 (8 bytes) or a pitch of 324 (648 bytes) is refused, and
+    every accepted placement (16-byte but not 32-byte aligned included) writes exactly the M x N window:
+    300 rows end inside a 32-row block, 296 columns end inside a 32-column slab."""
+    M, K, N = 300, 384, 296
+    spec = custom_spec(f"align{col0}_{pitch}_{int(dual)}", M, K, N, [0, K], [0, 160, N], dual, "int8", seed=77)
+    data = WL.make_layer(spec)
+    s_pos, s_neg, s_w, Wq, _ = oracle_scales(data)
+    layer = SegQuantLinear(data.W, data.bias, spec.kb, spec.nb, dual, "int8", DEV)
+    layer.calibrate(data.X_cal)
+    wide = torch.full((M + 2, pitch), -3.0, dtype=torch.bfloat16, device=DEV)
+    Y = wide[1:M + 1, col0:col0 + N]
+    c_pos, c_neg = B.segquant_quantize_act(data.X.to(DEV), layer.seg, layer.s_pos, layer.s_neg, "int8")
+    def call():
+        if dual:
+            B.segquant_dualscale_gemm(c_pos, c_neg, layer.Wq, layer.seg, "int8", layer.s_pos, layer.s_neg, layer.s_w,
+                                      layer.bias, layer.workspace, Y=Y)
+        else:
+            B.segquant_seglinear_gemm(c_pos, layer.Wq, layer.seg, "int8", layer.s_pos, layer.s_w, layer.bias,
+                                      layer.workspace, Y=Y)
+    if (col0 * 2) % 16 or (pitch * 2) % 16:
+        with pytest.raises(Exception, match="SQ_ERR_ALIGN"):
+            call()
+        torch.cuda.synchronize()
+        assert torch.all(wide == -3.0)
+        return
+    call()
+    layer.check_status()
+    torch.cuda.synchronize()
+    outside = wide.clone()
+    outside[1:M + 1, col0:col0 + N] = -3.0
+    assert torch.all(outside == -3.0), "wrote outside the M x N window"
+    res = O.layer_forward(to_f32_np(data.X), Wq, O.SegTable(spec.kb, spec.nb), s_pos, s_neg if dual else None, s_w,
+                          to_f32_np(data.bias))
+    check_bf16_output(Y.contiguous(), res.y64, res.y_abs, 2 if dual else 1)
+
+
 @pytest.mark.parametrize("code", ["int8", "e4m3"])
 @pytest.mark.parametrize("dual", [True, False])
 def test_quantizer_codes_equal_the_division_definition_on_adversarial_values(code, dual):
