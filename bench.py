@@ -446,9 +446,11 @@ def run_ours(args):
     layer_sets = [layers] + [[bl.device_copy() for bl in layers] for _ in range(n_sets - 1)]
 
     barrier()
+    sampler.start()                            # SM clock and throttle reasons over both timed passes
     step_ms, step_mode, launches = time_steps_back_to_back(layer_sets, args.steps, args.warmup)
     barrier()
-    q_ms, g_ms, clocks = time_workload(layers, args.steps, args.warmup, flush, sampler)
+    q_ms, g_ms, _ = time_workload(layers, args.steps, args.warmup, flush, None)
+    clocks = sampler.stop()
     barrier()
     for bl in layers:
         bl.layer.check_status()
