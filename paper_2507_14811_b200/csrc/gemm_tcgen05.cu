@@ -643,6 +643,12 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     tc_fence_after();
     const uint32_t tmem_base = hdr->tmem_base;
     const int acc_cols = (SEQ ? NPOL : prm.nacc) * TILE_N;     // TMEM columns of one accumulator set
+    // A dual 256-wide tile (one K-segment) fills TMEM, so there is one accumulator set and the tensor pipe would
+    // idle during the epilogue up to the set's release.  Instead the two polarities are released SEPARATELY
+    // (barrier tmem_empty[0] = positive accumulator free, tmem_empty[1] = negative one): the epilogue reads all
+    // positive columns first, and the MMA issuer starts the next tile with positive-only MMAs for as many
+    // K-blocks as the ring can hold back (stages - 1), then catches up on the negative ones.
+    constexpr bool kSplitRel = NPOL == 2 && TILE_N == 256 && !SEQ && !GENERIC;
 
     // The producer and the MMA issuer are single threads: their loops are kept to a few dozen
     // instructions per K-block (ring slot and phase advance incrementally, descriptors by addition).
@@ -704,6 +710,55 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
             uint32_t s = 0, ph = 0, as = 0, aph = 0;
             bool ok = true;
             for (int tile = unit; tile < num_tiles && ok; tile += num_units) {
+                if constexpr (kSplitRel) {
+                    constexpr uint64_t kANegDesc = uint64_t(a_bytes) >> 4;
+                    const int k_end = prm.sb.kb[1];
+                    const uint32_t nkb = uint32_t((k_end + BLOCK_K - 1) / BLOCK_K);
+                    const uint32_t ahead = nkb < stages - 1 ? nkb : stages - 1;
+                    if (!mbar_wait(smem_u32(&hdr->tmem_empty[0]), aph ^ 1, abort_flag, prm.status, kWhereMmaTmem)) break;
+                    tc_fence_after();
+                    // positive-only MMAs of the first `ahead` K-blocks; their ring slots stay taken
+                    uint32_t s1 = s, ph1 = ph;
+                    int k = 0;
+                    for (uint32_t j = 0; j < ahead && ok; j++, k += BLOCK_K) {
+                        if (!mbar_wait(full0 + 8 * s1, ph1, abort_flag, prm.status, kWhereMmaFull)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint64_t da = desc0 + s1 * kStageDesc;
+                        const int rem = k_end - k;
+                        const int nk = rem >= BLOCK_K ? BLOCK_K / MMA_K : (rem + MMA_K - 1) / MMA_K;
+                        issue_kblock<KIND, 1, TILE_N, CG>(tmem_base, da, da + kBDesc, idesc, nk, j > 0 ? 1u : 0u);
+                        if (++s1 == stages) { s1 = 0; ph1 ^= 1; }
+                    }
+                    if (!ok) break;
+                    if (!mbar_wait(smem_u32(&hdr->tmem_empty[1]), aph ^ 1, abort_flag, prm.status, kWhereMmaTmem)) break;
+                    tc_fence_after();
+                    // the negative MMAs of the same K-blocks, each freeing its slot
+                    k = 0;
+                    for (uint32_t j = 0; j < ahead; j++, k += BLOCK_K) {
+                        const uint64_t da = desc0 + s * kStageDesc;
+                        const int rem = k_end - k;
+                        const int nk = rem >= BLOCK_K ? BLOCK_K / MMA_K : (rem + MMA_K - 1) / MMA_K;
+                        issue_kblock<KIND, 1, TILE_N, CG>(tmem_base + TILE_N, da + kANegDesc, da + kBDesc, idesc, nk,
+                                                          j > 0 ? 1u : 0u);
+                        tc_commit<CG>(empty0 + 8 * s);
+                        if (++s == stages) { s = 0; ph ^= 1; }
+                    }
+                    // the rest of the tile: both polarities per K-step
+                    for (; k < k_end; k += BLOCK_K) {
+                        if (!mbar_wait(full0 + 8 * s, ph, abort_flag, prm.status, kWhereMmaFull)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint64_t da = desc0 + s * kStageDesc;
+                        const int rem = k_end - k;
+                        const int nk = rem >= BLOCK_K ? BLOCK_K / MMA_K : (rem + MMA_K - 1) / MMA_K;
+                        issue_kblock<KIND, NPOL, TILE_N, CG>(tmem_base, da, da + kBDesc, idesc, nk, 1u);
+                        tc_commit<CG>(empty0 + 8 * s);
+                        if (++s == stages) { s = 0; ph ^= 1; }
+                    }
+                    if (!ok) break;
+                    tc_commit<CG>(smem_u32(&hdr->tmem_full[0]));
+                    aph ^= 1;
+                    continue;
+                }
                 if (!SEQ) {
                     if (!mbar_wait(smem_u32(&hdr->tmem_empty[as]), aph ^ 1, abort_flag, prm.status, kWhereMmaTmem)) {
                         ok = false;
@@ -869,6 +924,37 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                 tc_fence_after();
                 const uint32_t t_row = tmem_base + (uint32_t(lane_grp * 32) << 16) + cur_as * acc_cols;
                 constexpr bool kEvenSplit = kSlabsPerWarp * kColGroups == kSlabs;
+                if constexpr (kSplitRel) {
+                    // four slabs per warp: all positive units first (then the positive accumulator goes back),
+                    // negative units as registers come free (then the negative one); five units live at most
+                    static_assert(!kSplitRel || kSlabsPerWarp == 4, "split release: 256-wide tile, 8 epilogue warps");
+                    const uint32_t t_pos = t_row + uint32_t(slab0 * 32), t_neg = t_pos + uint32_t(TILE_N);
+                    uint32_t pb[4][32], nbuf[4][32];
+                    uint64_t y2[16];
+#pragma unroll
+                    for (int sl = 0; sl < 4; sl++) tc_ld32(t_pos + uint32_t(sl * 32), pb[sl]);
+                    tc_wait_ld();
+                    release(0);
+                    tc_ld32(t_neg, nbuf[0]);
+                    tc_ld32(t_neg + 32u, nbuf[1]);
+#pragma unroll
+                    for (int sl = 0; sl < 4; sl++) {
+                        const int c0 = (slab0 + sl) * 32, nf = n0 + c0;
+                        const int q = seg_of_column(nf, Q, nb_addr, lane);
+                        scale_add_unit<KIND, false, true>(y2, pb[sl], 0, Q, q, q, nf, tab_addr, nb_addr,
+                                                          bias_addr + uint32_t(c0) * 4u);
+                        if (sl == 0) tc_wait_ld();
+                        scale_add_unit<KIND, false>(y2, nbuf[sl], 1, Q, q, q, nf, tab_addr, nb_addr);
+                        store_slab<GENERIC>(y2, prm, row, nf, yo);
+                        if (sl == 0) {                        // registers of slab 0 are free: the last two negative units
+                            tc_ld32(t_neg + 64u, nbuf[2]);
+                            tc_ld32(t_neg + 96u, nbuf[3]);
+                            tc_wait_ld();
+                            release(1);
+                        }
+                    }
+                    continue;
+                }
                 if (kEvenSplit && nacc == NPOL) {
                     // one K-segment (the usual case): the unit count is a compile-time constant, outputs slab by slab
                     constexpr int kUnits = kSlabsPerWarp * NPOL;
