@@ -626,6 +626,10 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    // Every thread arrives at the cluster barrier now (thread 0 after its barrier initialisation) and waits for it
+    // only after the TMEM allocation below, so the barrier's latency overlaps the allocation.
+    __syncwarp();
+    if (CG == 2) asm volatile("barrier.cluster.arrive.release;" ::: "memory");
     if (warp == 1) {
         if (CG == 1) {
             asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -639,7 +643,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     }
     tc_fence_before();
     __syncthreads();
-    if (CG == 2) cluster_sync_all();          // the peer's barriers are initialised before anyone signals them
+    if (CG == 2) asm volatile("barrier.cluster.wait.acquire;" ::: "memory");   // the peer's barriers are initialised
     tc_fence_after();
     const uint32_t tmem_base = hdr->tmem_base;
     const int acc_cols = (SEQ ? NPOL : prm.nacc) * TILE_N;     // TMEM columns of one accumulator set
