@@ -555,8 +555,8 @@ def run_ours(args):
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the GEMM launches of one step, from the ncu
 # capture summarised in profiles/gemm_pair_and_quantize_dit_xl2_sd3_mmdit.md; None = not captured for that workload.
-GEMM_DRAM_TRAFFIC = {"dit_xl2": 12770816 + 22784 + 24238848 + 0,
-                     "sd3_mmdit": 41511936 + 39289600 + 23185664 + 56704512 + 123792640 + 13555712}
+GEMM_DRAM_TRAFFIC = {"dit_xl2": 12765696 + 38912 + 24238592 + 1536,
+                     "sd3_mmdit": 41490944 + 38836736 + 23211008 + 56874752 + 123385344 + 13977600}
 
 
 # ------------------------------------------------------------------------------------ reference arm
