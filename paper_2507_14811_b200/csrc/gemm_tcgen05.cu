@@ -13,10 +13,10 @@
 //               accumulator in TMEM
 //   warps 2, 3  idle: they fill the first warpgroup, which hands most of its registers to the others
 //   warps 4..11 epilogue: tcgen05.ld of the accumulators of a 32-column slab, y = bias + sum over
-//               (segment, polarity) of factor * accumulator in fp32, -> bf16 / fp32, written from
-//               registers with 32-byte stores (every store covers whole 32-byte sectors of Y)
-// Registers: the kernel starts with 168 per thread; warps 0..3 drop to 72 (setmaxnreg.dec) and the epilogue
-// warps rise to 216 (setmaxnreg.inc): 128 x 72 + 256 x 216 = 384 x 168, the CTA's allocation.  The
+//               (segment, polarity) of factor * accumulator in fp32, -> bf16 (32 x 32 blocks staged in
+//               shared memory and written by TMA stores) or fp32 / unaligned output (plain stores)
+// Registers: the kernel starts with 168 per thread; warps 0..3 drop to 56 (setmaxnreg.dec) and the epilogue
+// warps rise to 224 (setmaxnreg.inc): 128 x 56 + 256 x 224 = 384 x 168, the CTA's allocation.  The
 // epilogue uses them to hold up to six 32-column accumulator loads at once, so that a tile's accumulators
 // are back with the MMA issuer early in the epilogue.
 // One K-segment: the npol accumulators (128 lanes x TILE_N columns each) of a tile stay in TMEM until the
