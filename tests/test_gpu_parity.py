@@ -187,6 +187,82 @@ def test_pipelined_host_call_equals_the_plain_one(chunks):
     check_bf16_output(Y_pipe, res.y64, res.y_abs, 4)
 
 
+def _codes_and_output_buffers(spec):
+    c_pos = B.new_codes(spec.M, spec.K, DEV)
+    c_neg = B.new_codes(spec.M, spec.K, DEV) if spec.dual else None
+    return c_pos, c_neg
+
+
+def test_back_to_back_calls_on_shared_code_buffers_do_not_race():
+    """Four quantize -> GEMM rounds on different inputs, issued without any synchronisation, all through the SAME
+    code matrices: the launches overlap (programmatic dependent launch), yet every round's output must be the one
+    of its own input, i.e. no quantize pass may overwrite codes that the previous GEMM is still reading."""
+    spec = custom_spec("b2b", 2300, 512, 768, [0, 512], [0, 256, 768], True, "int8", seed=11)
+    data = WL.make_layer(spec)
+    s_pos, s_neg, s_w, Wq, _ = oracle_scales(data)
+    layer = SegQuantLinear(data.W, data.bias, spec.kb, spec.nb, True, "int8", DEV)
+    layer.calibrate(data.X_cal)
+    rounds = 4
+    Xs = [torch.roll(data.X, shifts=17 * r, dims=0) * (1.0 + 0.25 * r) for r in range(rounds)]
+    Xd = [x.to(DEV) for x in Xs]
+    Ys = [torch.empty((spec.M, spec.N), dtype=torch.bfloat16, device=DEV) for _ in range(rounds)]
+    c_pos, c_neg = _codes_and_output_buffers(spec)
+    torch.cuda.synchronize()
+    for r in range(rounds):
+        B.segquant_quantize_act(Xd[r], layer.seg, layer.s_pos, layer.s_neg, "int8", 0, c_pos, c_neg)
+        B.segquant_dualscale_gemm(c_pos, c_neg, layer.Wq, layer.seg, "int8", layer.s_pos, layer.s_neg, layer.s_w,
+                                  layer.bias, layer.workspace, Y=Ys[r])
+    layer.check_status()
+    torch.cuda.synchronize()
+    rows = np.arange(0, spec.M, 37)
+    for r in range(rounds):
+        res = O.layer_forward(to_f32_np(Xs[r])[rows], Wq, O.SegTable(spec.kb, spec.nb), s_pos, s_neg, s_w,
+                              to_f32_np(data.bias))
+        check_bf16_output(Ys[r][torch.as_tensor(rows, device=DEV)], res.y64, res.y_abs, 2)
+
+
+def test_calls_can_be_captured_in_a_cuda_graph_and_replayed():
+    """quantize -> GEMM captured once into a CUDA graph (the calls allocate nothing and query nothing that a
+    capture forbids); two replays on changed input contents give the outputs of eager calls."""
+    spec = custom_spec("graph", 700, 384, 520, [0, 128, 384], [0, 256, 520], True, "int8", seed=12)
+    data = WL.make_layer(spec)
+    layer = SegQuantLinear(data.W, data.bias, spec.kb, spec.nb, True, "int8", DEV)
+    layer.calibrate(data.X_cal)
+    Xd = data.X.to(DEV)
+    X_in = Xd.clone()
+    c_pos, c_neg = _codes_and_output_buffers(spec)
+    Y = torch.empty((spec.M, spec.N), dtype=torch.bfloat16, device=DEV)
+
+    def calls():
+        B.segquant_quantize_act(X_in, layer.seg, layer.s_pos, layer.s_neg, "int8", 0, c_pos, c_neg)
+        B.segquant_dualscale_gemm(c_pos, c_neg, layer.Wq, layer.seg, "int8", layer.s_pos, layer.s_neg, layer.s_w,
+                                  layer.bias, layer.workspace, Y=Y)
+
+    calls()                                            # eager: loads the kernels, sets their attributes
+    torch.cuda.synchronize()
+    Y_eager0 = Y.clone()
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream, capture_error_mode="relaxed"):
+            calls()
+    torch.cuda.current_stream().wait_stream(stream)
+    Y.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(Y, Y_eager0)
+    X_in.copy_(torch.flip(Xd, dims=[0]) * 0.5)
+    graph.replay()
+    torch.cuda.synchronize()
+    Y_graph1 = Y.clone()
+    calls()
+    layer.check_status()
+    torch.cuda.synchronize()
+    assert torch.equal(Y_graph1, Y)
+    assert not torch.equal(Y_graph1, Y_eager0)
+
+
 def _random_case(i):
     rs = np.random.default_rng(1000 + i)
     P = int(rs.choice([1, 1, 2, 3, 5, 9, 17]))
