@@ -221,6 +221,37 @@ def test_back_to_back_calls_on_shared_code_buffers_do_not_race():
         check_bf16_output(Ys[r][torch.as_tensor(rows, device=DEV)], res.y64, res.y_abs, 2)
 
 
+@pytest.mark.parametrize("wl,idx", [("dit_xl2", 0), ("dit_xl2", 1), ("sdxl_skip", 0)])
+def test_repeated_full_size_launches_are_bitwise_identical(wl, idx):
+    """Forty back-to-back launches of a full-size benchmark layer (many tiles per CTA pair, so every hand-over
+    between the MMA issuer and the epilogue warps happens thousands of times) give the same bytes every time."""
+    spec = WL.WORKLOADS[wl][idx]
+    data = WL.make_layer(spec)
+    layer = SegQuantLinear(data.W, data.bias, spec.kb, spec.nb, spec.dual, spec.code, DEV)
+    layer.calibrate(data.X_cal)
+    c_pos, c_neg = B.segquant_quantize_act(data.X.to(DEV), layer.seg, layer.s_pos, layer.s_neg, spec.code)
+    Ys = [torch.empty((spec.M, spec.N), dtype=torch.bfloat16, device=DEV) for _ in range(3)]
+
+    def gemm(Y):
+        if spec.dual:
+            B.segquant_dualscale_gemm(c_pos, c_neg, layer.Wq, layer.seg, spec.code, layer.s_pos, layer.s_neg,
+                                      layer.s_w, layer.bias, layer.workspace, Y=Y)
+        else:
+            B.segquant_seglinear_gemm(c_pos, layer.Wq, layer.seg, spec.code, layer.s_pos, layer.s_w, layer.bias,
+                                      layer.workspace, Y=Y)
+    gemm(Ys[0])
+    torch.cuda.synchronize()
+    for r in range(20):
+        gemm(Ys[1])
+        gemm(Ys[2])
+        if r % 5 == 4:
+            torch.cuda.synchronize()
+            assert torch.equal(Ys[1], Ys[0]) and torch.equal(Ys[2], Ys[0]), f"launch {2 * r} differs"
+            Ys[1].zero_()
+            Ys[2].zero_()
+    layer.check_status()
+
+
 def test_calls_can_be_captured_in_a_cuda_graph_and_replayed():
     """quantize -> GEMM captured once into a CUDA graph (the calls allocate nothing and query nothing that a
     capture forbids); two replays on changed input contents give the outputs of eager calls."""
