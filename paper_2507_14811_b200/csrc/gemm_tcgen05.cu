@@ -8,10 +8,11 @@
 // kernel with one CTA per 128-row tile (used when M <= 128).
 //   warp 0      TMA producer (one lane): per 128-byte K-block, one tile of each activation code
 //               matrix and this CTA's part of ONE weight tile into a shared-memory ring
-//   warp 1      tcgen05.mma issuer (one lane, leader CTA only): for every 32-byte K-step one MMA per
-//               polarity against the same weight tile; every (K-segment, polarity) has its own
-//               accumulator in TMEM
-//   warps 2, 3  idle: they fill the first warpgroup, which hands most of its registers to the others
+//   warp 1      tcgen05.mma issuer (one lane, leader CTA only): for every 32-byte K-step one MMA of the
+//               positive (or only) code matrix against the weight tile; every (K-segment, polarity) has
+//               its own accumulator in TMEM
+//   warp 2      dual layers: the same for the negative code matrix, against the SAME weight tile
+//   warp 3      idle: it fills the first warpgroup, which hands most of its registers to the others
 //   warps 4..11 epilogue: tcgen05.ld of the accumulators of a 32-column slab, y = bias + sum over
 //               (segment, polarity) of factor * accumulator in fp32, -> bf16 (32 x 32 blocks staged in
 //               shared memory and written by TMA stores) or fp32 / unaligned output (plain stores)
@@ -616,10 +617,10 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     if (threadIdx.x == 0) {
         for (int s = 0; s < prm.stages; s++) {
             mbar_init(smem_u32(&hdr->full[s]), 1);
-            mbar_init(smem_u32(&hdr->empty[s]), 1);
+            mbar_init(smem_u32(&hdr->empty[s]), NPOL);          // one arrival per MMA-issuing thread
         }
         for (int s = 0; s < 2; s++) {
-            mbar_init(smem_u32(&hdr->tmem_full[s]), 1);
+            mbar_init(smem_u32(&hdr->tmem_full[s]), NPOL);
             mbar_init(smem_u32(&hdr->tmem_empty[s]), CG * kEpiWarps);
         }
         hdr->abort_flag = 0;
@@ -702,69 +703,29 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                 }
             }
         }
-      } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer (leader CTA)
+      } else if (warp == 1 || (NPOL == 2 && warp == 2)) {
+        // ------------------------------------------------------------------ MMA issuers (leader CTA)
+        // One thread per polarity: warp 1 issues the MMAs of the positive code matrix, warp 2 (dual layers)
+        // those of the negative one, each into its own accumulators.  A tcgen05.mma keeps its issuing thread
+        // busy for about 70 cycles, more than a 128-column MMA occupies the tensor pipe, so one thread cannot
+        // feed the pipe for narrow dual tiles.  Ring slots and accumulator sets are handed on when BOTH
+        // threads' MMAs have retired (barrier counts NPOL).  With the per-polarity release of a dual 256-wide
+        // tile each thread waits for its own accumulator only, so the positive thread starts the next tile
+        // while the negative accumulator is still being read (it can run ahead by the depth of the ring).
         if (lane == 0 && rank == 0) {
+            const uint32_t pol = uint32_t(warp - 1);
             constexpr uint32_t idesc = make_idesc(KIND, TILE_N, TILE_M * CG);
             const uint32_t stages = prm.stages, P = prm.sb.P, acc_stages = prm.acc_stages;
             const uint32_t full0 = smem_u32(&hdr->full[0]), empty0 = smem_u32(&hdr->empty[0]);
-            const uint64_t desc0 = make_smem_desc(smem_u32(smem));
+            const uint64_t desc0 = make_smem_desc(smem_u32(smem)) + pol * (uint64_t(a_bytes) >> 4);
             constexpr uint64_t kStageDesc = uint64_t(stage_bytes) >> 4;
-            constexpr uint64_t kBDesc = uint64_t(NPOL * a_bytes) >> 4;
+            const uint64_t b_off = (uint64_t(NPOL * a_bytes) >> 4) - pol * (uint64_t(a_bytes) >> 4);
             uint32_t s = 0, ph = 0, as = 0, aph = 0;
             bool ok = true;
             for (int tile = unit; tile < num_tiles && ok; tile += num_units) {
-                if constexpr (kSplitRel) {
-                    constexpr uint64_t kANegDesc = uint64_t(a_bytes) >> 4;
-                    const int k_end = prm.sb.kb[1];
-                    const uint32_t nkb = uint32_t((k_end + BLOCK_K - 1) / BLOCK_K);
-                    const uint32_t ahead = nkb < stages - 1 ? nkb : stages - 1;
-                    if (!mbar_wait(smem_u32(&hdr->tmem_empty[0]), aph ^ 1, abort_flag, prm.status, kWhereMmaTmem)) break;
-                    tc_fence_after();
-                    // positive-only MMAs of the first `ahead` K-blocks; their ring slots stay taken
-                    uint32_t s1 = s, ph1 = ph;
-                    int k = 0;
-                    for (uint32_t j = 0; j < ahead && ok; j++, k += BLOCK_K) {
-                        if (!mbar_wait(full0 + 8 * s1, ph1, abort_flag, prm.status, kWhereMmaFull)) { ok = false; break; }
-                        tc_fence_after();
-                        const uint64_t da = desc0 + s1 * kStageDesc;
-                        const int rem = k_end - k;
-                        const int nk = rem >= BLOCK_K ? BLOCK_K / MMA_K : (rem + MMA_K - 1) / MMA_K;
-                        issue_kblock<KIND, 1, TILE_N, CG>(tmem_base, da, da + kBDesc, idesc, nk, j > 0 ? 1u : 0u);
-                        if (++s1 == stages) { s1 = 0; ph1 ^= 1; }
-                    }
-                    if (!ok) break;
-                    if (!mbar_wait(smem_u32(&hdr->tmem_empty[1]), aph ^ 1, abort_flag, prm.status, kWhereMmaTmem)) break;
-                    tc_fence_after();
-                    // the negative MMAs of the same K-blocks, each freeing its slot
-                    k = 0;
-                    for (uint32_t j = 0; j < ahead; j++, k += BLOCK_K) {
-                        const uint64_t da = desc0 + s * kStageDesc;
-                        const int rem = k_end - k;
-                        const int nk = rem >= BLOCK_K ? BLOCK_K / MMA_K : (rem + MMA_K - 1) / MMA_K;
-                        issue_kblock<KIND, 1, TILE_N, CG>(tmem_base + TILE_N, da + kANegDesc, da + kBDesc, idesc, nk,
-                                                          j > 0 ? 1u : 0u);
-                        tc_commit<CG>(empty0 + 8 * s);
-                        if (++s == stages) { s = 0; ph ^= 1; }
-                    }
-                    // the rest of the tile: both polarities per K-step
-                    for (; k < k_end; k += BLOCK_K) {
-                        if (!mbar_wait(full0 + 8 * s, ph, abort_flag, prm.status, kWhereMmaFull)) { ok = false; break; }
-                        tc_fence_after();
-                        const uint64_t da = desc0 + s * kStageDesc;
-                        const int rem = k_end - k;
-                        const int nk = rem >= BLOCK_K ? BLOCK_K / MMA_K : (rem + MMA_K - 1) / MMA_K;
-                        issue_kblock<KIND, NPOL, TILE_N, CG>(tmem_base, da, da + kBDesc, idesc, nk, 1u);
-                        tc_commit<CG>(empty0 + 8 * s);
-                        if (++s == stages) { s = 0; ph ^= 1; }
-                    }
-                    if (!ok) break;
-                    tc_commit<CG>(smem_u32(&hdr->tmem_full[0]));
-                    aph ^= 1;
-                    continue;
-                }
                 if (!SEQ) {
-                    if (!mbar_wait(smem_u32(&hdr->tmem_empty[as]), aph ^ 1, abort_flag, prm.status, kWhereMmaTmem)) {
+                    const uint32_t bar = smem_u32(&hdr->tmem_empty[kSplitRel ? pol : as]);
+                    if (!mbar_wait(bar, aph ^ 1, abort_flag, prm.status, kWhereMmaTmem)) {
                         ok = false;
                         break;
                     }
@@ -778,7 +739,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                         }
                         tc_fence_after();
                     }
-                    const uint32_t d0 = tmem_base + as * acc_cols + (SEQ ? 0u : p * (NPOL * TILE_N));
+                    const uint32_t d0 = tmem_base + as * acc_cols + (SEQ ? 0u : p * (NPOL * TILE_N)) + pol * TILE_N;
                     const int k_end = prm.sb.kb[p + 1];
                     uint32_t accumulate = 0;
                     for (int k = prm.sb.kb[p]; k < k_end; k += BLOCK_K) {
@@ -790,9 +751,9 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                         const uint64_t da = desc0 + s * kStageDesc;
                         const int rem = k_end - k;
                         const int nk = rem >= BLOCK_K ? BLOCK_K / MMA_K : (rem + MMA_K - 1) / MMA_K;
-                        issue_kblock<KIND, NPOL, TILE_N, CG>(d0, da, da + kBDesc, idesc, nk, accumulate);
+                        issue_kblock<KIND, 1, TILE_N, CG>(d0, da, da + b_off, idesc, nk, accumulate);
                         accumulate = 1;
-                        tc_commit<CG>(empty0 + 8 * s);             // frees the ring slot when these MMAs retire
+                        tc_commit<CG>(empty0 + 8 * s);             // the slot is free when both threads' MMAs have retired
                         if (++s == stages) { s = 0; ph ^= 1; }
                     }
                     if (SEQ) {
