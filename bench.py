@@ -555,8 +555,8 @@ def run_ours(args):
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the GEMM launches of one step, from the ncu
 # capture summarised in profiles/gemm_pair_and_quantize_dit_xl2_sd3_mmdit.md; None = not captured for that workload.
-GEMM_DRAM_TRAFFIC = {"dit_xl2": 12765696 + 38912 + 24238592 + 1536,
-                     "sd3_mmdit": 41490944 + 38836736 + 23211008 + 56874752 + 123385344 + 13977600}
+GEMM_DRAM_TRAFFIC = {"dit_xl2": 12758528 + 12544 + 24237568 + 1792,
+                     "sd3_mmdit": 41486080 + 39151616 + 23182336 + 57289472 + 123912448 + 13631232}
 
 
 # ------------------------------------------------------------------------------------ reference arm
