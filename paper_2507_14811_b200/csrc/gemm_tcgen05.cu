@@ -651,8 +651,8 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     // A dual 256-wide tile (one K-segment) fills TMEM, so there is one accumulator set and the tensor pipe would
     // idle during the epilogue up to the set's release.  Instead the two polarities are released SEPARATELY
     // (barrier tmem_empty[0] = positive accumulator free, tmem_empty[1] = negative one): the epilogue reads all
-    // positive columns first, and the MMA issuer starts the next tile with positive-only MMAs for as many
-    // K-blocks as the ring can hold back (stages - 1), then catches up on the negative ones.
+    // positive columns first, and the thread that issues the positive MMAs starts the next tile as soon as they
+    // are in registers, ahead of the negative thread by at most the depth of the ring.
     constexpr bool kSplitRel = NPOL == 2 && TILE_N == 256 && !SEQ && !GENERIC;
 
     // The producer and the MMA issuer are single threads: their loops are kept to a few dozen
