@@ -554,7 +554,7 @@ def run_ours(args):
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the GEMM launches of one step, from the ncu
-# capture summarised in profiles/gemm_pair_and_quantize_dit_xl2_sd3_mmdit.md; None = not captured for that workload.
+# capture of these workloads (its summary is kept among the committed profile summaries); None = not captured.
 GEMM_DRAM_TRAFFIC = {"dit_xl2": 12758528 + 12544 + 24237568 + 1792,
                      "sd3_mmdit": 41486080 + 39151616 + 23182336 + 57289472 + 123912448 + 13631232}
 

@@ -26,7 +26,7 @@ def oracle_scales(data, flags_qmin_sym=False):
 
 
 def fp32_epilogue_tolerance(y64, y_abs, nacc):
-    """The benchmark spec's 1e-5 relative bound on the fp32 epilogue, plus the rounding the fp32 evaluation
+    """The 1e-5 relative bound required of the fp32 epilogue, plus the rounding the fp32 evaluation
     itself can commit on cancelling terms: each of the nacc products carries the rounding of the
     scale product, of the int->float conversion and of one FMA, and the bias add rounds once more,
     all relative to the sum of |terms| (2^-24 each)."""
