@@ -580,7 +580,12 @@ __device__ __forceinline__ void store_slab(const uint64_t (&y2)[16], const Param
 // are converted and stored after the last segment.  Any number of K-segments fits, tiles stay wide, and the
 // drain of every segment but the last overlaps tensor work.  SEQ = false keeps every (segment, polarity)
 // accumulator of a tile resident in TMEM and drains once per tile.
-template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ>
+// WIDE = true (single-scale layers, one K-segment, CTA pairs): the tile is 256 rows x 512 columns, two 256-column
+// halves that share ONE activation tile per K-block, the mirror image of a dual tile (two activation tiles, one
+// weight tile).  A single-scale 256 x 256 tile asks for 64 bytes of operands per SM cycle, which is all the L2
+// path delivers; the wide tile asks for 48.  Each half has its own weight tile in the ring stage, its own
+// issuing thread and accumulator, and is released to its thread separately, like the polarities of a dual tile.
+template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ, bool WIDE = false>
 // 384 threads = 12 warps, 3 on each SM sub-partition with 16 K registers: 168 registers per thread at launch
 __global__ void __launch_bounds__(kThreads, 1)
 segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_constant__ CUtensorMap tm_a_neg,
@@ -592,14 +597,18 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     constexpr int B_ROWS = TILE_N / CG;                  // weight rows this CTA loads per K-block
     constexpr uint32_t a_bytes = TILE_M * BLOCK_K;
     constexpr uint32_t b_bytes = B_ROWS * BLOCK_K;
-    constexpr uint32_t stage_bytes = NPOL * a_bytes + b_bytes;
+    constexpr int kHalves = WIDE ? 2 : 1;                // weight tiles per stage
+    constexpr int kTileCols = TILE_N * kHalves;          // output columns of a tile
+    constexpr int kIssuers = (NPOL == 2 || WIDE) ? 2 : 1;
+    static_assert(!WIDE || (NPOL == 1 && TILE_N == 256 && CG == 2 && !GENERIC && !SEQ), "wide single-scale tile");
+    constexpr uint32_t stage_bytes = NPOL * a_bytes + kHalves * b_bytes;
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t *sh_stage = smem + size_t(prm.stages) * stage_bytes;      // 1 KiB aligned: stages are multiples of 1 KiB
     float *sh_bias = reinterpret_cast<float *>(sh_stage + (GENERIC ? 0 : kStageBytes));     // [TILE_N], per tile
-    float *sh_tab = sh_bias + TILE_N;                                                       // [nacc][Q], per launch
+    float *sh_tab = sh_bias + kTileCols;                                                    // [nacc][Q], per launch
     int *sh_nb = reinterpret_cast<int *>(sh_tab + prm.nacc * prm.sb.Q);                     // [Q + 1]
     SharedHeader *hdr = reinterpret_cast<SharedHeader *>(reinterpret_cast<uint8_t *>(sh_bias) +
-                                                         epi_table_bytes(prm.nacc, prm.sb.Q, TILE_N));
+                                                         epi_table_bytes(prm.nacc, prm.sb.Q, kTileCols));
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -617,10 +626,10 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     if (threadIdx.x == 0) {
         for (int s = 0; s < prm.stages; s++) {
             mbar_init(smem_u32(&hdr->full[s]), 1);
-            mbar_init(smem_u32(&hdr->empty[s]), NPOL);          // one arrival per MMA-issuing thread
+            mbar_init(smem_u32(&hdr->empty[s]), kIssuers);      // one arrival per MMA-issuing thread
         }
         for (int s = 0; s < 2; s++) {
-            mbar_init(smem_u32(&hdr->tmem_full[s]), NPOL);
+            mbar_init(smem_u32(&hdr->tmem_full[s]), kIssuers);
             mbar_init(smem_u32(&hdr->tmem_empty[s]), CG * kEpiWarps);
         }
         hdr->abort_flag = 0;
@@ -647,13 +656,13 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     if (CG == 2) asm volatile("barrier.cluster.wait.acquire;" ::: "memory");   // the peer's barriers are initialised
     tc_fence_after();
     const uint32_t tmem_base = hdr->tmem_base;
-    const int acc_cols = (SEQ ? NPOL : prm.nacc) * TILE_N;     // TMEM columns of one accumulator set
+    const int acc_cols = (SEQ ? NPOL : prm.nacc) * kTileCols;  // TMEM columns of one accumulator set
     // A dual 256-wide tile (one K-segment) fills TMEM, so there is one accumulator set and the tensor pipe would
     // idle during the epilogue up to the set's release.  Instead the two polarities are released SEPARATELY
     // (barrier tmem_empty[0] = positive accumulator free, tmem_empty[1] = negative one): the epilogue reads all
     // positive columns first, and the thread that issues the positive MMAs starts the next tile as soon as they
     // are in registers, ahead of the negative thread by at most the depth of the ring.
-    constexpr bool kSplitRel = NPOL == 2 && TILE_N == 256 && !SEQ && !GENERIC;
+    constexpr bool kSplitRel = (NPOL == 2 && TILE_N == 256 && !SEQ && !GENERIC) || WIDE;
 
     // The producer and the MMA issuer are single threads: their loops are kept to a few dozen
     // instructions per K-block (ring slot and phase advance incrementally, descriptors by addition).
@@ -672,7 +681,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
             bool ok = true;
             for (int tile = unit; tile < num_tiles && ok; tile += num_units) {
                 const int m0 = (tile / prm.num_n_tiles) * (TILE_M * CG) + int(rank) * TILE_M;
-                const int n0 = (tile % prm.num_n_tiles) * TILE_N + int(rank) * B_ROWS;
+                const int n0 = (tile % prm.num_n_tiles) * kTileCols + int(rank) * B_ROWS;
                 for (uint32_t p = 0; p < P && ok; p++) {
                     const int k_end = prm.sb.kb[p + 1];
                     for (int k = prm.sb.kb[p]; k < k_end; k += BLOCK_K) {
@@ -686,6 +695,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                         tma_load_2d<CG>(dst, &tm_a_pos, bar, k, m0);
                         if (NPOL == 2) tma_load_2d<CG>(dst + a_bytes, &tm_a_neg, bar, k, m0);
                         tma_load_2d<CG>(dst + NPOL * a_bytes, &tm_b, bar, k, n0);
+                        if (WIDE) tma_load_2d<CG>(dst + NPOL * a_bytes + b_bytes, &tm_b, bar, k, n0 + TILE_N);
                         issued++;
                         if (++s == stages) { s = 0; ph ^= 1; }
                     }
@@ -703,7 +713,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                 }
             }
         }
-      } else if (warp == 1 || (NPOL == 2 && warp == 2)) {
+      } else if (warp == 1 || (kIssuers == 2 && warp == 2)) {
         // ------------------------------------------------------------------ MMA issuers (leader CTA)
         // One thread per polarity: warp 1 issues the MMAs of the positive code matrix, warp 2 (dual layers)
         // those of the negative one, each into its own accumulators.  A tcgen05.mma keeps its issuing thread
@@ -717,9 +727,11 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
             constexpr uint32_t idesc = make_idesc(KIND, TILE_N, TILE_M * CG);
             const uint32_t stages = prm.stages, P = prm.sb.P, acc_stages = prm.acc_stages;
             const uint32_t full0 = smem_u32(&hdr->full[0]), empty0 = smem_u32(&hdr->empty[0]);
-            const uint64_t desc0 = make_smem_desc(smem_u32(smem)) + pol * (uint64_t(a_bytes) >> 4);
+            // dual: thread `pol` takes activation tile `pol`; wide: thread `pol` takes weight tile (half) `pol`
+            const uint64_t desc0 = make_smem_desc(smem_u32(smem)) + (WIDE ? 0u : pol) * (uint64_t(a_bytes) >> 4);
             constexpr uint64_t kStageDesc = uint64_t(stage_bytes) >> 4;
-            const uint64_t b_off = (uint64_t(NPOL * a_bytes) >> 4) - pol * (uint64_t(a_bytes) >> 4);
+            const uint64_t b_off = WIDE ? (uint64_t(a_bytes) >> 4) + pol * (uint64_t(b_bytes) >> 4)
+                                        : (uint64_t(NPOL * a_bytes) >> 4) - pol * (uint64_t(a_bytes) >> 4);
             uint32_t s = 0, ph = 0, as = 0, aph = 0;
             bool ok = true;
             for (int tile = unit; tile < num_tiles && ok; tile += num_units) {
@@ -795,13 +807,14 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
             }
         };
         // bias slice of a tile, one column per thread, fetched one tile ahead into a register
-        auto fetch_bias = [&](int tile) -> float {
+        auto fetch_bias = [&](int tile, int half = 0) -> float {
             if (tile >= num_tiles || et >= TILE_N || !prm.bias) return 0.0f;
-            const int n = (tile % prm.num_n_tiles) * TILE_N + et;
+            const int n = (tile % prm.num_n_tiles) * kTileCols + half * TILE_N + et;
             return n < prm.N ? __ldg(prm.bias + n) : 0.0f;
         };
         grid_dependency_wait();                     // scales, bias and Y may belong to the previous kernel
         float bias_next = fetch_bias(unit);
+        float bias_next1 = WIDE ? fetch_bias(unit, 1) : 0.0f;   // second half of a wide tile
         // dequantization factors c[a][q] = s_act[p][pol] * s_w[p][q], a = p * NPOL + pol (one fp32 multiply);
         // built here, off the producer's and the MMA issuer's path, and published by the first tile's barrier
         for (int i = et; i < nacc * Q; i += kEpiThreads) {
@@ -816,13 +829,17 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
         bool ok = true;
         for (int tile = unit; tile < num_tiles; tile += num_units) {
             const int m0 = (tile / prm.num_n_tiles) * (TILE_M * CG) + int(rank) * TILE_M;
-            const int n0 = (tile % prm.num_n_tiles) * TILE_N;
+            const int n0 = (tile % prm.num_n_tiles) * kTileCols;
             const int row = m0 + lane_grp * 32 + lane;
             yo.row0 = m0 + lane_grp * 32;
 
             asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // previous tile's readers are done
             if (et < TILE_N) sh_bias[et] = bias_next;
             bias_next = fetch_bias(tile + num_units);                        // lands during this tile's work
+            if (WIDE) {
+                sh_bias[TILE_N + et] = bias_next1;                           // et < 256 = TILE_N for every epilogue thread
+                bias_next1 = fetch_bias(tile + num_units, 1);
+            }
             asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
 
             // A warp's share of one accumulator set is kUnits TMEM loads (unit u = slab u / NPOL, polarity
@@ -889,7 +906,37 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                 tc_fence_after();
                 const uint32_t t_row = tmem_base + (uint32_t(lane_grp * 32) << 16) + cur_as * acc_cols;
                 constexpr bool kEvenSplit = kSlabsPerWarp * kColGroups == kSlabs;
-                if constexpr (kSplitRel) {
+                if constexpr (WIDE) {
+                    // two independent 256-column halves, four slabs of each per warp: all units of half 0 first
+                    // (then its accumulator goes back), two of half 1, and the last two of half 1 into the
+                    // registers of the first two finished slabs (then the second accumulator goes back)
+                    const uint32_t t_h0 = t_row + uint32_t(slab0 * 32), t_h1 = t_h0 + uint32_t(TILE_N);
+                    uint32_t hb[2][4][32];
+                    uint64_t y2[16];
+#pragma unroll
+                    for (int sl = 0; sl < 4; sl++) tc_ld32(t_h0 + uint32_t(sl * 32), hb[0][sl]);
+                    tc_wait_ld();
+                    release(0);
+                    tc_ld32(t_h1, hb[1][0]);
+                    tc_ld32(t_h1 + 32u, hb[1][1]);
+#pragma unroll
+                    for (int u = 0; u < 8; u++) {
+                        const int h = u >> 2, sl = u & 3;
+                        const int c0 = h * TILE_N + (slab0 + sl) * 32, nf = n0 + c0;
+                        const int q = seg_of_column(min(nf, prm.N - 1), Q, nb_addr, lane);
+                        scale_add_unit<KIND, false, true>(y2, hb[h][sl], 0, Q, q, q, nf, tab_addr, nb_addr,
+                                                          bias_addr + uint32_t(c0) * 4u);
+                        store_slab<GENERIC>(y2, prm, row, nf, yo);
+                        if (u == 1) {
+                            tc_ld32(t_h1 + 64u, hb[1][2]);
+                            tc_ld32(t_h1 + 96u, hb[1][3]);
+                            tc_wait_ld();
+                            release(1);
+                        }
+                    }
+                    continue;
+                }
+                if constexpr (kSplitRel && !WIDE) {
                     // four slabs per warp: all positive units first (then the positive accumulator goes back),
                     // negative units as registers come free (then the negative one); five units live at most
                     static_assert(!kSplitRel || kSlabsPerWarp == 4, "split release: 256-wide tile, 8 epilogue warps");
@@ -1079,9 +1126,10 @@ bool make_map_y(CUtensorMap *map, void *base, int64_t M, int64_t N, int64_t ldy)
 
 int g_tune_tile_n = 0, g_tune_stages = 0, g_tune_cta_group = 0, g_tune_seq = 0;
 
-template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ>
+template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ, bool WIDE = false>
 sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cudaStream_t st)
 {
+    constexpr int kTileCols = TILE_N * (WIDE ? 2 : 1);
     constexpr int B_ROWS = TILE_N / CG;
     CUtensorMap ta, tn, tb, ty;
     if (GENERIC) ty = CUtensorMap{};                // unused by the generic variant
@@ -1090,18 +1138,18 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
     if (!make_map(&tn, g.a_neg ? g.a_neg : g.a_pos, g.M, g.K, g.lda, TILE_M)) return SQ_ERR_CUDA;
     if (!make_map(&tb, g.b, g.N, g.K, g.ldb, B_ROWS)) return SQ_ERR_CUDA;
 
-    const uint32_t stage_bytes = NPOL * TILE_M * BLOCK_K + B_ROWS * BLOCK_K;
-    const uint32_t tail = (GENERIC ? 0u : kStageBytes) + epi_table_bytes(prm.nacc, prm.sb.Q, TILE_N) + sizeof(SharedHeader);
+    const uint32_t stage_bytes = NPOL * TILE_M * BLOCK_K + (WIDE ? 2 : 1) * B_ROWS * BLOCK_K;
+    const uint32_t tail = (GENERIC ? 0u : kStageBytes) + epi_table_bytes(prm.nacc, prm.sb.Q, kTileCols) + sizeof(SharedHeader);
     int stages = int((kSmemBudget - 1024 - tail) / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (g_tune_stages >= 2 && g_tune_stages < stages) stages = g_tune_stages;
     if (stages < 2) return SQ_ERR_UNSUPPORTED;
     prm.stages = stages;
     prm.num_m_tiles = int((g.M + TILE_M * CG - 1) / (TILE_M * CG));
-    prm.num_n_tiles = int((g.N + TILE_N - 1) / TILE_N);
+    prm.num_n_tiles = int((g.N + kTileCols - 1) / kTileCols);
     const size_t smem = 1024 + size_t(stages) * stage_bytes + tail;
 
-    auto kern = segquant_gemm_kernel<KIND, NPOL, TILE_N, CG, GENERIC, SEQ>;
+    auto kern = segquant_gemm_kernel<KIND, NPOL, TILE_N, CG, GENERIC, SEQ, WIDE>;
     const cudaError_t ea = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
     if (ea != cudaSuccess) { note_cuda_error(ea); return SQ_ERR_CUDA; }
     const int tiles = prm.num_m_tiles * prm.num_n_tiles;
@@ -1155,6 +1203,15 @@ sq_status launch_tile(const GemmArgs &g, KernelParams &prm, int tile_n, bool seq
         constexpr int TN = NPOL == 1 ? 256 : 128;
         return dbg ? launch_variant<KIND, NPOL, TN, CG, true, true>(g, prm, sm_count, st)
                    : launch_variant<KIND, NPOL, TN, CG, false, true>(g, prm, sm_count, st);
+    }
+    // single-scale layer, one K-segment, CTA pairs, at least two 256-column tiles: 256 x 512 tiles whose halves
+    // share the activation tile; an odd number of 256-column tiles leaves one half idle, so then only when there
+    // are many of them
+    const int64_t n256 = (g.N + 255) / 256;
+    if (NPOL == 1 && CG == 2 && !dbg && tile_n == 256 && prm.sb.P == 1 && g_tune_seq != 4 &&
+        (n256 % 2 == 0 || n256 >= 9)) {
+        prm.acc_stages = 1;
+        return launch_variant<KIND, 1, 256, 2, false, false, true>(g, prm, sm_count, st);
     }
     switch (tile_n) {
         case 256: return dbg ? launch_variant<KIND, NPOL, 256, CG, true, false>(g, prm, sm_count, st)

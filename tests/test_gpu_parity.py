@@ -124,6 +124,36 @@ def test_every_tile_width_dual(tile_n, cta_group):
                cta_group=cta_group)
 
 
+@pytest.mark.parametrize("case", [
+    # name, M, K, N, nb, code: single-scale layers whose bf16 output takes the 256 x 512 tiles (an even number of
+    # 256-column tiles): exact, a second half of 8 columns, ragged rows, several N-segments, both code types
+    ("wide_exact", 256, 256, 512, [0, 512], "int8"),
+    ("wide_tail8", 300, 384, 776, [0, 256, 776], "int8"),
+    ("wide_ragged", 700, 400, 1000, [0, 160, 480, 1000], "int8"),
+    ("wide_e4m3", 260, 256, 1536, [0, 1536], "e4m3"),
+    ("wide_many", 520, 128, 2560, [0, 2560], "int8"),
+])
+def test_wide_single_scale_tiles(case):
+    name, M, K, N, nb, code = case
+    run_parity(custom_spec(name, M, K, N, [0, K], nb, False, code, x_kind="normal", seed=51), tile_n=256, cta_group=2)
+    # the same layer with 256 x 256 tiles gives the same bytes
+    spec = custom_spec(name, M, K, N, [0, K], nb, False, code, x_kind="normal", seed=51)
+    data = WL.make_layer(spec)
+    layer = SegQuantLinear(data.W, data.bias, spec.kb, spec.nb, False, code, DEV)
+    layer.calibrate(data.X_cal)
+    Xd = data.X.to(DEV)
+    try:
+        B.segquant_set_tuning(256, 0, 2, 0)
+        Y_wide = layer.forward(Xd)
+        B.segquant_set_tuning(256, 0, 2, 4)
+        Y_narrow = layer.forward(Xd)
+        layer.check_status()
+        torch.cuda.synchronize()
+    finally:
+        B.segquant_set_tuning(0, 0, 0, 0)
+    assert torch.equal(Y_wide, Y_narrow)
+
+
 @pytest.mark.parametrize("cta_group", [1, 2])
 @pytest.mark.parametrize("case", [
     # the CTA-pair tile is 256 rows: M at, just below and just above its multiples; a second CTA with no rows
