@@ -556,7 +556,7 @@ def run_ours(args):
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the GEMM launches of one step, from the ncu
 # capture of these workloads (its summary is kept among the committed profile summaries); None = not captured.
 GEMM_DRAM_TRAFFIC = {"dit_xl2": 12758528 + 12544 + 24237568 + 1792,
-                     "sd3_mmdit": 41486080 + 39151616 + 23182336 + 57289472 + 123912448 + 13631232}
+                     "sd3_mmdit": 41489152 + 38824960 + 23200512 + 56566784 + 123355648 + 13652992}
 
 
 # ------------------------------------------------------------------------------------ reference arm

@@ -204,7 +204,8 @@ sq_status segquant_last_device_status(void *workspace, void *stream, uint32_t *d
  * 1 (one CTA per 128-row tile) or 2; segment_mode for layers with several K-segments: 0 (automatic:
  * segments pass through tensor memory one after the other, running sums in registers), 1 (all
  * accumulators of a tile resident in tensor memory; at most 16 of them), 2 (sequential) or 4
- * (automatic, but single-scale layers keep 256 x 256 tiles instead of 256 x 512 ones).
+ * (automatic, but single-scale layers keep 256 x 256 tiles instead of 256 x 512 ones) or 5 (256 x 512
+ * tiles for single-scale layers even where the automatic choice expects no gain from them).
  * Process-wide; meant for benchmarking sweeps and tests.  Values the layer cannot use are replaced by
  * the automatic choice. */
 sq_status segquant_set_tuning(int tile_n, int stages, int cta_group, int segment_mode);

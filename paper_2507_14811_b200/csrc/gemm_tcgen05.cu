@@ -1206,10 +1206,13 @@ sq_status launch_tile(const GemmArgs &g, KernelParams &prm, int tile_n, bool seq
     }
     // single-scale layer, one K-segment, CTA pairs, at least two 256-column tiles: 256 x 512 tiles whose halves
     // share the activation tile; an odd number of 256-column tiles leaves one half idle, so then only when there
-    // are many of them
-    const int64_t n256 = (g.N + 255) / 256;
+    // are many of them; and a wide tile is two tiles' work, so it must not cost more waves than it saves time
+    // (measured gain per unit of work: 5-6 %)
+    const int64_t n256 = (g.N + 255) / 256, m_pairs = (g.M + 2 * TILE_M - 1) / (2 * TILE_M), units = sm_count / 2;
+    const int64_t waves_256 = (m_pairs * n256 + units - 1) / units;
+    const int64_t waves_wide = (m_pairs * ((n256 + 1) / 2) + units - 1) / units;
     if (NPOL == 1 && CG == 2 && !dbg && tile_n == 256 && prm.sb.P == 1 && g_tune_seq != 4 &&
-        (n256 % 2 == 0 || n256 >= 9)) {
+        (n256 % 2 == 0 || n256 >= 9) && (g_tune_seq == 5 || 2 * waves_wide * 94 < waves_256 * 100)) {
         prm.acc_stages = 1;
         return launch_variant<KIND, 1, 256, 2, false, false, true>(g, prm, sm_count, st);
     }

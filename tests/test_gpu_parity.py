@@ -135,7 +135,8 @@ def test_every_tile_width_dual(tile_n, cta_group):
 ])
 def test_wide_single_scale_tiles(case):
     name, M, K, N, nb, code = case
-    run_parity(custom_spec(name, M, K, N, [0, K], nb, False, code, x_kind="normal", seed=51), tile_n=256, cta_group=2)
+    run_parity(custom_spec(name, M, K, N, [0, K], nb, False, code, x_kind="normal", seed=51), tile_n=256, cta_group=2,
+               segment_mode=5)
     # the same layer with 256 x 256 tiles gives the same bytes
     spec = custom_spec(name, M, K, N, [0, K], nb, False, code, x_kind="normal", seed=51)
     data = WL.make_layer(spec)
@@ -143,7 +144,7 @@ def test_wide_single_scale_tiles(case):
     layer.calibrate(data.X_cal)
     Xd = data.X.to(DEV)
     try:
-        B.segquant_set_tuning(256, 0, 2, 0)
+        B.segquant_set_tuning(256, 0, 2, 5)
         Y_wide = layer.forward(Xd)
         B.segquant_set_tuning(256, 0, 2, 4)
         Y_narrow = layer.forward(Xd)
