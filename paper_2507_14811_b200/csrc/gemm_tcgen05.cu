@@ -22,7 +22,9 @@
 // are back with the MMA issuer early in the epilogue.
 // One K-segment: the npol accumulators (128 lanes x TILE_N columns each) of a tile stay in TMEM until the
 // tile's epilogue; if they use at most half of TMEM there are two sets, and the epilogue of one tile
-// overlaps the main loop of the next.  Several K-segments: see SEQ below.
+// overlaps the main loop of the next.  A dual 256-wide tile fills TMEM: its two polarities are handed back
+// to their issuing threads separately.  Single-scale layers may use 256 x 512 tiles built the same way
+// (WIDE below).  Several K-segments: see SEQ below.
 // Every wait on an mbarrier is bounded (SM cycle counter, about 2 s); on expiry the CTA records
 // which wait gave up in the status word, stops issuing work, lets its own copies land and leaves
 // normally.  No load uses cluster multicast.
