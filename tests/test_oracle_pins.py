@@ -251,6 +251,49 @@ def test_e4m3_activation_codes_match_library_cast():
     assert (cp == 0x7E).any()                                           # the clamp was exercised
 
 
+def test_e4m3_single_scale_activation_codes_match_library_cast():
+    """Single-scale branch of the e4m3 activation quantizer (Sec. 3 quantizer with z = 0, Table 1 "8/8 (fp)"):
+    one signed code matrix, clip to [-448, 448], against torch's float8 cast of the fp32 quotient."""
+    r = rng(31)
+    X = r.standard_t(4, (40, 96)).astype(np.float32)
+    X[0, :6] = [0.0, -0.0, 1e-30, -1e-30, 1e6, -1e6]
+    kb = [0, 32, 96]
+    s, _ = O.calib_act(X[:6], kb, False, q_max=448.0, q_min_abs=448.0)    # few rows: runtime exceeds the range
+    c, none = O.quantize_act(X, kb, s, None, code="e4m3")
+    assert none is None
+    sv = torch.zeros(96)
+    for p in range(2):
+        sv[kb[p]:kb[p + 1]] = float(s[p])
+    t = torch.clamp(torch.from_numpy(X) / sv, -448, 448).to(torch.float8_e4m3fn).view(torch.uint8).numpy().copy()
+    t[t == 0x80] = 0
+    assert np.array_equal(c, t)
+    assert (c == 0x7E).any() and (c == 0xFE).any()                       # both ends of the clip were exercised
+    assert ((c & 0x80) != 0).any()                                       # negative codes exist (not clipped to [0, 448])
+
+
+def test_e4m3_weight_codes_match_library_cast_per_block():
+    """FP8 weight codes, one scale per (K-segment, N-segment) block (Sec. 4.2.2: every W_i is quantized
+    separately; Sec. 3 quantizer): each block against torch's float8 cast of W / s_w[p][q].  P = 2 and Q = 3
+    with P != Q and blocks of very different ranges, so that a transposed scale index cannot pass."""
+    r = rng(32)
+    kb, nb = [0, 24, 64], [0, 8, 20, 28]
+    W = r.normal(0, 0.02, (28, 64)).astype(np.float32)
+    for p in range(2):
+        for q in range(3):
+            W[nb[q]:nb[q + 1], kb[p]:kb[p + 1]] *= 3.0 ** (p * 3 + q)
+    s_w = O.calib_weight(W, kb, nb, w_max=448.0)
+    assert s_w.shape == (2, 3) and len(np.unique(s_w)) == 6
+    Wq = O.quantize_weight(W, kb, nb, s_w, code="e4m3")
+    for p in range(2):
+        for q in range(3):
+            blk = torch.from_numpy(W[nb[q]:nb[q + 1], kb[p]:kb[p + 1]].copy())
+            assert np.float32(blk.abs().max()) / np.float32(448.0) == s_w[p, q]
+            t = torch.clamp(blk / float(s_w[p, q]), -448, 448).to(torch.float8_e4m3fn).view(torch.uint8).numpy().copy()
+            t[t == 0x80] = 0
+            assert np.array_equal(Wq[nb[q]:nb[q + 1], kb[p]:kb[p + 1]], t)
+            assert (t & 0x7F).max() == 0x7E                               # the block's extremum sits on 448
+
+
 # --------------------------------------------------------------- accumulators
 
 def test_int8_accumulators_brute_force_tiny():
@@ -392,6 +435,73 @@ def test_recombination_equals_brute_force_dot_of_dequantized_operands():
                 wdq = float(s_w[p, q]) * int(Wq[n, k])
                 tot += xdq * wdq
             assert math.isclose(res.y64[m, n], tot, rel_tol=1e-12, abs_tol=1e-15)
+
+
+@pytest.mark.parametrize("dual", [False, True])
+def test_sum_of_absolute_terms_equals_brute_force(dual):
+    """The oracle also reports, per output, sum over (segment, polarity) of |term| + |bias|: the magnitude
+    against which an fp32 evaluation of the recombination is judged in the GPU parity tests (it sets their
+    tolerance, so it is pinned like a result).  Brute force on a tiny layer with terms of both signs."""
+    r = rng(33)
+    M, N, K = 4, 5, 24
+    kb, nb = [0, 8, 24], [0, 2, 5]
+    X = gelu(r.normal(0, 1.5, (M, K))).astype(np.float32)
+    W = r.normal(0, 0.02, (N, K)).astype(np.float32)
+    bias = r.normal(0, 0.1, N).astype(np.float32)
+    res, (sp, sn, s_w, Wq) = oracle_layer(X, W, kb, nb, dual, bias)
+    for m in range(M):
+        for n in range(N):
+            q = 0 if n < 2 else 1
+            tot = abs(float(bias[n]))
+            for p in range(2):
+                ap = sum(int(res.c_pos[m, k]) * int(Wq[n, k]) for k in range(kb[p], kb[p + 1]))
+                tot += abs(float(sp[p]) * float(s_w[p, q]) * ap)
+                if dual:
+                    an = sum(int(res.c_neg[m, k]) * int(Wq[n, k]) for k in range(kb[p], kb[p + 1]))
+                    tot += abs(float(sn[p]) * float(s_w[p, q]) * an)
+            assert math.isclose(res.y_abs[m, n], tot, rel_tol=1e-12, abs_tol=0)
+    assert np.all(res.y_abs >= np.abs(res.y64) * (1 - 1e-12))
+    assert (res.y_abs > np.abs(res.y64) * 1.5).any()                    # terms do cancel somewhere
+    none_bias = O.layer_forward(X, Wq, O.SegTable(kb, nb), sp, sn, s_w, None)
+    assert np.allclose(none_bias.y_abs, res.y_abs - np.abs(bias.astype(np.float64))[None, :], rtol=1e-12, atol=1e-18)
+
+
+def per_tensor_layer_e4m3(X, W, dual):
+    """Unsegmented per-tensor FP8 layer from torch library ops only: abs-max / 448 scales, float8 casts,
+    fp64 matmul of the decoded codes (exact), fp64 recovery."""
+    X = torch.from_numpy(np.asarray(X, np.float32)); W = torch.from_numpy(np.asarray(W, np.float32))
+    f8 = lambda t: t.to(torch.float8_e4m3fn).double()
+    s_w = np.float32(W.abs().max()) / np.float32(448.0)
+    Wd = f8(torch.clamp(W / float(s_w), -448, 448))
+    if dual:
+        sp = np.float32(max(float(X.max()), 0)) / np.float32(448.0)
+        sn = np.float32(max(-float(X.min()), 0)) / np.float32(448.0)
+        xp = f8(torch.clamp(torch.clamp(X, min=0) / float(sp), 0, 448))
+        xn = f8(torch.clamp(torch.clamp(X, max=0) / float(sn), -448, 0))
+        return ((float(sp) * float(s_w)) * (xp @ Wd.T) + (float(sn) * float(s_w)) * (xn @ Wd.T)).numpy()
+    s = np.float32(X.abs().max()) / np.float32(448.0)
+    return ((float(s) * float(s_w)) * (f8(torch.clamp(X / float(s), -448, 448)) @ Wd.T)).numpy()
+
+
+@pytest.mark.parametrize("dual", [False, True])
+def test_e4m3_layer_compositions(dual):
+    """The FP8 layer through the same reductions as the int8 one: one segment = per-tensor layer,
+    output-segmented = concatenation, input-segmented = sum of independent per-tensor layers (Sec. 4.2.2)."""
+    r = rng(34)
+    X = gelu(r.standard_t(4, (12, 56))).astype(np.float32)
+    W = r.normal(0, 0.02, (30, 56)).astype(np.float32)
+    W[8:24] *= 7.0
+    res, _ = oracle_layer(X, W, [0, 56], [0, 30], dual, code="e4m3")
+    assert np.allclose(res.y64, per_tensor_layer_e4m3(X, W, dual), rtol=1e-13, atol=1e-18)
+    nb = [0, 8, 24, 30]
+    res, _ = oracle_layer(X, W, [0, 56], nb, dual, code="e4m3")
+    ref = np.concatenate([per_tensor_layer_e4m3(X, W[nb[q]:nb[q + 1]], dual) for q in range(3)], axis=1)
+    assert np.allclose(res.y64, ref, rtol=1e-13, atol=1e-18)
+    kb = [0, 16, 24, 56]
+    X2 = X.copy(); X2[:, 16:24] *= 6.0
+    res, _ = oracle_layer(X2, W, kb, [0, 30], dual, code="e4m3")
+    ref = sum(per_tensor_layer_e4m3(X2[:, kb[p]:kb[p + 1]], W[:, kb[p]:kb[p + 1]], dual) for p in range(3))
+    assert np.allclose(res.y64, ref, rtol=1e-12, atol=1e-18)
 
 
 def test_power_of_two_scales_and_on_grid_inputs_give_exact_linear_layer():
