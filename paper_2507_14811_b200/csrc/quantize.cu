@@ -1,8 +1,9 @@
 // Activation / weight quantization kernels (Sec. 3 uniform quantizer, Sec. 4.3.2 Q_dual and polarity
 // split, Sec. 4.2.2 one scale per segment).  HBM-streaming: every thread converts 16 consecutive
-// elements of one row (128-bit loads, one 128-bit store per code matrix).  The codes are those of
-// "one IEEE fp32 division, round half to even, clip"; the common case computes them with a handful of
-// full-rate fp32 instructions per element (see SegConst) so that the pass stays memory bound.
+// elements per row (128-bit loads, one 128-bit store per code matrix) and walks down the rows with that column
+// chunk.  The codes are those of "one IEEE fp32 division, round half to even, clip"; the common case computes
+// them with a handful of full-rate fp32 instructions per element (see SegConst) so that the pass stays memory
+// bound.
 #include <cuda_bf16.h>
 #include "sq_common.cuh"
 
@@ -10,31 +11,41 @@ namespace sq {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kVec = 16;   // elements per thread
+constexpr int kVec = 16;             // elements per thread and row
+#ifndef SQ_QUANT_BLOCKS_PER_SM
+#define SQ_QUANT_BLOCKS_PER_SM 4
+#endif
+constexpr int kBlocksPerSm = SQ_QUANT_BLOCKS_PER_SM;   // resident blocks per SM the kernel is compiled for (4: at most 64 registers)
+constexpr int kThreadsPerSm = kThreads * kBlocksPerSm;
 
-__device__ __forceinline__ void load16(const float *p, float (&x)[kVec])
+// 16 consecutive elements of a row as loaded (fp32: four 128-bit words, bf16: two), converted when used
+template <typename Tin> struct Raw16;
+template <> struct Raw16<float> { float4 v[4]; };
+template <> struct Raw16<__nv_bfloat16> { uint4 v[2]; };
+
+__device__ __forceinline__ void load16(const float *p, Raw16<float> &r)
 {
     const float4 *q = reinterpret_cast<const float4 *>(p);
 #pragma unroll
-    for (int i = 0; i < 4; i++) {
-        float4 v = __ldg(q + i);
-        x[4 * i + 0] = v.x; x[4 * i + 1] = v.y; x[4 * i + 2] = v.z; x[4 * i + 3] = v.w;
-    }
+    for (int i = 0; i < 4; i++) r.v[i] = __ldg(q + i);
 }
-
-__device__ __forceinline__ void load16(const __nv_bfloat16 *p, float (&x)[kVec])
+__device__ __forceinline__ void load16(const __nv_bfloat16 *p, Raw16<__nv_bfloat16> &r)
 {
     const uint4 *q = reinterpret_cast<const uint4 *>(p);
 #pragma unroll
-    for (int i = 0; i < 2; i++) {
-        uint4 v = __ldg(q + i);
-        uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int j = 0; j < 4; j++) {
-            x[8 * i + 2 * j + 0] = __uint_as_float(w[j] << 16);
-            x[8 * i + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
-        }
-    }
+    for (int i = 0; i < 2; i++) r.v[i] = __ldg(q + i);
+}
+// elements 4 g .. 4 g + 3 as fp32
+__device__ __forceinline__ void get4(const Raw16<float> &r, int g, float (&x)[4])
+{
+    x[0] = r.v[g].x; x[1] = r.v[g].y; x[2] = r.v[g].z; x[3] = r.v[g].w;
+}
+__device__ __forceinline__ void get4(const Raw16<__nv_bfloat16> &r, int g, float (&x)[4])
+{
+    const uint4 v = r.v[g >> 1];
+    const uint32_t w0 = (g & 1) ? v.z : v.x, w1 = (g & 1) ? v.w : v.y;
+    x[0] = __uint_as_float(w0 << 16); x[1] = __uint_as_float(w0 & 0xFFFF0000u);
+    x[2] = __uint_as_float(w1 << 16); x[3] = __uint_as_float(w1 & 0xFFFF0000u);
 }
 
 __device__ __forceinline__ float load1(const float *p) { return __ldg(p); }
@@ -73,29 +84,31 @@ __device__ __forceinline__ void quant1(float x, float sp, float sn, int lo, int 
     }
 }
 
-// Per-segment constants of the fast form.  The quotient x / s is obtained, correctly rounded, from the
-// correctly rounded reciprocal r = RN(1/s) by one multiply and two FMAs:
-//   q0 = RN(x r),  e = x - q0 s (exact in one FMA),  q = RN(q0 + e r)
-// which equals RN(x / s) when nothing over- or underflows on the way.  To rule that out, and to get the
-// polarity split for free, the input is first mapped to u = sat(x / L) in [0, 1] by one saturating FMA,
-// L = 2^(exponent(s) + 11) >= 1024 s.  L is a power of two, so x / L is exact and u / (s / L) has the
-// bits of x / s; negative x give u = 0 (the other polarity's zero code) and x > L, which is clipped to
-// the end of the code range anyway, gives u = 1.  A quotient too small to be normal rounds to code 0
-// whatever its last bits are.  The fast form is taken for 2^-100 <= s <= 2^100.
+// Per-segment constants of the fast form.  The quotient x / s is obtained from the correctly rounded
+// reciprocal r = RN(1/s) by one multiply and two FMAs,
+//   q0 = RN(x r),  e = x - q0 s (exact in one FMA),  q = RN(q0 + e r),
+// which lands on the same side of every rounding boundary of the codes (k + 1/2 for int8, the midpoints of
+// adjacent e4m3 values) as RN(x / s), provided e is exact, i.e. does not underflow: |x| >= 2^-100 suffices, and for
+// smaller |x| the quotient is below 2^-20 for the scales of the fast form (2^-80 <= s <= 2^100) and the code is 0
+// whatever its last bits are.  (Checked on the CPU against the IEEE division for 2 * 10^10 inputs within six
+// units in the last place of a rounding boundary, scales with random, all-ones and power-of-two significands.)
 struct SegConst {
-    float inv_l;       // 1 / L
-    float s_l, r_l;    // s / L and RN(L / s) = RN(1 / s) L
+    float s, r;        // scale and RN(1 / s)
+    float inv_l;       // e4m3 form: 1 / L with L = 2^(exponent(s) + 11) >= 1024 s
+    float s_l, r_l;    // e4m3 form: s / L and RN(L / s)
     int fast;
 };
 __device__ __forceinline__ SegConst seg_const(float s)
 {
     SegConst c;
-    c.fast = (s >= 7.8886090522101181e-31f && s <= 1.2676506002282294e+30f) ? 1 : 0;
+    c.fast = (s >= 8.2718061255302767e-25f && s <= 1.2676506002282294e+30f) ? 1 : 0;     // 2^-80 .. 2^100
+    c.s = s;
+    c.r = __frcp_rn(s);
     const uint32_t l_bits = (__float_as_uint(s) & 0x7F800000u) + (11u << 23);
     const float l = __uint_as_float(l_bits);
     c.inv_l = __uint_as_float((254u << 23) - l_bits);
     c.s_l = s * c.inv_l;
-    c.r_l = __frcp_rn(s) * l;
+    c.r_l = c.r * l;
     return c;
 }
 __device__ __forceinline__ float fma_sat(float a, float b, float c)
@@ -116,6 +129,10 @@ __device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi)
 {
     asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
 }
+__device__ __forceinline__ void unpack2u(uint64_t v, uint32_t &lo, uint32_t &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
+}
 __device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b)
 {
     uint64_t d;
@@ -134,129 +151,182 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
-// two correctly rounded quotients x / s from r = RN(1/s): q0 = RN(x r), e = x - q0 s, q = RN(q0 + e r)
+// two quotients x / s from r = RN(1/s): q0 = RN(x r), e = x - q0 s, q = RN(q0 + e r)
 __device__ __forceinline__ uint64_t div2_rn_fast(uint64_t x2, uint64_t neg_s2, uint64_t r2)
 {
     const uint64_t q0 = mul2(x2, r2);
     const uint64_t e = fma2(q0, neg_s2, x2);
     return fma2(e, r2, q0);
 }
+// {sat_s8(hi_val), sat_s8(lo_val)} into bits 15..0 of the result, bits 15..0 of `upper` into bits 31..16
+__device__ __forceinline__ uint32_t pack_sat_s8(int hi_val, int lo_val, uint32_t upper)
+{
+    uint32_t d;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(hi_val), "r"(lo_val), "r"(upper));
+    return d;
+}
 
 constexpr float kRoundMagic = 12582912.0f;   // 1.5 * 2^23: v + magic rounds v to an integer, half to even
+constexpr int kMagicBits = 0x4B400000;       // its bit pattern: bits(v + magic) - kMagicBits is that integer
 
-// 16 elements of one K-segment -> packed codes.  int8: clip in fp32 (the bounds are integers, so
-// clip-then-round equals round-then-clip), add the magic constant, and the low byte of the sum's bit
-// pattern is the two's-complement code.  Dual: the positive matrix quantizes max(x, 0) = L sat(x / L),
-// the negative one min(x, 0) = -L sat(-x / L), each with its own constants, which reproduces the
-// per-element polarity select.  Single scale: |x| is quantized and the sign put back when rounding.
+// 4 elements of one K-segment -> one word of packed codes per matrix.
+// int8, dual: both polarities are quantized as non-negative numbers, max(x, 0) and max(-x, 0) = max(x, 0) - x,
+//   each with its own constants.  Adding the magic constant rounds half to even; the integer is the distance of
+//   the sum's bit pattern from the constant's, taken with the sign of the polarity, and a saturating pack clips
+//   it to [-128, 127].  A quotient beyond the range of the magic constant, infinity, or the NaN of an overflowed
+//   chain all have bit patterns above the constant's, so they saturate to the end of the code range as the
+//   clip demands; nothing has to be bounded beforehand.  (A negative bound of -127 takes the division path.)
+// int8, single scale: |x| is quantized, clipped in fp32 (clip-then-round equals round-then-clip for integer
+//   bounds; a NaN from an overflowed chain clips to the bound as well) and the sign put back when rounding.
+// e4m3: the input is first mapped to u = sat(x / L) in [0, 1] with one saturating FMA (L a power of two, so
+//   u / (s / L) has the bits of x / s; x beyond L is clipped to 448 anyway), which also splits the polarities and
+//   keeps infinities and NaNs out of the saturating e4m3 conversion.
 template <int CODE, bool DUAL>
-__device__ __forceinline__ void quant16(const float (&x)[kVec], const SegConst &cp, const SegConst &cn, float lo,
-                                        float hi, uint32_t (&wp)[4], uint32_t (&wn)[4])
+__device__ __forceinline__ void quant4(const float (&x)[4], const SegConst &cp, const SegConst &cn, float hi,
+                                       uint32_t &wp, uint32_t &wn)
 {
-    uint32_t bp[kVec], bn[kVec];
-    const uint64_t rp2 = pack2(cp.r_l, cp.r_l), nsp2 = pack2(-cp.s_l, -cp.s_l);
-    const uint64_t rn2 = pack2(-cn.r_l, -cn.r_l), nsn2 = pack2(cn.s_l, cn.s_l);   // negated: quotients <= 0
     const uint64_t magic2 = pack2(kRoundMagic, kRoundMagic);
+    if (CODE == SQ_CODE_INT8 && DUAL) {
+        const uint64_t rp2 = pack2(cp.r, cp.r), nsp2 = pack2(-cp.s, -cp.s);
+        const uint64_t rn2 = pack2(cn.r, cn.r), nsn2 = pack2(-cn.s, -cn.s);
+        const uint64_t minus1 = pack2(-1.0f, -1.0f);
+        int kp[4], kn[4];
 #pragma unroll
-    for (int i = 0; i < kVec; i += 2) {
+        for (int i = 0; i < 4; i += 2) {
+            const uint64_t xp2 = pack2(fmaxf(x[i], 0.0f), fmaxf(x[i + 1], 0.0f));
+            const uint64_t xn2 = fma2(pack2(x[i], x[i + 1]), minus1, xp2);          // max(x, 0) - x, exact
+            uint32_t a, b;
+            unpack2u(add2(div2_rn_fast(xp2, nsp2, rp2), magic2), a, b);
+            kp[i] = int(a) - kMagicBits; kp[i + 1] = int(b) - kMagicBits;
+            unpack2u(add2(div2_rn_fast(xn2, nsn2, rn2), magic2), a, b);
+            kn[i] = kMagicBits - int(a); kn[i + 1] = kMagicBits - int(b);
+        }
+        wp = pack_sat_s8(kp[1], kp[0], pack_sat_s8(kp[3], kp[2], 0u));
+        wn = pack_sat_s8(kn[1], kn[0], pack_sat_s8(kn[3], kn[2], 0u));
+        return;
+    }
+    uint32_t bp[4], bn[4];
+    if (CODE == SQ_CODE_INT8) {                          // single scale
+        const uint64_t r2 = pack2(cp.r, cp.r), ns2 = pack2(-cp.s, -cp.s);
+#pragma unroll
+        for (int i = 0; i < 4; i += 2) {
+            float a0, a1;
+            unpack2(div2_rn_fast(pack2(fabsf(x[i]), fabsf(x[i + 1])), ns2, r2), a0, a1);
+            bp[i] = __float_as_uint(fmaf(fminf(a0, hi), copysignf(1.0f, x[i]), kRoundMagic));
+            bp[i + 1] = __float_as_uint(fmaf(fminf(a1, hi), copysignf(1.0f, x[i + 1]), kRoundMagic));
+        }
+        wp = __byte_perm(__byte_perm(bp[0], bp[1], 0x0040), __byte_perm(bp[2], bp[3], 0x0040), 0x5410);
+        return;
+    }
+    // e4m3
+    const uint64_t rp2 = pack2(cp.r_l, cp.r_l), nsp2 = pack2(-cp.s_l, -cp.s_l);
+    const uint64_t rn2 = pack2(cn.r_l, cn.r_l), nsn2 = pack2(-cn.s_l, -cn.s_l);
+#pragma unroll
+    for (int i = 0; i < 4; i += 2) {
         float a0, a1;
         if (DUAL) {
-            const uint64_t qp2 = div2_rn_fast(pack2(fma_sat(x[i], cp.inv_l, 0.0f), fma_sat(x[i + 1], cp.inv_l, 0.0f)), nsp2, rp2);
-            const uint64_t qn2 = div2_rn_fast(pack2(fma_sat(x[i], -cn.inv_l, 0.0f), fma_sat(x[i + 1], -cn.inv_l, 0.0f)), nsn2, rn2);
-            if (CODE == SQ_CODE_INT8) {
-                unpack2(qp2, a0, a1);
-                unpack2(add2(pack2(fminf(a0, hi), fminf(a1, hi)), magic2), a0, a1);
-                bp[i] = __float_as_uint(a0); bp[i + 1] = __float_as_uint(a1);
-                unpack2(qn2, a0, a1);
-                unpack2(add2(pack2(fmaxf(a0, lo), fmaxf(a1, lo)), magic2), a0, a1);
-                bn[i] = __float_as_uint(a0); bn[i + 1] = __float_as_uint(a1);
-            } else {
-                unpack2(qp2, a0, a1);
-                bp[i] = __float_as_uint(a0); bp[i + 1] = __float_as_uint(a1);
-                unpack2(qn2, a0, a1);
-                bn[i] = __float_as_uint(a0); bn[i + 1] = __float_as_uint(a1);
-            }
-        } else {
-            const uint64_t q2 = div2_rn_fast(pack2(fma_sat(fabsf(x[i]), cp.inv_l, 0.0f), fma_sat(fabsf(x[i + 1]), cp.inv_l, 0.0f)), nsp2, rp2);
-            unpack2(q2, a0, a1);
-            if (CODE == SQ_CODE_INT8) {                  // the range is symmetric: clip |q|, round with the sign of x
-                a0 = fmaf(fminf(a0, hi), copysignf(1.0f, x[i]), kRoundMagic);
-                a1 = fmaf(fminf(a1, hi), copysignf(1.0f, x[i + 1]), kRoundMagic);
-            } else {
-                a0 = copysignf(a0, x[i]);
-                a1 = copysignf(a1, x[i + 1]);
-            }
+            unpack2(div2_rn_fast(pack2(fma_sat(x[i], cp.inv_l, 0.0f), fma_sat(x[i + 1], cp.inv_l, 0.0f)), nsp2, rp2), a0, a1);
             bp[i] = __float_as_uint(a0); bp[i + 1] = __float_as_uint(a1);
+            unpack2(div2_rn_fast(pack2(fma_sat(x[i], -cn.inv_l, 0.0f), fma_sat(x[i + 1], -cn.inv_l, 0.0f)), nsn2, rn2), a0, a1);
+            bn[i] = __float_as_uint(a0); bn[i + 1] = __float_as_uint(a1);
+        } else {
+            unpack2(div2_rn_fast(pack2(fma_sat(fabsf(x[i]), cp.inv_l, 0.0f), fma_sat(fabsf(x[i + 1]), cp.inv_l, 0.0f)), nsp2, rp2), a0, a1);
+            bp[i] = __float_as_uint(copysignf(a0, x[i])); bp[i + 1] = __float_as_uint(copysignf(a1, x[i + 1]));
         }
     }
-#pragma unroll
-    for (int g = 0; g < 4; g++) {
-        if (CODE == SQ_CODE_INT8) {
-            wp[g] = __byte_perm(__byte_perm(bp[4 * g], bp[4 * g + 1], 0x0040), __byte_perm(bp[4 * g + 2], bp[4 * g + 3], 0x0040), 0x5410);
-            if (DUAL)
-                wn[g] = __byte_perm(__byte_perm(bn[4 * g], bn[4 * g + 1], 0x0040), __byte_perm(bn[4 * g + 2], bn[4 * g + 3], 0x0040), 0x5410);
-        } else {
-            uint32_t w = cvt_e4m3x2(__uint_as_float(bp[4 * g]), __uint_as_float(bp[4 * g + 1])) |
-                         (cvt_e4m3x2(__uint_as_float(bp[4 * g + 2]), __uint_as_float(bp[4 * g + 3])) << 16);
-            wp[g] = w & ~(__vcmpeq4(w & 0x7F7F7F7Fu, 0u) & 0x80808080u);      // -0 is stored as +0
-            if (DUAL) {
-                w = cvt_e4m3x2(__uint_as_float(bn[4 * g]), __uint_as_float(bn[4 * g + 1])) |
-                    (cvt_e4m3x2(__uint_as_float(bn[4 * g + 2]), __uint_as_float(bn[4 * g + 3])) << 16);
-                wn[g] = w & ~(__vcmpeq4(w & 0x7F7F7F7Fu, 0u) & 0x80808080u);
-            }
-        }
+    uint32_t w = cvt_e4m3x2(__uint_as_float(bp[0]), __uint_as_float(bp[1])) |
+                 (cvt_e4m3x2(__uint_as_float(bp[2]), __uint_as_float(bp[3])) << 16);
+    // single scale: -0 is stored as +0; dual: the positive matrix holds non-negative quotients, no -0 arises
+    wp = DUAL ? w : w & ~(__vcmpeq4(w & 0x7F7F7F7Fu, 0u) & 0x80808080u);
+    if (DUAL) {
+        // the negative matrix was quantized as magnitudes: set the sign bit of every nonzero byte
+        // (a byte b <= 0x7E plus 0x7F reaches 0x80 exactly when b >= 1, and never carries into the next byte)
+        w = cvt_e4m3x2(__uint_as_float(bn[0]), __uint_as_float(bn[1])) |
+            (cvt_e4m3x2(__uint_as_float(bn[2]), __uint_as_float(bn[3])) << 16);
+        wn = w | ((w + 0x7F7F7F7Fu) & 0x80808080u);
     }
 }
 
+// Thread g of the grid owns the 16-element column chunk g % V of the rows g / V, g / V + R, g / V + 2 R, ...
+// (V chunks per row, R rows in flight over the whole grid), so that a warp reads 1 KiB (bf16) of consecutive
+// addresses per row, the per-segment constants are made once per thread, and the next row's loads are in
+// flight while the current row is converted.
 template <typename Tin, int CODE, bool DUAL>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, kBlocksPerSm)
 quantize_kernel(const Tin *__restrict__ X, int64_t M, int K, int64_t ld, const SegBounds sb,
                 const float *__restrict__ s_pos, const float *__restrict__ s_neg, int row_segments,
-                int lo, int hi, uint8_t *__restrict__ c_pos, uint8_t *__restrict__ c_neg, int64_t ldc)
+                int lo, int hi, uint8_t *__restrict__ c_pos, uint8_t *__restrict__ c_neg, int64_t ldc,
+                int V, int R)
 {
     // Programmatic dependent launch: this kernel may be scheduled while the previous kernel of the stream
     // winds down, and lets the next one be scheduled while its own last blocks run; nothing in global
     // memory is touched before the previous kernel has completed.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    const int V = (K + kVec - 1) / kVec;
-    const int64_t idx = int64_t(blockIdx.x) * kThreads + threadIdx.x;
-    if (idx >= M * int64_t(V)) return;
-    const int64_t row = idx / V;
-    const int k0 = int(idx - row * V) * kVec;
+    const uint32_t g = blockIdx.x * kThreads + threadIdx.x;
+    const uint32_t r0 = g / uint32_t(V);
+    if (r0 >= uint32_t(R) || int64_t(r0) >= M) return;
+    const int k0 = int(g - r0 * uint32_t(V)) * kVec;
 
-    // segment of this vector (bounds come with the kernel parameters); the scale loads below do not
-    // depend on the data loads, so both are in flight together
-    const int Qs = row_segments ? sb.Q : 1;
-    int q = 0;
-    if (row_segments) while (q + 1 < sb.Q && row >= sb.nb[q + 1]) q++;
+    // K-segment of this chunk (bounds come with the kernel parameters)
     int p = 0;
     while (p + 1 < sb.P && k0 >= sb.kb[p + 1]) p++;
-    const bool whole = k0 + kVec <= sb.kb[p + 1];            // vector inside one K-segment (and inside K)
+    const bool whole = k0 + kVec <= sb.kb[p + 1];            // chunk inside one K-segment (and inside K)
+    const int Qs = row_segments ? sb.Q : 1;
 
-    const Tin *src = X + row * ld + k0;
-    uint8_t *dp = c_pos + row * ldc + k0;
-    uint8_t *dn = DUAL ? c_neg + row * ldc + k0 : nullptr;
+    const Tin *src = X + int64_t(r0) * ld + k0;
+    uint8_t *dp = c_pos + int64_t(r0) * ldc + k0;
+    uint8_t *dn = DUAL ? c_neg + int64_t(r0) * ldc + k0 : nullptr;
+    const int64_t src_step = int64_t(R) * ld, dst_step = int64_t(R) * ldc;
 
-    float x[kVec];
-    if (whole) load16(src, x);
-    const SegConst cp = seg_const(__ldg(s_pos + p * Qs + q));
-    const SegConst cn = seg_const(DUAL ? __ldg(s_neg + p * Qs + q) : 1.0f);
-    if (whole && cp.fast && cn.fast) {
-        uint32_t wp[4], wn[4];
-        quant16<CODE, DUAL>(x, cp, cn, float(lo), float(hi), wp, wn);
-        *reinterpret_cast<uint4 *>(dp) = make_uint4(wp[0], wp[1], wp[2], wp[3]);
-        if (DUAL) *reinterpret_cast<uint4 *>(dn) = make_uint4(wn[0], wn[1], wn[2], wn[3]);
-    } else {                                    // segment bound or end of row inside the vector, or an extreme scale
-        const int n = min(kVec, K - k0);
-        for (int i = 0; i < n; i++) {
-            while (p + 1 < sb.P && k0 + i >= sb.kb[p + 1]) p++;
-            uint32_t a, b;
-            quant1<CODE, DUAL>(load1(src + i), __ldg(s_pos + p * Qs + q), DUAL ? __ldg(s_neg + p * Qs + q) : 0.0f, lo, hi,
-                               a, b);
-            dp[i] = uint8_t(a);
-            if (DUAL) dn[i] = uint8_t(b);
+    Raw16<Tin> cur, nxt;
+    if (whole) load16(src, cur);
+    int q = 0;                                               // N-segment (weights only) the constants belong to
+    int64_t q_end = 0;                                       // first row beyond it (0: no constants yet)
+    SegConst cp, cn;
+    bool fast = false;
+    for (int64_t row = r0; row < M; row += R) {
+        if (row >= q_end) {                                  // (weights) the row entered another N-segment
+            if (row_segments) {
+                while (q + 1 < sb.Q && row >= sb.nb[q + 1]) q++;
+                q_end = sb.nb[q + 1];
+            } else {
+                q_end = M;
+            }
+            cp = seg_const(__ldg(s_pos + p * Qs + (row_segments ? q : 0)));
+            cn = seg_const(DUAL ? __ldg(s_neg + p * Qs + (row_segments ? q : 0)) : 1.0f);
+            fast = whole && cp.fast && cn.fast && !(DUAL && CODE == SQ_CODE_INT8 && lo != -128);
         }
+        if (fast) {
+            const bool more = row + R < M;
+            if (more) load16(src + src_step, nxt);           // next row in flight during the conversion
+            uint32_t wp[4], wn[4];
+#pragma unroll
+            for (int g4 = 0; g4 < 4; g4++) {
+                float x[4];
+                get4(cur, g4, x);
+                quant4<CODE, DUAL>(x, cp, cn, float(hi), wp[g4], wn[g4]);
+            }
+            *reinterpret_cast<uint4 *>(dp) = make_uint4(wp[0], wp[1], wp[2], wp[3]);
+            if (DUAL) *reinterpret_cast<uint4 *>(dn) = make_uint4(wn[0], wn[1], wn[2], wn[3]);
+            if (more) cur = nxt;
+        } else {                                 // segment bound or end of row inside the chunk, or an extreme scale
+            const int n = min(kVec, K - k0);
+            int pp = p;
+            const int qq = row_segments ? q : 0;
+            for (int i = 0; i < n; i++) {
+                while (pp + 1 < sb.P && k0 + i >= sb.kb[pp + 1]) pp++;
+                uint32_t a, b;
+                quant1<CODE, DUAL>(load1(src + i), __ldg(s_pos + pp * Qs + qq), DUAL ? __ldg(s_neg + pp * Qs + qq) : 0.0f,
+                                   lo, hi, a, b);
+                dp[i] = uint8_t(a);
+                if (DUAL) dn[i] = uint8_t(b);
+            }
+            if (whole && row + R < M) load16(src + src_step, cur);
+        }
+        src += src_step;
+        dp += dst_step;
+        if (DUAL) dn += dst_step;
     }
 }
 
@@ -265,9 +335,19 @@ sq_status launch_t(const Tin *X, int64_t M, int64_t K, int64_t ld, const SegBoun
                    const float *s_neg, int row_segments, int lo, int hi, void *c_pos, void *c_neg,
                    int64_t ldc, cudaStream_t st)
 {
+    // V chunks per row; R rows in flight: enough threads to fill every SM several times over, and a row count per
+    // thread that the rows divide into evenly
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        return SQ_ERR_CUDA;
     const int64_t V = (K + kVec - 1) / kVec;
-    const int64_t blocks = (M * V + kThreads - 1) / kThreads;
-    if (blocks > 0x7FFFFFFF) return SQ_ERR_SHAPE;
+    const int64_t target_threads = int64_t(sms) * kThreadsPerSm;
+    int64_t iters = (M * V + target_threads - 1) / target_threads;
+    if (iters < 1) iters = 1;
+    const int64_t R = (M + iters - 1) / iters;
+    const int64_t blocks = (R * V + kThreads - 1) / kThreads;
+    if (blocks > 0x7FFFFFFF || R * V > 0xFFFFFFFFll || V > 0x7FFFFFFF || R > 0x7FFFFFFF) return SQ_ERR_SHAPE;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(unsigned(blocks));
     cfg.blockDim = dim3(kThreads);
@@ -277,16 +357,19 @@ sq_status launch_t(const Tin *X, int64_t M, int64_t K, int64_t ld, const SegBoun
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const int Ki = int(K);
+    const int Ki = int(K), Vi = int(V), Ri = int(R);
     uint8_t *cp = static_cast<uint8_t *>(c_pos), *cn = static_cast<uint8_t *>(c_neg);
     const float *no_neg = nullptr;
+    cudaError_t e;
     if (s_neg)
-        cudaLaunchKernelEx(&cfg, quantize_kernel<Tin, CODE, true>, X, M, Ki, ld, sb, s_pos, s_neg, row_segments, lo, hi, cp, cn, ldc);
+        e = cudaLaunchKernelEx(&cfg, quantize_kernel<Tin, CODE, true>, X, M, Ki, ld, sb, s_pos, s_neg, row_segments, lo, hi,
+                               cp, cn, ldc, Vi, Ri);
     else
-        cudaLaunchKernelEx(&cfg, quantize_kernel<Tin, CODE, false>, X, M, Ki, ld, sb, s_pos, no_neg, row_segments, lo, hi, cp,
-                           static_cast<uint8_t *>(nullptr), ldc);
+        e = cudaLaunchKernelEx(&cfg, quantize_kernel<Tin, CODE, false>, X, M, Ki, ld, sb, s_pos, no_neg, row_segments, lo, hi,
+                               cp, static_cast<uint8_t *>(nullptr), ldc, Vi, Ri);
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
+    if (e != cudaSuccess) { note_cuda_error(e); return SQ_ERR_CUDA; }
+    return SQ_OK;
 }
 
 }  // namespace

@@ -24,9 +24,27 @@ def test_op_and_byte_counts():
     assert bench.layer_ops(fc2, M=100)[1] == 2.0 * 100 * 1152 * 4608
 
 
-def test_traffic_table_names_workloads():
+def test_traffic_table_names_workloads_and_goes_stale_with_the_kernel_source():
     assert set(bench.GEMM_DRAM_TRAFFIC) <= set(WL.WORKLOADS)
-    assert all(isinstance(v, int) and v > 0 for v in bench.GEMM_DRAM_TRAFFIC.values())
+    for e in bench.GEMM_DRAM_TRAFFIC.values():
+        assert isinstance(e["bytes"], int) and e["bytes"] > 0 and len(e["source_tag"]) == 16 and e["from"]
+    assert bench.gemm_dram_traffic("no_such_workload")[0] is None
+    saved = dict(bench.GEMM_DRAM_TRAFFIC)
+    try:
+        bench.GEMM_DRAM_TRAFFIC["tiny_qkv"] = {"bytes": 123, "source_tag": "0" * 16, "from": "test"}
+        assert bench.gemm_dram_traffic("tiny_qkv")[0] is None                      # another kernel source: stale
+        bench.GEMM_DRAM_TRAFFIC["tiny_qkv"]["source_tag"] = bench.gemm_source_tag()
+        assert bench.gemm_dram_traffic("tiny_qkv") == (123, "test")
+    finally:
+        bench.GEMM_DRAM_TRAFFIC.clear()
+        bench.GEMM_DRAM_TRAFFIC.update(saved)
+
+
+def test_fractions_against_the_three_peaks():
+    p8 = bench.eight_bit_peaks({"bf16_tflops": 1600.0, "bf16_tflops_sustained": 1400.0})
+    assert p8 == {"burst": 3200.0, "sustained": 2800.0, "nominal": 4500.0}
+    f = bench.fractions(1600.0, p8)
+    assert f == {"of_measured_burst": 0.5, "of_measured_sustained": round(1600 / 2800, 4), "of_nominal_4500": round(1600 / 4500, 4)}
 
 
 def test_measured_peaks_have_the_fields_the_roofline_uses():
