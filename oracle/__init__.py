@@ -53,6 +53,10 @@ def lib():
         _lib.sqo_bf16_from_f64.argtypes = [C.c_double]
         _lib.sqo_accumulate_i8.restype = C.c_int64
         _lib.sqo_num_threads.restype = C.c_int
+        _lib.sqo_silu.restype = C.c_double
+        _lib.sqo_silu.argtypes = [C.c_double]
+        _lib.sqo_gelu.restype = C.c_double
+        _lib.sqo_gelu.argtypes = [C.c_double]
     return _lib
 
 
@@ -225,6 +229,115 @@ def e4m3_encode(values):
     v = _f32(values)
     f = lib().sqo_e4m3_encode
     return np.array([f(float(x)) for x in v.ravel()], np.uint8).reshape(v.shape)
+
+
+# ------------------------------------------- comparison scheme: zero-point quantization (App. A)
+
+def calib_act_asym(X, kb, q_min=-128.0, q_max=127.0):
+    """(s [P] fp32, z [P] int32) per K-segment from strict min/max with the range widened to contain 0."""
+    X = _f32(X)
+    kb = _i32(kb)
+    P = len(kb) - 1
+    s = np.zeros(P, np.float32)
+    z = np.zeros(P, np.int32)
+    lib().sqo_calib_act_asym(_p(X), C.c_int64(X.shape[0]), C.c_int64(X.shape[1]), C.c_int64(X.shape[1]),
+                             C.c_int(P), _p(kb), C.c_float(q_min), C.c_float(q_max), _p(s), _p(z))
+    return s, z
+
+
+def quantize_act_asym(X, kb, s, z, q_min=-128.0, q_max=127.0):
+    """int8 codes clip(round(x / s[p]) + z[p], q_min, q_max)."""
+    X = _f32(X)
+    kb = _i32(kb)
+    M, K = X.shape
+    c = np.zeros((M, K), np.int8)
+    lib().sqo_quantize_act_asym_i8(_p(X), C.c_int64(M), C.c_int64(K), C.c_int64(K), C.c_int(len(kb) - 1), _p(kb),
+                                   _p(_f32(s)), _p(_i32(z)), C.c_float(q_min), C.c_float(q_max), _p(c), C.c_int64(K))
+    return c
+
+
+def segment_sums(A, kb):
+    """out[p, r] = sum over K-segment p of the int8 codes A[r, k] (exact)."""
+    A = np.ascontiguousarray(A, np.int8)
+    kb = _i32(kb)
+    out = np.zeros((len(kb) - 1, A.shape[0]), np.int64)
+    lib().sqo_segment_sums_i8(_p(A), C.c_int64(A.shape[1]), C.c_int64(A.shape[0]), C.c_int(len(kb) - 1), _p(kb), _p(out))
+    return out
+
+
+def dequant_asym(acc, xsum, wsum, kb, nb, s_x, z_x, s_w, z_w=None, bias=None):
+    """App. A asymmetric recovery in fp64; returns (y, sum of |terms|)."""
+    kb, nb = _i32(kb), _i32(nb)
+    P, M, N = acc.shape
+    Q = len(nb) - 1
+    acc = np.ascontiguousarray(acc, np.float64)
+    xsum = np.ascontiguousarray(xsum, np.int64)
+    wsum = np.ascontiguousarray(wsum, np.int64)
+    y = np.zeros((M, N), np.float64)
+    ya = np.zeros((M, N), np.float64)
+    zw = None if z_w is None else _i32(np.asarray(z_w).reshape(P, Q))
+    b = None if bias is None else _f32(bias)
+    lib().sqo_dequant_asym(_p(acc), _p(xsum), _p(wsum), C.c_int64(M), C.c_int64(N), C.c_int(P), _p(kb), C.c_int(Q),
+                           _p(nb), _p(_f32(s_x)), _p(_i32(z_x)), _p(_f32(s_w).reshape(P, Q)), _p(zw), _p(b), _p(y), _p(ya))
+    return y, ya
+
+
+def fold_zero_point(wsum, nb, s_x, z_x, s_w, bias=None):
+    """bias'[n] = bias[n] - sum_p s_x[p] s_w[p][q(n)] z_x[p] wsum[p][n] in fp64 (symmetric weights)."""
+    nb = _i32(nb)
+    wsum = np.ascontiguousarray(wsum, np.int64)
+    P, N = wsum.shape
+    Q = len(nb) - 1
+    out = np.zeros(N, np.float64)
+    b = None if bias is None else _f32(bias)
+    lib().sqo_fold_zero_point(_p(wsum), C.c_int64(N), C.c_int(P), C.c_int(Q), _p(nb), _p(_f32(s_x)), _p(_i32(z_x)),
+                              _p(_f32(s_w).reshape(P, Q)), _p(b), _p(out))
+    return out
+
+
+@dataclass
+class AsymResult:
+    codes: np.ndarray
+    acc: np.ndarray
+    wsum: np.ndarray
+    bias_folded: np.ndarray
+    y64: np.ndarray
+    y_abs: np.ndarray
+
+
+def layer_forward_asym(X, Wq, seg: SegTable, s_x, z_x, s_w, bias=None) -> AsymResult:
+    """The zero-point scheme for one layer with symmetric weight codes: codes, accumulators, the unfolded
+    App. A recovery in fp64 and the folded bias."""
+    codes = quantize_act_asym(X, seg.kb, s_x, z_x)
+    acc = accumulate(codes, Wq, seg.kb, "int8")
+    xsum = segment_sums(codes, seg.kb)
+    wsum = segment_sums(Wq, seg.kb)
+    y64, y_abs = dequant_asym(acc, xsum, wsum, seg.kb, seg.nb, s_x, z_x, s_w, None, bias)
+    return AsymResult(codes, acc, wsum, fold_zero_point(wsum, seg.nb, s_x, z_x, s_w, bias), y64, y_abs)
+
+
+# ------------------------------------------- act-to-linear segment in front of the quantizer
+
+ACT = {"silu": 1, "gelu": 2}
+
+
+def activation(H, act: str, stored="bf16"):
+    """act(H) evaluated in fp64 and rounded once to the stored dtype; returns (fp32 array, fp64 exact values)."""
+    H = _f32(H)
+    out = np.zeros(H.shape, np.float32)
+    exact = np.zeros(H.shape, np.float64)
+    lib().sqo_activation(_p(H), C.c_int64(H.size), C.c_int(ACT[act]), C.c_int(int(stored == "bf16")), _p(out), _p(exact))
+    return out, exact
+
+
+def smooth(X, mult):
+    """fl32(x * mult[k]) per element."""
+    X = _f32(X)
+    mult = _f32(mult)
+    out = np.zeros(X.shape, np.float32)
+    lib().sqo_smooth(_p(X), C.c_int64(X.shape[0]), C.c_int64(X.shape[1]), C.c_int64(X.shape[1]), _p(mult), _p(out),
+                     C.c_int64(X.shape[1]))
+    return out
 
 
 # ----------------------------------------------------------- whole layer

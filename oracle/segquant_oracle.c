@@ -28,6 +28,10 @@
  * same precision on both sides of a parity test.  Everything after the codes is
  * exact integer arithmetic (int8 codes) or fp64 (e4m3 codes, dequantization).
  *
+ * Also here, for the rows next to the main path: the zero-point (asymmetric) scheme of App. A that DualScale is
+ * compared with, and the activation / per-channel multiplier of the act-to-linear segment in front of the
+ * quantizer (Sec. 4.3.2, Sec. 4.2.2 last paragraph).
+ *
  * Pins (see tests/test_oracle_pins.py): library quantizers of torch on CPU,
  * on-grid exact reconstruction, brute-force dot products, reduction of one
  * segment to per-tensor, reduction of equal dual scales to symmetric, the
@@ -306,6 +310,146 @@ void sqo_dequant(const double *acc_pos, const double *acc_neg,
             y[m * N + n] = v;
             if (ysum_abs) ysum_abs[m * N + n] = av;
         }
+}
+
+uint16_t sqo_bf16_from_f64(double v);
+
+/* ------------------------------------------- comparison scheme: zero-point (asymmetric) quantization */
+
+/* App. A writes the asymmetric quantizer as X^ = round(X / s_X) + z_X with an integer zero-point, recovered by
+ * X ~ s_X (X^ - z_X); this is the form taken here (the Sec. 3 display puts z inside the quotient instead, and
+ * its inverse does not match it).  One (s, z) pair per K-segment, from strict min/max over the calibration
+ * rows with the range widened to contain 0:
+ *   lo = min(min x, 0), hi = max(max x, 0), s = (hi - lo) / (q_max - q_min), z = q_min - round(lo / s)
+ * so that lo maps to q_min.  A zero range gives s = 1, z = 0.                                              */
+void sqo_calib_act_asym(const float *X, int64_t rows, int64_t K, int64_t ld,
+                        int P, const int32_t *kb, float q_min, float q_max,
+                        float *s, int32_t *z)
+{
+    (void)K;
+    for (int p = 0; p < P; p++) {
+        float hi = 0.0f, lo = 0.0f;
+        for (int64_t r = 0; r < rows; r++)
+            for (int64_t k = kb[p]; k < kb[p + 1]; k++) {
+                float x = X[r * ld + k];
+                if (x > hi) hi = x;
+                if (x < lo) lo = x;
+            }
+        float range = hi - lo;
+        if (range > 0.0f) {
+            s[p] = range / (q_max - q_min);
+            float zf = q_min - rne(lo / s[p]);
+            z[p] = (int32_t)clampf(zf, q_min, q_max);
+        } else {
+            s[p] = 1.0f;
+            z[p] = 0;
+        }
+    }
+}
+
+/* X^ = clip(round(x / s[p]) + z[p], q_min, q_max)   (App. A asymmetric quantizer, Sec. 3 clip), int8 codes. */
+void sqo_quantize_act_asym_i8(const float *X, int64_t M, int64_t K, int64_t ld,
+                              int P, const int32_t *kb, const float *s, const int32_t *z,
+                              float q_min, float q_max, int8_t *c, int64_t ldc)
+{
+    for (int64_t m = 0; m < M; m++)
+        for (int64_t k = 0; k < K; k++) {
+            int p = seg_of(k, P, kb);
+            float v = rne(X[m * ld + k] / s[p]);
+            v = clampf(v, -1.0e6f, 1.0e6f);                     /* keeps the integer sum below in range */
+            c[m * ldc + k] = (int8_t)clampf(v + (float)z[p], q_min, q_max);
+        }
+}
+
+/* xsum[p][m] = sum over K-segment p of X^[m][k];  wsum[p][n] = sum over K-segment p of W^[n][k]
+ * (the rowsum terms of the App. A recovery; "rowsum(W^)" there sums W in R^{k x n} over k).               */
+void sqo_segment_sums_i8(const int8_t *A, int64_t lda, int64_t rows, int P, const int32_t *kb, int64_t *out)
+{
+    for (int p = 0; p < P; p++)
+        for (int64_t r = 0; r < rows; r++) {
+            int64_t t = 0;
+            for (int64_t k = kb[p]; k < kb[p + 1]; k++) t += A[r * lda + k];
+            out[(int64_t)p * rows + r] = t;
+        }
+}
+
+/* App. A asymmetric recovery, per (K-segment, N-segment) block and summed over K-segments, in fp64:
+ *   y[m][n] = sum_p s_x[p] s_w[p][q] ( acc[p][m][n] - z_x[p] wsum[p][n] - z_w[p][q] xsum[p][m]
+ *                                      + k_p z_x[p] z_w[p][q] ) + bias[n],      k_p = kb[p+1] - kb[p].
+ * z_w may be NULL (symmetric weights).  ysum_abs as in sqo_dequant, every term counted separately.        */
+void sqo_dequant_asym(const double *acc, const int64_t *xsum, const int64_t *wsum,
+                      int64_t M, int64_t N, int P, const int32_t *kb, int Q, const int32_t *nb,
+                      const float *s_x, const int32_t *z_x, const float *s_w, const int32_t *z_w,
+                      const float *bias, double *y, double *ysum_abs)
+{
+    for (int64_t m = 0; m < M; m++)
+        for (int64_t n = 0; n < N; n++) {
+            int q = seg_of(n, Q, nb);
+            double v = 0.0, av = 0.0;
+            for (int p = 0; p < P; p++) {
+                double c = (double)s_x[p] * (double)s_w[p * Q + q];
+                double zx = (double)z_x[p], zw = z_w ? (double)z_w[p * Q + q] : 0.0;
+                double kp = (double)(kb[p + 1] - kb[p]);
+                double t0 = c * acc[((int64_t)p * M + m) * N + n];
+                double t1 = c * zx * (double)wsum[(int64_t)p * N + n];
+                double t2 = c * zw * (double)xsum[(int64_t)p * M + m];
+                double t3 = c * kp * zx * zw;
+                v += t0 - t1 - t2 + t3;
+                av += fabs(t0) + fabs(t1) + fabs(t2) + fabs(t3);
+            }
+            if (bias) { v += (double)bias[n]; av += fabs((double)bias[n]); }
+            y[m * N + n] = v;
+            if (ysum_abs) ysum_abs[m * N + n] = av;
+        }
+}
+
+/* With symmetric weights the zero-point term does not depend on the row and folds into the bias offline:
+ *   bias'[n] = bias[n] - sum_p s_x[p] s_w[p][q(n)] z_x[p] wsum[p][n]      (fp64)                          */
+void sqo_fold_zero_point(const int64_t *wsum, int64_t N, int P, int Q, const int32_t *nb,
+                         const float *s_x, const int32_t *z_x, const float *s_w, const float *bias,
+                         double *bias_folded)
+{
+    for (int64_t n = 0; n < N; n++) {
+        int q = seg_of(n, Q, nb);
+        double v = bias ? (double)bias[n] : 0.0;
+        for (int p = 0; p < P; p++)
+            v -= (double)s_x[p] * (double)s_w[p * Q + q] * (double)z_x[p] * (double)wsum[(int64_t)p * N + n];
+        bias_folded[n] = v;
+    }
+}
+
+/* --------------------------------------------- act-to-linear segment in front of the quantizer (Sec. 4.3.2) */
+
+/* The activation functions DualScale is applied behind (App. B: SiLU, GELU), in fp64 from their definitions:
+ *   SiLU(h) = h / (1 + exp(-h)),   GELU(h) = h Phi(h) = (h / 2) erfc(-h / sqrt 2).                          */
+double sqo_silu(double h) { return h / (1.0 + exp(-h)); }
+double sqo_gelu(double h) { return 0.5 * h * erfc(-h / sqrt(2.0)); }
+
+/* act: 1 = SiLU, 2 = GELU.  The value is rounded ONCE from fp64 to the dtype the unfused graph would have
+ * stored it in (bf16 if stored_bf16, else fp32) and returned as fp32; `exact` (optional) receives the fp64 value. */
+void sqo_activation(const float *H, int64_t n, int act, int stored_bf16, float *out, double *exact)
+{
+    for (int64_t i = 0; i < n; i++) {
+        double a = act == 1 ? sqo_silu((double)H[i]) : sqo_gelu((double)H[i]);
+        if (exact) exact[i] = a;
+        if (stored_bf16) {
+            uint32_t bits = (uint32_t)sqo_bf16_from_f64(a) << 16;
+            float f;
+            memcpy(&f, &bits, 4);
+            out[i] = f;
+        } else {
+            out[i] = (float)a;
+        }
+    }
+}
+
+/* Per-channel multiplier in front of the quantizer (Sec. 4.2.2 last paragraph: SmoothQuant's migration, one
+ * strength per segment; the multiplier m[k] = 1 / smoothing factor is made offline): out = fl32(x * m[k]).   */
+void sqo_smooth(const float *X, int64_t M, int64_t K, int64_t ld, const float *mult, float *out, int64_t ldo)
+{
+    for (int64_t m = 0; m < M; m++)
+        for (int64_t k = 0; k < K; k++)
+            out[m * ldo + k] = X[m * ld + k] * mult[k];
 }
 
 /* fp64 -> bf16 bit pattern, round-to-nearest-even directly from the fp64 value

@@ -39,6 +39,23 @@ MUTATIONS = {
     "abs_sum_misses_bias": ("av += fabs((double)bias[n]); }", "}"),
     "abs_sum_misses_negative_path": ("v += u; av += fabs(u);", "v += u;"),
     "e4m3_weight_not_clipped": ("sqo_e4m3_encode(clampf(v, -448.0f, 448.0f))", "sqo_e4m3_encode(v * 0.5f)"),
+    "asym_zero_point_wrong_sign": ("float zf = q_min - rne(lo / s[p]);", "float zf = q_min + rne(lo / s[p]);"),
+    "asym_range_not_widened_to_zero": ("float hi = 0.0f, lo = 0.0f;\n        for (int64_t r = 0; r < rows; r++)",
+                                       "float hi = -INFINITY, lo = INFINITY;\n        for (int64_t r = 0; r < rows; r++)"),
+    "asym_zero_point_subtracted_in_codes": ("c[m * ldc + k] = (int8_t)clampf(v + (float)z[p], q_min, q_max);",
+                                            "c[m * ldc + k] = (int8_t)clampf(v - (float)z[p], q_min, q_max);"),
+    "asym_weight_sum_term_added": ("v += t0 - t1 - t2 + t3;", "v += t0 + t1 - t2 + t3;"),
+    "asym_constant_term_dropped": ("v += t0 - t1 - t2 + t3;", "v += t0 - t1 - t2;"),
+    "asym_row_sum_term_dropped": ("v += t0 - t1 - t2 + t3;", "v += t0 - t1 + t3;"),
+    "asym_fold_added": ("v -= (double)s_x[p] * (double)s_w[p * Q + q] * (double)z_x[p]", "v += (double)s_x[p] * (double)s_w[p * Q + q] * (double)z_x[p]"),
+    "asym_fold_scale_index_transposed": ("v -= (double)s_x[p] * (double)s_w[p * Q + q] * (double)z_x[p]", "v -= (double)s_x[p] * (double)s_w[q * P + p] * (double)z_x[p]"),
+    "segment_sum_skips_first": ("for (int64_t k = kb[p]; k < kb[p + 1]; k++) t += A[r * lda + k];",
+                                "for (int64_t k = kb[p] + 1; k < kb[p + 1]; k++) t += A[r * lda + k];"),
+    "silu_exponent_sign": ("return h / (1.0 + exp(-h));", "return h / (1.0 + exp(h));"),
+    "gelu_half_dropped": ("return 0.5 * h * erfc(-h / sqrt(2.0));", "return h * erfc(-h / sqrt(2.0));"),
+    "gelu_tanh_like_argument": ("return 0.5 * h * erfc(-h / sqrt(2.0));", "return 0.5 * h * erfc(-h / 2.0);"),
+    "activation_rounded_twice": ("uint32_t bits = (uint32_t)sqo_bf16_from_f64(a) << 16;", "uint32_t bits = (uint32_t)sqo_bf16_from_f64((double)(float)a + 1e-3 * a) << 16;"),
+    "smooth_indexed_by_row": ("out[m * ldo + k] = X[m * ld + k] * mult[k];", "out[m * ldo + k] = X[m * ld + k] * mult[m % K];"),
     "bf16_truncates": ("double q = nearbyint((f * 2.0 - 1.0) * 128.0);", "double q = floor((f * 2.0 - 1.0) * 128.0);"),
 }
 

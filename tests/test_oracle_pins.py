@@ -588,3 +588,185 @@ def test_bf16_rounding_matches_torch_on_fp32_inputs_and_ties():
     assert O.bf16_bits(np.array([tie + 2.0 ** -40]))[0] == 0x3F81
     assert O.bf16_bits(np.array([tie]))[0] == 0x3F80                  # tie -> even
     assert np.float32(tie + 2.0 ** -40) == np.float32(tie)            # fp32 cannot see the difference
+
+
+# --------------------------------------------------------------- zero-point (asymmetric) comparison scheme, App. A
+
+def torch_asym_codes(X, kb, s, z):
+    X = torch.from_numpy(np.asarray(X, np.float32))
+    sv = torch.zeros(X.shape[1]); zv = torch.zeros(X.shape[1])
+    for p in range(len(kb) - 1):
+        sv[kb[p]:kb[p + 1]] = float(s[p]); zv[kb[p]:kb[p + 1]] = float(z[p])
+    return torch.clamp(torch.round(X / sv) + zv, -128, 127).numpy().astype(np.int8)
+
+
+def test_asym_calibration_closed_form_and_range_ends():
+    r = rng(40)
+    kb = [0, 16, 48, 64]
+    X = gelu(r.normal(0, 1.5, (40, 64))).astype(np.float32)
+    X[:, 16:48] = np.abs(X[:, 16:48]) + 0.25                       # a segment without negative values
+    X[:, 48:] = 0.0                                                # an all-zero segment
+    s, z = O.calib_act_asym(X, kb)
+    lo, hi = min(float(X[:, :16].min()), 0.0), max(float(X[:, :16].max()), 0.0)
+    assert s[0] == (np.float32(hi) - np.float32(lo)) / np.float32(255.0)
+    assert z[0] == int(-128 - np.round(np.float32(lo) / s[0]))
+    assert s[1] == np.float32(X[:, 16:48].max()) / np.float32(255.0) and z[1] == -128     # range [0, max]
+    assert s[2] == 1.0 and z[2] == 0
+    c = O.quantize_act_asym(X, kb, s, z)
+    i_lo, i_hi = np.unravel_index(np.argmin(X[:, :16]), (40, 16)), np.unravel_index(np.argmax(X[:, :16]), (40, 16))
+    assert c[i_lo] == -128 and c[i_hi] in (126, 127)               # the ends of the range sit on the ends of the code range
+    assert np.all(c[:, 48:] == 0)
+    # inside the calibrated range the reconstruction s (c - z) is within half a step
+    for p in range(2):
+        ks = slice(kb[p], kb[p + 1])
+        rec = float(s[p]) * (c[:, ks].astype(np.float64) - int(z[p]))
+        assert np.all(np.abs(rec - X[:, ks]) <= float(s[p]) / 2 * (1 + 1e-6))
+
+
+def test_asym_codes_match_library_quantizer():
+    r = rng(41)
+    kb = [0, 24, 64]
+    X = gelu(r.standard_t(4, (60, 64))).astype(np.float32)
+    s, z = O.calib_act_asym(X[:6], kb)                              # few rows: run-time values exceed the range
+    assert len(set(z.tolist())) == 2
+    X[0, :6] = [0.0, -0.0, 1e30, -1e30, 2.5 * s[0], -0.5 * s[0]]    # clip far outside, exact ties
+    c = O.quantize_act_asym(X, kb, s, z)
+    assert np.array_equal(c, torch_asym_codes(X, kb, s, z))
+    assert (c == 127).any() and (c == -128).any()
+
+
+def asym_layer(X, W, kb, nb, bias=None):
+    s_x, z_x = O.calib_act_asym(X, kb)
+    s_w = O.calib_weight(W, kb, nb)
+    Wq = O.quantize_weight(W, kb, nb, s_w)
+    return O.layer_forward_asym(X, Wq, O.SegTable(kb, nb), s_x, z_x, s_w, bias), (s_x, z_x, s_w, Wq)
+
+
+def test_asym_recovery_equals_brute_force_with_both_zero_points():
+    r = rng(42)
+    M, N, K = 5, 6, 24
+    kb, nb = [0, 8, 24], [0, 2, 6]
+    P, Q = 2, 2
+    Xq = r.integers(-128, 128, (M, K)).astype(np.int8)
+    Wq = r.integers(-128, 128, (N, K)).astype(np.int8)
+    s_x = np.array([0.011, 0.37], np.float32); z_x = np.array([-77, 13], np.int32)
+    s_w = np.array([[0.002, 0.0031], [0.0007, 0.0013]], np.float32); z_w = np.array([[5, -9], [-3, 21]], np.int32)
+    bias = r.normal(0, 0.1, N).astype(np.float32)
+    acc = O.accumulate(Xq, Wq, kb)
+    xsum, wsum = O.segment_sums(Xq, kb), O.segment_sums(Wq, kb)
+    for p in range(P):
+        assert np.array_equal(xsum[p], Xq[:, kb[p]:kb[p + 1]].astype(np.int64).sum(axis=1))
+        assert np.array_equal(wsum[p], Wq[:, kb[p]:kb[p + 1]].astype(np.int64).sum(axis=1))
+    y, ya = O.dequant_asym(acc, xsum, wsum, kb, nb, s_x, z_x, s_w, z_w, bias)
+    for m in range(M):
+        for n in range(N):
+            q = 0 if n < 2 else 1
+            tot, tot_abs = float(bias[n]), abs(float(bias[n]))
+            for k in range(K):
+                p = 0 if k < 8 else 1
+                tot += float(s_x[p]) * (int(Xq[m, k]) - int(z_x[p])) * float(s_w[p, q]) * (int(Wq[n, k]) - int(z_w[p, q]))
+            for p in range(P):
+                c = float(s_x[p]) * float(s_w[p, q])
+                kp = kb[p + 1] - kb[p]
+                tot_abs += abs(c * int(acc[p, m, n])) + abs(c * int(z_x[p]) * int(wsum[p, n])) + \
+                    abs(c * int(z_w[p, q]) * int(xsum[p, m])) + abs(c * kp * int(z_x[p]) * int(z_w[p, q]))
+            assert math.isclose(y[m, n], tot, rel_tol=1e-11, abs_tol=1e-13)
+            assert math.isclose(ya[m, n], tot_abs, rel_tol=1e-12)
+
+
+def test_asym_with_zero_zero_points_is_the_symmetric_recovery():
+    r = rng(43)
+    kb, nb = [0, 32, 64], [0, 8, 16]
+    X = r.normal(0, 1, (12, 64)).astype(np.float32)
+    W = r.normal(0, 0.02, (16, 64)).astype(np.float32)
+    s, _ = O.calib_act(X, kb, dual=False)
+    s_w = O.calib_weight(W, kb, nb)
+    Wq = O.quantize_weight(W, kb, nb, s_w)
+    bias = r.normal(0, 0.1, 16).astype(np.float32)
+    sym = O.layer_forward(X, Wq, O.SegTable(kb, nb), s, None, s_w, bias)
+    z0 = np.zeros(2, np.int32)
+    asym = O.layer_forward_asym(X, Wq, O.SegTable(kb, nb), s, z0, s_w, bias)
+    assert np.array_equal(asym.codes, sym.c_pos) and np.array_equal(asym.acc, sym.acc_pos)
+    assert np.array_equal(asym.y64, sym.y64) and np.allclose(asym.y_abs, sym.y_abs, rtol=1e-14)
+    assert np.array_equal(asym.bias_folded, bias.astype(np.float64))
+
+
+def test_asym_folded_bias_gives_the_unfolded_recovery():
+    r = rng(44)
+    kb, nb = [0, 16, 56], [0, 8, 24, 30]
+    X = gelu(r.normal(0, 1.5, (14, 56))).astype(np.float32)
+    X[:, 16:] *= 4.0
+    W = r.normal(0, 0.02, (30, 56)).astype(np.float32)
+    W[8:24] *= 5.0
+    bias = r.normal(0, 0.1, 30).astype(np.float32)
+    res, (s_x, z_x, s_w, Wq) = asym_layer(X, W, kb, nb, bias)
+    assert (z_x != 0).all()
+    # symmetric recovery of the same accumulators with the folded bias (the form the GPU path runs)
+    folded = O.dequant(res.acc.astype(np.float64), None, nb, s_x, None, s_w, None) + res.bias_folded[None, :]
+    assert np.allclose(folded, res.y64, rtol=1e-11, atol=1e-13)
+    # the fold itself, term by term
+    for n in (0, 9, 29):
+        q = 0 if n < 8 else (1 if n < 24 else 2)
+        t = float(bias[n]) - sum(float(s_x[p]) * float(s_w[p, q]) * int(z_x[p]) *
+                                 int(Wq[n, kb[p]:kb[p + 1]].astype(np.int64).sum()) for p in range(2))
+        assert math.isclose(res.bias_folded[n], t, rel_tol=1e-12, abs_tol=1e-15)
+    # and the layer approximates the real one within the half-step bound of both operands
+    exact = X.astype(np.float64) @ W.astype(np.float64).T + bias
+    assert np.abs(res.y64 - exact).max() < 0.05 * np.abs(exact).max()
+
+
+def test_zero_point_lowers_error_on_polarity_asymmetric_input_like_dual_scale():
+    # App. A: the asymmetric scheme "can improve accuracy when data distributions are significantly shifted";
+    # Sec. 4.3.1: even so its uniform bins resolve the narrow negative range worse than two scales do.
+    r = rng(45)
+    X = gelu(r.normal(0, 1.5, (128, 256))).astype(np.float32)
+    W = r.normal(0, 0.02, (64, 256)).astype(np.float32)
+    exact = X.astype(np.float64) @ W.astype(np.float64).T
+    single, _ = oracle_layer(X, W, [0, 256], [0, 64], False)
+    dual, _ = oracle_layer(X, W, [0, 256], [0, 64], True)
+    asym, _ = asym_layer(X, W, [0, 256], [0, 64])
+    assert rel_fnorm(asym.y64, exact) < rel_fnorm(single.y64, exact)
+    assert rel_fnorm(dual.y64, exact) < rel_fnorm(single.y64, exact)
+
+
+# --------------------------------------------------------------- act-to-linear segment: activation and multiplier
+
+def test_activation_functions_match_library_and_identities():
+    import scipy.special
+    h = np.concatenate([np.linspace(-12, 12, 4801), rng(46).normal(0, 3, 2000)])
+    L = O.lib()
+    silu = np.array([L.sqo_silu(float(v)) for v in h])
+    gel = np.array([L.sqo_gelu(float(v)) for v in h])
+    ht = torch.from_numpy(h)
+    assert np.allclose(silu, torch.nn.functional.silu(ht).numpy(), rtol=1e-13, atol=1e-300)
+    assert np.allclose(gel, h * scipy.special.ndtr(h), rtol=1e-12, atol=1e-300)        # GELU(h) = h Phi(h)
+    assert np.allclose(gel, torch.nn.functional.gelu(ht).numpy(), rtol=1e-9, atol=1e-14)
+    # odd-part identities: f(h) - f(-h) = h for both functions
+    for f in (L.sqo_silu, L.sqo_gelu):
+        for v in (0.3, 1.0, 2.5, 7.0):
+            assert math.isclose(f(v) - f(-v), v, rel_tol=1e-14)
+        assert f(0.0) == 0.0
+    assert math.isclose(L.sqo_silu(1.0), 1.0 / (1.0 + math.exp(-1.0)), rel_tol=1e-15)
+    assert math.isclose(L.sqo_gelu(1.0), 0.5 * (1.0 + math.erf(1.0 / math.sqrt(2.0))), rel_tol=1e-15)
+    assert L.sqo_silu(-5.0) < 0 and L.sqo_gelu(-5.0) < 0 and abs(L.sqo_gelu(-5.0)) < 2e-6
+
+
+@pytest.mark.parametrize("act", ["silu", "gelu"])
+def test_activation_is_rounded_once_to_the_stored_dtype(act):
+    h = torch.from_numpy(rng(47).normal(0, 2.5, 4000).astype(np.float32)).to(torch.bfloat16).float().numpy()
+    out, exact = O.activation(h, act, "bf16")
+    bits = out.view(np.uint32)
+    assert np.all((bits & 0xFFFF) == 0)                                      # bf16 values
+    assert np.array_equal((bits >> 16).astype(np.uint16), O.bf16_bits(exact))  # = the pinned fp64 -> bf16 rounding
+    ulp = 2.0 ** (np.floor(np.log2(np.abs(exact) + 1e-300)) - 7)
+    assert np.all(np.abs(out - exact) <= ulp / 2)
+    out32, exact32 = O.activation(h, act, "f32")
+    assert np.array_equal(out32, exact32.astype(np.float32)) and np.array_equal(exact32, exact)
+
+
+def test_smoothing_multiplier_is_one_fp32_multiply():
+    r = rng(48)
+    X = r.normal(0, 1, (9, 40)).astype(np.float32)
+    m = r.uniform(0.1, 4.0, 40).astype(np.float32)
+    assert np.array_equal(O.smooth(X, m), X * m[None, :])
+    assert O.smooth(X, m).dtype == np.float32
