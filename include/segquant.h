@@ -46,6 +46,7 @@ typedef enum {
 
 typedef enum { SQ_CODE_INT8 = 0, SQ_CODE_E4M3 = 1 } sq_code;   /* 8-bit code type */
 typedef enum { SQ_F32 = 0, SQ_BF16 = 1 } sq_dtype;             /* real-valued element type */
+typedef enum { SQ_ACT_NONE = 0, SQ_ACT_SILU = 1, SQ_ACT_GELU = 2 } sq_act;   /* activation in front of the quantizer */
 
 /* flags */
 #define SQ_FLAG_QMIN_SYM 1u  /* int8 DualScale: clamp the negative path to -127 instead of -128 */
@@ -77,7 +78,7 @@ size_t segquant_workspace_bytes(void);
  *       dual == 0: s_pos[p] = max|x|/q_max; s_neg is ignored (may be NULL).
  *   is_weight = 1: X is the weight matrix [rows=N,K]; s_pos[p*Q+q] = max|W block(p,q)|/q_max.
  *   q_max = 127 (int8) or 448 (e4m3); |q_min| = 128 (int8; 127 with SQ_FLAG_QMIN_SYM) or 448.
- *   A segment whose extremum is 0 gets scale 1.  Inputs must be finite.
+ *   A segment whose extremum is 0 gets scale 1.  Inputs must be finite.  rows < 2^37, K <= 16 776 960.
  *   s_pos / s_neg: dev float arrays written by the call.  Alignment: X 16 bytes, ld*sizeof(dt)
  *   a multiple of 16 bytes. */
 sq_status segquant_calib_scales(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld,
@@ -119,6 +120,46 @@ sq_status segquant_quantize_act(const void *X, sq_dtype dt, int64_t M, int64_t K
                                 const sq_segtable *seg, const float *s_pos, const float *s_neg,
                                 sq_code code, uint32_t flags, void *c_pos, void *c_neg, int64_t ldc,
                                 void *stream);
+
+/* The act-to-linear segment fused into the quantizer -- Sec. 4.3.2 ("the computation path from an activation
+ * function to its subsequent linear operator"), App. B (DualScale is applied behind SiLU and GELU), Sec. 4.2.2 last
+ * paragraph with App. B "Extra Hyperparameter Settings" (SmoothQuant's migration with one strength per segment: a
+ * per-channel multiplier in front of the quantizer, the reciprocal smoothing factor, made offline).
+ *   H [M,K] dev is the PRE-activation; per element a = act(h) (SQ_ACT_SILU: h / (1 + exp(-h)); SQ_ACT_GELU:
+ *   (h / 2) erfc(-h / sqrt 2); SQ_ACT_NONE: a = h), rounded once to dtype dt (the dtype the unfused graph would
+ *   have stored it in), then x = a * mult[k] as one fp32 multiply (mult dev [K] fp32, or NULL), then the codes
+ *   of segquant_quantize_act for x.  The activation never goes through device memory.
+ *   Accuracy of the activation: evaluated in fp32 with relative error <= 2^-20 (SiLU) and (2 h^2 + 32) 2^-24
+ *   (GELU); where the exact value lies that close to a rounding boundary of dt the stored value, and with it the
+ *   code, may be that of the neighbouring dt value.  With SQ_ACT_NONE the codes are exact.
+ *   Everything else as for segquant_quantize_act. */
+sq_status segquant_quantize_act_fused(const void *H, sq_dtype dt, int64_t M, int64_t K, int64_t ld,
+                                      const sq_segtable *seg, const float *s_pos, const float *s_neg,
+                                      sq_code code, uint32_t flags, sq_act act, const float *mult,
+                                      void *c_pos, void *c_neg, int64_t ldc, void *stream);
+
+/* Comparison scheme: zero-point (asymmetric) quantization, App. A -- X^ = round(X / s_X) + z_X with an integer
+ * zero-point, recovered by s_X s_W (X^ W^ - z_X rowsum(W^)) for symmetric weight codes (the paper's rowsum runs
+ * over the input dimension).  int8 codes only.
+ *   segquant_calib_zero_point: per K-segment p, from strict min/max over the calibration batch with the range
+ *     widened to contain 0:  s_x[p] = (hi - lo) / 255,  z_x[p] = -128 - round(lo / s_x[p])  (lo maps to -128);
+ *     a zero range gives s = 1, z = 0.  s_x dev float [P], z_x dev int32 [P].
+ *   segquant_quantize_act_zero_point: codes[m][k] = clip(round(x / s_x[p]) + z_x[p], -128, 127), one IEEE fp32
+ *     division, round half to even.  codes [M,K] dev, ldc bytes.
+ *   segquant_fold_zero_point (offline): the correction term does not depend on the token, so it is folded into
+ *     the bias:  bias_folded[n] = bias[n] - sum_p s_x[p] s_w[p*Q+q(n)] z_x[p] * (sum over K-segment p of Wq[n][k]),
+ *     evaluated in fp32 (exact integer sums; per K-segment one product of the two scales and one FMA, ascending p).
+ *     bias may be NULL (zero).  The layer then runs as segquant_seglinear_gemm(codes, ..., s_x, s_w, bias_folded).
+ *   Alignment and limits as for the corresponding symmetric calls. */
+sq_status segquant_calib_zero_point(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld,
+                                    const sq_segtable *seg, float *s_x, int32_t *z_x,
+                                    void *workspace, size_t ws_bytes, void *stream);
+sq_status segquant_quantize_act_zero_point(const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld,
+                                           const sq_segtable *seg, const float *s_x, const int32_t *z_x,
+                                           void *codes, int64_t ldc, void *stream);
+sq_status segquant_fold_zero_point(const void *Wq, int64_t ldw, int64_t N, int64_t K, const sq_segtable *seg,
+                                   const float *s_x, const int32_t *z_x, const float *s_w, const float *bias,
+                                   float *bias_folded, void *stream);
 
 /* Step "weight quantization" (offline) -- Sec. 4.2.2: every block W(p,q) is quantized separately,
  * W^ = clip(round(W / s_w[p*Q+q]), -q_max, q_max) (App. A symmetric case).

@@ -26,7 +26,8 @@ EXPORTS = [
     "segquant_workspace_bytes", "segquant_calib_scales", "segquant_calib_scales_static", "segquant_quantize_act", "segquant_quantize_weight",
     "segquant_seglinear_gemm", "segquant_dualscale_gemm", "segquant_layer_scratch_bytes",
     "segquant_layer_forward", "segquant_layer_forward_pipelined", "segquant_last_device_status", "segquant_set_tuning", "segquant_launch_count", "segquant_last_cuda_error",
-    "segquant_status_string",
+    "segquant_status_string", "segquant_quantize_act_fused", "segquant_calib_zero_point",
+    "segquant_quantize_act_zero_point", "segquant_fold_zero_point",
 ]
 
 
@@ -169,6 +170,57 @@ def segquant_quantize_act(X: torch.Tensor, seg: SegTable, s_pos, s_neg, code: st
                                      _ptr(c_pos), _ptr(c_neg), C.c_int64(c_pos.stride(0)), _stream())
     _check(st, "segquant_quantize_act")
     return c_pos, (c_neg if s_neg is not None else None)
+
+
+SQ_ACT = {None: 0, "none": 0, "silu": 1, "gelu": 2}
+
+
+def segquant_quantize_act_fused(H: torch.Tensor, seg: SegTable, s_pos, s_neg, code: str, act=None, mult=None,
+                                flags: int = 0, c_pos=None, c_neg=None):
+    """Activation function and / or per-channel multiplier in front of the quantizer, in one pass over H."""
+    M, K = H.shape
+    if c_pos is None:
+        c_pos = new_codes(M, K, H.device)
+    if s_neg is not None and c_neg is None:
+        c_neg = new_codes(M, K, H.device)
+    st = lib().segquant_quantize_act_fused(_ptr(H), C.c_int(_dt(H)), C.c_int64(M), C.c_int64(K), C.c_int64(H.stride(0)),
+                                           seg.ref(), _ptr(s_pos), _ptr(s_neg), C.c_int(SQ_CODE[code]), C.c_uint32(flags),
+                                           C.c_int(SQ_ACT[act]), _ptr(mult), _ptr(c_pos), _ptr(c_neg),
+                                           C.c_int64(c_pos.stride(0)), _stream())
+    _check(st, "segquant_quantize_act_fused")
+    return c_pos, (c_neg if s_neg is not None else None)
+
+
+def segquant_calib_zero_point(X: torch.Tensor, seg: SegTable, workspace: torch.Tensor):
+    """(s_x [P] fp32, z_x [P] int32) of the zero-point comparison scheme."""
+    rows, K = X.shape
+    s_x = torch.empty(seg.P, dtype=torch.float32, device=X.device)
+    z_x = torch.empty(seg.P, dtype=torch.int32, device=X.device)
+    st = lib().segquant_calib_zero_point(_ptr(X), C.c_int(_dt(X)), C.c_int64(rows), C.c_int64(K), C.c_int64(X.stride(0)),
+                                         seg.ref(), _ptr(s_x), _ptr(z_x), _ptr(workspace), C.c_size_t(workspace.numel()),
+                                         _stream())
+    _check(st, "segquant_calib_zero_point")
+    return s_x, z_x
+
+
+def segquant_quantize_act_zero_point(X: torch.Tensor, seg: SegTable, s_x, z_x, codes=None):
+    M, K = X.shape
+    if codes is None:
+        codes = new_codes(M, K, X.device)
+    st = lib().segquant_quantize_act_zero_point(_ptr(X), C.c_int(_dt(X)), C.c_int64(M), C.c_int64(K),
+                                                C.c_int64(X.stride(0)), seg.ref(), _ptr(s_x), _ptr(z_x), _ptr(codes),
+                                                C.c_int64(codes.stride(0)), _stream())
+    _check(st, "segquant_quantize_act_zero_point")
+    return codes
+
+
+def segquant_fold_zero_point(Wq: torch.Tensor, seg: SegTable, s_x, z_x, s_w, bias=None):
+    N, K = Wq.shape
+    out = torch.empty(N, dtype=torch.float32, device=Wq.device)
+    st = lib().segquant_fold_zero_point(_ptr(Wq), C.c_int64(Wq.stride(0)), C.c_int64(N), C.c_int64(K), seg.ref(),
+                                        _ptr(s_x), _ptr(z_x), _ptr(s_w), _ptr(bias), _ptr(out), _stream())
+    _check(st, "segquant_fold_zero_point")
+    return out
 
 
 def segquant_quantize_weight(W: torch.Tensor, seg: SegTable, s_w, code: str, flags: int = 0, Wq=None):

@@ -140,8 +140,71 @@ sq_status segquant_quantize_act(const void *X, sq_dtype dt, int64_t M, int64_t K
     if (s_neg && (st = check_matrix(c_neg, M, K, ldc, 1)) != SQ_OK) return st;
     HostSeg hs = load_segtable(seg, K, seg && seg->nb && seg->Q >= 1 ? seg->nb[seg->Q] : 0);
     if (hs.status != SQ_OK) return hs.status;
-    return launch_quantize(X, dt, M, K, ld, hs.b, s_pos, s_neg, 0, code, code_qmax(code),
-                           code_qmin_abs(code, flags), c_pos, c_neg, ldc, static_cast<cudaStream_t>(stream));
+    return launch_quantize(X, dt, M, K, ld, hs.b, s_pos, s_neg, nullptr, 0, code, code_qmax(code),
+                           code_qmin_abs(code, flags), 0, nullptr, c_pos, c_neg, ldc, static_cast<cudaStream_t>(stream));
+}
+
+sq_status segquant_quantize_act_fused(const void *H, sq_dtype dt, int64_t M, int64_t K, int64_t ld,
+                                      const sq_segtable *seg, const float *s_pos, const float *s_neg, sq_code code,
+                                      uint32_t flags, sq_act act, const float *mult, void *c_pos, void *c_neg,
+                                      int64_t ldc, void *stream)
+{
+    if (!s_pos || (s_neg && !c_neg)) return SQ_ERR_NULL;
+    if (!valid_dt(dt) || !valid_code(code)) return SQ_ERR_UNSUPPORTED;
+    if (act != SQ_ACT_NONE && act != SQ_ACT_SILU && act != SQ_ACT_GELU) return SQ_ERR_UNSUPPORTED;
+    sq_status st;
+    if ((st = check_matrix(H, M, K, ld, dt_size(dt))) != SQ_OK) return st;
+    if ((st = check_matrix(c_pos, M, K, ldc, 1)) != SQ_OK) return st;
+    if (s_neg && (st = check_matrix(c_neg, M, K, ldc, 1)) != SQ_OK) return st;
+    HostSeg hs = load_segtable(seg, K, seg && seg->nb && seg->Q >= 1 ? seg->nb[seg->Q] : 0);
+    if (hs.status != SQ_OK) return hs.status;
+    return launch_quantize(H, dt, M, K, ld, hs.b, s_pos, s_neg, nullptr, 0, code, code_qmax(code),
+                           code_qmin_abs(code, flags), int(act), mult, c_pos, c_neg, ldc,
+                           static_cast<cudaStream_t>(stream));
+}
+
+sq_status segquant_calib_zero_point(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld,
+                                    const sq_segtable *seg, float *s_x, int32_t *z_x, void *workspace,
+                                    size_t ws_bytes, void *stream)
+{
+    if (!s_x || !z_x) return SQ_ERR_NULL;
+    if (!valid_dt(dt)) return SQ_ERR_UNSUPPORTED;
+    sq_status st = check_matrix(X, rows, K, ld, dt_size(dt));
+    if (st != SQ_OK) return st;
+    HostSeg hs = load_segtable(seg, K, seg && seg->nb && seg->Q >= 1 ? seg->nb[seg->Q] : 0);
+    if (hs.status != SQ_OK) return hs.status;
+    if ((st = check_ws(workspace, ws_bytes)) != SQ_OK) return st;
+    uint32_t *partials = reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(workspace) + kWsStatusBytes);
+    return launch_calib_zero_point(X, dt, rows, K, ld, hs.b, s_x, z_x, partials, static_cast<cudaStream_t>(stream));
+}
+
+sq_status segquant_quantize_act_zero_point(const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld,
+                                           const sq_segtable *seg, const float *s_x, const int32_t *z_x,
+                                           void *codes, int64_t ldc, void *stream)
+{
+    if (!s_x || !z_x) return SQ_ERR_NULL;
+    if (!valid_dt(dt)) return SQ_ERR_UNSUPPORTED;
+    sq_status st;
+    if ((st = check_matrix(X, M, K, ld, dt_size(dt))) != SQ_OK) return st;
+    if ((st = check_matrix(codes, M, K, ldc, 1)) != SQ_OK) return st;
+    HostSeg hs = load_segtable(seg, K, seg && seg->nb && seg->Q >= 1 ? seg->nb[seg->Q] : 0);
+    if (hs.status != SQ_OK) return hs.status;
+    return launch_quantize(X, dt, M, K, ld, hs.b, s_x, nullptr, z_x, 0, SQ_CODE_INT8, 127.0f, 128.0f, 0, nullptr, codes,
+                           nullptr, ldc, static_cast<cudaStream_t>(stream));
+}
+
+sq_status segquant_fold_zero_point(const void *Wq, int64_t ldw, int64_t N, int64_t K, const sq_segtable *seg,
+                                   const float *s_x, const int32_t *z_x, const float *s_w, const float *bias,
+                                   float *bias_folded, void *stream)
+{
+    if (!s_x || !z_x || !s_w || !bias_folded) return SQ_ERR_NULL;
+    sq_status st;
+    if ((st = check_matrix(Wq, N, K, ldw, 1)) != SQ_OK) return st;
+    if (K > kMaxK) return SQ_ERR_SHAPE;
+    HostSeg hs = load_segtable(seg, K, N);
+    if (hs.status != SQ_OK) return hs.status;
+    return launch_fold_zero_point(Wq, ldw, N, K, hs.b, s_x, z_x, s_w, bias, bias_folded,
+                                  static_cast<cudaStream_t>(stream));
 }
 
 sq_status segquant_quantize_weight(const void *W, sq_dtype dt, int64_t N, int64_t K, int64_t ld,
@@ -156,8 +219,8 @@ sq_status segquant_quantize_weight(const void *W, sq_dtype dt, int64_t N, int64_
     if ((st = check_matrix(Wq, N, K, ldq, 1)) != SQ_OK) return st;
     HostSeg hs = load_segtable(seg, K, N);
     if (hs.status != SQ_OK) return hs.status;
-    return launch_quantize(W, dt, N, K, ld, hs.b, s_w, nullptr, 1, code, code_qmax(code), code_qmax(code), Wq,
-                           nullptr, ldq, static_cast<cudaStream_t>(stream));
+    return launch_quantize(W, dt, N, K, ld, hs.b, s_w, nullptr, nullptr, 1, code, code_qmax(code), code_qmax(code), 0,
+                           nullptr, Wq, nullptr, ldq, static_cast<cudaStream_t>(stream));
 }
 
 sq_status segquant_seglinear_gemm(const void *Xq, int64_t ldx, const void *Wq, int64_t ldw, int64_t M, int64_t N,

@@ -36,7 +36,7 @@ __global__ void calib_init_kernel(uint32_t *partials, int nblocks)
     if (i < nblocks) { partials[2 * i] = 0u; partials[2 * i + 1] = 0xFFFFFFFFu; }
 }
 
-// grid.x covers columns (one column per thread), grid.y covers chunks of kRowsPerBlock rows.
+// grid.y covers columns (one column per thread), grid.x covers chunks of kRowsPerBlock rows.
 // Consecutive threads read consecutive columns of the same row: coalesced.
 template <typename Tin>
 __global__ void __launch_bounds__(kThreads)
@@ -50,8 +50,8 @@ calib_reduce_kernel(const Tin *__restrict__ X, int64_t rows, int K, int64_t ld, 
     for (int i = threadIdx.x; i < nblk; i += kThreads) { sh_max[i] = 0u; sh_min[i] = 0xFFFFFFFFu; }
     __syncthreads();
 
-    const int k = blockIdx.x * kThreads + threadIdx.x;
-    const int64_t r0 = int64_t(blockIdx.y) * kRowsPerBlock;
+    const int k = blockIdx.y * kThreads + threadIdx.x;
+    const int64_t r0 = int64_t(blockIdx.x) * kRowsPerBlock;
     const int64_t r1 = min(rows, r0 + kRowsPerBlock);
     if (k < K && r0 < r1) {
         int p = 0;
@@ -99,6 +99,50 @@ __global__ void calib_finalize_kernel(const uint32_t *__restrict__ partials, int
     }
 }
 
+// App. A asymmetric quantizer: s = (hi - lo) / 255 and z = -128 - round(lo / s) from the extrema widened to
+// contain 0 (one fp32 subtraction, two IEEE divisions, round half to even); a zero range gives s = 1, z = 0.
+__global__ void calib_finalize_zero_point_kernel(const uint32_t *__restrict__ partials, int nblocks,
+                                                 float *__restrict__ s_x, int32_t *__restrict__ z_x)
+{
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= nblocks) return;
+    const uint32_t emx = partials[2 * i], emn = partials[2 * i + 1];
+    const float mx = (emx == 0u || emx == enc(-INFINITY)) ? 0.0f : dec(emx);
+    const float mn = (emn == 0xFFFFFFFFu || emn == enc(INFINITY)) ? 0.0f : dec(emn);
+    const float hi = fmaxf(mx, 0.0f), lo = fminf(mn, 0.0f);
+    const float range = __fsub_rn(hi, lo);
+    if (range > 0.0f) {
+        const float s = __fdiv_rn(range, 255.0f);
+        const float zf = __fsub_rn(-128.0f, rintf(__fdiv_rn(lo, s)));
+        s_x[i] = s;
+        z_x[i] = int(fminf(fmaxf(zf, -128.0f), 127.0f));
+    } else {
+        s_x[i] = 1.0f;
+        z_x[i] = 0;
+    }
+}
+
+// Launch shape of the reduction; false if the matrix is beyond what one grid covers (checked before any launch).
+bool calib_grid(int64_t rows, int64_t K, dim3 *grid)
+{
+    const int64_t gx = (rows + kRowsPerBlock - 1) / kRowsPerBlock, gy = (K + kThreads - 1) / kThreads;
+    if (gx < 1 || gy < 1 || gx > 0x7FFFFFFFll || gy > 65535) return false;
+    *grid = dim3(unsigned(gx), unsigned(gy));
+    return true;
+}
+
+void launch_reduce(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld, const SegBounds &sb, int is_weight,
+                   int nblocks, uint32_t *partials, dim3 grid, cudaStream_t st)
+{
+    calib_init_kernel<<<(nblocks + 255) / 256, 256, 0, st>>>(partials, nblocks);
+    if (dt == SQ_F32)
+        calib_reduce_kernel<float><<<grid, kThreads, 0, st>>>(static_cast<const float *>(X), rows, int(K), ld, sb,
+                                                              is_weight, partials);
+    else
+        calib_reduce_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(static_cast<const __nv_bfloat16 *>(X), rows,
+                                                                      int(K), ld, sb, is_weight, partials);
+}
+
 }  // namespace
 
 sq_status launch_calib(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld, const SegBounds &sb,
@@ -106,20 +150,27 @@ sq_status launch_calib(const void *X, sq_dtype dt, int64_t rows, int64_t K, int6
                        uint32_t *partials, cudaStream_t st)
 {
     const int nblocks = sb.P * (is_weight ? sb.Q : 1);
-    calib_init_kernel<<<(nblocks + 255) / 256, 256, 0, st>>>(partials, nblocks);
-    dim3 grid(unsigned((K + kThreads - 1) / kThreads), unsigned((rows + kRowsPerBlock - 1) / kRowsPerBlock));
-    if (grid.y > 65535) return SQ_ERR_SHAPE;
-    if (dt == SQ_F32)
-        calib_reduce_kernel<float><<<grid, kThreads, 0, st>>>(static_cast<const float *>(X), rows, int(K), ld, sb,
-                                                              is_weight, partials);
-    else
-        calib_reduce_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(static_cast<const __nv_bfloat16 *>(X), rows,
-                                                                      int(K), ld, sb, is_weight, partials);
+    dim3 grid;
+    if (!calib_grid(rows, K, &grid)) return SQ_ERR_SHAPE;      // nothing has been launched yet
+    launch_reduce(X, dt, rows, K, ld, sb, is_weight, nblocks, partials, grid, st);
     calib_finalize_kernel<<<(nblocks + 255) / 256, 256, 0, st>>>(partials, nblocks, is_weight, dual, q_max, q_min_abs,
                                                                  s_pos, s_neg);
     count_launch(3);
     return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
 }
+
+sq_status launch_calib_zero_point(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld, const SegBounds &sb,
+                                  float *s_x, int32_t *z_x, uint32_t *partials, cudaStream_t st)
+{
+    dim3 grid;
+    if (!calib_grid(rows, K, &grid)) return SQ_ERR_SHAPE;
+    launch_reduce(X, dt, rows, K, ld, sb, 0, sb.P, partials, grid, st);
+    calib_finalize_zero_point_kernel<<<(sb.P + 255) / 256, 256, 0, st>>>(partials, sb.P, s_x, z_x);
+    count_launch(3);
+    return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
+}
+
+namespace {
 
 // ----------------------------------------------------------------------------- built-in scratch
 // Reduction partials for callers that have no device allocator to take a workspace from: 2 words per
@@ -146,6 +197,8 @@ static sq_status static_partials_address(uint32_t **out)
     *out = addr[dev];
     return SQ_OK;
 }
+
+}  // namespace
 
 sq_status launch_calib_static(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld, const SegBounds &sb,
                               int is_weight, int dual, float q_max, float q_min_abs, float *s_pos, float *s_neg,

@@ -16,7 +16,6 @@ constexpr int kVec = 16;             // elements per thread and row
 #define SQ_QUANT_BLOCKS_PER_SM 4
 #endif
 constexpr int kBlocksPerSm = SQ_QUANT_BLOCKS_PER_SM;   // resident blocks per SM the kernel is compiled for (4: at most 64 registers)
-constexpr int kThreadsPerSm = kThreads * kBlocksPerSm;
 
 // 16 consecutive elements of a row as loaded (fp32: four 128-bit words, bf16: two), converted when used
 template <typename Tin> struct Raw16;
@@ -62,15 +61,20 @@ __device__ __forceinline__ uint32_t cvt_e4m3x2(float a, float b)
     return r;
 }
 
+enum : int { kSingle = 0, kDual = 1, kZeroPoint = 2 };   // quantizer modes
+
 // One element -> (code for the positive / only matrix, code for the negative matrix), as bytes.
 // Reference form: one IEEE division, round half to even, clip.  Used where a vector straddles a
 // segment bound or the end of a row, and for scales outside the range of the fast form below.
-template <int CODE, bool DUAL>
-__device__ __forceinline__ void quant1(float x, float sp, float sn, int lo, int hi, uint32_t &cp, uint32_t &cn)
+// Zero-point mode (App. A asymmetric quantizer): clip(round(x / s) + z, lo, hi), z passed in `zp`.
+template <int CODE, int MODE>
+__device__ __forceinline__ void quant1(float x, float sp, float sn, int zp, int lo, int hi, uint32_t &cp, uint32_t &cn)
 {
+    constexpr bool DUAL = MODE == kDual;
     if (CODE == SQ_CODE_INT8) {
         float s = DUAL ? (x >= 0.0f ? sp : sn) : sp;
         int c = __float2int_rn(__fdiv_rn(x, s));      // IEEE divide, round half to even, saturating convert
+        if (MODE == kZeroPoint) c = max(min(c, 1000000), -1000000) + zp;
         c = max(min(c, hi), lo);
         if (DUAL) { cp = uint32_t(max(c, 0)) & 0xFFu; cn = uint32_t(min(c, 0)) & 0xFFu; }
         else      { cp = uint32_t(c) & 0xFFu; cn = 0; }
@@ -82,6 +86,33 @@ __device__ __forceinline__ void quant1(float x, float sp, float sn, int lo, int 
         if (DUAL) { cp = pos ? c : 0u; cn = pos ? 0u : c; }
         else      { cp = c; cn = 0; }
     }
+}
+
+// The act-to-linear segment in front of the quantizer (Sec. 4.3.2; App. B: SiLU and GELU feed DualScale layers),
+// evaluated in fp32 and rounded once to the dtype the unfused graph would have stored the activation in.
+// SiLU(h) = h sigma(h) with z = exp(-|h|): sigma = 1 / (1 + z) for h >= 0, z / (1 + z) below (no overflow);
+// relative error <= 2^-20 (exp 2 ulp, one add, one multiply, one IEEE division).
+// GELU(h) = (h / 2) erfc(-h / sqrt 2): relative error <= (2 h^2 + 32) 2^-24 (erfc 4 ulp; the rounding of its
+// argument is amplified by about 2 t^2 in the negative tail).
+__device__ __forceinline__ float silu_f32(float h)
+{
+    const float z = expf(-fabsf(h));
+    const float num = h >= 0.0f ? h : __fmul_rn(h, z);
+    return __fdiv_rn(num, __fadd_rn(1.0f, z));
+}
+__device__ __forceinline__ float gelu_f32(float h)
+{
+    return __fmul_rn(__fmul_rn(0.5f, h), erfcf(__fmul_rn(-h, 0.70710678118654752440f)));
+}
+template <typename Tin>
+__device__ __forceinline__ float pre1(float h, int act, float mult)
+{
+    float a = h;
+    if (act) {
+        a = act == 1 ? silu_f32(h) : gelu_f32(h);
+        if (sizeof(Tin) == 2) a = __bfloat162float(__float2bfloat16_rn(a));      // stored as bf16 in the unfused graph
+    }
+    return __fmul_rn(a, mult);                                // the per-channel multiplier: one fp32 multiply
 }
 
 // Per-segment constants of the fast form.  The quotient x / s is obtained from the correctly rounded
@@ -181,11 +212,28 @@ constexpr int kMagicBits = 0x4B400000;       // its bit pattern: bits(v + magic)
 // e4m3: the input is first mapped to u = sat(x / L) in [0, 1] with one saturating FMA (L a power of two, so
 //   u / (s / L) has the bits of x / s; x beyond L is clipped to 448 anyway), which also splits the polarities and
 //   keeps infinities and NaNs out of the saturating e4m3 conversion.
-template <int CODE, bool DUAL>
-__device__ __forceinline__ void quant4(const float (&x)[4], const SegConst &cp, const SegConst &cn, float hi,
+template <int CODE, int MODE>
+__device__ __forceinline__ void quant4(const float (&x)[4], const SegConst &cp, const SegConst &cn, float hi, int zp,
                                        uint32_t &wp, uint32_t &wn)
 {
+    constexpr bool DUAL = MODE == kDual;
     const uint64_t magic2 = pack2(kRoundMagic, kRoundMagic);
+    if (MODE == kZeroPoint) {
+        // round(|x| / s) with the sign of x (the magnitude clipped at 256: anything beyond leaves the code range
+        // whatever z is; a NaN from an overflowed chain clips the same way), plus z, saturated to [-128, 127]
+        const uint64_t r2 = pack2(cp.r, cp.r), ns2 = pack2(-cp.s, -cp.s);
+        const int off = zp - kMagicBits;
+        int k[4];
+#pragma unroll
+        for (int i = 0; i < 4; i += 2) {
+            float a0, a1;
+            unpack2(div2_rn_fast(pack2(fabsf(x[i]), fabsf(x[i + 1])), ns2, r2), a0, a1);
+            k[i] = int(__float_as_uint(fmaf(fminf(a0, 256.0f), copysignf(1.0f, x[i]), kRoundMagic))) + off;
+            k[i + 1] = int(__float_as_uint(fmaf(fminf(a1, 256.0f), copysignf(1.0f, x[i + 1]), kRoundMagic))) + off;
+        }
+        wp = pack_sat_s8(k[1], k[0], pack_sat_s8(k[3], k[2], 0u));
+        return;
+    }
     if (CODE == SQ_CODE_INT8 && DUAL) {
         const uint64_t rp2 = pack2(cp.r, cp.r), nsp2 = pack2(-cp.s, -cp.s);
         const uint64_t rn2 = pack2(cn.r, cn.r), nsn2 = pack2(-cn.s, -cn.s);
@@ -247,26 +295,46 @@ __device__ __forceinline__ void quant4(const float (&x)[4], const SegConst &cp, 
     }
 }
 
+struct QuantParams {
+    const void *X;
+    int64_t M;
+    int K;
+    int64_t ld;
+    SegBounds sb;
+    const float *s_pos, *s_neg;
+    const int32_t *zp;        // zero-point mode: z per K-segment
+    int row_segments;         // weights: the scale also depends on the row's N-segment
+    int lo, hi;
+    uint8_t *c_pos, *c_neg;
+    int64_t ldc;
+    int V, R;
+    int act;                  // PRE: 0 = none, 1 = SiLU, 2 = GELU applied to the input first
+    const float *mult;        // PRE: per-channel multiplier [K] applied after it, or nullptr
+};
+
 // Thread g of the grid owns the 16-element column chunk g % V of the rows g / V, g / V + R, g / V + 2 R, ...
 // (V chunks per row, R rows in flight over the whole grid), so that a warp reads 1 KiB (bf16) of consecutive
 // addresses per row, the per-segment constants are made once per thread, and the next row's loads are in
 // flight while the current row is converted.
-template <typename Tin, int CODE, bool DUAL>
-__global__ void __launch_bounds__(kThreads, kBlocksPerSm)
-quantize_kernel(const Tin *__restrict__ X, int64_t M, int K, int64_t ld, const SegBounds sb,
-                const float *__restrict__ s_pos, const float *__restrict__ s_neg, int row_segments,
-                int lo, int hi, uint8_t *__restrict__ c_pos, uint8_t *__restrict__ c_neg, int64_t ldc,
-                int V, int R)
+// PRE compiles in the act-to-linear prologue: activation function and per-channel multiplier in front of the
+// quantizer, so that the activation's output never goes through HBM.
+template <typename Tin, int CODE, int MODE, bool PRE>
+__global__ void __launch_bounds__(kThreads, PRE ? 3 : kBlocksPerSm)
+quantize_kernel(const __grid_constant__ QuantParams prm)
 {
+    constexpr bool DUAL = MODE == kDual;
     // Programmatic dependent launch: this kernel may be scheduled while the previous kernel of the stream
     // winds down, and lets the next one be scheduled while its own last blocks run; nothing in global
     // memory is touched before the previous kernel has completed.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    const SegBounds &sb = prm.sb;
+    const int64_t M = prm.M;
+    const int K = prm.K, R = prm.R, lo = prm.lo, hi = prm.hi, row_segments = prm.row_segments;
     const uint32_t g = blockIdx.x * kThreads + threadIdx.x;
-    const uint32_t r0 = g / uint32_t(V);
+    const uint32_t r0 = g / uint32_t(prm.V);
     if (r0 >= uint32_t(R) || int64_t(r0) >= M) return;
-    const int k0 = int(g - r0 * uint32_t(V)) * kVec;
+    const int k0 = int(g - r0 * uint32_t(prm.V)) * kVec;
 
     // K-segment of this chunk (bounds come with the kernel parameters)
     int p = 0;
@@ -274,16 +342,23 @@ quantize_kernel(const Tin *__restrict__ X, int64_t M, int K, int64_t ld, const S
     const bool whole = k0 + kVec <= sb.kb[p + 1];            // chunk inside one K-segment (and inside K)
     const int Qs = row_segments ? sb.Q : 1;
 
-    const Tin *src = X + int64_t(r0) * ld + k0;
-    uint8_t *dp = c_pos + int64_t(r0) * ldc + k0;
-    uint8_t *dn = DUAL ? c_neg + int64_t(r0) * ldc + k0 : nullptr;
-    const int64_t src_step = int64_t(R) * ld, dst_step = int64_t(R) * ldc;
+    const Tin *src = static_cast<const Tin *>(prm.X) + int64_t(r0) * prm.ld + k0;
+    uint8_t *dp = prm.c_pos + int64_t(r0) * prm.ldc + k0;
+    uint8_t *dn = DUAL ? prm.c_neg + int64_t(r0) * prm.ldc + k0 : nullptr;
+    const int64_t src_step = int64_t(R) * prm.ld, dst_step = int64_t(R) * prm.ldc;
+
+    float mreg[PRE ? kVec : 1];                              // this chunk's multipliers, loaded once
+    if (PRE) {
+#pragma unroll
+        for (int i = 0; i < kVec; i++) mreg[i] = (prm.mult && k0 + i < K) ? __ldg(prm.mult + k0 + i) : 1.0f;
+    }
 
     Raw16<Tin> cur, nxt;
     if (whole) load16(src, cur);
     int q = 0;                                               // N-segment (weights only) the constants belong to
     int64_t q_end = 0;                                       // first row beyond it (0: no constants yet)
     SegConst cp, cn;
+    int zp = 0;
     bool fast = false;
     for (int64_t row = r0; row < M; row += R) {
         if (row >= q_end) {                                  // (weights) the row entered another N-segment
@@ -293,8 +368,9 @@ quantize_kernel(const Tin *__restrict__ X, int64_t M, int K, int64_t ld, const S
             } else {
                 q_end = M;
             }
-            cp = seg_const(__ldg(s_pos + p * Qs + (row_segments ? q : 0)));
-            cn = seg_const(DUAL ? __ldg(s_neg + p * Qs + (row_segments ? q : 0)) : 1.0f);
+            cp = seg_const(__ldg(prm.s_pos + p * Qs + (row_segments ? q : 0)));
+            cn = seg_const(DUAL ? __ldg(prm.s_neg + p * Qs + (row_segments ? q : 0)) : 1.0f);
+            if (MODE == kZeroPoint) zp = __ldg(prm.zp + p);
             fast = whole && cp.fast && cn.fast && !(DUAL && CODE == SQ_CODE_INT8 && lo != -128);
         }
         if (fast) {
@@ -305,7 +381,11 @@ quantize_kernel(const Tin *__restrict__ X, int64_t M, int K, int64_t ld, const S
             for (int g4 = 0; g4 < 4; g4++) {
                 float x[4];
                 get4(cur, g4, x);
-                quant4<CODE, DUAL>(x, cp, cn, float(hi), wp[g4], wn[g4]);
+                if (PRE) {
+#pragma unroll
+                    for (int i = 0; i < 4; i++) x[i] = pre1<Tin>(x[i], prm.act, mreg[PRE ? 4 * g4 + i : 0]);
+                }
+                quant4<CODE, MODE>(x, cp, cn, float(hi), zp, wp[g4], wn[g4]);
             }
             *reinterpret_cast<uint4 *>(dp) = make_uint4(wp[0], wp[1], wp[2], wp[3]);
             if (DUAL) *reinterpret_cast<uint4 *>(dn) = make_uint4(wn[0], wn[1], wn[2], wn[3]);
@@ -317,8 +397,10 @@ quantize_kernel(const Tin *__restrict__ X, int64_t M, int K, int64_t ld, const S
             for (int i = 0; i < n; i++) {
                 while (pp + 1 < sb.P && k0 + i >= sb.kb[pp + 1]) pp++;
                 uint32_t a, b;
-                quant1<CODE, DUAL>(load1(src + i), __ldg(s_pos + pp * Qs + qq), DUAL ? __ldg(s_neg + pp * Qs + qq) : 0.0f,
-                                   lo, hi, a, b);
+                float x = load1(src + i);
+                if (PRE) x = pre1<Tin>(x, prm.act, prm.mult ? __ldg(prm.mult + k0 + i) : 1.0f);
+                quant1<CODE, MODE>(x, __ldg(prm.s_pos + pp * Qs + qq), DUAL ? __ldg(prm.s_neg + pp * Qs + qq) : 0.0f,
+                                   MODE == kZeroPoint ? __ldg(prm.zp + pp) : 0, lo, hi, a, b);
                 dp[i] = uint8_t(a);
                 if (DUAL) dn[i] = uint8_t(b);
             }
@@ -330,10 +412,8 @@ quantize_kernel(const Tin *__restrict__ X, int64_t M, int K, int64_t ld, const S
     }
 }
 
-template <typename Tin, int CODE>
-sq_status launch_t(const Tin *X, int64_t M, int64_t K, int64_t ld, const SegBounds &sb, const float *s_pos,
-                   const float *s_neg, int row_segments, int lo, int hi, void *c_pos, void *c_neg,
-                   int64_t ldc, cudaStream_t st)
+template <typename Tin, int CODE, int MODE>
+sq_status launch_t(QuantParams &prm, cudaStream_t st)
 {
     // V chunks per row; R rows in flight: enough threads to fill every SM several times over, and a row count per
     // thread that the rows divide into evenly
@@ -341,13 +421,16 @@ sq_status launch_t(const Tin *X, int64_t M, int64_t K, int64_t ld, const SegBoun
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
         return SQ_ERR_CUDA;
-    const int64_t V = (K + kVec - 1) / kVec;
-    const int64_t target_threads = int64_t(sms) * kThreadsPerSm;
-    int64_t iters = (M * V + target_threads - 1) / target_threads;
+    const bool pre = prm.act != 0 || prm.mult != nullptr;
+    const int64_t V = (prm.K + kVec - 1) / kVec;
+    const int64_t target_threads = int64_t(sms) * kThreads * (pre ? 3 : kBlocksPerSm);
+    int64_t iters = (prm.M * V + target_threads - 1) / target_threads;
     if (iters < 1) iters = 1;
-    const int64_t R = (M + iters - 1) / iters;
+    const int64_t R = (prm.M + iters - 1) / iters;
     const int64_t blocks = (R * V + kThreads - 1) / kThreads;
     if (blocks > 0x7FFFFFFF || R * V > 0xFFFFFFFFll || V > 0x7FFFFFFF || R > 0x7FFFFFFF) return SQ_ERR_SHAPE;
+    prm.V = int(V);
+    prm.R = int(R);
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(unsigned(blocks));
     cfg.blockDim = dim3(kThreads);
@@ -357,40 +440,41 @@ sq_status launch_t(const Tin *X, int64_t M, int64_t K, int64_t ld, const SegBoun
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const int Ki = int(K), Vi = int(V), Ri = int(R);
-    uint8_t *cp = static_cast<uint8_t *>(c_pos), *cn = static_cast<uint8_t *>(c_neg);
-    const float *no_neg = nullptr;
-    cudaError_t e;
-    if (s_neg)
-        e = cudaLaunchKernelEx(&cfg, quantize_kernel<Tin, CODE, true>, X, M, Ki, ld, sb, s_pos, s_neg, row_segments, lo, hi,
-                               cp, cn, ldc, Vi, Ri);
-    else
-        e = cudaLaunchKernelEx(&cfg, quantize_kernel<Tin, CODE, false>, X, M, Ki, ld, sb, s_pos, no_neg, row_segments, lo, hi,
-                               cp, static_cast<uint8_t *>(nullptr), ldc, Vi, Ri);
+    const cudaError_t e = pre ? cudaLaunchKernelEx(&cfg, quantize_kernel<Tin, CODE, MODE, true>, prm)
+                              : cudaLaunchKernelEx(&cfg, quantize_kernel<Tin, CODE, MODE, false>, prm);
     count_launch();
     if (e != cudaSuccess) { note_cuda_error(e); return SQ_ERR_CUDA; }
     return SQ_OK;
 }
 
+template <typename Tin>
+sq_status launch_mode(QuantParams &prm, sq_code code, int mode, cudaStream_t st)
+{
+    if (mode == kZeroPoint) return launch_t<Tin, SQ_CODE_INT8, kZeroPoint>(prm, st);
+    if (code == SQ_CODE_INT8)
+        return mode == kDual ? launch_t<Tin, SQ_CODE_INT8, kDual>(prm, st) : launch_t<Tin, SQ_CODE_INT8, kSingle>(prm, st);
+    return mode == kDual ? launch_t<Tin, SQ_CODE_E4M3, kDual>(prm, st) : launch_t<Tin, SQ_CODE_E4M3, kSingle>(prm, st);
+}
+
 }  // namespace
 
 sq_status launch_quantize(const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld, const SegBounds &sb,
-                          const float *s_pos, const float *s_neg, int row_segments, sq_code code,
-                          float q_max, float q_min_abs, void *c_pos, void *c_neg, int64_t ldc, cudaStream_t st)
+                          const float *s_pos, const float *s_neg, const int32_t *zero_point, int row_segments,
+                          sq_code code, float q_max, float q_min_abs, int act, const float *mult,
+                          void *c_pos, void *c_neg, int64_t ldc, cudaStream_t st)
 {
-    // dual: codes in [-|q_min|, q_max]; single scale: symmetric [-q_max, q_max]
-    const int hi = int(q_max);
-    const int lo = s_neg ? -int(q_min_abs) : -int(q_max);
-    if (dt == SQ_F32) {
-        const float *x = static_cast<const float *>(X);
-        return code == SQ_CODE_INT8
-                   ? launch_t<float, SQ_CODE_INT8>(x, M, K, ld, sb, s_pos, s_neg, row_segments, lo, hi, c_pos, c_neg, ldc, st)
-                   : launch_t<float, SQ_CODE_E4M3>(x, M, K, ld, sb, s_pos, s_neg, row_segments, lo, hi, c_pos, c_neg, ldc, st);
-    }
-    const __nv_bfloat16 *x = static_cast<const __nv_bfloat16 *>(X);
-    return code == SQ_CODE_INT8
-               ? launch_t<__nv_bfloat16, SQ_CODE_INT8>(x, M, K, ld, sb, s_pos, s_neg, row_segments, lo, hi, c_pos, c_neg, ldc, st)
-               : launch_t<__nv_bfloat16, SQ_CODE_E4M3>(x, M, K, ld, sb, s_pos, s_neg, row_segments, lo, hi, c_pos, c_neg, ldc, st);
+    QuantParams prm{};
+    prm.X = X; prm.M = M; prm.K = int(K); prm.ld = ld;
+    prm.sb = sb;
+    prm.s_pos = s_pos; prm.s_neg = s_neg; prm.zp = zero_point;
+    prm.row_segments = row_segments;
+    // dual: codes in [-|q_min|, q_max]; single scale: symmetric [-q_max, q_max]; zero-point: the whole int8 range
+    prm.hi = int(q_max);
+    prm.lo = (s_neg || zero_point) ? -int(q_min_abs) : -int(q_max);
+    prm.c_pos = static_cast<uint8_t *>(c_pos); prm.c_neg = static_cast<uint8_t *>(c_neg); prm.ldc = ldc;
+    prm.act = act; prm.mult = mult;
+    const int mode = zero_point ? kZeroPoint : (s_neg ? kDual : kSingle);
+    return dt == SQ_F32 ? launch_mode<float>(prm, code, mode, st) : launch_mode<__nv_bfloat16>(prm, code, mode, st);
 }
 
 }  // namespace sq

@@ -51,9 +51,19 @@ sq_status launch_calib_static(const void *X, sq_dtype dt, int64_t rows, int64_t 
                               int is_weight, int dual, float q_max, float q_min_abs, float *s_pos, float *s_neg,
                               cudaStream_t st);
 
+// zero_point != nullptr selects the App. A asymmetric quantizer (int8); act / mult: optional activation
+// function (0 none, 1 SiLU, 2 GELU) and per-channel multiplier [K] applied in front of the quantizer
 sq_status launch_quantize(const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld, const SegBounds &sb,
-                          const float *s_pos, const float *s_neg, int row_segments, sq_code code,
-                          float q_max, float q_min_abs, void *c_pos, void *c_neg, int64_t ldc, cudaStream_t st);
+                          const float *s_pos, const float *s_neg, const int32_t *zero_point, int row_segments,
+                          sq_code code, float q_max, float q_min_abs, int act, const float *mult,
+                          void *c_pos, void *c_neg, int64_t ldc, cudaStream_t st);
+
+sq_status launch_calib_zero_point(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld, const SegBounds &sb,
+                                  float *s_x, int32_t *z_x, uint32_t *partials, cudaStream_t st);
+
+sq_status launch_fold_zero_point(const void *Wq, int64_t ldw, int64_t N, int64_t K, const SegBounds &sb,
+                                 const float *s_x, const int32_t *z_x, const float *s_w, const float *bias,
+                                 float *bias_folded, cudaStream_t st);
 
 struct GemmArgs {
     const void *a_pos, *a_neg;   // code matrices [M,K]; a_neg == nullptr: single path

@@ -1,0 +1,257 @@
+"""GPU parity of the rows next to the main path: the zero-point (asymmetric) comparison scheme of App. A and
+the act-to-linear prologue (activation function and per-channel multiplier in front of the quantizer), each
+against the CPU oracle on the same seeded inputs, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from paper_2507_14811_b200 import binding as B
+from paper_2507_14811_b200 import workloads as WL
+from paper_2507_14811_b200.layer import SegQuantLinear
+
+from parity_util import QRANGE, check_bf16_output, to_f32_np
+from test_gpu_parity import custom_spec
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+# ------------------------------------------------------------------ zero-point scheme (App. A)
+
+def run_zero_point_parity(spec):
+    data = WL.make_layer(spec)
+    kb, nb, P = spec.kb, spec.nb, spec.P
+    Xn, Wn, bn = to_f32_np(data.X), to_f32_np(data.W), to_f32_np(data.bias)
+    s_x, z_x = O.calib_act_asym(to_f32_np(data.X_cal), kb)
+    s_w = O.calib_weight(Wn, kb, nb)
+    Wq = O.quantize_weight(Wn, kb, nb, s_w)
+    res = O.layer_forward_asym(Xn, Wq, O.SegTable(kb, nb), s_x, z_x, s_w, bn)
+
+    layer = SegQuantLinear(data.W, data.bias, kb, nb, False, "int8", DEV)
+    seg, ws = layer.seg, layer.workspace
+    g_s, g_z = B.segquant_calib_zero_point(data.X_cal.to(DEV), seg, ws)
+    assert np.array_equal(g_s.cpu().numpy(), s_x) and np.array_equal(g_z.cpu().numpy(), z_x)       # bit-exact
+    assert np.array_equal(layer.Wq.cpu().numpy().view(np.int8), Wq)
+    codes = B.segquant_quantize_act_zero_point(data.X.to(DEV), seg, g_s, g_z)
+    assert np.array_equal(codes.cpu().numpy().view(np.int8), res.codes)                           # bit-exact
+    bias_f = B.segquant_fold_zero_point(layer.Wq, seg, g_s, g_z, layer.s_w, layer.bias)
+    # the fold in fp32: per K-segment one scale product, one int -> float conversion and one FMA, plus the bias
+    fold_abs = np.abs(bn.astype(np.float64))
+    for p in range(P):
+        q_of_n = np.searchsorted(np.asarray(nb), np.arange(spec.N), side="right") - 1
+        fold_abs = fold_abs + np.abs(float(s_x[p]) * s_w[p, q_of_n].astype(np.float64) * int(z_x[p]) * res.wsum[p])
+    err = np.abs(bias_f.cpu().numpy().astype(np.float64) - res.bias_folded)
+    assert np.all(err <= (3 * P + 1) * 2.0 ** -24 * fold_abs)
+    Y32, dump = B.segquant_seglinear_gemm(codes, layer.Wq, seg, "int8", g_s, layer.s_w, bias_f, ws,
+                                          y_dtype=torch.float32, dump_acc=True)
+    Ybf = B.segquant_seglinear_gemm(codes, layer.Wq, seg, "int8", g_s, layer.s_w, bias_f, ws)
+    layer.check_status()
+    torch.cuda.synchronize()
+    assert np.array_equal(dump.cpu().numpy(), res.acc)                                            # bit-exact
+    # the output against the UNFOLDED recovery in fp64: accumulator terms and fold terms each round three times
+    tol = 1e-5 * np.abs(res.y64) + (6 * P + 2) * 2.0 ** -24 * res.y_abs
+    assert np.all(np.abs(Y32.cpu().numpy().astype(np.float64) - res.y64) <= tol)
+    check_bf16_output(Ybf, res.y64, res.y_abs, 2 * P + 1)
+    return res
+
+
+@pytest.mark.parametrize("case", [
+    ("zp_small", 200, 256, 136, [0, 256], [0, 136]),
+    ("zp_k_segments", 300, 512, 264, [0, 128, 224, 512], [0, 64, 264]),
+    ("zp_ragged_tail", 129, 208, 200, [0, 96, 208], [0, 8, 200]),
+    ("zp_many_n_segments", 260, 384, 768, [0, 384], [0, 128, 256, 384, 512, 640, 768]),
+])
+@pytest.mark.parametrize("x_kind", ["normal+gelu", "normal"])
+def test_zero_point_scheme_small_shapes(case, x_kind):
+    name, M, K, N, kb, nb = case
+    run_zero_point_parity(custom_spec(name, M, K, N, kb, nb, False, "int8", x_kind=x_kind,
+                                      x_seg_std=[1.0 + 2 * i for i in range(len(kb) - 1)], seed=61))
+
+
+def test_zero_point_scheme_nonnegative_and_zero_segments():
+    """A segment without negative values gets z = -128; an all-zero calibration segment gets s = 1, z = 0."""
+    spec = custom_spec("zp_degenerate", 140, 256, 64, [0, 128, 256], [0, 64], False, "int8", x_kind="normal")
+    data = WL.make_layer(spec)
+    data.X[:, :128] = data.X[:, :128].abs(); data.X_cal[:, :128] = data.X_cal[:, :128].abs()
+    data.X_cal[:, 128:] = 0
+    s_x, z_x = O.calib_act_asym(to_f32_np(data.X_cal), spec.kb)
+    assert z_x[0] == -128 and s_x[1] == 1.0 and z_x[1] == 0
+    ws = B.new_workspace(DEV)
+    seg = B.SegTable(spec.kb, spec.nb)
+    g_s, g_z = B.segquant_calib_zero_point(data.X_cal.to(DEV), seg, ws)
+    assert np.array_equal(g_s.cpu().numpy(), s_x) and np.array_equal(g_z.cpu().numpy(), z_x)
+    codes = B.segquant_quantize_act_zero_point(data.X.to(DEV), seg, g_s, g_z)
+    assert np.array_equal(codes.cpu().numpy().view(np.int8), O.quantize_act_asym(to_f32_np(data.X), spec.kb, s_x, z_x))
+
+
+def test_zero_point_codes_on_adversarial_values():
+    """Exact ties, far-out-of-range inputs, tiny quotients and extreme scales (which take the division path),
+    odd and even zero-points."""
+    rs = np.random.default_rng(6)
+    M, P, seg_len = 512, 8, 256
+    K = P * seg_len
+    kb = [i * seg_len for i in range(P + 1)]
+    exps = [0, -7, 13, -30, 40, -90, 105, 3]
+    s = (rs.uniform(1.0, 2.0, P) * np.exp2(exps)).astype(np.float32)
+    z = np.array([-128, -77, -1, 0, 1, 64, 127, 13], np.int32)
+    X = np.empty((M, K), np.float32)
+    for p in range(P):
+        blk = rs.uniform(-300, 300, (M, seg_len))
+        blk[:, :64] = np.round(blk[:, :64]) + 0.5
+        blk[:, 64:96] *= 1e-3
+        blk[:, 96:100] *= 1e6
+        with np.errstate(over="ignore"):
+            X[:, kb[p]:kb[p + 1]] = (blk * float(s[p])).astype(np.float32)
+    X[~np.isfinite(X)] = 0.0
+    seg = B.SegTable(kb, [0, 8])
+    codes = B.segquant_quantize_act_zero_point(torch.from_numpy(X).to(DEV), seg, torch.from_numpy(s).to(DEV),
+                                               torch.from_numpy(z).to(DEV))
+    torch.cuda.synchronize()
+    assert np.array_equal(codes.cpu().numpy().view(np.int8), O.quantize_act_asym(X, kb, s, z))
+
+
+@pytest.mark.parametrize("wl,idx", [("dit_xl2", 0), ("dit_xl2", 1), ("sd3_mmdit", 2), ("sdxl_skip", 0)])
+def test_zero_point_scheme_full_size_dual_layers(wl, idx):
+    """The int8 DualScale layers of the benchmark run as zero-point layers instead (what the benchmark times
+    next to them), every row."""
+    sp = WL.WORKLOADS[wl][idx]
+    run_zero_point_parity(WL.LayerSpec(name=sp.name + "_zp", M=sp.M, K=sp.K, N=sp.N, kb=sp.kb, nb=sp.nb, dual=False,
+                                       code="int8", x_dtype=sp.x_dtype, x_kind=sp.x_kind, w_kind=sp.w_kind, seed=sp.seed,
+                                       cal_rows=sp.cal_rows, x_seg_std=list(sp.x_seg_std)))
+
+
+def test_zero_point_calls_reject_bad_arguments_before_launch():
+    seg = B.SegTable([0, 128], [0, 64])
+    X = torch.zeros((16, 128), dtype=torch.bfloat16, device=DEV)
+    ws = B.new_workspace(DEV)
+    n0 = B.segquant_launch_count()
+    with pytest.raises(B.SegquantError) as e:
+        B.segquant_calib_zero_point(X, B.SegTable([0, 64, 32, 128], [0, 64]), ws)
+    assert e.value.status == 3
+    with pytest.raises(B.SegquantError) as e:
+        B.segquant_calib_zero_point(X, seg, torch.zeros(8, dtype=torch.uint8, device=DEV))
+    assert e.value.status == 8
+    with pytest.raises(B.SegquantError) as e:
+        B.segquant_quantize_act_zero_point(X[:, 1:], B.SegTable([0, 127], [0, 64]), torch.ones(1, device=DEV),
+                                           torch.zeros(1, dtype=torch.int32, device=DEV))
+    assert e.value.status == 4
+    assert B.segquant_launch_count() == n0
+
+
+# ------------------------------------------------------------------ act-to-linear prologue, step 1: the multiplier
+
+@pytest.mark.parametrize("code", ["int8", "e4m3"])
+@pytest.mark.parametrize("dual", [True, False])
+@pytest.mark.parametrize("x_dtype", ["bf16", "f32"])
+def test_per_channel_multiplier_codes_are_exact(code, dual, x_dtype):
+    """code = Q(fl32(x * mult[k]) / s): the multiplier is one fp32 multiply on both sides, so the codes are compared
+    bit for bit; K-segments, a ragged row end and a chunk that straddles a segment bound included."""
+    rs = np.random.default_rng(8)
+    spec = custom_spec("mult", 300, 456, 64, [0, 104, 456], [0, 64], dual, code, x_dtype=x_dtype, seed=62,
+                       x_seg_std=[1.0, 3.0])
+    data = WL.make_layer(spec)
+    mult = rs.uniform(0.05, 8.0, spec.K).astype(np.float32)
+    Xs = O.smooth(to_f32_np(data.X), mult)
+    qmax, qmin_abs = QRANGE[code]
+    s_pos, s_neg = O.calib_act(O.smooth(to_f32_np(data.X_cal), mult), spec.kb, dual, q_max=qmax, q_min_abs=qmin_abs)
+    r_pos, r_neg = O.quantize_act(Xs, spec.kb, s_pos, s_neg, code=code, q_max=qmax, q_min_abs=qmin_abs)
+    seg = B.SegTable(spec.kb, spec.nb)
+    c_pos, c_neg = B.segquant_quantize_act_fused(data.X.to(DEV), seg, torch.from_numpy(s_pos).to(DEV),
+                                                 torch.from_numpy(s_neg).to(DEV) if dual else None, code,
+                                                 act=None, mult=torch.from_numpy(mult).to(DEV))
+    torch.cuda.synchronize()
+    dt = np.int8 if code == "int8" else np.uint8
+    assert np.array_equal(c_pos.cpu().numpy().view(dt), r_pos)
+    if dual:
+        assert np.array_equal(c_neg.cpu().numpy().view(dt), r_neg)
+    # without activation and multiplier the fused entry point is the plain quantizer
+    p_pos, p_neg = B.segquant_quantize_act_fused(data.X.to(DEV), seg, torch.from_numpy(s_pos).to(DEV),
+                                                 torch.from_numpy(s_neg).to(DEV) if dual else None, code)
+    q_pos, q_neg = B.segquant_quantize_act(data.X.to(DEV), seg, torch.from_numpy(s_pos).to(DEV),
+                                           torch.from_numpy(s_neg).to(DEV) if dual else None, code)
+    assert torch.equal(p_pos, q_pos) and (not dual or torch.equal(p_neg, q_neg))
+
+
+# ------------------------------------------------------------------ step 2: the activation function
+
+def act_rel_eps(h, act):
+    """Relative error bound of the kernel's fp32 evaluation of the activation (stated in the C header)."""
+    return np.full(h.shape, 2.0 ** -20) if act == "silu" else (2.0 * h.astype(np.float64) ** 2 + 32.0) * 2.0 ** -24
+
+
+def stored_candidates(h, act, stored):
+    """The values the stored activation may take: the oracle's (fp64 evaluation rounded once to the stored dtype)
+    and, where the exact value lies within the kernel's error bound of a rounding boundary, its neighbour."""
+    a_ref, exact = O.activation(h, act, stored)
+    eps = act_rel_eps(h, act)
+    lo, hi = exact * (1 - np.sign(exact) * eps), exact * (1 + np.sign(exact) * eps)
+    if stored == "bf16":
+        rnd = lambda v: (O.bf16_bits(v).astype(np.uint32) << 16).view(np.float32)
+    else:
+        rnd = lambda v: v.astype(np.float32)
+    tiny = np.abs(exact) < 2.0 ** -100                   # below any code's first step: the kernel may flush to zero
+    cands = [a_ref, rnd(lo), rnd(hi)]
+    return cands, tiny
+
+
+@pytest.mark.parametrize("act", ["silu", "gelu"])
+@pytest.mark.parametrize("code,dual", [("int8", True), ("int8", False), ("e4m3", True)])
+def test_fused_activation_codes_are_valid(act, code, dual):
+    """H (bf16 pre-activation) -> act -> bf16 -> (multiplier) -> codes in one kernel.  The oracle evaluates the
+    activation in fp64 and rounds once; a GPU code must be the oracle's code, or the code of the neighbouring
+    bf16 value where the exact activation lies within the kernel's stated error bound of a bf16 rounding
+    boundary.  Almost every element must take the first branch."""
+    rs = np.random.default_rng(9)
+    spec = custom_spec("fact", 700, 512, 64, [0, 192, 512], [0, 64], dual, code, x_kind="normal", seed=63,
+                       x_seg_std=[1.5, 3.0])
+    data = WL.make_layer(spec)
+    H = to_f32_np(data.X)
+    H[0, :12] = [0.0, -0.0, 11.5, -11.5, 30.0, -30.0, -60.0, -100.0, 1e-20, -1e-20, 88.0, -88.0]
+    Hb = torch.from_numpy(H).to(torch.bfloat16)
+    H = Hb.float().numpy()
+    mult = rs.uniform(0.5, 2.0, spec.K).astype(np.float32)
+    qmax, qmin_abs = QRANGE[code]
+    cal, _ = O.activation(to_f32_np(data.X_cal), act, "bf16")
+    s_pos, s_neg = O.calib_act(O.smooth(cal, mult), spec.kb, dual, q_max=qmax, q_min_abs=qmin_abs)
+    seg = B.SegTable(spec.kb, spec.nb)
+    c_pos, c_neg = B.segquant_quantize_act_fused(Hb.to(DEV), seg, torch.from_numpy(s_pos).to(DEV),
+                                                 torch.from_numpy(s_neg).to(DEV) if dual else None, code, act=act,
+                                                 mult=torch.from_numpy(mult).to(DEV))
+    torch.cuda.synchronize()
+    dt = np.int8 if code == "int8" else np.uint8
+    g_pos = c_pos.cpu().numpy().view(dt)
+    g_neg = c_neg.cpu().numpy().view(dt) if dual else None
+    cands, tiny = stored_candidates(H, act, "bf16")
+    ok = np.zeros(H.shape, bool)
+    first = None
+    for a in cands + [np.zeros_like(cands[0])]:
+        r_pos, r_neg = O.quantize_act(O.smooth(a, mult), spec.kb, s_pos, s_neg, code=code, q_max=qmax, q_min_abs=qmin_abs)
+        same = (g_pos == r_pos) & ((g_neg == r_neg) if dual else True)
+        if first is None:
+            first = same
+        if a is cands[0] or a is cands[1] or a is cands[2]:
+            ok |= same
+        else:
+            ok |= same & tiny
+    assert ok.all(), f"{(~ok).sum()} codes are neither the oracle's nor a neighbour's"
+    assert first.mean() > 0.999, f"only {first.mean():.5f} of the codes equal the oracle's"
+
+
+@pytest.mark.parametrize("act", ["silu", "gelu"])
+def test_fused_activation_equals_the_unfused_pair_when_the_stored_values_agree(act):
+    """Feeding the oracle's stored activation through the plain quantizer gives the codes of the fused call
+    wherever the two stored values agree: the quantizer behind the prologue is the same arithmetic."""
+    spec = custom_spec("fact2", 400, 384, 64, [0, 384], [0, 64], True, "int8", x_kind="normal", seed=64, x_seg_std=[2.0])
+    data = WL.make_layer(spec)
+    Hb = data.X
+    a_ref, _ = O.activation(to_f32_np(Hb), act, "bf16")
+    s_pos, s_neg = O.calib_act(a_ref[:64], spec.kb, True)
+    seg = B.SegTable(spec.kb, spec.nb)
+    sp, sn = torch.from_numpy(s_pos).to(DEV), torch.from_numpy(s_neg).to(DEV)
+    f_pos, f_neg = B.segquant_quantize_act_fused(Hb.to(DEV), seg, sp, sn, "int8", act=act)
+    A = torch.from_numpy(a_ref).to(torch.bfloat16)
+    assert torch.equal(A.float(), torch.from_numpy(a_ref))             # the oracle's values are bf16 values
+    u_pos, u_neg = B.segquant_quantize_act(A.to(DEV), seg, sp, sn, "int8")
+    agree = ((f_pos == u_pos) & (f_neg == u_neg)).float().mean().item()
+    assert agree > 0.999
