@@ -143,6 +143,15 @@ class BenchLayer:
         self.y_stage = torch.empty_like(self.Y)
         self.Y_host = torch.empty((self.M, spec.N), dtype=torch.bfloat16).pin_memory()
         self.layer.scratch_for(self.M)
+        # comparison variants of DualScale layers: the zero-point scheme (int8) and the fused activation
+        self.act = spec.x_kind.partition("+")[2] or None
+        self.zp = None
+        if spec.dual and spec.code == "int8":
+            L = self.layer
+            s_x, z_x = B.segquant_calib_zero_point(data.X_cal.to(device), L.seg, L.workspace)
+            self.zp = {"s_x": s_x, "z_x": z_x, "codes": B.new_codes(self.M, spec.K, device),
+                       "bias": B.segquant_fold_zero_point(L.Wq, L.seg, s_x, z_x, L.s_w, L.bias)}
+        self.a_stage = torch.empty_like(self.X) if (spec.dual and self.act) else None
 
     def quantize(self):
         L = self.layer
@@ -156,6 +165,35 @@ class BenchLayer:
         else:
             self.B.segquant_seglinear_gemm(self.c_pos, L.Wq, L.seg, L.code, L.s_pos, L.s_w, L.bias, L.workspace,
                                            Y=self.Y)
+
+    def quantize_plain(self):
+        """Single-scale codes of the same input (the plain W8A8 layer's quantize pass).  Timing only."""
+        L = self.layer
+        self.B.segquant_quantize_act(self.X, L.seg, L.s_pos, None, L.code, L.flags, self.c_pos, None)
+
+    def quantize_zero_point(self):
+        self.B.segquant_quantize_act_zero_point(self.X, self.layer.seg, self.zp["s_x"], self.zp["z_x"], self.zp["codes"])
+
+    def gemm_zero_point(self):
+        """The zero-point layer: its codes and the folded bias through the single-scale GEMM."""
+        L = self.layer
+        self.B.segquant_seglinear_gemm(self.zp["codes"], L.Wq, L.seg, L.code, self.zp["s_x"], L.s_w, self.zp["bias"],
+                                       L.workspace, Y=self.Y)
+
+    def quantize_fused_act(self):
+        """Pre-activation -> activation -> codes in one pass.  Timing only: the layer's input stands in for the
+        pre-activation (the cost does not depend on the values)."""
+        L = self.layer
+        self.B.segquant_quantize_act_fused(self.X, L.seg, L.s_pos, L.s_neg, L.code, act=self.act, c_pos=self.c_pos,
+                                           c_neg=self.c_neg)
+
+    def act_unfused(self):
+        """The activation as its own elementwise pass (a library kernel, comparison only): reads the
+        pre-activation, writes the activation that the quantize pass then reads."""
+        if self.act == "silu":
+            torch.nn.functional.silu(self.X, inplace=False) if self.a_stage is None else torch.ops.aten.silu.out(self.X, out=self.a_stage)
+        else:
+            torch.ops.aten.gelu.out(self.X, out=self.a_stage)
 
     def gemm_plain(self):
         """The same shape as a plain single-scale W8A8 layer (one code matrix): the denominator of the
@@ -186,9 +224,11 @@ class BenchLayer:
         for name in ("Wq", "s_w", "bias", "s_pos", "s_neg", "workspace"):
             t = getattr(self.layer, name)
             setattr(other.layer, name, None if t is None else t.clone())
-        for name in ("X", "c_pos", "c_neg", "Y"):
+        for name in ("X", "c_pos", "c_neg", "Y", "a_stage"):
             t = getattr(self, name)
             setattr(other, name, None if t is None else t.clone())
+        if self.zp is not None:
+            other.zp = {k: v.clone() for k, v in self.zp.items()}
         return other
 
     def device_bytes(self):
@@ -236,7 +276,8 @@ def time_kernels(layers, launches=48, max_copies=96):
     its own pair of events cannot be used for this: the event timer of these GPUs ticks in steps of 2 us and an
     event pair around one small kernel reads 6-8 us more than the kernel's own span.
     Returns lists (quantize_us, gemm_us, plain_us | None, unsegmented_us | None, copies)."""
-    out = {"q": [], "g": [], "plain": [], "unseg": [], "copies": []}
+    out = {"q": [], "g": [], "plain": [], "unseg": [], "copies": [], "q_plain": [], "q_zp": [], "g_zp": [], "q_fused": [],
+           "act": []}
     for bl in layers:
         s = bl.spec
         foot = min(quant_bytes(s, bl.M), gemm_bytes(s, bl.M))
@@ -249,6 +290,12 @@ def time_kernels(layers, launches=48, max_copies=96):
         out["plain"].append(graph_time_per_launch([c.gemm_plain for c in copies], rounds) if s.dual else None)
         out["unseg"].append(graph_time_per_launch([c.gemm_unsegmented for c in copies], rounds)
                             if (s.P > 1 or s.Q > 1) else None)
+        out["q_plain"].append(graph_time_per_launch([c.quantize_plain for c in copies], rounds) if s.dual else None)
+        out["q_zp"].append(graph_time_per_launch([c.quantize_zero_point for c in copies], rounds) if bl.zp else None)
+        out["g_zp"].append(graph_time_per_launch([c.gemm_zero_point for c in copies], rounds) if bl.zp else None)
+        fused = s.dual and bl.act
+        out["q_fused"].append(graph_time_per_launch([c.quantize_fused_act for c in copies], rounds) if fused else None)
+        out["act"].append(graph_time_per_launch([c.act_unfused for c in copies], rounds) if fused else None)
         del copies
         torch.cuda.empty_cache()
     return out
@@ -307,6 +354,31 @@ def time_steps_back_to_back(layer_sets, steps, warmup, min_region_s=0.0):
             launches = (B.segquant_launch_count() - n0) // reps
     torch.cuda.current_stream().wait_stream(stream)
     return e0.elapsed_time(e1) / (steps * reps), mode, launches, reps
+
+
+def time_steps_planned(layer_sets, steps, min_region_s=0.02):
+    """The same whole steps issued from the host through prepared calls (one plan per layer and buffer set, built
+    outside the timed region; a step's host cost is one call per layer = two kernel launches each), no CUDA graph.
+    Returns ms per step."""
+    R = len(layer_sets)
+    plans = [[bl.layer.plan(bl.X, bl.Y) for bl in layers] for layers in layer_sets]
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        def issue(n):
+            for i in range(n):
+                for p in plans[i % R]:
+                    p.run()
+        issue(max(R, 3))
+        stream.synchronize()
+        e0.record(stream); issue(steps); e1.record(stream)
+        stream.synchronize()
+        n = max(steps, int(np.ceil(steps * min_region_s / max(e0.elapsed_time(e1) * 1e-3, 1e-9))))
+        e0.record(stream); issue(n); e1.record(stream)
+        stream.synchronize()
+    torch.cuda.current_stream().wait_stream(stream)
+    return e0.elapsed_time(e1) / n
 
 
 def time_e2e(layers, steps, warmup, flush, chunks=0):
@@ -441,6 +513,24 @@ def layer_table(specs, kt, peaks):
             "unsegmented_gemm_us": None if un is None else round(un * 1e3, 2),
             "seglinear_gemm_time_over_unsegmented": None if un is None else round(float(g) / un, 3),
         })
+        i = len(rows) - 1
+        r, us = rows[-1], lambda v: None if v is None else round(v, 2)
+        layer_us = (q + g) * 1e3
+        if kt["q_plain"][i] is not None:
+            plain_us = kt["q_plain"][i] + kt["plain"][i]
+            r.update({"plain_w8a8_quant_us": us(kt["q_plain"][i]),
+                      "dual_layer_time_over_plain_layer": round(layer_us / plain_us, 3)})
+            if kt["q_zp"][i] is not None:
+                zp_us = kt["q_zp"][i] + kt["g_zp"][i]
+                r.update({"asym_quant_us": us(kt["q_zp"][i]), "asym_gemm_us": us(kt["g_zp"][i]),
+                          "dual_layer_time_over_asym_layer": round(layer_us / zp_us, 3),
+                          "asym_layer_time_over_plain_layer": round(zp_us / plain_us, 3)})
+        if kt["q_fused"][i] is not None:
+            r["fused_act"] = {"act": s.x_kind.partition("+")[2], "fused_quant_us": us(kt["q_fused"][i]),
+                              "unfused_act_us": us(kt["act"][i]), "unfused_pair_us": us(kt["act"][i] + q * 1e3),
+                              "fused_time_over_unfused_pair": round(kt["q_fused"][i] / (kt["act"][i] + q * 1e3), 3),
+                              "hbm_bytes_saved": 4 * s.M * s.K,
+                              "note": "the unfused activation is a library elementwise kernel (comparison only)"}
     return rows
 
 
@@ -464,10 +554,12 @@ def measure_side_workload(name, dev, args, peaks):
     sets, set_bytes, n_sets = buffer_sets(layers)
     steps = max(3, min(args.steps, 50))
     step_ms, mode, launches, reps = time_steps_back_to_back(sets, steps, max(3, min(args.warmup, 5)), 0.05)
+    planned_ms = time_steps_planned(sets, steps)
     del sets
     exec_ops = sum(layer_ops(s)[0] for s in specs)
     tops = exec_ops / (step_ms * 1e-3) / 1e12
-    out = {"ms_per_step": round(step_ms, 5), "exec_tops": round(tops, 1),
+    out = {"ms_per_step": round(step_ms, 5), "ms_per_step_planned_calls_from_host": round(planned_ms, 5),
+           "exec_tops": round(tops, 1),
            "whole_step": fractions(tops, eight_bit_peaks(peaks)),
            "timed_region": f"{reps} replay(s) of a CUDA graph of {steps} steps over {n_sets} buffer sets "
                            f"({n_sets * set_bytes / 2**20:.0f} MiB)",
@@ -534,6 +626,8 @@ def run_ours(args):
     step_ms, step_mode, launches, reps = time_steps_back_to_back(layer_sets, args.steps, args.warmup, args.min_region_s)
     clocks = sampler.stop()
     barrier()
+    time.sleep(COOL_DOWN_S)
+    planned_ms = time_steps_planned(layer_sets, args.steps)
     del layer_sets
     torch.cuda.empty_cache()
     time.sleep(COOL_DOWN_S)
@@ -602,6 +696,9 @@ def run_ours(args):
                                note="quantize + GEMM of every layer inside a long back-to-back region: the sustained "
                                     "peak is the fair denominator; the quantize passes are HBM work inside it"),
             "ms_per_step_kernels_timed_alone": round(split_ms, 5),
+            "ms_per_step_planned_calls_from_host": round(planned_ms, 5),
+            "planned_calls_note": "the same steps without a CUDA graph: every layer issued from the host through its "
+                                  "prepared call (segquant_plan_run: two launches, no checks or queries), short region",
             "frac_of_nominal_4500_tops": round(step_tops / NOMINAL_8BIT_TOPS, 4),
             "e2e": {"value": round(world * exec_ops / (e2e_step_ms * 1e-3) / 1e12, 2), "unit": "TOPS",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_step_ms, 4),

@@ -16,11 +16,15 @@
  *   - "dev" pointers are CUDA device pointers of the current device, "host" pointers are
  *     ordinary host memory that is only read during the call.
  *   - The caller owns every buffer.  The library allocates no device memory and keeps no
- *     state between calls other than cached driver entry points and per-device attributes.
+ *     state between calls other than a cached driver entry point, per-device kernel attributes (both
+ *     guarded for concurrent callers) and the test-only overrides of segquant_set_tuning.
  *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*, NULL = default
  *     stream) and return without synchronizing, except segquant_last_device_status.
  *   - Every entry point returns an sq_status.  Anything checkable on the host is rejected
  *     before any launch; nothing aborts or throws.  There is no CPU fallback.
+ *   - SQ_OK from a launching call means the work was enqueued.  A bounded wait inside a kernel that
+ *     expires is reported only through segquant_last_device_status; Y is undefined unless that call
+ *     returns SQ_OK as well.
  */
 #ifndef SEGQUANT_H_
 #define SEGQUANT_H_
@@ -235,6 +239,26 @@ sq_status segquant_layer_forward_pipelined(const void *X, void *x_stage, sq_dtyp
                                            void *workspace, size_t ws_bytes, int chunks, void *stream,
                                            void *stream_in, void *stream_out);
 
+/* A layer call prepared once and replayed.  segquant_plan_layer does everything segquant_layer_forward does on
+ * the host for device X and Y -- argument checks, tile plan, kernel choice, tensor-map encoding, attribute set-up --
+ * and stores the result in caller-owned memory instead of launching; segquant_plan_run then issues the layer's
+ * two kernels (quantize, GEMM + epilogue) on `stream` with no further checks, queries or encoding, for callers
+ * that run the same layer on the same buffers again and again (its host cost is two kernel launches).
+ *   The plan is plain data: it may be copied or freed at will and owns nothing.  It refers to the buffers by
+ *   address: X, Wq, the scale tables, bias, Y, scratch and workspace must stay where they were (their CONTENTS
+ *   may change between runs); after any pointer, shape or pitch change build a new plan.  A plan belongs to the
+ *   device that was current when it was built and to this process; segquant_plan_run on a zeroed or failed
+ *   plan, or with another device current, returns SQ_ERR_UNSUPPORTED.  Arguments as for segquant_layer_forward
+ *   with device X and Y. */
+#define SQ_PLAN_BYTES 4096
+typedef struct { uint64_t opaque[SQ_PLAN_BYTES / 8]; } sq_plan;
+sq_status segquant_plan_layer(sq_plan *plan, const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld,
+                              const void *Wq, int64_t ldw, int64_t N, const sq_segtable *seg, sq_code code,
+                              const float *s_pos, const float *s_neg, const float *s_w, const float *bias,
+                              uint32_t flags, void *Y, sq_dtype y_dtype, int64_t ldy,
+                              void *scratch, size_t scratch_bytes, void *workspace, size_t ws_bytes);
+sq_status segquant_plan_run(const sq_plan *plan, void *stream);
+
 /* Synchronizes `stream`, reads the device status word of `workspace` and clears it.  Returns SQ_OK,
  * SQ_ERR_TIMEOUT (a bounded wait inside a kernel expired; *detail, if not NULL, receives a code that
  * names the wait) or SQ_ERR_CUDA. */
@@ -247,8 +271,9 @@ sq_status segquant_last_device_status(void *workspace, void *stream, uint32_t *d
  * accumulators of a tile resident in tensor memory; at most 16 of them), 2 (sequential) or 4
  * (automatic, but single-scale layers keep 256 x 256 tiles instead of 256 x 512 ones) or 5 (256 x 512
  * tiles for single-scale layers even where the automatic choice expects no gain from them).
- * Process-wide; meant for benchmarking sweeps and tests.  Values the layer cannot use are replaced by
- * the automatic choice. */
+ * Process-wide (atomic words read when a launch or a plan is prepared); meant for benchmarking sweeps and
+ * tests only: production callers leave everything automatic.  Values the layer cannot use are replaced by the
+ * automatic choice. */
 sq_status segquant_set_tuning(int tile_n, int stages, int cta_group, int segment_mode);
 
 /* Text of the CUDA error behind the most recent SQ_ERR_CUDA of a GEMM launch ("no error" if none). */

@@ -27,7 +27,7 @@ EXPORTS = [
     "segquant_seglinear_gemm", "segquant_dualscale_gemm", "segquant_layer_scratch_bytes",
     "segquant_layer_forward", "segquant_layer_forward_pipelined", "segquant_last_device_status", "segquant_set_tuning", "segquant_launch_count", "segquant_last_cuda_error",
     "segquant_status_string", "segquant_quantize_act_fused", "segquant_calib_zero_point",
-    "segquant_quantize_act_zero_point", "segquant_fold_zero_point",
+    "segquant_quantize_act_zero_point", "segquant_fold_zero_point", "segquant_plan_layer", "segquant_plan_run",
 ]
 
 
@@ -310,6 +310,32 @@ def segquant_layer_forward_pipelined(X, Wq, seg: SegTable, code: str, s_pos, s_n
         C.c_void_p(stream_in.cuda_stream), C.c_void_p(stream_out.cuda_stream))
     _check(st, "segquant_layer_forward_pipelined")
     return Y
+
+
+SQ_PLAN_BYTES = 4096
+
+
+class LayerPlan:
+    """A prepared layer call (segquant_plan_layer): holds the plan's storage and the tensors it refers to."""
+
+    def __init__(self, X, Wq, seg: SegTable, code, s_pos, s_neg, s_w, bias, Y, scratch, workspace, flags: int = 0):
+        M, K = X.shape
+        N = Wq.shape[0]
+        self._keep = (X, Wq, seg, s_pos, s_neg, s_w, bias, Y, scratch, workspace)
+        self._buf = (C.c_uint64 * (SQ_PLAN_BYTES // 8))()
+        st = lib().segquant_plan_layer(
+            C.byref(self._buf), _ptr(X), C.c_int(_dt(X)), C.c_int64(M), C.c_int64(K), C.c_int64(X.stride(0)), _ptr(Wq),
+            C.c_int64(Wq.stride(0)), C.c_int64(N), seg.ref(), C.c_int(SQ_CODE[code]), _ptr(s_pos), _ptr(s_neg), _ptr(s_w),
+            _ptr(bias), C.c_uint32(flags), _ptr(Y), C.c_int(_dt(Y)), C.c_int64(Y.stride(0)), _ptr(scratch),
+            C.c_size_t(scratch.numel()), _ptr(workspace), C.c_size_t(workspace.numel()))
+        _check(st, "segquant_plan_layer")
+        self._run = lib().segquant_plan_run
+        self._ref = C.byref(self._buf)
+
+    def run(self):
+        st = self._run(self._ref, _stream())
+        if st != SQ_OK:
+            _check(st, "segquant_plan_run")
 
 
 def segquant_last_device_status(workspace) -> tuple[int, int]:

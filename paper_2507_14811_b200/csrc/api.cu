@@ -1,5 +1,6 @@
 // C ABI: host-side validation and dispatch.  Every argument error is reported before any launch.
 #include <atomic>
+#include <cstring>
 #include "sq_common.cuh"
 
 namespace sq {
@@ -53,11 +54,12 @@ static sq_status check_matrix(const void *p, int64_t rows, int64_t cols, int64_t
     return SQ_OK;
 }
 
-static sq_status gemm_common(const void *a_pos, const void *a_neg, int dual, int64_t ldx, const void *Wq, int64_t ldw,
-                             int64_t M, int64_t N, int64_t K, const sq_segtable *seg, sq_code code,
-                             const float *s_pos, const float *s_neg, const float *s_w, const float *bias, void *Y,
-                             sq_dtype y_dtype, int64_t ldy, void *acc_dump, void *workspace, size_t ws_bytes,
-                             void *stream)
+// Validation shared by the GEMM entry points and the plan; fills `g` when everything is in order.
+static sq_status gemm_args(const void *a_pos, const void *a_neg, int dual, int64_t ldx, const void *Wq, int64_t ldw,
+                           int64_t M, int64_t N, int64_t K, const sq_segtable *seg, sq_code code,
+                           const float *s_pos, const float *s_neg, const float *s_w, const float *bias, void *Y,
+                           sq_dtype y_dtype, int64_t ldy, void *acc_dump, void *workspace, size_t ws_bytes,
+                           GemmArgs *out)
 {
     if (!s_pos || !s_w || (dual && (!a_neg || !s_neg))) return SQ_ERR_NULL;
     if (!valid_code(code) || !valid_dt(y_dtype)) return SQ_ERR_UNSUPPORTED;
@@ -76,7 +78,8 @@ static sq_status gemm_common(const void *a_pos, const void *a_neg, int dual, int
     if (hs.b.P * (dual ? 2 : 1) * hs.b.Q > 2048) return SQ_ERR_UNSUPPORTED;   // dequantization factors kept in shared memory
     if ((st = check_ws(workspace, ws_bytes)) != SQ_OK) return st;
 
-    GemmArgs g{};
+    GemmArgs &g = *out;
+    g = GemmArgs{};
     g.a_pos = a_pos; g.a_neg = dual ? a_neg : nullptr; g.lda = ldx;
     g.b = Wq; g.ldb = ldw;
     g.M = M; g.N = N; g.K = K;
@@ -86,8 +89,29 @@ static sq_status gemm_common(const void *a_pos, const void *a_neg, int dual, int
     g.Y = Y; g.y_dtype = y_dtype; g.ldy = ldy;
     g.acc_dump = acc_dump;
     g.status = static_cast<uint32_t *>(workspace);
-    return launch_gemm(g, static_cast<cudaStream_t>(stream));
+    return SQ_OK;
 }
+
+static sq_status gemm_common(const void *a_pos, const void *a_neg, int dual, int64_t ldx, const void *Wq, int64_t ldw,
+                             int64_t M, int64_t N, int64_t K, const sq_segtable *seg, sq_code code,
+                             const float *s_pos, const float *s_neg, const float *s_w, const float *bias, void *Y,
+                             sq_dtype y_dtype, int64_t ldy, void *acc_dump, void *workspace, size_t ws_bytes,
+                             void *stream)
+{
+    GemmArgs g;
+    const sq_status st = gemm_args(a_pos, a_neg, dual, ldx, Wq, ldw, M, N, K, seg, code, s_pos, s_neg, s_w, bias, Y,
+                                   y_dtype, ldy, acc_dump, workspace, ws_bytes, &g);
+    return st == SQ_OK ? launch_gemm(g, static_cast<cudaStream_t>(stream)) : st;
+}
+
+// What an sq_plan holds (copied in and out of the caller's storage, which need not be aligned for it).
+struct LayerPlan {
+    uint64_t magic;
+    QuantLaunch quant;
+    GemmLaunch gemm;
+};
+constexpr uint64_t kPlanMagic = 0x53514C41594552ull;   // "SQLAYER"
+static_assert(sizeof(LayerPlan) <= sizeof(sq_plan), "sq_plan is too small for a layer plan");
 
 }  // namespace sq
 
@@ -361,6 +385,51 @@ sq_status segquant_layer_forward_pipelined(const void *X, void *x_stage, sq_dtyp
         fail(SQ_ERR_CUDA);
     for (int i = 0; i < nev; i++) cudaEventDestroy(ev[i]);
     return r;
+}
+
+sq_status segquant_plan_layer(sq_plan *plan, const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld,
+                              const void *Wq, int64_t ldw, int64_t N, const sq_segtable *seg, sq_code code,
+                              const float *s_pos, const float *s_neg, const float *s_w, const float *bias,
+                              uint32_t flags, void *Y, sq_dtype y_dtype, int64_t ldy, void *scratch,
+                              size_t scratch_bytes, void *workspace, size_t ws_bytes)
+{
+    if (!plan || !X || !Y || !scratch || !s_pos) return SQ_ERR_NULL;
+    std::memset(plan, 0, sizeof(*plan));
+    if (!valid_dt(dt) || !valid_dt(y_dtype) || !valid_code(code)) return SQ_ERR_UNSUPPORTED;
+    const int dual = s_neg != nullptr;
+    sq_status st;
+    if ((st = check_matrix(X, M, K, ld, dt_size(dt))) != SQ_OK) return st;
+    if (scratch_bytes < segquant_layer_scratch_bytes(M, K, dual)) return SQ_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(scratch) & 255u) return SQ_ERR_ALIGN;
+    const int64_t ldc = (K + 127) & ~int64_t(127);
+    uint8_t *c_pos = static_cast<uint8_t *>(scratch);
+    uint8_t *c_neg = dual ? c_pos + ((size_t(M) * ldc + 255) & ~size_t(255)) : nullptr;
+    GemmArgs g;
+    if ((st = gemm_args(c_pos, c_neg, dual, ldc, Wq, ldw, M, N, K, seg, code, s_pos, s_neg, s_w, bias, Y, y_dtype, ldy,
+                        nullptr, workspace, ws_bytes, &g)) != SQ_OK)
+        return st;
+    LayerPlan lp{};
+    if ((st = prepare_quantize(X, dt, M, K, ld, g.sb, s_pos, s_neg, nullptr, 0, code, code_qmax(code),
+                               code_qmin_abs(code, flags), 0, nullptr, c_pos, c_neg, ldc, &lp.quant)) != SQ_OK)
+        return st;
+    if ((st = prepare_gemm(g, &lp.gemm)) != SQ_OK) return st;
+    lp.magic = kPlanMagic;
+    std::memcpy(plan, &lp, sizeof(lp));
+    return SQ_OK;
+}
+
+sq_status segquant_plan_run(const sq_plan *plan, void *stream)
+{
+    if (!plan) return SQ_ERR_NULL;
+    LayerPlan lp;
+    std::memcpy(&lp, plan, sizeof(lp));
+    if (lp.magic != kPlanMagic) return SQ_ERR_UNSUPPORTED;     // never built, or a failed segquant_plan_layer
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SQ_ERR_CUDA;
+    if (dev != lp.gemm.device) return SQ_ERR_UNSUPPORTED;      // plans belong to the device they were built on
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const sq_status r = run_quantize(lp.quant, st);
+    return r == SQ_OK ? run_gemm(lp.gemm, st) : r;
 }
 
 sq_status segquant_last_device_status(void *workspace, void *stream, uint32_t *detail)

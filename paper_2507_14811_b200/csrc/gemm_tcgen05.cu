@@ -28,7 +28,9 @@
 // Every wait on an mbarrier is bounded (SM cycle counter, about 2 s); on expiry the CTA records
 // which wait gave up in the status word, stops issuing work, lets its own copies land and leaves
 // normally.  No load uses cluster multicast.
-#include <cuda.h>
+#include <atomic>
+#include <mutex>
+#include <vector>
 #include <cuda_bf16.h>
 #include "sq_common.cuh"
 
@@ -58,22 +60,6 @@ constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s
 constexpr uint32_t kStageBytesPerWarp = 32 * 64;       // one 32 x 32 bf16 output block per epilogue warp
 constexpr uint32_t kStageBytes = kEpiWarps * kStageBytesPerWarp;
 constexpr int kMaxFactorTable = 2048;                  // (K-segments x polarities) x N-segments factors in shared memory
-
-struct KernelParams {
-    int M, N, K;
-    int nacc;          // P * npol
-    int acc_stages;    // 1 or 2 accumulator sets in TMEM
-    int stages;        // shared-memory ring depth
-    int num_m_tiles, num_n_tiles;
-    SegBounds sb;
-    const float *s_pos, *s_neg, *s_w, *bias;
-    void *Y;
-    long long ldy;     // elements
-    int y_is_f32;
-    int y_wide;        // rows of Y are 32-byte aligned: 256-bit stores allowed
-    void *acc_dump;
-    uint32_t *status;
-};
 
 // ----------------------------------------------------------------------------- PTX wrappers
 
@@ -1080,17 +1066,18 @@ using EncodeFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, vo
                               const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                               CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// The driver's tensor-map encoder, looked up once per process.
 EncodeFn get_encode_fn()
 {
+    static std::once_flag once;
     static EncodeFn fn = nullptr;
-    if (!fn) {
+    std::call_once(once, [] {
         void *p = nullptr;
         cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess)
-            return nullptr;
-        fn = reinterpret_cast<EncodeFn>(p);
-    }
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeFn>(p);
+    });
     return fn;
 }
 
@@ -1126,25 +1113,63 @@ bool make_map_y(CUtensorMap *map, void *base, int64_t M, int64_t N, int64_t ldy)
     return r == CUDA_SUCCESS;
 }
 
-int g_tune_tile_n = 0, g_tune_stages = 0, g_tune_cta_group = 0, g_tune_seq = 0;
+// Tile-plan overrides for benchmarking sweeps and tests (segquant_set_tuning); 0 = automatic.
+std::atomic<int> g_tune_tile_n{0}, g_tune_stages{0}, g_tune_cta_group{0}, g_tune_seq{0};
+
+// What has been found out per (device, kernel instantiation, dynamic shared-memory size): how many CTA pairs can
+// be resident; and per (device, kernel instantiation) the largest dynamic shared-memory size the kernel's
+// attribute has been raised to (it is only ever raised, so that earlier plans stay launchable).  Guarded by a
+// mutex; a handful of entries.
+struct KernelFacts { int device; const void *kernel; size_t smem; int clusters; };
+struct KernelSmem { int device; const void *kernel; size_t max_smem; };
+std::mutex g_facts_mu;
+std::vector<KernelFacts> g_facts;
+std::vector<KernelSmem> g_smem;
+
+template <typename Kern>
+sq_status kernel_facts(int device, Kern kern, size_t smem, int cg, const cudaLaunchConfig_t &cfg, int *clusters)
+{
+    const void *key = reinterpret_cast<const void *>(kern);
+    std::lock_guard<std::mutex> lock(g_facts_mu);
+    KernelSmem *ks = nullptr;
+    for (KernelSmem &e : g_smem)
+        if (e.device == device && e.kernel == key) ks = &e;
+    if (!ks || ks->max_smem < smem) {
+        const cudaError_t ea = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        if (ea != cudaSuccess) { note_cuda_error(ea); return SQ_ERR_CUDA; }
+        if (ks) ks->max_smem = smem;
+        else g_smem.push_back({device, key, smem});
+    }
+    for (const KernelFacts &f : g_facts)
+        if (f.device == device && f.kernel == key && f.smem == smem) { *clusters = f.clusters; return SQ_OK; }
+    int n = 0;
+    if (cg == 2) {
+        const cudaError_t eo = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+        if (eo != cudaSuccess || n <= 0) { note_cuda_error(eo != cudaSuccess ? eo : cudaErrorLaunchOutOfResources); return SQ_ERR_CUDA; }
+    }
+    g_facts.push_back({device, key, smem, n});
+    *clusters = n;
+    return SQ_OK;
+}
 
 template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ, bool WIDE = false>
-sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cudaStream_t st)
+sq_status prepare_variant(const GemmArgs &g, GemmLaunch &L, int device, int sm_count)
 {
     constexpr int kTileCols = TILE_N * (WIDE ? 2 : 1);
     constexpr int B_ROWS = TILE_N / CG;
-    CUtensorMap ta, tn, tb, ty;
-    if (GENERIC) ty = CUtensorMap{};                // unused by the generic variant
-    else if (!make_map_y(&ty, g.Y, g.M, g.N, g.ldy)) return SQ_ERR_CUDA;
-    if (!make_map(&ta, g.a_pos, g.M, g.K, g.lda, TILE_M)) return SQ_ERR_CUDA;
-    if (!make_map(&tn, g.a_neg ? g.a_neg : g.a_pos, g.M, g.K, g.lda, TILE_M)) return SQ_ERR_CUDA;
-    if (!make_map(&tb, g.b, g.N, g.K, g.ldb, B_ROWS)) return SQ_ERR_CUDA;
+    KernelParams &prm = L.prm;
+    if (GENERIC) L.ty = CUtensorMap{};                // unused by the generic variant
+    else if (!make_map_y(&L.ty, g.Y, g.M, g.N, g.ldy)) return SQ_ERR_CUDA;
+    if (!make_map(&L.ta, g.a_pos, g.M, g.K, g.lda, TILE_M)) return SQ_ERR_CUDA;
+    if (!make_map(&L.tn, g.a_neg ? g.a_neg : g.a_pos, g.M, g.K, g.lda, TILE_M)) return SQ_ERR_CUDA;
+    if (!make_map(&L.tb, g.b, g.N, g.K, g.ldb, B_ROWS)) return SQ_ERR_CUDA;
 
     const uint32_t stage_bytes = NPOL * TILE_M * BLOCK_K + (WIDE ? 2 : 1) * B_ROWS * BLOCK_K;
     const uint32_t tail = (GENERIC ? 0u : kStageBytes) + epi_table_bytes(prm.nacc, prm.sb.Q, kTileCols) + sizeof(SharedHeader);
     int stages = int((kSmemBudget - 1024 - tail) / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
-    if (g_tune_stages >= 2 && g_tune_stages < stages) stages = g_tune_stages;
+    const int tune_stages = g_tune_stages.load(std::memory_order_relaxed);
+    if (tune_stages >= 2 && tune_stages < stages) stages = tune_stages;
     if (stages < 2) return SQ_ERR_UNSUPPORTED;
     prm.stages = stages;
     prm.num_m_tiles = int((g.M + TILE_M * CG - 1) / (TILE_M * CG));
@@ -1152,109 +1177,98 @@ sq_status launch_variant(const GemmArgs &g, KernelParams &prm, int sm_count, cud
     const size_t smem = 1024 + size_t(stages) * stage_bytes + tail;
 
     auto kern = segquant_gemm_kernel<KIND, NPOL, TILE_N, CG, GENERIC, SEQ, WIDE>;
-    const cudaError_t ea = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-    if (ea != cudaSuccess) { note_cuda_error(ea); return SQ_ERR_CUDA; }
-    const int tiles = prm.num_m_tiles * prm.num_n_tiles;
-
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(unsigned(sm_count / CG * CG));
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[2];
+    cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = CG;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = CG == 2 ? attr : attr + 1;          // the cluster attribute only for CTA pairs
-    cfg.numAttrs = CG == 2 ? 2 : 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = CG == 2 ? 1 : 0;
 
     // persistent grid: one CTA (pair) per SM (pair) that can be resident at the same time
-    int units = sm_count / CG;
-    if (CG == 2) {
-        static size_t cached_smem = 0;          // per kernel instantiation
-        static int cached_clusters = 0;
-        if (cached_smem != smem) {
-            int n = 0;
-            const cudaError_t eo = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
-            if (eo != cudaSuccess || n <= 0) { note_cuda_error(eo != cudaSuccess ? eo : cudaErrorLaunchOutOfResources); return SQ_ERR_CUDA; }
-            cached_clusters = n;
-            cached_smem = smem;
-        }
-        if (cached_clusters < units) units = cached_clusters;
-    }
-    const int grid = (tiles < units ? tiles : units) * CG;
-    cfg.gridDim = dim3(unsigned(grid));
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ta, tn, tb, ty, prm);
-    count_launch();
-    const cudaError_t e2 = cudaGetLastError();
-    if (e != cudaSuccess || e2 != cudaSuccess) { note_cuda_error(e != cudaSuccess ? e : e2); return SQ_ERR_CUDA; }
+    int units = sm_count / CG, clusters = 0;
+    const sq_status fs = kernel_facts(device, kern, smem, CG, cfg, &clusters);
+    if (fs != SQ_OK) return fs;
+    if (CG == 2 && clusters < units) units = clusters;
+    const int tiles = prm.num_m_tiles * prm.num_n_tiles;
+    L.kernel = reinterpret_cast<const void *>(kern);
+    L.grid = unsigned((tiles < units ? tiles : units) * CG);
+    L.cluster = CG;
+    L.smem = smem;
+    L.device = device;
     return SQ_OK;
 }
 
 template <int KIND, int NPOL, int CG>
-sq_status launch_tile(const GemmArgs &g, KernelParams &prm, int tile_n, bool seq, int sm_count, cudaStream_t st)
+sq_status prepare_tile(const GemmArgs &g, GemmLaunch &L, int tile_n, bool seq, int device, int sm_count)
 {
+    KernelParams &prm = L.prm;
     bool dbg = prm.y_is_f32 || prm.acc_dump != nullptr;
     // the production variant writes Y with TMA stores: 16-byte aligned base and row pitch
     dbg = dbg || reinterpret_cast<uintptr_t>(g.Y) % 16 != 0 || (size_t(g.ldy) * 2) % 16 != 0;
     for (int q = 1; q < prm.sb.Q; q++) dbg = dbg || (prm.sb.nb[q] % 32 != 0);
     if (seq) {      // sequential K-segments: one tile width per polarity count
         constexpr int TN = NPOL == 1 ? 256 : 128;
-        return dbg ? launch_variant<KIND, NPOL, TN, CG, true, true>(g, prm, sm_count, st)
-                   : launch_variant<KIND, NPOL, TN, CG, false, true>(g, prm, sm_count, st);
+        return dbg ? prepare_variant<KIND, NPOL, TN, CG, true, true>(g, L, device, sm_count)
+                   : prepare_variant<KIND, NPOL, TN, CG, false, true>(g, L, device, sm_count);
     }
     // single-scale layer, one K-segment, CTA pairs, at least two 256-column tiles: 256 x 512 tiles whose halves
     // share the activation tile; an odd number of 256-column tiles leaves one half idle, so then only when there
     // are many of them; and a wide tile is two tiles' work, so it must not cost more waves than it saves time
     // (measured gain per unit of work: 5-6 %)
+    const int tune_seq = g_tune_seq.load(std::memory_order_relaxed);
     const int64_t n256 = (g.N + 255) / 256, m_pairs = (g.M + 2 * TILE_M - 1) / (2 * TILE_M), units = sm_count / 2;
     const int64_t waves_256 = (m_pairs * n256 + units - 1) / units;
     const int64_t waves_wide = (m_pairs * ((n256 + 1) / 2) + units - 1) / units;
-    if (NPOL == 1 && CG == 2 && !dbg && tile_n == 256 && prm.sb.P == 1 && g_tune_seq != 4 &&
-        (n256 % 2 == 0 || n256 >= 9) && (g_tune_seq == 5 || 2 * waves_wide * 94 < waves_256 * 100)) {
+    if (NPOL == 1 && CG == 2 && !dbg && tile_n == 256 && prm.sb.P == 1 && tune_seq != 4 &&
+        (n256 % 2 == 0 || n256 >= 9) && (tune_seq == 5 || 2 * waves_wide * 94 < waves_256 * 100)) {
         prm.acc_stages = 1;
-        return launch_variant<KIND, 1, 256, 2, false, false, true>(g, prm, sm_count, st);
+        return prepare_variant<KIND, 1, 256, 2, false, false, true>(g, L, device, sm_count);
     }
     switch (tile_n) {
-        case 256: return dbg ? launch_variant<KIND, NPOL, 256, CG, true, false>(g, prm, sm_count, st)
-                             : launch_variant<KIND, NPOL, 256, CG, false, false>(g, prm, sm_count, st);
-        case 128: return dbg ? launch_variant<KIND, NPOL, 128, CG, true, false>(g, prm, sm_count, st)
-                             : launch_variant<KIND, NPOL, 128, CG, false, false>(g, prm, sm_count, st);
-        case 64: return dbg ? launch_variant<KIND, NPOL, 64, CG, true, false>(g, prm, sm_count, st)
-                            : launch_variant<KIND, NPOL, 64, CG, false, false>(g, prm, sm_count, st);
-        case 32: return dbg ? launch_variant<KIND, NPOL, 32, CG, true, false>(g, prm, sm_count, st)
-                            : launch_variant<KIND, NPOL, 32, CG, false, false>(g, prm, sm_count, st);
+        case 256: return dbg ? prepare_variant<KIND, NPOL, 256, CG, true, false>(g, L, device, sm_count)
+                             : prepare_variant<KIND, NPOL, 256, CG, false, false>(g, L, device, sm_count);
+        case 128: return dbg ? prepare_variant<KIND, NPOL, 128, CG, true, false>(g, L, device, sm_count)
+                             : prepare_variant<KIND, NPOL, 128, CG, false, false>(g, L, device, sm_count);
+        case 64: return dbg ? prepare_variant<KIND, NPOL, 64, CG, true, false>(g, L, device, sm_count)
+                            : prepare_variant<KIND, NPOL, 64, CG, false, false>(g, L, device, sm_count);
+        case 32: return dbg ? prepare_variant<KIND, NPOL, 32, CG, true, false>(g, L, device, sm_count)
+                            : prepare_variant<KIND, NPOL, 32, CG, false, false>(g, L, device, sm_count);
     }
     return SQ_ERR_UNSUPPORTED;
 }
 
 template <int KIND>
-sq_status launch_kind(const GemmArgs &g, KernelParams &prm, int npol, int cg, int tile_n, bool seq, int sm_count,
-                      cudaStream_t st)
+sq_status prepare_kind(const GemmArgs &g, GemmLaunch &L, int npol, int cg, int tile_n, bool seq, int device, int sm_count)
 {
     if (npol == 2)
-        return cg == 2 ? launch_tile<KIND, 2, 2>(g, prm, tile_n, seq, sm_count, st)
-                       : launch_tile<KIND, 2, 1>(g, prm, tile_n, seq, sm_count, st);
-    return cg == 2 ? launch_tile<KIND, 1, 2>(g, prm, tile_n, seq, sm_count, st)
-                   : launch_tile<KIND, 1, 1>(g, prm, tile_n, seq, sm_count, st);
+        return cg == 2 ? prepare_tile<KIND, 2, 2>(g, L, tile_n, seq, device, sm_count)
+                       : prepare_tile<KIND, 2, 1>(g, L, tile_n, seq, device, sm_count);
+    return cg == 2 ? prepare_tile<KIND, 1, 2>(g, L, tile_n, seq, device, sm_count)
+                   : prepare_tile<KIND, 1, 1>(g, L, tile_n, seq, device, sm_count);
 }
 
 }  // namespace
 
 void set_gemm_tuning(int tile_n, int stages, int cta_group, int segment_mode)
 {
-    g_tune_tile_n = tile_n;
-    g_tune_stages = stages;
-    g_tune_cta_group = cta_group;
-    g_tune_seq = segment_mode;
+    g_tune_tile_n.store(tile_n, std::memory_order_relaxed);
+    g_tune_stages.store(stages, std::memory_order_relaxed);
+    g_tune_cta_group.store(cta_group, std::memory_order_relaxed);
+    g_tune_seq.store(segment_mode, std::memory_order_relaxed);
 }
 
-sq_status launch_gemm(const GemmArgs &g, cudaStream_t st)
+// Everything a GEMM launch needs that can be worked out ahead of it: tile plan, kernel instantiation, tensor
+// maps, shared-memory size and grid.  Launches nothing.
+sq_status prepare_gemm(const GemmArgs &g, GemmLaunch *out)
 {
-    KernelParams prm{};
+    GemmLaunch &L = *out;
+    KernelParams &prm = L.prm;
+    prm = KernelParams{};
     prm.M = int(g.M); prm.N = int(g.N); prm.K = int(g.K);
     const int npol = g.a_neg ? 2 : 1;
     prm.nacc = g.sb.P * npol;
@@ -1270,22 +1284,25 @@ sq_status launch_gemm(const GemmArgs &g, cudaStream_t st)
     if (cudaGetDevice(&dev) != cudaSuccess) return SQ_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
         return SQ_ERR_CUDA;
+    const int tune_tile_n = g_tune_tile_n.load(std::memory_order_relaxed);
+    const int tune_cta_group = g_tune_cta_group.load(std::memory_order_relaxed);
+    const int tune_seq = g_tune_seq.load(std::memory_order_relaxed);
 
     // CTA pairs whenever a tile has more than 128 rows to work on
     int cg = g.M > TILE_M ? 2 : 1;
-    if (g_tune_cta_group == 1 || g_tune_cta_group == 2) cg = g_tune_cta_group;
+    if (tune_cta_group == 1 || tune_cta_group == 2) cg = tune_cta_group;
     if (sm_count < 2) cg = 1;
 
     // More than one K-segment: segments go through TMEM one after the other (SEQ) unless the caller asks for
     // all accumulators of a tile to stay resident, which needs 32 columns for each of them.
     bool seq = g.sb.P > 1;
-    if (g_tune_seq == 1 && prm.nacc * 32 <= kTmemCols) seq = false;
-    if (g_tune_seq == 2) seq = true;
+    if (tune_seq == 1 && prm.nacc * 32 <= kTmemCols) seq = false;
+    if (tune_seq == 2) seq = true;
     if (prm.nacc * g.sb.Q > kMaxFactorTable) return SQ_ERR_UNSUPPORTED;
     if (seq) {
         prm.acc_stages = 2;
-        return g.code == SQ_CODE_INT8 ? launch_kind<0>(g, prm, npol, cg, 0, true, sm_count, st)
-                                      : launch_kind<1>(g, prm, npol, cg, 0, true, sm_count, st);
+        return g.code == SQ_CODE_INT8 ? prepare_kind<0>(g, L, npol, cg, 0, true, dev, sm_count)
+                                      : prepare_kind<1>(g, L, npol, cg, 0, true, dev, sm_count);
     }
 
     // Tile width: the widest tile whose accumulators fit the 512 TMEM columns, unless half that width
@@ -1305,12 +1322,44 @@ sq_status launch_gemm(const GemmArgs &g, cudaStream_t st)
         };
         if (score(tile_max / 2, 0.75) > score(tile_max, 1.0)) tile_n = tile_max / 2;
     }
-    if (g_tune_tile_n >= 32 && g_tune_tile_n <= tile_max && (g_tune_tile_n & (g_tune_tile_n - 1)) == 0)
-        tile_n = g_tune_tile_n;
+    if (tune_tile_n >= 32 && tune_tile_n <= tile_max && (tune_tile_n & (tune_tile_n - 1)) == 0)
+        tile_n = tune_tile_n;
     prm.acc_stages = (2 * tile_n * prm.nacc <= kTmemCols) ? 2 : 1;
 
-    return g.code == SQ_CODE_INT8 ? launch_kind<0>(g, prm, npol, cg, tile_n, false, sm_count, st)
-                                  : launch_kind<1>(g, prm, npol, cg, tile_n, false, sm_count, st);
+    return g.code == SQ_CODE_INT8 ? prepare_kind<0>(g, L, npol, cg, tile_n, false, dev, sm_count)
+                                  : prepare_kind<1>(g, L, npol, cg, tile_n, false, dev, sm_count);
+}
+
+// One launch from a prepared plan: no queries, no encoding.
+sq_status run_gemm(const GemmLaunch &L, cudaStream_t st)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(L.grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = L.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = L.cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = L.cluster == 2 ? attr : attr + 1;          // the cluster attribute only for CTA pairs
+    cfg.numAttrs = L.cluster == 2 ? 2 : 1;
+    void *args[5] = {const_cast<CUtensorMap *>(&L.ta), const_cast<CUtensorMap *>(&L.tn), const_cast<CUtensorMap *>(&L.tb),
+                     const_cast<CUtensorMap *>(&L.ty), const_cast<KernelParams *>(&L.prm)};
+    const cudaError_t e = cudaLaunchKernelExC(&cfg, L.kernel, args);
+    count_launch();
+    if (e != cudaSuccess) { note_cuda_error(e); return SQ_ERR_CUDA; }
+    return SQ_OK;
+}
+
+sq_status launch_gemm(const GemmArgs &g, cudaStream_t st)
+{
+    GemmLaunch L;
+    const sq_status s = prepare_gemm(g, &L);
+    return s == SQ_OK ? run_gemm(L, st) : s;
 }
 
 }  // namespace sq

@@ -295,23 +295,6 @@ __device__ __forceinline__ void quant4(const float (&x)[4], const SegConst &cp, 
     }
 }
 
-struct QuantParams {
-    const void *X;
-    int64_t M;
-    int K;
-    int64_t ld;
-    SegBounds sb;
-    const float *s_pos, *s_neg;
-    const int32_t *zp;        // zero-point mode: z per K-segment
-    int row_segments;         // weights: the scale also depends on the row's N-segment
-    int lo, hi;
-    uint8_t *c_pos, *c_neg;
-    int64_t ldc;
-    int V, R;
-    int act;                  // PRE: 0 = none, 1 = SiLU, 2 = GELU applied to the input first
-    const float *mult;        // PRE: per-channel multiplier [K] applied after it, or nullptr
-};
-
 // Thread g of the grid owns the 16-element column chunk g % V of the rows g / V, g / V + R, g / V + 2 R, ...
 // (V chunks per row, R rows in flight over the whole grid), so that a warp reads 1 KiB (bf16) of consecutive
 // addresses per row, the per-segment constants are made once per thread, and the next row's loads are in
@@ -413,10 +396,11 @@ quantize_kernel(const __grid_constant__ QuantParams prm)
 }
 
 template <typename Tin, int CODE, int MODE>
-sq_status launch_t(QuantParams &prm, cudaStream_t st)
+sq_status prepare_t(QuantLaunch &L)
 {
     // V chunks per row; R rows in flight: enough threads to fill every SM several times over, and a row count per
     // thread that the rows divide into evenly
+    QuantParams &prm = L.prm;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
@@ -431,39 +415,30 @@ sq_status launch_t(QuantParams &prm, cudaStream_t st)
     if (blocks > 0x7FFFFFFF || R * V > 0xFFFFFFFFll || V > 0x7FFFFFFF || R > 0x7FFFFFFF) return SQ_ERR_SHAPE;
     prm.V = int(V);
     prm.R = int(R);
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(unsigned(blocks));
-    cfg.blockDim = dim3(kThreads);
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    const cudaError_t e = pre ? cudaLaunchKernelEx(&cfg, quantize_kernel<Tin, CODE, MODE, true>, prm)
-                              : cudaLaunchKernelEx(&cfg, quantize_kernel<Tin, CODE, MODE, false>, prm);
-    count_launch();
-    if (e != cudaSuccess) { note_cuda_error(e); return SQ_ERR_CUDA; }
+    L.blocks = unsigned(blocks);
+    L.kernel = pre ? reinterpret_cast<const void *>(quantize_kernel<Tin, CODE, MODE, true>)
+                   : reinterpret_cast<const void *>(quantize_kernel<Tin, CODE, MODE, false>);
     return SQ_OK;
 }
 
 template <typename Tin>
-sq_status launch_mode(QuantParams &prm, sq_code code, int mode, cudaStream_t st)
+sq_status prepare_mode(QuantLaunch &L, sq_code code, int mode)
 {
-    if (mode == kZeroPoint) return launch_t<Tin, SQ_CODE_INT8, kZeroPoint>(prm, st);
+    if (mode == kZeroPoint) return prepare_t<Tin, SQ_CODE_INT8, kZeroPoint>(L);
     if (code == SQ_CODE_INT8)
-        return mode == kDual ? launch_t<Tin, SQ_CODE_INT8, kDual>(prm, st) : launch_t<Tin, SQ_CODE_INT8, kSingle>(prm, st);
-    return mode == kDual ? launch_t<Tin, SQ_CODE_E4M3, kDual>(prm, st) : launch_t<Tin, SQ_CODE_E4M3, kSingle>(prm, st);
+        return mode == kDual ? prepare_t<Tin, SQ_CODE_INT8, kDual>(L) : prepare_t<Tin, SQ_CODE_INT8, kSingle>(L);
+    return mode == kDual ? prepare_t<Tin, SQ_CODE_E4M3, kDual>(L) : prepare_t<Tin, SQ_CODE_E4M3, kSingle>(L);
 }
 
 }  // namespace
 
-sq_status launch_quantize(const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld, const SegBounds &sb,
-                          const float *s_pos, const float *s_neg, const int32_t *zero_point, int row_segments,
-                          sq_code code, float q_max, float q_min_abs, int act, const float *mult,
-                          void *c_pos, void *c_neg, int64_t ldc, cudaStream_t st)
+sq_status prepare_quantize(const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld, const SegBounds &sb,
+                           const float *s_pos, const float *s_neg, const int32_t *zero_point, int row_segments,
+                           sq_code code, float q_max, float q_min_abs, int act, const float *mult,
+                           void *c_pos, void *c_neg, int64_t ldc, QuantLaunch *out)
 {
-    QuantParams prm{};
+    QuantParams &prm = out->prm;
+    prm = QuantParams{};
     prm.X = X; prm.M = M; prm.K = int(K); prm.ld = ld;
     prm.sb = sb;
     prm.s_pos = s_pos; prm.s_neg = s_neg; prm.zp = zero_point;
@@ -474,7 +449,36 @@ sq_status launch_quantize(const void *X, sq_dtype dt, int64_t M, int64_t K, int6
     prm.c_pos = static_cast<uint8_t *>(c_pos); prm.c_neg = static_cast<uint8_t *>(c_neg); prm.ldc = ldc;
     prm.act = act; prm.mult = mult;
     const int mode = zero_point ? kZeroPoint : (s_neg ? kDual : kSingle);
-    return dt == SQ_F32 ? launch_mode<float>(prm, code, mode, st) : launch_mode<__nv_bfloat16>(prm, code, mode, st);
+    return dt == SQ_F32 ? prepare_mode<float>(*out, code, mode) : prepare_mode<__nv_bfloat16>(*out, code, mode);
+}
+
+sq_status run_quantize(const QuantLaunch &L, cudaStream_t st)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(L.blocks);
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    void *args[1] = {const_cast<QuantParams *>(&L.prm)};
+    const cudaError_t e = cudaLaunchKernelExC(&cfg, L.kernel, args);
+    count_launch();
+    if (e != cudaSuccess) { note_cuda_error(e); return SQ_ERR_CUDA; }
+    return SQ_OK;
+}
+
+sq_status launch_quantize(const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld, const SegBounds &sb,
+                          const float *s_pos, const float *s_neg, const int32_t *zero_point, int row_segments,
+                          sq_code code, float q_max, float q_min_abs, int act, const float *mult,
+                          void *c_pos, void *c_neg, int64_t ldc, cudaStream_t st)
+{
+    QuantLaunch L;
+    const sq_status s = prepare_quantize(X, dt, M, K, ld, sb, s_pos, s_neg, zero_point, row_segments, code, q_max,
+                                         q_min_abs, act, mult, c_pos, c_neg, ldc, &L);
+    return s == SQ_OK ? run_quantize(L, st) : s;
 }
 
 }  // namespace sq

@@ -1,5 +1,6 @@
 // Internal declarations shared by the CUDA translation units of the library.
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include "segquant.h"
@@ -51,12 +52,43 @@ sq_status launch_calib_static(const void *X, sq_dtype dt, int64_t rows, int64_t 
                               int is_weight, int dual, float q_max, float q_min_abs, float *s_pos, float *s_neg,
                               cudaStream_t st);
 
+// Parameters of the quantize kernel (by value, constant bank).
+struct QuantParams {
+    const void *X;
+    int64_t M;
+    int K;
+    int64_t ld;
+    SegBounds sb;
+    const float *s_pos, *s_neg;
+    const int32_t *zp;        // zero-point mode: z per K-segment
+    int row_segments;         // weights: the scale also depends on the row's N-segment
+    int lo, hi;
+    uint8_t *c_pos, *c_neg;
+    int64_t ldc;
+    int V, R;
+    int act;                  // PRE: 0 = none, 1 = SiLU, 2 = GELU applied to the input first
+    const float *mult;        // PRE: per-channel multiplier [K] applied after it, or nullptr
+};
+
+// A quantize launch worked out ahead of time.
+struct QuantLaunch {
+    QuantParams prm;
+    const void *kernel;
+    unsigned blocks;
+};
+
 // zero_point != nullptr selects the App. A asymmetric quantizer (int8); act / mult: optional activation
 // function (0 none, 1 SiLU, 2 GELU) and per-channel multiplier [K] applied in front of the quantizer
 sq_status launch_quantize(const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld, const SegBounds &sb,
                           const float *s_pos, const float *s_neg, const int32_t *zero_point, int row_segments,
                           sq_code code, float q_max, float q_min_abs, int act, const float *mult,
                           void *c_pos, void *c_neg, int64_t ldc, cudaStream_t st);
+
+sq_status prepare_quantize(const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld, const SegBounds &sb,
+                           const float *s_pos, const float *s_neg, const int32_t *zero_point, int row_segments,
+                           sq_code code, float q_max, float q_min_abs, int act, const float *mult,
+                           void *c_pos, void *c_neg, int64_t ldc, QuantLaunch *out);    // launches nothing
+sq_status run_quantize(const QuantLaunch &l, cudaStream_t st);                          // one launch, no queries
 
 sq_status launch_calib_zero_point(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld, const SegBounds &sb,
                                   float *s_x, int32_t *z_x, uint32_t *partials, cudaStream_t st);
@@ -80,7 +112,35 @@ struct GemmArgs {
     void *acc_dump;
     uint32_t *status;
 };
-sq_status launch_gemm(const GemmArgs &g, cudaStream_t st);
+// Parameters of the GEMM kernel (by value, constant bank).
+struct KernelParams {
+    int M, N, K;
+    int nacc;          // P * npol
+    int acc_stages;    // 1 or 2 accumulator sets in TMEM
+    int stages;        // shared-memory ring depth
+    int num_m_tiles, num_n_tiles;
+    SegBounds sb;
+    const float *s_pos, *s_neg, *s_w, *bias;
+    void *Y;
+    long long ldy;     // elements
+    int y_is_f32;
+    int y_wide;        // rows of Y are 32-byte aligned: 256-bit stores allowed
+    void *acc_dump;
+    uint32_t *status;
+};
+
+// A GEMM launch worked out ahead of time: kernel instantiation, tensor maps, parameters, grid.
+struct GemmLaunch {
+    CUtensorMap ta, tn, tb, ty;
+    KernelParams prm;
+    const void *kernel;
+    unsigned grid, cluster;
+    size_t smem;
+    int device;
+};
+sq_status prepare_gemm(const GemmArgs &g, GemmLaunch *out);    // launches nothing
+sq_status run_gemm(const GemmLaunch &l, cudaStream_t st);      // one launch, no queries
+sq_status launch_gemm(const GemmArgs &g, cudaStream_t st);     // prepare + run
 void set_gemm_tuning(int tile_n, int stages, int cta_group, int segment_mode);
 
 }  // namespace sq

@@ -48,6 +48,11 @@ class SegQuantLinear:
                                         self.bias, Y, self.scratch_for(M), self.workspace,
                                         x_stage=x_stage, y_stage=y_stage, flags=self.flags)
 
+    def plan(self, X: torch.Tensor, Y: torch.Tensor) -> "B.LayerPlan":
+        """A prepared call for these device buffers: plan.run() issues the layer's two kernels and nothing else."""
+        return B.LayerPlan(X, self.Wq, self.seg, self.code, self.s_pos, self.s_neg, self.s_w, self.bias, Y,
+                           self.scratch_for(X.shape[0]), self.workspace, self.flags)
+
     def forward_pipelined(self, X_host: torch.Tensor, Y_host: torch.Tensor, x_stage, y_stage, chunks, stream_in, stream_out):
         """Pinned-host X -> pinned-host Y with the copies overlapped with the kernels (see the C header)."""
         M = X_host.shape[0]

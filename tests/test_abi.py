@@ -113,3 +113,29 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError):
         B.lib()
+
+
+def test_plan_calls_reject_on_the_host(L):
+    plan = (C.c_uint64 * (B.SQ_PLAN_BYTES // 8))()
+    # a plan that was never built (all zero) does not run
+    assert L.segquant_plan_run(C.byref(plan), None) == 5
+    assert L.segquant_plan_run(None, None) == 1
+    seg = _seg([0, 128], [0, 64])
+
+    def plan_layer(x=FAKE, y=FAKE, scratch=FAKE, scratch_bytes=1 << 20, K=128, ld=128, kb=(0, 128), s=FAKE, dt=1, code=0):
+        sg = _seg(list(kb), [0, 64])
+        return L.segquant_plan_layer(C.byref(plan), C.c_void_p(x), C.c_int(dt), C.c_int64(128), C.c_int64(K), C.c_int64(ld),
+                                     C.c_void_p(FAKE), C.c_int64(128), C.c_int64(64), sg.ref(), C.c_int(code), C.c_void_p(s),
+                                     None, C.c_void_p(FAKE), None, C.c_uint32(0), C.c_void_p(y), C.c_int(1), C.c_int64(64),
+                                     C.c_void_p(scratch), C.c_size_t(scratch_bytes), C.c_void_p(FAKE),
+                                     C.c_size_t(B.workspace_bytes()))
+    assert plan_layer(x=0) == 1 and plan_layer(y=0) == 1 and plan_layer(scratch=0) == 1 and plan_layer(s=0) == 1
+    assert plan_layer(dt=7) == 5 and plan_layer(code=9) == 5
+    assert plan_layer(ld=64) == 2                                 # pitch below K
+    assert plan_layer(scratch_bytes=100) == 8                     # code matrices do not fit
+    assert plan_layer(scratch=FAKE + 16) == 4
+    assert plan_layer(kb=(0, 40, 128)) == 4                       # interior K-bound not a multiple of 32
+    assert plan_layer(kb=(0, 64, 32, 128)) == 3
+    # a failed build leaves a plan that does not run
+    assert L.segquant_plan_run(C.byref(plan), None) == 5
+    assert seg.P == 1 and B.SQ_PLAN_BYTES == 4096

@@ -588,3 +588,75 @@ def test_argument_errors_are_reported_before_launch():
                                   None, torch.zeros(16, dtype=torch.uint8, device=DEV))
     assert e.value.status == 8
     assert B.segquant_launch_count() == n1 and n1 == n0 + 1
+
+
+# ------------------------------------------------------------------ prepared calls (plans)
+
+@pytest.mark.parametrize("case", [
+    ("plan_dual", 700, 384, 520, [0, 384], [0, 256, 520], True, "int8"),
+    ("plan_single_k_segments", 333, 512, 768, [0, 256, 512], [0, 256, 512, 768], False, "int8"),
+    ("plan_e4m3", 300, 256, 264, [0, 256], [0, 264], True, "e4m3"),
+])
+def test_planned_layer_call_equals_the_checked_call(case):
+    """segquant_plan_layer + segquant_plan_run give the bytes of segquant_layer_forward; a replay after the
+    input's contents changed gives the new input's output; building and running launch exactly 0 and 2 kernels;
+    the run can be captured into a CUDA graph."""
+    name, M, K, N, kb, nb, dual, code = case
+    spec = custom_spec(name, M, K, N, kb, nb, dual, code, seed=71)
+    data = WL.make_layer(spec)
+    layer = SegQuantLinear(data.W, data.bias, kb, nb, dual, code, DEV)
+    layer.calibrate(data.X_cal)
+    Xd = data.X.to(DEV)
+    Y_ref = layer.forward(Xd).clone()
+    X_in = Xd.clone()
+    Y = torch.zeros((M, N), dtype=torch.bfloat16, device=DEV)
+    torch.cuda.synchronize()
+    n0 = B.segquant_launch_count()
+    plan = layer.plan(X_in, Y)
+    assert B.segquant_launch_count() == n0                       # building launches nothing
+    plan.run()
+    assert B.segquant_launch_count() == n0 + 2
+    layer.check_status()
+    torch.cuda.synchronize()
+    assert torch.equal(Y, Y_ref)
+    X_in.copy_(torch.flip(Xd, dims=[0]) * 0.5)
+    Y_ref2 = layer.forward(X_in).clone()
+    Y.zero_()
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream, capture_error_mode="relaxed"):
+            plan.run()
+    torch.cuda.current_stream().wait_stream(stream)
+    graph.replay()
+    layer.check_status()
+    torch.cuda.synchronize()
+    assert torch.equal(Y, Y_ref2) and not torch.equal(Y_ref2, Y_ref)
+    res = O.layer_forward(to_f32_np(X_in.cpu()), oracle_scales(data)[3], O.SegTable(kb, nb), *oracle_scales(data)[:3],
+                          to_f32_np(data.bias), code=code, q_max=QRANGE[code][0], q_min_abs=QRANGE[code][1])
+    if code == "int8":
+        check_bf16_output(Y, res.y64, res.y_abs, (2 if dual else 1) * (len(kb) - 1))
+
+
+def test_calibration_beyond_one_grid_is_refused_without_a_launch():
+    """A matrix with more columns than the reduction's grid covers (65535 blocks of 256 columns) is refused
+    on the host: no kernel is launched and the partials are not touched."""
+    K = 65536 * 256
+    X = torch.zeros((1, K), dtype=torch.bfloat16, device=DEV)
+    ws = B.new_workspace(DEV)
+    ws[256:320] = 7
+    n0 = B.segquant_launch_count()
+    with pytest.raises(B.SegquantError) as e:
+        B.segquant_calib_scales(X, B.SegTable([0, K], [0, 8]), "int8", False, True, ws)
+    assert e.value.status == 2
+    with pytest.raises(B.SegquantError) as e:
+        B.segquant_calib_scales_static(X, B.SegTable([0, K], [0, 8]), "int8", False, True)
+    assert e.value.status == 2
+    torch.cuda.synchronize()
+    assert B.segquant_launch_count() == n0 and bool(torch.all(ws[256:320] == 7))
+    # one block of columns fewer is accepted
+    X2 = X[:, :K - 256]
+    s_pos, s_neg = B.segquant_calib_scales(X2, B.SegTable([0, K - 256], [0, 8]), "int8", False, True, ws)
+    torch.cuda.synchronize()
+    assert float(s_pos[0]) == 1.0 and float(s_neg[0]) == 1.0

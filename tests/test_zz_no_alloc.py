@@ -74,3 +74,38 @@ def test_static_calibration_refuses_more_blocks_than_it_holds():
     s_w, _ = B.segquant_calib_scales(X, seg, "int8", True, False, B.new_workspace(DEV))
     torch.cuda.synchronize()
     assert s_w.numel() == P * Q and bool(torch.all(s_w == 1.0))       # all-zero blocks: unit scale
+
+
+def test_static_calibration_allocates_nothing_and_takes_exactly_its_limit():
+    """The reason this entry point exists is that its caller cannot allocate: after one warm-up call (which looks
+    up the built-in array's address) a call leaves torch's allocator counters and the device's free memory
+    untouched.  And the limit is exact: 32 x 32 = 1024 weight blocks are accepted and give the workspace
+    version's scales; an activation table with more K- than N-segments (P > Q) goes through the same array."""
+    rs = np.random.default_rng(21)
+    P, Q = 32, 32
+    K, N = 32 * P, 8 * Q
+    W = torch.from_numpy(rs.normal(0, 0.02, (N, K)).astype(np.float32)).to(DEV)
+    W *= torch.linspace(0.5, 20.0, N, device=DEV)[:, None]
+    seg = B.SegTable(list(range(0, K + 1, 32)), list(range(0, N + 1, 8)))
+    out = torch.empty(P * Q, dtype=torch.float32, device=DEV)
+    B.segquant_calib_scales_static(W, seg, "int8", True, False, s_pos=out)            # warm-up call
+    torch.cuda.synchronize()
+    before = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), torch.cuda.mem_get_info()[0])
+    B.segquant_calib_scales_static(W, seg, "int8", True, False, s_pos=out)
+    torch.cuda.synchronize()
+    after = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), torch.cuda.mem_get_info()[0])
+    assert after == before
+    ref, _ = B.segquant_calib_scales(W, seg, "int8", True, False, B.new_workspace(DEV))
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy(), ref.cpu().numpy()) and len(np.unique(out.cpu().numpy())) > 100
+
+    # activations: 40 K-segments, 1 N-segment (P > Q)
+    Pa = 40
+    X = torch.from_numpy(rs.normal(0, 1, (50, 32 * Pa)).astype(np.float32)).to(DEV)
+    X *= torch.linspace(0.1, 30.0, 32 * Pa, device=DEV)[None, :]
+    seg_a = B.SegTable(list(range(0, 32 * Pa + 1, 32)), [0, 8])
+    sp, sn = torch.empty(Pa, device=DEV), torch.empty(Pa, device=DEV)
+    B.segquant_calib_scales_static(X, seg_a, "int8", False, True, s_pos=sp, s_neg=sn)
+    rp, rn = B.segquant_calib_scales(X, seg_a, "int8", False, True, B.new_workspace(DEV))
+    torch.cuda.synchronize()
+    assert torch.equal(sp, rp) and torch.equal(sn, rn)
