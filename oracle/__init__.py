@@ -340,6 +340,75 @@ def smooth(X, mult):
     return out
 
 
+# ------------------------------------------- W4A8: per-channel 4-bit weights, per-token activation scales
+
+def quantize_per_row(X, kb, dual, q_max=INT8_QMAX, q_min_abs=INT8_QMIN_ABS):
+    """One scale per (row, K-segment) from the row's own extrema, and the codes quantized with it.
+    Returns (s_pos [M,P], s_neg [M,P] | None, c_pos, c_neg | None)."""
+    X = _f32(X)
+    kb = _i32(kb)
+    M, K = X.shape
+    P = len(kb) - 1
+    s_pos = np.zeros((M, P), np.float32)
+    s_neg = np.zeros((M, P), np.float32) if dual else None
+    c_pos = np.zeros((M, K), np.int8)
+    c_neg = np.zeros((M, K), np.int8) if dual else None
+    lib().sqo_quantize_per_row_i8(_p(X), C.c_int64(M), C.c_int64(K), C.c_int64(K), C.c_int(P), _p(kb), C.c_int(int(dual)),
+                                  C.c_float(q_max), C.c_float(q_min_abs), _p(s_pos), _p(s_neg), _p(c_pos), _p(c_neg),
+                                  C.c_int64(K))
+    return s_pos, s_neg, c_pos, c_neg
+
+
+def pack_w4(Wq):
+    Wq = np.ascontiguousarray(Wq, np.int8)
+    N, K = Wq.shape
+    out = np.zeros((N, K // 2), np.uint8)
+    lib().sqo_pack_w4(_p(Wq), C.c_int64(N), C.c_int64(K), C.c_int64(K), _p(out), C.c_int64(K // 2))
+    return out
+
+
+def unpack_w4(packed):
+    packed = np.ascontiguousarray(packed, np.uint8)
+    N, K2 = packed.shape
+    out = np.zeros((N, 2 * K2), np.int8)
+    lib().sqo_unpack_w4(_p(packed), C.c_int64(N), C.c_int64(2 * K2), C.c_int64(K2), _p(out), C.c_int64(2 * K2))
+    return out
+
+
+def dequant_per_token(acc_pos, acc_neg, s_pos, s_neg, s_w, bias=None):
+    """fp64 recombination with per-token activation scales [M,P] and per-channel weight scales [N,P]."""
+    P, M, N = acc_pos.shape
+    a_pos = np.ascontiguousarray(acc_pos, np.float64)
+    a_neg = None if acc_neg is None else np.ascontiguousarray(acc_neg, np.float64)
+    y = np.zeros((M, N), np.float64)
+    ya = np.zeros((M, N), np.float64)
+    b = None if bias is None else _f32(bias)
+    lib().sqo_dequant_per_token(_p(a_pos), _p(a_neg), C.c_int64(M), C.c_int64(N), C.c_int(P), _p(_f32(s_pos)),
+                                _p(None if s_neg is None else _f32(s_neg)), _p(_f32(s_w)), _p(b), _p(y), _p(ya))
+    return y, ya
+
+
+@dataclass
+class W4A8Result:
+    s_pos: np.ndarray
+    s_neg: np.ndarray | None
+    c_pos: np.ndarray
+    c_neg: np.ndarray | None
+    acc_pos: np.ndarray
+    acc_neg: np.ndarray | None
+    y64: np.ndarray
+    y_abs: np.ndarray
+
+
+def layer_forward_w4a8(X, Wq, s_w, kb, dual, bias=None) -> W4A8Result:
+    """Per-token quantization of X, accumulation against the (unpacked) 4-bit weight codes, recombination."""
+    s_pos, s_neg, c_pos, c_neg = quantize_per_row(X, kb, dual)
+    acc_pos = accumulate(c_pos, Wq, kb, "int8")
+    acc_neg = accumulate(c_neg, Wq, kb, "int8") if dual else None
+    y64, y_abs = dequant_per_token(acc_pos, acc_neg, s_pos, s_neg, s_w, bias)
+    return W4A8Result(s_pos, s_neg, c_pos, c_neg, acc_pos, acc_neg, y64, y_abs)
+
+
 # ----------------------------------------------------------- whole layer
 
 @dataclass

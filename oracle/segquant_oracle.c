@@ -452,6 +452,69 @@ void sqo_smooth(const float *X, int64_t M, int64_t K, int64_t ld, const float *m
             out[m * ldo + k] = X[m * ld + k] * mult[k];
 }
 
+/* ---------------------------------- 4-bit weights with per-channel scales, per-token activation scales (W4A8) */
+
+/* App. B "Extra Hyperparameter Settings": in the 4-bit settings weights are quantized per channel and
+ * activations dynamically per token.  Combined with input segmentation (Sec. 4.2.2 item 2) every row r of a
+ * matrix gets one scale per K-segment p from its own extrema:
+ *   dual:   s_pos[r*P+p] = max(max x, 0) / q_max,  s_neg[r*P+p] = max(-min x, 0) / q_min_abs   (Sec. 4.3.2)
+ *   single: s_pos[r*P+p] = max|x| / q_max
+ * (an extremum of 0 gives scale 1) and is quantized with it by the same quantizer as everywhere else.
+ * Activations: rows are tokens, q_max = 127.  Weights: rows are output channels, q_max = 7 (symmetric 4-bit
+ * codes in [-7, 7]), single scale.                                                                          */
+void sqo_quantize_per_row_i8(const float *X, int64_t M, int64_t K, int64_t ld,
+                             int P, const int32_t *kb, int dual, float q_max, float q_min_abs,
+                             float *s_pos, float *s_neg, int8_t *c_pos, int8_t *c_neg, int64_t ldc)
+{
+    for (int64_t m = 0; m < M; m++) {
+        sqo_calib_act(X + m * ld, 1, K, ld, P, kb, dual, q_max, q_min_abs, s_pos + m * P, dual ? s_neg + m * P : NULL);
+        sqo_quantize_act_i8(X + m * ld, 1, K, ld, P, kb, s_pos + m * P, dual ? s_neg + m * P : NULL, q_max, q_min_abs,
+                            c_pos + m * ldc, dual ? c_neg + m * ldc : NULL, ldc);
+    }
+}
+
+/* Two 4-bit codes per byte: code 2j in the low nibble, code 2j+1 in the high nibble, two's complement. */
+void sqo_pack_w4(const int8_t *Wq, int64_t N, int64_t K, int64_t ld, uint8_t *out, int64_t ldo)
+{
+    for (int64_t n = 0; n < N; n++)
+        for (int64_t j = 0; j < K / 2; j++)
+            out[n * ldo + j] = (uint8_t)((Wq[n * ld + 2 * j] & 0xF) | ((Wq[n * ld + 2 * j + 1] & 0xF) << 4));
+}
+void sqo_unpack_w4(const uint8_t *in, int64_t N, int64_t K, int64_t ldi, int8_t *Wq, int64_t ld)
+{
+    for (int64_t n = 0; n < N; n++)
+        for (int64_t j = 0; j < K / 2; j++) {
+            uint8_t b = in[n * ldi + j];
+            Wq[n * ld + 2 * j] = (int8_t)(((b & 0xF) ^ 8) - 8);
+            Wq[n * ld + 2 * j + 1] = (int8_t)(((b >> 4) ^ 8) - 8);
+        }
+}
+
+/* y[m][n] = sum_p ( s_pos[m*P+p] s_w[n*P+p] acc_pos[p][m][n] + s_neg[m*P+p] s_w[n*P+p] acc_neg[p][m][n] ) + bias[n]
+ * in fp64 (Sec. 4.3.2 recombination with per-token and per-channel scales).                                  */
+void sqo_dequant_per_token(const double *acc_pos, const double *acc_neg, int64_t M, int64_t N, int P,
+                           const float *s_pos, const float *s_neg, const float *s_w, const float *bias,
+                           double *y, double *ysum_abs)
+{
+    for (int64_t m = 0; m < M; m++)
+        for (int64_t n = 0; n < N; n++) {
+            double v = 0.0, av = 0.0;
+            for (int p = 0; p < P; p++) {
+                int64_t i = ((int64_t)p * M + m) * N + n;
+                double sw = (double)s_w[n * P + p];
+                double t = (double)s_pos[m * P + p] * sw * acc_pos[i];
+                v += t; av += fabs(t);
+                if (acc_neg) {
+                    double u = (double)s_neg[m * P + p] * sw * acc_neg[i];
+                    v += u; av += fabs(u);
+                }
+            }
+            if (bias) { v += (double)bias[n]; av += fabs((double)bias[n]); }
+            y[m * N + n] = v;
+            if (ysum_abs) ysum_abs[m * N + n] = av;
+        }
+}
+
 /* fp64 -> bf16 bit pattern, round-to-nearest-even directly from the fp64 value
  * (no intermediate fp32 rounding).  Finite inputs within bf16 range only.    */
 uint16_t sqo_bf16_from_f64(double v)

@@ -56,6 +56,14 @@ MUTATIONS = {
     "gelu_tanh_like_argument": ("return 0.5 * h * erfc(-h / sqrt(2.0));", "return 0.5 * h * erfc(-h / 2.0);"),
     "activation_rounded_twice": ("uint32_t bits = (uint32_t)sqo_bf16_from_f64(a) << 16;", "uint32_t bits = (uint32_t)sqo_bf16_from_f64((double)(float)a + 1e-3 * a) << 16;"),
     "smooth_indexed_by_row": ("out[m * ldo + k] = X[m * ld + k] * mult[k];", "out[m * ldo + k] = X[m * ld + k] * mult[m % K];"),
+    "per_row_uses_first_rows_scales": ("sqo_quantize_act_i8(X + m * ld, 1, K, ld, P, kb, s_pos + m * P,", "sqo_quantize_act_i8(X + m * ld, 1, K, ld, P, kb, s_pos,"),
+    "per_row_scales_from_whole_matrix": ("sqo_calib_act(X + m * ld, 1, K, ld, P, kb, dual,", "sqo_calib_act(X, M, K, ld, P, kb, dual,"),
+    "w4_nibbles_swapped": ("out[n * ldo + j] = (uint8_t)((Wq[n * ld + 2 * j] & 0xF) | ((Wq[n * ld + 2 * j + 1] & 0xF) << 4));",
+                           "out[n * ldo + j] = (uint8_t)((Wq[n * ld + 2 * j + 1] & 0xF) | ((Wq[n * ld + 2 * j] & 0xF) << 4));"),
+    "w4_unpack_without_sign": ("Wq[n * ld + 2 * j] = (int8_t)(((b & 0xF) ^ 8) - 8);", "Wq[n * ld + 2 * j] = (int8_t)(b & 0xF);"),
+    "per_token_weight_scale_index_transposed": ("double sw = (double)s_w[n * P + p];", "double sw = (double)s_w[p * N + n];"),
+    "per_token_act_scale_of_wrong_token": ("double t = (double)s_pos[m * P + p] * sw * acc_pos[i];", "double t = (double)s_pos[p] * sw * acc_pos[i];"),
+    "per_token_negative_path_uses_positive_scale": ("double u = (double)s_neg[m * P + p] * sw * acc_neg[i];", "double u = (double)s_pos[m * P + p] * sw * acc_neg[i];"),
     "bf16_truncates": ("double q = nearbyint((f * 2.0 - 1.0) * 128.0);", "double q = floor((f * 2.0 - 1.0) * 128.0);"),
 }
 

@@ -770,3 +770,121 @@ def test_smoothing_multiplier_is_one_fp32_multiply():
     m = r.uniform(0.1, 4.0, 40).astype(np.float32)
     assert np.array_equal(O.smooth(X, m), X * m[None, :])
     assert O.smooth(X, m).dtype == np.float32
+
+
+# --------------------------------------------------------------- W4A8: per-channel 4-bit weights, per-token scales
+
+def test_per_row_scales_and_codes_match_closed_form_and_library_quantizer():
+    r = rng(50)
+    kb = [0, 24, 64]
+    X = gelu(r.normal(0, 1.5, (20, 64))).astype(np.float32)
+    X[3] = 0.0                                                      # an all-zero token
+    X[4, :24] = np.abs(X[4, :24])                                   # a token without negative values in segment 0
+    for dual in (False, True):
+        s_pos, s_neg, c_pos, c_neg = O.quantize_per_row(X, kb, dual)
+        for m in range(20):
+            for p in range(2):
+                seg = X[m, kb[p]:kb[p + 1]]
+                if dual:
+                    hi, lo = max(float(seg.max()), 0.0), max(float(-seg.min()), 0.0)
+                    assert s_pos[m, p] == (np.float32(hi) / np.float32(127.0) if hi > 0 else 1.0)
+                    assert s_neg[m, p] == (np.float32(lo) / np.float32(128.0) if lo > 0 else 1.0)
+                else:
+                    a = float(np.abs(seg).max())
+                    assert s_pos[m, p] == (np.float32(a) / np.float32(127.0) if a > 0 else 1.0)
+            # the row's codes are those of the library quantizer with the row's own scales
+            if dual:
+                tp, tn = torch_dual_codes(X[m:m + 1], kb, s_pos[m], s_neg[m])
+                assert np.array_equal(c_pos[m:m + 1], tp) and np.array_equal(c_neg[m:m + 1], tn)
+            else:
+                assert np.array_equal(c_pos[m:m + 1], torch_sym_codes(X[m:m + 1], kb, s_pos[m]))
+        # every token uses its full range: the row extremum sits on the end of the code range
+        assert np.all(np.abs(c_pos[[0, 1, 2, 5]].astype(int)).max(axis=1) == 127)
+    # 4-bit weights: the same quantizer with q_max = 7
+    W = r.normal(0, 0.02, (12, 64)).astype(np.float32)
+    s_w, _, Wq, _ = O.quantize_per_row(W, kb, False, q_max=7.0, q_min_abs=7.0)
+    assert Wq.min() == -7 and Wq.max() == 7
+    for n in range(12):
+        assert np.array_equal(Wq[n:n + 1], torch_sym_codes(W[n:n + 1], kb, s_w[n], qmax=7.0))
+        assert s_w[n, 1] == np.float32(np.abs(W[n, 24:]).max()) / np.float32(7.0)
+
+
+def test_w4_pack_roundtrip_and_nibble_order():
+    r = rng(51)
+    Wq = r.integers(-8, 8, (9, 32)).astype(np.int8)
+    packed = O.pack_w4(Wq)
+    assert packed.shape == (9, 16)
+    assert np.array_equal(O.unpack_w4(packed), Wq)
+    one = np.zeros((1, 4), np.int8); one[0] = [1, -1, 7, -8]
+    assert O.pack_w4(one).tolist() == [[0xF1, 0x87]]                  # even code in the low nibble, two's complement
+
+
+@pytest.mark.parametrize("dual", [False, True])
+def test_w4a8_recombination_equals_brute_force_and_exact_on_grid(dual):
+    r = rng(52)
+    M, N, K = 5, 6, 24
+    kb = [0, 8, 24]
+    X = gelu(r.normal(0, 1.5, (M, K))).astype(np.float32)
+    W = r.normal(0, 0.02, (N, K)).astype(np.float32)
+    bias = r.normal(0, 0.1, N).astype(np.float32)
+    s_w, _, Wq, _ = O.quantize_per_row(W, kb, False, q_max=7.0, q_min_abs=7.0)
+    res = O.layer_forward_w4a8(X, O.unpack_w4(O.pack_w4(Wq)), s_w, kb, dual, bias)
+    for m in range(M):
+        for n in range(N):
+            tot, tot_abs = float(bias[n]), abs(float(bias[n]))
+            for p in range(2):
+                ks = range(kb[p], kb[p + 1])
+                ap = sum(int(res.c_pos[m, k]) * int(Wq[n, k]) for k in ks)
+                t = float(res.s_pos[m, p]) * float(s_w[n, p]) * ap
+                tot += t; tot_abs += abs(t)
+                if dual:
+                    an = sum(int(res.c_neg[m, k]) * int(Wq[n, k]) for k in ks)
+                    u = float(res.s_neg[m, p]) * float(s_w[n, p]) * an
+                    tot += u; tot_abs += abs(u)
+            assert math.isclose(res.y64[m, n], tot, rel_tol=1e-12, abs_tol=1e-15)
+            assert math.isclose(res.y_abs[m, n], tot_abs, rel_tol=1e-12)
+    # the layer approximates X W^T + b within the half-step bounds of both operands
+    exact = X.astype(np.float64) @ W.astype(np.float64).T + bias
+    ex = np.zeros((M, K)); ew = np.zeros((N, K))
+    for p in range(2):
+        ks = slice(kb[p], kb[p + 1])
+        sp = res.s_pos[:, p:p + 1].astype(np.float64)
+        sn = res.s_neg[:, p:p + 1].astype(np.float64) if dual else sp
+        ex[:, ks] = np.where(X[:, ks] >= 0, sp, sn) / 2
+        ew[:, ks] = s_w[:, p:p + 1].astype(np.float64) / 2
+    bound = ex @ np.abs(W.astype(np.float64)).T + (np.abs(X.astype(np.float64)) + ex) @ ew.T
+    assert np.all(np.abs(res.y64 - exact) <= bound * (1 + 1e-9))
+    # power-of-two scales and on-grid operands: exact
+    cx = r.integers(-127, 128, (M, K)); cw = r.integers(-7, 8, (N, K))
+    cx[:, 0] = 127; cx[:, 8] = -127 if not dual else 127; cw[:, 0] = 7; cw[:, 8] = -7
+    if dual:
+        cx[:, 1] = -128; cx[:, 9] = -128
+    Xg = np.where(cx >= 0, cx * 2.0 ** -5, cx * (2.0 ** -9 if dual else 2.0 ** -5)).astype(np.float32)
+    Wg = (cw * 2.0 ** -6).astype(np.float32)
+    s_wg, _, Wqg, _ = O.quantize_per_row(Wg, kb, False, q_max=7.0, q_min_abs=7.0)
+    assert np.array_equal(Wqg, cw) and np.all(s_wg == 2.0 ** -6)
+    resg = O.layer_forward_w4a8(Xg, Wqg, s_wg, kb, dual, None)
+    assert np.array_equal(resg.c_pos.astype(int) + (resg.c_neg.astype(int) if dual else 0), cx)
+    assert np.array_equal(resg.y64, Xg.astype(np.float64) @ Wg.astype(np.float64).T)
+
+
+def test_per_token_scales_lower_error_against_one_scale_for_all_tokens():
+    # tokens whose magnitudes differ by orders of magnitude: one scale for all of them leaves the small tokens
+    # a handful of codes, a scale per token gives every token the full range
+    r = rng(53)
+    X = r.normal(0, 1, (64, 128)).astype(np.float32) * (10.0 ** r.uniform(-2.0, 1.3, (64, 1))).astype(np.float32)
+    s_tok, _, c_tok, _ = O.quantize_per_row(X, [0, 128], False)
+    s_all, _ = O.calib_act(X, [0, 128], False)
+    c_all, _ = O.quantize_act(X, [0, 128], s_all)
+    row_err = lambda rec: np.linalg.norm(rec - X, axis=1) / np.linalg.norm(X, axis=1)
+    e_tok = row_err(s_tok.astype(np.float64) * c_tok)
+    e_all = row_err(float(s_all[0]) * c_all.astype(np.float64))
+    assert np.all(e_tok <= e_all * 1.0001) and np.median(e_tok) < 0.2 * np.median(e_all)
+    # and through a layer with 8-bit per-channel weights the output error follows
+    W = r.normal(0, 0.02, (32, 128)).astype(np.float32)
+    exact = X.astype(np.float64) @ W.astype(np.float64).T
+    s_w, _, Wq, _ = O.quantize_per_row(W, [0, 128], False)
+    y_tok = O.layer_forward_w4a8(X, Wq, s_w, [0, 128], False).y64
+    y_all, _ = O.dequant_per_token(O.accumulate(c_all, Wq, [0, 128]), None, np.full((64, 1), s_all[0], np.float32), None, s_w)
+    out_err = lambda y: np.linalg.norm(y - exact, axis=1) / np.linalg.norm(exact, axis=1)
+    assert np.median(out_err(y_tok)) < 0.5 * np.median(out_err(y_all))
