@@ -152,6 +152,15 @@ class BenchLayer:
             self.zp = {"s_x": s_x, "z_x": z_x, "codes": B.new_codes(self.M, spec.K, device),
                        "bias": B.segquant_fold_zero_point(L.Wq, L.seg, s_x, z_x, L.s_w, L.bias)}
         self.a_stage = torch.empty_like(self.X) if (spec.dual and self.act) else None
+        # the same layer as W4A8: per-channel 4-bit weights (kept packed), per-token activation scales
+        self.w4 = None
+        if spec.code == "int8" and spec.K <= 16384:
+            seg4 = B.SegTable(spec.kb, [0, spec.N])
+            s_w4, _, w8, _ = B.segquant_quantize_per_row(data.W.to(device), seg4, False, bits=4)
+            self.w4 = {"s_w": s_w4, "packed": B.segquant_pack_w4(w8), "w8": w8,
+                       "s_pos": torch.empty((self.M, spec.P), dtype=torch.float32, device=device),
+                       "s_neg": torch.empty((self.M, spec.P), dtype=torch.float32, device=device) if spec.dual else None}
+            self.seg4 = seg4
 
     def quantize(self):
         L = self.layer
@@ -195,6 +204,25 @@ class BenchLayer:
         else:
             torch.ops.aten.gelu.out(self.X, out=self.a_stage)
 
+    def w4_unpack(self):
+        self.B.segquant_unpack_w4(self.w4["packed"], out=self.w4["w8"])
+
+    def w4_quantize(self):
+        """Per-token scales and codes (one kernel)."""
+        L, w = self.B.lib(), self.w4
+        import ctypes as C
+        from paper_2507_14811_b200.binding import _ptr, _dt, _stream, _check
+        st = L.segquant_quantize_per_row(_ptr(self.X), C.c_int(_dt(self.X)), C.c_int64(self.M), C.c_int64(self.spec.K),
+                                         C.c_int64(self.X.stride(0)), self.seg4.ref(), C.c_int(8), C.c_uint32(0),
+                                         _ptr(w["s_pos"]), _ptr(w["s_neg"]), _ptr(self.c_pos), _ptr(self.c_neg),
+                                         C.c_int64(self.c_pos.stride(0)), _stream())
+        _check(st, "segquant_quantize_per_row")
+
+    def w4_gemm(self):
+        w = self.w4
+        self.B.segquant_w4a8_gemm(self.c_pos, self.c_neg, w["w8"], self.seg4, w["s_pos"], w["s_neg"], w["s_w"],
+                                  self.layer.bias, self.layer.workspace, Y=self.Y)
+
     def gemm_plain(self):
         """The same shape as a plain single-scale W8A8 layer (one code matrix): the denominator of the
         DualScale overhead.  Timing only; its output is not checked."""
@@ -229,6 +257,8 @@ class BenchLayer:
             setattr(other, name, None if t is None else t.clone())
         if self.zp is not None:
             other.zp = {k: v.clone() for k, v in self.zp.items()}
+        if self.w4 is not None:
+            other.w4 = {k: (None if v is None else v.clone()) for k, v in self.w4.items()}
         return other
 
     def device_bytes(self):
@@ -269,7 +299,7 @@ def graph_time_per_launch(calls, rounds):
     return e0.elapsed_time(e1) * 1e3 / (rounds * len(calls))
 
 
-def time_kernels(layers, launches=48, max_copies=96):
+def time_kernels(layers, launches=48, max_copies=96, with_w4a8=True):
     """Per-layer device time of each kernel, timed alone: a CUDA graph of >= `launches` launches of that one
     kernel, launch i on copy i mod C of the layer's device buffers, C chosen so that the copies the kernel walks
     through are at least twice the L2 capacity (every launch finds its operands in HBM).  A single launch between
@@ -277,7 +307,7 @@ def time_kernels(layers, launches=48, max_copies=96):
     event pair around one small kernel reads 6-8 us more than the kernel's own span.
     Returns lists (quantize_us, gemm_us, plain_us | None, unsegmented_us | None, copies)."""
     out = {"q": [], "g": [], "plain": [], "unseg": [], "copies": [], "q_plain": [], "q_zp": [], "g_zp": [], "q_fused": [],
-           "act": []}
+           "act": [], "w4_q": [], "w4_unpack": [], "w4_g": []}
     for bl in layers:
         s = bl.spec
         foot = min(quant_bytes(s, bl.M), gemm_bytes(s, bl.M))
@@ -296,6 +326,10 @@ def time_kernels(layers, launches=48, max_copies=96):
         fused = s.dual and bl.act
         out["q_fused"].append(graph_time_per_launch([c.quantize_fused_act for c in copies], rounds) if fused else None)
         out["act"].append(graph_time_per_launch([c.act_unfused for c in copies], rounds) if fused else None)
+        w4 = bl.w4 is not None and with_w4a8
+        out["w4_q"].append(graph_time_per_launch([c.w4_quantize for c in copies], rounds) if w4 else None)
+        out["w4_unpack"].append(graph_time_per_launch([c.w4_unpack for c in copies], rounds) if w4 else None)
+        out["w4_g"].append(graph_time_per_launch([c.w4_gemm for c in copies], rounds) if w4 else None)
         del copies
         torch.cuda.empty_cache()
     return out
@@ -525,6 +559,12 @@ def layer_table(specs, kt, peaks):
                 r.update({"asym_quant_us": us(kt["q_zp"][i]), "asym_gemm_us": us(kt["g_zp"][i]),
                           "dual_layer_time_over_asym_layer": round(layer_us / zp_us, 3),
                           "asym_layer_time_over_plain_layer": round(zp_us / plain_us, 3)})
+        if kt["w4_q"][i] is not None:
+            w4_us = kt["w4_q"][i] + kt["w4_unpack"][i] + kt["w4_g"][i]
+            r["w4a8"] = {"per_token_quant_us": us(kt["w4_q"][i]), "unpack_us": us(kt["w4_unpack"][i]),
+                         "gemm_us": us(kt["w4_g"][i]), "layer_time_over_w8a8_layer": round(w4_us / layer_us, 3),
+                         "note": "per-channel 4-bit weights kept packed and unpacked in front of the GEMM, per-token "
+                                 "activation scales; the GEMM runs the variant with per-(token, channel) factors"}
         if kt["q_fused"][i] is not None:
             r["fused_act"] = {"act": s.x_kind.partition("+")[2], "fused_quant_us": us(kt["q_fused"][i]),
                               "unfused_act_us": us(kt["act"][i]), "unfused_pair_us": us(kt["act"][i] + q * 1e3),
@@ -548,7 +588,7 @@ def measure_side_workload(name, dev, args, peaks):
     specs = WL.WORKLOADS[name]
     layers = [BenchLayer(s, dev) for s in specs]
     time.sleep(COOL_DOWN_S)                    # the power state of the previous long region must not leak in
-    kt = time_kernels(layers)
+    kt = time_kernels(layers, with_w4a8=name in ("dit_xl2", "sd3_heads"))
     for bl in layers:
         bl.layer.check_status()
     sets, set_bytes, n_sets = buffer_sets(layers)

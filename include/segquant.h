@@ -239,6 +239,39 @@ sq_status segquant_layer_forward_pipelined(const void *X, void *x_stage, sq_dtyp
                                            void *workspace, size_t ws_bytes, int chunks, void *stream,
                                            void *stream_in, void *stream_out);
 
+/* 4-bit weights with per-channel scales, 8-bit activations with dynamic per-token scales -- App. B "Extra
+ * Hyperparameter Settings" ("In 4-bit settings, weights are quantized per-channel, and activations are quantized
+ * dynamically per-token"), Table 1 rows "4/8 (int)"; combined with input segmentation (Sec. 4.2.2 item 2) and
+ * DualScale (Sec. 4.3.2) every row gets one scale per K-segment (and polarity) from its own extrema.
+ *   segquant_quantize_per_row: for every row r of X [rows,K] and K-segment p
+ *       s_neg == NULL: s_pos[r*P+p] = max|x| / q_max,  codes clip(round(x / s), -q_max, q_max) into c_pos;
+ *       s_neg != NULL: s_pos[r*P+p] = max(max x, 0) / 127, s_neg[r*P+p] = max(-min x, 0) / 128 and the DualScale codes
+ *                      of segquant_quantize_act into c_pos / c_neg (bits = 8 only);
+ *     bits = 8: q_max = 127 (tokens of an activation matrix); bits = 4: q_max = 7 (output channels of a weight
+ *     matrix; symmetric 4-bit codes in [-7, 7], one int8 per code, to be packed by segquant_pack_w4).
+ *     An extremum of 0 gives scale 1.  s_pos / s_neg: dev float [rows*P], written.  K <= 16384 (a row is held in
+ *     one thread block's registers); more is refused with SQ_ERR_UNSUPPORTED.  Alignment as segquant_quantize_act.
+ *   segquant_pack_w4 / segquant_unpack_w4: int8 codes in [-8, 7] <-> two 4-bit two's-complement codes per byte,
+ *     code 2j in the low nibble of byte j.  Wq8 [N,K] (ld8 bytes, 16-byte aligned), Wq4 [N,K/2] (ld4 bytes, 8-byte
+ *     aligned, a multiple of 8); K a multiple of 16.  The GEMM reads 8-bit operands, so a layer keeps its weights
+ *     packed (half the bytes) and unpacks them into an int8 scratch matrix in front of the GEMM.
+ *   segquant_w4a8_gemm: y[m][n] = sum_p ( s_pos[m*P+p] s_w[n*P+p] acc_pos[p][m][n]
+ *                                        + s_neg[m*P+p] s_w[n*P+p] acc_neg[p][m][n] ) + bias[n]
+ *     with the accumulators of segquant_dualscale_gemm (Xq_neg == NULL: single path, s_neg ignored).  s_pos / s_neg
+ *     dev [M*P], s_w dev [N*P] as written by segquant_quantize_per_row; the segment table must have Q = 1.  Per
+ *     term one fp32 product of the two scales and one FMA, ascending p.  Other arguments, alignment and limits
+ *     as segquant_dualscale_gemm. */
+sq_status segquant_quantize_per_row(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld,
+                                    const sq_segtable *seg, int bits, uint32_t flags, float *s_pos, float *s_neg,
+                                    void *c_pos, void *c_neg, int64_t ldc, void *stream);
+sq_status segquant_pack_w4(const void *Wq8, int64_t ld8, int64_t N, int64_t K, void *Wq4, int64_t ld4, void *stream);
+sq_status segquant_unpack_w4(const void *Wq4, int64_t ld4, int64_t N, int64_t K, void *Wq8, int64_t ld8, void *stream);
+sq_status segquant_w4a8_gemm(const void *Xq_pos, const void *Xq_neg, int64_t ldx, const void *Wq8, int64_t ldw,
+                             int64_t M, int64_t N, int64_t K, const sq_segtable *seg,
+                             const float *s_pos, const float *s_neg, const float *s_w, const float *bias,
+                             void *Y, sq_dtype y_dtype, int64_t ldy, void *acc_dump,
+                             void *workspace, size_t ws_bytes, void *stream);
+
 /* A layer call prepared once and replayed.  segquant_plan_layer does everything segquant_layer_forward does on
  * the host for device X and Y -- argument checks, tile plan, kernel choice, tensor-map encoding, attribute set-up --
  * and stores the result in caller-owned memory instead of launching; segquant_plan_run then issues the layer's

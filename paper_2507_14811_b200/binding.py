@@ -28,6 +28,7 @@ EXPORTS = [
     "segquant_layer_forward", "segquant_layer_forward_pipelined", "segquant_last_device_status", "segquant_set_tuning", "segquant_launch_count", "segquant_last_cuda_error",
     "segquant_status_string", "segquant_quantize_act_fused", "segquant_calib_zero_point",
     "segquant_quantize_act_zero_point", "segquant_fold_zero_point", "segquant_plan_layer", "segquant_plan_run",
+    "segquant_quantize_per_row", "segquant_pack_w4", "segquant_unpack_w4", "segquant_w4a8_gemm",
 ]
 
 
@@ -310,6 +311,56 @@ def segquant_layer_forward_pipelined(X, Wq, seg: SegTable, code: str, s_pos, s_n
         C.c_void_p(stream_in.cuda_stream), C.c_void_p(stream_out.cuda_stream))
     _check(st, "segquant_layer_forward_pipelined")
     return Y
+
+
+def segquant_quantize_per_row(X: torch.Tensor, seg: SegTable, dual: bool, bits: int = 8, flags: int = 0):
+    """Per-row scales [rows, P] (per token, or per output channel for bits = 4) and the int8 codes made with them."""
+    rows, K = X.shape
+    s_pos = torch.empty((rows, seg.P), dtype=torch.float32, device=X.device)
+    s_neg = torch.empty((rows, seg.P), dtype=torch.float32, device=X.device) if dual else None
+    c_pos = new_codes(rows, K, X.device)
+    c_neg = new_codes(rows, K, X.device) if dual else None
+    st = lib().segquant_quantize_per_row(_ptr(X), C.c_int(_dt(X)), C.c_int64(rows), C.c_int64(K), C.c_int64(X.stride(0)),
+                                         seg.ref(), C.c_int(bits), C.c_uint32(flags), _ptr(s_pos), _ptr(s_neg), _ptr(c_pos),
+                                         _ptr(c_neg), C.c_int64(c_pos.stride(0)), _stream())
+    _check(st, "segquant_quantize_per_row")
+    return s_pos, s_neg, c_pos, c_neg
+
+
+def segquant_pack_w4(Wq8: torch.Tensor):
+    N, K = Wq8.shape
+    out = torch.empty((N, K // 2), dtype=torch.uint8, device=Wq8.device)
+    st = lib().segquant_pack_w4(_ptr(Wq8), C.c_int64(Wq8.stride(0)), C.c_int64(N), C.c_int64(K), _ptr(out),
+                                C.c_int64(out.stride(0)), _stream())
+    _check(st, "segquant_pack_w4")
+    return out
+
+
+def segquant_unpack_w4(Wq4: torch.Tensor, out=None):
+    N, K2 = Wq4.shape
+    if out is None:
+        out = new_codes(N, 2 * K2, Wq4.device)
+    st = lib().segquant_unpack_w4(_ptr(Wq4), C.c_int64(Wq4.stride(0)), C.c_int64(N), C.c_int64(2 * K2), _ptr(out),
+                                  C.c_int64(out.stride(0)), _stream())
+    _check(st, "segquant_unpack_w4")
+    return out
+
+
+def segquant_w4a8_gemm(Xq_pos, Xq_neg, Wq8, seg: SegTable, s_pos, s_neg, s_w, bias, workspace,
+                       y_dtype=torch.bfloat16, Y=None, dump_acc=False):
+    M, K = Xq_pos.shape
+    N = Wq8.shape[0]
+    dual = Xq_neg is not None
+    if Y is None:
+        Y = _new_y(M, N, y_dtype, Xq_pos.device)
+    dump = _new_dump(seg.P * (2 if dual else 1), M, N, "int8", Xq_pos.device) if dump_acc else None
+    st = lib().segquant_w4a8_gemm(_ptr(Xq_pos), _ptr(Xq_neg), C.c_int64(Xq_pos.stride(0)), _ptr(Wq8),
+                                  C.c_int64(Wq8.stride(0)), C.c_int64(M), C.c_int64(N), C.c_int64(K), seg.ref(),
+                                  _ptr(s_pos), _ptr(s_neg), _ptr(s_w), _ptr(bias), _ptr(Y), C.c_int(_dt(Y)),
+                                  C.c_int64(Y.stride(0)), _ptr(dump), _ptr(workspace), C.c_size_t(workspace.numel()),
+                                  _stream())
+    _check(st, "segquant_w4a8_gemm")
+    return (Y, dump) if dump_acc else Y
 
 
 SQ_PLAN_BYTES = 4096

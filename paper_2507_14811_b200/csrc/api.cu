@@ -59,7 +59,7 @@ static sq_status gemm_args(const void *a_pos, const void *a_neg, int dual, int64
                            int64_t M, int64_t N, int64_t K, const sq_segtable *seg, sq_code code,
                            const float *s_pos, const float *s_neg, const float *s_w, const float *bias, void *Y,
                            sq_dtype y_dtype, int64_t ldy, void *acc_dump, void *workspace, size_t ws_bytes,
-                           GemmArgs *out)
+                           GemmArgs *out, int per_token = 0)
 {
     if (!s_pos || !s_w || (dual && (!a_neg || !s_neg))) return SQ_ERR_NULL;
     if (!valid_code(code) || !valid_dt(y_dtype)) return SQ_ERR_UNSUPPORTED;
@@ -85,7 +85,12 @@ static sq_status gemm_args(const void *a_pos, const void *a_neg, int dual, int64
     g.M = M; g.N = N; g.K = K;
     g.sb = hs.b;
     g.code = code;
-    g.s_pos = s_pos; g.s_neg = dual ? s_neg : nullptr; g.s_w = s_w; g.bias = bias;
+    if (per_token) {     // s_pos / s_neg are [M][P] token scales, s_w is [N][P] channel scales
+        g.row_pos = s_pos; g.row_neg = dual ? s_neg : nullptr; g.col_scale = s_w;
+    } else {
+        g.s_pos = s_pos; g.s_neg = dual ? s_neg : nullptr; g.s_w = s_w;
+    }
+    g.bias = bias;
     g.Y = Y; g.y_dtype = y_dtype; g.ldy = ldy;
     g.acc_dump = acc_dump;
     g.status = static_cast<uint32_t *>(workspace);
@@ -385,6 +390,58 @@ sq_status segquant_layer_forward_pipelined(const void *X, void *x_stage, sq_dtyp
         fail(SQ_ERR_CUDA);
     for (int i = 0; i < nev; i++) cudaEventDestroy(ev[i]);
     return r;
+}
+
+sq_status segquant_quantize_per_row(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld,
+                                    const sq_segtable *seg, int bits, uint32_t flags, float *s_pos, float *s_neg,
+                                    void *c_pos, void *c_neg, int64_t ldc, void *stream)
+{
+    if (!s_pos || (s_neg && !c_neg)) return SQ_ERR_NULL;
+    if (!valid_dt(dt) || (bits != 8 && bits != 4) || (bits == 4 && s_neg)) return SQ_ERR_UNSUPPORTED;
+    sq_status st;
+    if ((st = check_matrix(X, rows, K, ld, dt_size(dt))) != SQ_OK) return st;
+    if ((st = check_matrix(c_pos, rows, K, ldc, 1)) != SQ_OK) return st;
+    if (s_neg && (st = check_matrix(c_neg, rows, K, ldc, 1)) != SQ_OK) return st;
+    HostSeg hs = load_segtable(seg, K, seg && seg->nb && seg->Q >= 1 ? seg->nb[seg->Q] : 0);
+    if (hs.status != SQ_OK) return hs.status;
+    const float q_max = bits == 4 ? 7.0f : 127.0f;
+    const float q_min_abs = bits == 4 ? 7.0f : code_qmin_abs(SQ_CODE_INT8, flags);
+    return launch_quantize_per_row(X, dt, rows, K, ld, hs.b, s_neg != nullptr, q_max, q_min_abs, s_pos, s_neg, c_pos,
+                                   c_neg, ldc, static_cast<cudaStream_t>(stream));
+}
+
+static sq_status w4_common(const void *w8, int64_t ld8, void *w4, int64_t ld4, int64_t N, int64_t K, int unpack, void *stream)
+{
+    sq_status st;
+    if ((st = check_matrix(w8, N, K, ld8, 1)) != SQ_OK) return st;
+    if (K % 16 != 0) return SQ_ERR_ALIGN;
+    if (!w4) return SQ_ERR_NULL;
+    if (ld4 < K / 2) return SQ_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(w4) & 7u) || ld4 % 8 != 0) return SQ_ERR_ALIGN;
+    return launch_pack_w4(w8, ld8, N, K, w4, ld4, unpack, static_cast<cudaStream_t>(stream));
+}
+
+sq_status segquant_pack_w4(const void *Wq8, int64_t ld8, int64_t N, int64_t K, void *Wq4, int64_t ld4, void *stream)
+{
+    return w4_common(Wq8, ld8, Wq4, ld4, N, K, 0, stream);
+}
+
+sq_status segquant_unpack_w4(const void *Wq4, int64_t ld4, int64_t N, int64_t K, void *Wq8, int64_t ld8, void *stream)
+{
+    return w4_common(Wq8, ld8, const_cast<void *>(Wq4), ld4, N, K, 1, stream);
+}
+
+sq_status segquant_w4a8_gemm(const void *Xq_pos, const void *Xq_neg, int64_t ldx, const void *Wq8, int64_t ldw,
+                             int64_t M, int64_t N, int64_t K, const sq_segtable *seg, const float *s_pos,
+                             const float *s_neg, const float *s_w, const float *bias, void *Y, sq_dtype y_dtype,
+                             int64_t ldy, void *acc_dump, void *workspace, size_t ws_bytes, void *stream)
+{
+    const int dual = Xq_neg != nullptr;
+    if (seg && seg->Q != 1) return SQ_ERR_SEGTABLE;             // per-channel scales subsume output segments
+    GemmArgs g;
+    const sq_status st = gemm_args(Xq_pos, Xq_neg, dual, ldx, Wq8, ldw, M, N, K, seg, SQ_CODE_INT8, s_pos, s_neg, s_w,
+                                   bias, Y, y_dtype, ldy, acc_dump, workspace, ws_bytes, &g, 1);
+    return st == SQ_OK ? launch_gemm(g, static_cast<cudaStream_t>(stream)) : st;
 }
 
 sq_status segquant_plan_layer(sq_plan *plan, const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld,

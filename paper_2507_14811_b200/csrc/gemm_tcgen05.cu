@@ -406,11 +406,39 @@ __device__ __forceinline__ int seg_of_column(int n, int Q, uint32_t nb_addr, int
 // raw accumulator words of one TMEM load.  A slab that lies in one N-segment (q_lo == q_hi; always so in the
 // production variant) takes one factor; otherwise the factor is looked up per column.
 // INIT: y starts from the bias slice at shared address bias_slab (32 floats) instead of its old value.
+// Per-token x per-channel factors (4-bit weights with per-channel scales, activations with per-token scales):
+// the factor of column n is row_factor * col_scale[n * col_stride], row_factor being the token's scale for this
+// accumulator.  col_scale == nullptr: factors come from the table.  Only the checking variant carries this.
+struct TokenScale {
+    float row_factor;
+    const float *col_scale;      // already offset to the accumulator's K-segment
+    int col_stride, N;
+};
+
 template <int KIND, bool GENERIC, bool INIT = false>
 __device__ __forceinline__ void scale_add_unit(uint64_t (&y2)[16], const uint32_t (&r)[32], int a, int Q, int q_lo,
                                                int q_hi, int nf, uint32_t tab_addr, uint32_t nb_addr,
-                                               uint32_t bias_slab = 0)
+                                               uint32_t bias_slab = 0, const TokenScale *ts = nullptr)
 {
+    if (GENERIC && ts && ts->col_scale) {
+        if (INIT) {
+#pragma unroll
+            for (int j4 = 0; j4 < 8; j4++) ld_shared_2x64(bias_slab + uint32_t(16 * j4), y2[2 * j4], y2[2 * j4 + 1]);
+        }
+#pragma unroll
+        for (int j = 0; j < 16; j++) {
+            float cc[2];
+#pragma unroll
+            for (int t = 0; t < 2; t++) {
+                const int n = nf + 2 * j + t;
+                cc[t] = n < ts->N ? __fmul_rn(ts->row_factor, __ldg(ts->col_scale + size_t(n) * ts->col_stride)) : 0.0f;
+            }
+            const uint64_t v2 = KIND == 0 ? pack_f32x2(__int2float_rn(int(r[2 * j])), __int2float_rn(int(r[2 * j + 1])))
+                                          : pack_b32x2(r[2 * j], r[2 * j + 1]);
+            y2[j] = fma_f32x2(pack_f32x2(cc[0], cc[1]), v2, y2[j]);
+        }
+        return;
+    }
     if (!GENERIC || q_lo == q_hi) {
         const float c = ld_shared_f32(tab_addr + uint32_t(a * Q + q_lo) * 4u);
         const uint64_t c2 = pack_f32x2(c, c);
@@ -805,11 +833,24 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
         float bias_next1 = WIDE ? fetch_bias(unit, 1) : 0.0f;   // second half of a wide tile
         // dequantization factors c[a][q] = s_act[p][pol] * s_w[p][q], a = p * NPOL + pol (one fp32 multiply);
         // built here, off the producer's and the MMA issuer's path, and published by the first tile's barrier
-        for (int i = et; i < nacc * Q; i += kEpiThreads) {
+        const bool per_token = GENERIC && prm.col_scale != nullptr;      // factors per (token, channel), no table
+        for (int i = et; i < nacc * Q && !per_token; i += kEpiThreads) {
             const int a = i / Q, q = i - a * Q, p = a / NPOL;
             const float s_act = (NPOL == 2 && (a & 1)) ? prm.s_neg[p] : prm.s_pos[p];
             sh_tab[i] = s_act * prm.s_w[p * Q + q];
         }
+        // (per-token mode) this thread's token scale for accumulator a = p * NPOL + pol, and the channel scales of p
+        auto token_scale = [&](int a, int row_) -> TokenScale {
+            TokenScale t{0.0f, nullptr, 0, prm.N};
+            if (per_token) {
+                const int p = a / NPOL;
+                const float *rs = (NPOL == 2 && (a & 1)) ? prm.row_neg : prm.row_pos;
+                t.row_factor = row_ < prm.M ? __ldg(rs + size_t(row_) * P + p) : 0.0f;
+                t.col_scale = prm.col_scale + p;
+                t.col_stride = P;
+            }
+            return t;
+        };
         for (int i = et; i <= Q; i += kEpiThreads) sh_nb[i] = prm.sb.nb[i];
 
         YOut yo{&tm_y, smem_u32(sh_stage) + uint32_t(ew) * kStageBytesPerWarp, lane, 0};
@@ -875,7 +916,8 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                                     buf[(u - 1) % NB]);
                         const int a = p * NPOL + pol;
                         const int nf = n0 + (slab0 + sl) * 32;
-                        scale_add_unit<KIND, GENERIC>(y2[sl], buf[u % NB], a, Q, q_lo[sl], q_hi[sl], nf, tab_addr, nb_addr);
+                        const TokenScale tk = token_scale(a, row);
+                        scale_add_unit<KIND, GENERIC>(y2[sl], buf[u % NB], a, Q, q_lo[sl], q_hi[sl], nf, tab_addr, nb_addr, 0, &tk);
                         if (GENERIC && prm.acc_dump && row < prm.M)
                             dump_unit(prm.acc_dump, buf[u % NB], a, row, nf, prm.M, prm.N);
                     }
@@ -985,10 +1027,12 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                         if (pol == 0) {
                             q_lo = seg_of_column(nf, Q, nb_addr, lane);
                             q_hi = GENERIC ? seg_of_column(min(nf + 31, prm.N - 1), Q, nb_addr, lane) : q_lo;
+                            const TokenScale tk = token_scale(pol, row);
                             scale_add_unit<KIND, GENERIC, true>(y2, buf[u % NB], pol, Q, q_lo, q_hi, nf, tab_addr, nb_addr,
-                                                                bias_addr + uint32_t(c0) * 4u);
+                                                                bias_addr + uint32_t(c0) * 4u, &tk);
                         } else {
-                            scale_add_unit<KIND, GENERIC>(y2, buf[u % NB], pol, Q, q_lo, q_hi, nf, tab_addr, nb_addr);
+                            const TokenScale tk = token_scale(pol, row);
+                            scale_add_unit<KIND, GENERIC>(y2, buf[u % NB], pol, Q, q_lo, q_hi, nf, tab_addr, nb_addr, 0, &tk);
                         }
                         if (GENERIC && prm.acc_dump && row < prm.M)
                             dump_unit(prm.acc_dump, buf[u % NB], pol, row, nf, prm.M, prm.N);
@@ -1020,7 +1064,8 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                         for (int j4 = 0; j4 < 8; j4++)
                             ld_shared_2x64(bias_addr + uint32_t(c0 + 4 * j4) * 4u, y2[2 * j4], y2[2 * j4 + 1]);
                     }
-                    scale_add_unit<KIND, GENERIC>(y2, r, c_a, Q, q_lo, q_hi, nf, tab_addr, nb_addr);
+                    const TokenScale tk = token_scale(c_a, row);
+                    scale_add_unit<KIND, GENERIC>(y2, r, c_a, Q, q_lo, q_hi, nf, tab_addr, nb_addr, 0, &tk);
                     if (GENERIC && prm.acc_dump && row < prm.M) dump_unit(prm.acc_dump, r, c_a, row, nf, prm.M, prm.N);
                     if (++c_a < nacc) return;
                     c_a = 0;
@@ -1207,7 +1252,7 @@ template <int KIND, int NPOL, int CG>
 sq_status prepare_tile(const GemmArgs &g, GemmLaunch &L, int tile_n, bool seq, int device, int sm_count)
 {
     KernelParams &prm = L.prm;
-    bool dbg = prm.y_is_f32 || prm.acc_dump != nullptr;
+    bool dbg = prm.y_is_f32 || prm.acc_dump != nullptr || prm.col_scale != nullptr;
     // the production variant writes Y with TMA stores: 16-byte aligned base and row pitch
     dbg = dbg || reinterpret_cast<uintptr_t>(g.Y) % 16 != 0 || (size_t(g.ldy) * 2) % 16 != 0;
     for (int q = 1; q < prm.sb.Q; q++) dbg = dbg || (prm.sb.nb[q] % 32 != 0);
@@ -1274,6 +1319,7 @@ sq_status prepare_gemm(const GemmArgs &g, GemmLaunch *out)
     prm.nacc = g.sb.P * npol;
     prm.sb = g.sb;
     prm.s_pos = g.s_pos; prm.s_neg = g.s_neg; prm.s_w = g.s_w; prm.bias = g.bias;
+    prm.row_pos = g.row_pos; prm.row_neg = g.row_neg; prm.col_scale = g.col_scale;
     prm.Y = g.Y; prm.ldy = g.ldy;
     prm.y_is_f32 = g.y_dtype == SQ_F32;
     prm.y_wide = (reinterpret_cast<uintptr_t>(g.Y) % 32 == 0) && ((size_t(g.ldy) * (prm.y_is_f32 ? 4 : 2)) % 32 == 0);

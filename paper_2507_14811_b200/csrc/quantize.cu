@@ -395,6 +395,167 @@ quantize_kernel(const __grid_constant__ QuantParams prm)
     }
 }
 
+// ----------------------------------------------------------------------------- per-row scales (W4A8)
+// App. B "Extra Hyperparameter Settings": 4-bit weights are quantized per channel, activations dynamically per
+// token.  One CTA per row: the row is read once into registers (up to kRowChunks 16-element chunks per thread),
+// its extrema per K-segment are reduced in shared memory, the scales (one IEEE division each) are written out,
+// and the codes are made from the registers with the same quantizer as everywhere else.
+constexpr int kRowChunks = 4;                       // K <= 256 threads x 4 chunks x 16 = 16384
+
+__device__ __forceinline__ uint32_t ord_enc(float f)     // monotone map float -> uint32
+{
+    const uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float ord_dec(uint32_t u)
+{
+    return __uint_as_float((u & 0x80000000u) ? (u & 0x7FFFFFFFu) : ~u);
+}
+
+template <typename Tin, bool DUAL>
+__global__ void __launch_bounds__(kThreads)
+quantize_per_row_kernel(const Tin *__restrict__ X, int K, int64_t ld, const SegBounds sb, float q_max, float q_min_abs,
+                        float *__restrict__ s_pos, float *__restrict__ s_neg, uint8_t *__restrict__ c_pos,
+                        uint8_t *__restrict__ c_neg, int64_t ldc)
+{
+    __shared__ uint32_t sh_max[SQ_MAX_P], sh_min[SQ_MAX_P];
+    __shared__ float sh_sp[SQ_MAX_P], sh_sn[SQ_MAX_P];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int64_t row = blockIdx.x;
+    const int P = sb.P;
+    for (int i = threadIdx.x; i < P; i += blockDim.x) { sh_max[i] = 0u; sh_min[i] = 0xFFFFFFFFu; }
+    __syncthreads();
+    const Tin *src = X + row * ld;
+    Raw16<Tin> raw[kRowChunks];
+    int seg[kRowChunks];                            // K-segment of a whole chunk, -1: straddles a bound or the row end
+#pragma unroll
+    for (int c = 0; c < kRowChunks; c++) {
+        const int k0 = (int(threadIdx.x) + c * int(blockDim.x)) * kVec;
+        seg[c] = -2;                                // beyond the row
+        if (k0 >= K) continue;
+        int p = 0;
+        while (p + 1 < P && k0 >= sb.kb[p + 1]) p++;
+        if (k0 + kVec <= sb.kb[p + 1]) {
+            seg[c] = p;
+            load16(src + k0, raw[c]);
+            float mx = -INFINITY, mn = INFINITY;
+#pragma unroll
+            for (int g4 = 0; g4 < 4; g4++) {
+                float x[4];
+                get4(raw[c], g4, x);
+#pragma unroll
+                for (int i = 0; i < 4; i++) { mx = fmaxf(mx, x[i]); mn = fminf(mn, x[i]); }
+            }
+            atomicMax(&sh_max[p], ord_enc(mx));
+            atomicMin(&sh_min[p], ord_enc(mn));
+        } else {
+            seg[c] = -1;
+            const int n = min(kVec, K - k0);
+            for (int i = 0; i < n; i++) {
+                while (p + 1 < P && k0 + i >= sb.kb[p + 1]) p++;
+                const float x = load1(src + k0 + i);
+                atomicMax(&sh_max[p], ord_enc(x));
+                atomicMin(&sh_min[p], ord_enc(x));
+            }
+        }
+    }
+    __syncthreads();
+    for (int p = threadIdx.x; p < P; p += blockDim.x) {
+        const float mx = ord_dec(sh_max[p]), mn = ord_dec(sh_min[p]);
+        float sp, sn = 1.0f;
+        if (DUAL) {
+            const float hi = fmaxf(mx, 0.0f), lo = fmaxf(-mn, 0.0f);
+            sp = hi > 0.0f ? __fdiv_rn(hi, q_max) : 1.0f;
+            sn = lo > 0.0f ? __fdiv_rn(lo, q_min_abs) : 1.0f;
+            s_neg[row * P + p] = sn;
+        } else {
+            const float a = fmaxf(fabsf(mx), fabsf(mn));
+            sp = a > 0.0f ? __fdiv_rn(a, q_max) : 1.0f;
+        }
+        s_pos[row * P + p] = sp;
+        sh_sp[p] = sp;
+        sh_sn[p] = sn;
+    }
+    __syncthreads();
+    const int hi = int(q_max), lo = DUAL ? -int(q_min_abs) : -int(q_max);
+    constexpr int MODE = DUAL ? kDual : kSingle;
+#pragma unroll
+    for (int c = 0; c < kRowChunks; c++) {
+        const int k0 = (int(threadIdx.x) + c * int(blockDim.x)) * kVec;
+        if (seg[c] == -2) continue;
+        uint8_t *dp = c_pos + row * ldc + k0;
+        uint8_t *dn = DUAL ? c_neg + row * ldc + k0 : nullptr;
+        bool done = false;
+        if (seg[c] >= 0) {
+            const SegConst cp = seg_const(sh_sp[seg[c]]);
+            const SegConst cn = seg_const(DUAL ? sh_sn[seg[c]] : 1.0f);
+            if (cp.fast && cn.fast && !(DUAL && lo != -128)) {
+                uint32_t wp[4], wn[4];
+#pragma unroll
+                for (int g4 = 0; g4 < 4; g4++) {
+                    float x[4];
+                    get4(raw[c], g4, x);
+                    quant4<SQ_CODE_INT8, MODE>(x, cp, cn, float(hi), 0, wp[g4], wn[g4]);
+                }
+                *reinterpret_cast<uint4 *>(dp) = make_uint4(wp[0], wp[1], wp[2], wp[3]);
+                if (DUAL) *reinterpret_cast<uint4 *>(dn) = make_uint4(wn[0], wn[1], wn[2], wn[3]);
+                done = true;
+            }
+        }
+        if (!done) {
+            const int n = min(kVec, K - k0);
+            int p = 0;
+            for (int i = 0; i < n; i++) {
+                while (p + 1 < P && k0 + i >= sb.kb[p + 1]) p++;
+                uint32_t a, b;
+                quant1<SQ_CODE_INT8, MODE>(load1(src + k0 + i), sh_sp[p], sh_sn[p], 0, lo, hi, a, b);
+                dp[i] = uint8_t(a);
+                if (DUAL) dn[i] = uint8_t(b);
+            }
+        }
+    }
+}
+
+// int8 codes in [-8, 7] <-> two 4-bit codes per byte (code 2j in the low nibble); 16 codes per thread
+__global__ void __launch_bounds__(kThreads)
+pack_w4_kernel(uint8_t *__restrict__ w8, int64_t ld8, int64_t N, int K, uint8_t *__restrict__ w4, int64_t ld4, int unpack)
+{
+    const int V = K / kVec;
+    const int64_t idx = int64_t(blockIdx.x) * kThreads + threadIdx.x;
+    if (idx >= N * V) return;
+    const int64_t n = idx / V;
+    const int k0 = int(idx - n * V) * kVec;
+    if (!unpack) {
+        const uint4 v = *reinterpret_cast<const uint4 *>(w8 + n * ld8 + k0);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint32_t o[2];
+#pragma unroll
+        for (int h = 0; h < 2; h++) {
+            const uint32_t a = w[2 * h], b = w[2 * h + 1];          // 4 codes each
+            const uint32_t pa = (a & 0xF) | ((a >> 4) & 0xF0) | ((a >> 8) & 0xF00) | ((a >> 12) & 0xF000);
+            const uint32_t pb = (b & 0xF) | ((b >> 4) & 0xF0) | ((b >> 8) & 0xF00) | ((b >> 12) & 0xF000);
+            o[h] = pa | (pb << 16);
+        }
+        *reinterpret_cast<uint2 *>(w4 + n * ld4 + k0 / 2) = make_uint2(o[0], o[1]);
+    } else {
+        const uint2 v = *reinterpret_cast<const uint2 *>(w4 + n * ld4 + k0 / 2);
+        const uint32_t in[2] = {v.x, v.y};
+        uint32_t o[4];
+#pragma unroll
+        for (int h = 0; h < 2; h++) {
+#pragma unroll
+            for (int t = 0; t < 2; t++) {
+                const uint32_t hw = (in[h] >> (16 * t)) & 0xFFFFu;   // 4 nibbles
+                uint32_t bytes = (hw & 0xF) | ((hw & 0xF0) << 4) | ((hw & 0xF00) << 8) | ((hw & 0xF000) << 12);
+                bytes |= (bytes & 0x08080808u) * 0x1Eu;              // sign-extend each nibble: bit 3 copied into bits 4..7
+                o[2 * h + t] = bytes;
+            }
+        }
+        *reinterpret_cast<uint4 *>(w8 + n * ld8 + k0) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
 template <typename Tin, int CODE, int MODE>
 sq_status prepare_t(QuantLaunch &L)
 {
@@ -479,6 +640,55 @@ sq_status launch_quantize(const void *X, sq_dtype dt, int64_t M, int64_t K, int6
     const sq_status s = prepare_quantize(X, dt, M, K, ld, sb, s_pos, s_neg, zero_point, row_segments, code, q_max,
                                          q_min_abs, act, mult, c_pos, c_neg, ldc, &L);
     return s == SQ_OK ? run_quantize(L, st) : s;
+}
+
+sq_status launch_quantize_per_row(const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld, const SegBounds &sb,
+                                  int dual, float q_max, float q_min_abs, float *s_pos, float *s_neg,
+                                  void *c_pos, void *c_neg, int64_t ldc, cudaStream_t st)
+{
+    const int64_t V = (K + kVec - 1) / kVec;
+    if (V > int64_t(kThreads) * kRowChunks) return SQ_ERR_UNSUPPORTED;      // the row is held in registers
+    if (M > 0x7FFFFFFF) return SQ_ERR_SHAPE;
+    int threads = int((V + kRowChunks - 1) / kRowChunks);
+    threads = (threads + 31) / 32 * 32;
+    if (threads < 32) threads = 32;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(unsigned(M));
+    cfg.blockDim = dim3(unsigned(threads));
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    uint8_t *cp = static_cast<uint8_t *>(c_pos), *cn = static_cast<uint8_t *>(c_neg);
+    const int Ki = int(K);
+    cudaError_t e;
+    if (dt == SQ_F32) {
+        const float *x = static_cast<const float *>(X);
+        e = dual ? cudaLaunchKernelEx(&cfg, quantize_per_row_kernel<float, true>, x, Ki, ld, sb, q_max, q_min_abs, s_pos, s_neg, cp, cn, ldc)
+                 : cudaLaunchKernelEx(&cfg, quantize_per_row_kernel<float, false>, x, Ki, ld, sb, q_max, q_min_abs, s_pos, s_neg, cp, cn, ldc);
+    } else {
+        const __nv_bfloat16 *x = static_cast<const __nv_bfloat16 *>(X);
+        e = dual ? cudaLaunchKernelEx(&cfg, quantize_per_row_kernel<__nv_bfloat16, true>, x, Ki, ld, sb, q_max, q_min_abs, s_pos, s_neg, cp, cn, ldc)
+                 : cudaLaunchKernelEx(&cfg, quantize_per_row_kernel<__nv_bfloat16, false>, x, Ki, ld, sb, q_max, q_min_abs, s_pos, s_neg, cp, cn, ldc);
+    }
+    count_launch();
+    if (e != cudaSuccess) { note_cuda_error(e); return SQ_ERR_CUDA; }
+    return SQ_OK;
+}
+
+sq_status launch_pack_w4(const void *Wq8, int64_t ld8, int64_t N, int64_t K, void *Wq4, int64_t ld4, int unpack,
+                         cudaStream_t st)
+{
+    const int64_t blocks = (N * (K / kVec) + kThreads - 1) / kThreads;
+    if (blocks > 0x7FFFFFFF) return SQ_ERR_SHAPE;
+    pack_w4_kernel<<<unsigned(blocks), kThreads, 0, st>>>(static_cast<uint8_t *>(const_cast<void *>(Wq8)), ld8, N, int(K),
+                                                          static_cast<uint8_t *>(Wq4), ld4, unpack);
+    count_launch();
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { note_cuda_error(e); return SQ_ERR_CUDA; }
+    return SQ_OK;
 }
 
 }  // namespace sq

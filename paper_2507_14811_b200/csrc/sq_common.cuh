@@ -90,6 +90,14 @@ sq_status prepare_quantize(const void *X, sq_dtype dt, int64_t M, int64_t K, int
                            void *c_pos, void *c_neg, int64_t ldc, QuantLaunch *out);    // launches nothing
 sq_status run_quantize(const QuantLaunch &l, cudaStream_t st);                          // one launch, no queries
 
+// One scale per (row, K-segment) from the row's own extrema, written to s_pos / s_neg [rows][P], and the int8 codes
+// quantized with them (per-token activations, q_max 127; per-channel 4-bit weights, q_max 7).
+sq_status launch_quantize_per_row(const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld, const SegBounds &sb,
+                                  int dual, float q_max, float q_min_abs, float *s_pos, float *s_neg,
+                                  void *c_pos, void *c_neg, int64_t ldc, cudaStream_t st);
+sq_status launch_pack_w4(const void *Wq8, int64_t ld8, int64_t N, int64_t K, void *Wq4, int64_t ld4, int unpack,
+                         cudaStream_t st);
+
 sq_status launch_calib_zero_point(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld, const SegBounds &sb,
                                   float *s_x, int32_t *z_x, uint32_t *partials, cudaStream_t st);
 
@@ -106,6 +114,7 @@ struct GemmArgs {
     SegBounds sb;
     sq_code code;
     const float *s_pos, *s_neg, *s_w, *bias;
+    const float *row_pos, *row_neg, *col_scale;   // W4A8: per-token and per-channel scales (then s_pos / s_neg / s_w unused)
     void *Y;
     sq_dtype y_dtype;
     int64_t ldy;
@@ -121,6 +130,7 @@ struct KernelParams {
     int num_m_tiles, num_n_tiles;
     SegBounds sb;
     const float *s_pos, *s_neg, *s_w, *bias;
+    const float *row_pos, *row_neg, *col_scale;   // per-token [M][P] and per-channel [N][P] scales instead of the tables
     void *Y;
     long long ldy;     // elements
     int y_is_f32;

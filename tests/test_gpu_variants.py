@@ -255,3 +255,97 @@ def test_fused_activation_equals_the_unfused_pair_when_the_stored_values_agree(a
     u_pos, u_neg = B.segquant_quantize_act(A.to(DEV), seg, sp, sn, "int8")
     agree = ((f_pos == u_pos) & (f_neg == u_neg)).float().mean().item()
     assert agree > 0.999
+
+
+# ------------------------------------------------------------------ W4A8: per-channel 4-bit weights, per-token scales
+
+def run_w4a8_parity(spec):
+    data = WL.make_layer(spec)
+    kb, P = spec.kb, spec.P
+    Xn, Wn, bn = to_f32_np(data.X), to_f32_np(data.W), to_f32_np(data.bias)
+    s_w, _, Wq, _ = O.quantize_per_row(Wn, kb, False, q_max=7.0, q_min_abs=7.0)
+    res = O.layer_forward_w4a8(Xn, Wq, s_w, kb, spec.dual, bn)
+
+    seg = B.SegTable(kb, [0, spec.N])
+    ws = B.new_workspace(DEV)
+    # offline: per-channel scales, 4-bit codes, packed
+    g_sw, _, g_w8, _ = B.segquant_quantize_per_row(data.W.to(DEV), seg, False, bits=4)
+    assert np.array_equal(g_sw.cpu().numpy(), s_w) and np.array_equal(g_w8.cpu().numpy().view(np.int8), Wq)
+    packed = B.segquant_pack_w4(g_w8)
+    assert np.array_equal(packed.cpu().numpy(), O.pack_w4(Wq))
+    # per call: unpack, per-token quantize, GEMM with per-token x per-channel factors
+    w8 = B.segquant_unpack_w4(packed)
+    assert np.array_equal(w8.cpu().numpy().view(np.int8), Wq)
+    g_sp, g_sn, c_pos, c_neg = B.segquant_quantize_per_row(data.X.to(DEV), seg, spec.dual, bits=8)
+    assert np.array_equal(g_sp.cpu().numpy(), res.s_pos)
+    assert np.array_equal(c_pos.cpu().numpy().view(np.int8), res.c_pos)
+    if spec.dual:
+        assert np.array_equal(g_sn.cpu().numpy(), res.s_neg)
+        assert np.array_equal(c_neg.cpu().numpy().view(np.int8), res.c_neg)
+    bias = data.bias.to(DEV)
+    Y32, dump = B.segquant_w4a8_gemm(c_pos, c_neg, w8, seg, g_sp, g_sn, g_sw, bias, ws, y_dtype=torch.float32, dump_acc=True)
+    Ybf = B.segquant_w4a8_gemm(c_pos, c_neg, w8, seg, g_sp, g_sn, g_sw, bias, ws)
+    B.check_device_status(ws)
+    torch.cuda.synchronize()
+    npol = 2 if spec.dual else 1
+    acc = dump.cpu().numpy().reshape(P, npol, spec.M, spec.N)
+    assert np.array_equal(acc[:, 0], res.acc_pos)
+    if spec.dual:
+        assert np.array_equal(acc[:, 1], res.acc_neg)
+    from parity_util import check_fp32_output
+    check_fp32_output(Y32, res.y64, res.y_abs, P * npol)
+    check_bf16_output(Ybf, res.y64, res.y_abs, P * npol)
+
+
+@pytest.mark.parametrize("dual", [True, False])
+@pytest.mark.parametrize("case", [
+    ("w4_small", 200, 256, 136, [0, 256]),
+    ("w4_k_segments", 300, 512, 264, [0, 128, 224, 512]),
+    ("w4_ragged", 129, 208, 200, [0, 96, 208]),
+    ("w4_long_row", 70, 16384, 64, [0, 4096, 16384]),
+    ("w4_heads", 260, 1536, 320, list(range(0, 1537, 64))),
+])
+def test_w4a8_layer_parity(case, dual):
+    name, M, K, N, kb = case
+    run_w4a8_parity(custom_spec(name, M, K, N, kb, [0, N], dual, "int8", seed=81,
+                                x_seg_std=[1.0 + (i % 7) for i in range(len(kb) - 1)]))
+
+
+def test_w4a8_tokens_of_very_different_magnitude_and_degenerate_rows():
+    """Per-token scales: tokens spread over five orders of magnitude, an all-zero token, a token without
+    negative values; fp32 input."""
+    spec = custom_spec("w4_tokens", 160, 384, 72, [0, 128, 384], [0, 72], True, "int8", x_dtype="f32", seed=82)
+    data = WL.make_layer(spec)
+    mult = (10.0 ** torch.linspace(-3, 2, spec.M))[:, None]
+    data.X = (data.X * mult).contiguous()
+    data.X[5] = 0.0
+    data.X[6] = data.X[6].abs()
+    WL_make = WL.make_layer
+    try:
+        WL.make_layer = lambda s, M=None: data
+        run_w4a8_parity(spec)
+    finally:
+        WL.make_layer = WL_make
+
+
+def test_w4a8_full_size_layer_every_row():
+    sp = WL.WORKLOADS["dit_xl2"][1]
+    run_w4a8_parity(WL.LayerSpec(name="dit_fc2_w4a8", M=sp.M, K=sp.K, N=sp.N, kb=sp.kb, nb=[0, sp.N], dual=True,
+                                 code="int8", x_dtype=sp.x_dtype, x_kind=sp.x_kind, w_kind=sp.w_kind, seed=sp.seed,
+                                 cal_rows=sp.cal_rows, x_seg_std=list(sp.x_seg_std)))
+
+
+def test_w4a8_calls_reject_bad_arguments_before_launch():
+    X = torch.zeros((16, 16400), dtype=torch.bfloat16, device=DEV)
+    n0 = B.segquant_launch_count()
+    with pytest.raises(B.SegquantError) as e:
+        B.segquant_quantize_per_row(X, B.SegTable([0, 16400], [0, 8]), False)       # longer than a block holds
+    assert e.value.status == 5
+    seg2 = B.SegTable([0, 128], [0, 32, 64])
+    z = torch.zeros((16, 128), dtype=torch.uint8, device=DEV)
+    one = torch.ones(64, device=DEV)
+    with pytest.raises(B.SegquantError) as e:
+        B.segquant_w4a8_gemm(z, None, torch.zeros((64, 128), dtype=torch.uint8, device=DEV), seg2, one, None, one, None,
+                             B.new_workspace(DEV))
+    assert e.value.status == 3                                                      # output segments: not with per-channel scales
+    assert B.segquant_launch_count() == n0
