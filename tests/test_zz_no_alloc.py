@@ -90,11 +90,13 @@ def test_static_calibration_allocates_nothing_and_takes_exactly_its_limit():
     out = torch.empty(P * Q, dtype=torch.float32, device=DEV)
     B.segquant_calib_scales_static(W, seg, "int8", True, False, s_pos=out)            # warm-up call
     torch.cuda.synchronize()
-    before = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), torch.cuda.mem_get_info()[0])
+    # cumulative allocation and segment counts of torch's allocator, its reserved bytes, the device's free bytes
+    snap = lambda: (torch.cuda.memory_stats()["allocation.all.allocated"], torch.cuda.memory_stats()["segment.all.allocated"],
+                    torch.cuda.memory_reserved(), torch.cuda.mem_get_info()[0])
+    before = snap()
     B.segquant_calib_scales_static(W, seg, "int8", True, False, s_pos=out)
     torch.cuda.synchronize()
-    after = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), torch.cuda.mem_get_info()[0])
-    assert after == before
+    assert snap() == before
     ref, _ = B.segquant_calib_scales(W, seg, "int8", True, False, B.new_workspace(DEV))
     torch.cuda.synchronize()
     assert np.array_equal(out.cpu().numpy(), ref.cpu().numpy()) and len(np.unique(out.cpu().numpy())) > 100
