@@ -90,15 +90,18 @@ __device__ __forceinline__ void quant1(float x, float sp, float sn, int zp, int 
 
 // The act-to-linear segment in front of the quantizer (Sec. 4.3.2; App. B: SiLU and GELU feed DualScale layers),
 // evaluated in fp32 and rounded once to the dtype the unfused graph would have stored the activation in.
-// SiLU(h) = h sigma(h) with z = exp(-|h|): sigma = 1 / (1 + z) for h >= 0, z / (1 + z) below (no overflow);
-// relative error <= 2^-20 (exp 2 ulp, one add, one multiply, one IEEE division).
+// SiLU(h) = h sigma(h) with z = exp(-|h|): sigma = 1 / (1 + z) for h >= 0, z / (1 + z) below (no overflow).  The
+// exponential is the hardware base-2 approximation of h log2(e) (the rounding of that product costs |h| 2^-24
+// relative, the approximation itself about one unit in the last place) and the division the hardware's fast one
+// (2 units in the last place for a divisor in [1, 2]): relative error <= (|h| + 8) 2^-23, a fraction of a bf16
+// half-step (2^-9) for every |h| below the underflow of the result.
 // GELU(h) = (h / 2) erfc(-h / sqrt 2): relative error <= (2 h^2 + 32) 2^-24 (erfc 4 ulp; the rounding of its
 // argument is amplified by about 2 t^2 in the negative tail).
 __device__ __forceinline__ float silu_f32(float h)
 {
-    const float z = expf(-fabsf(h));
+    const float z = __expf(-fabsf(h));
     const float num = h >= 0.0f ? h : __fmul_rn(h, z);
-    return __fdiv_rn(num, __fadd_rn(1.0f, z));
+    return __fdividef(num, __fadd_rn(1.0f, z));
 }
 __device__ __forceinline__ float gelu_f32(float h)
 {
