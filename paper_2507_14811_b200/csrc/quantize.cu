@@ -34,6 +34,13 @@ __device__ __forceinline__ void load16(const __nv_bfloat16 *p, Raw16<__nv_bfloat
 #pragma unroll
     for (int i = 0; i < 2; i++) r.v[i] = __ldg(q + i);
 }
+// piece v (16 bytes) of a row chunk
+__device__ __forceinline__ void set_piece(Raw16<float> &r, int v, uint4 w)
+{
+    r.v[v] = make_float4(__uint_as_float(w.x), __uint_as_float(w.y), __uint_as_float(w.z), __uint_as_float(w.w));
+}
+__device__ __forceinline__ void set_piece(Raw16<__nv_bfloat16> &r, int v, uint4 w) { r.v[v] = w; }
+
 // elements 4 g .. 4 g + 3 as fp32
 __device__ __forceinline__ void get4(const Raw16<float> &r, int g, float (&x)[4])
 {
@@ -304,7 +311,9 @@ __device__ __forceinline__ void quant4(const float (&x)[4], const SegConst &cp, 
 // flight while the current row is converted.
 // PRE compiles in the act-to-linear prologue: activation function and per-channel multiplier in front of the
 // quantizer, so that the activation's output never goes through HBM.
-template <typename Tin, int CODE, int MODE, bool PRE>
+// RING: depth of the shared-memory ring the rows travel through (see below); 4 when a thread has many rows to
+// walk (large inputs: more bytes in flight), 2 otherwise (less shared memory, more L1 for the copies).
+template <typename Tin, int CODE, int MODE, bool PRE, int RING>
 __global__ void __launch_bounds__(kThreads, PRE ? 3 : kBlocksPerSm)
 quantize_kernel(const __grid_constant__ QuantParams prm)
 {
@@ -339,13 +348,43 @@ quantize_kernel(const __grid_constant__ QuantParams prm)
         for (int i = 0; i < kVec; i++) mreg[i] = (prm.mult && k0 + i < K) ? __ldg(prm.mult + k0 + i) : 1.0f;
     }
 
-    Raw16<Tin> cur, nxt;
-    if (whole) load16(src, cur);
+    // The rows of this chunk travel through a thread-private ring in shared memory: asynchronous 16-byte copies
+    // (global -> shared without passing through registers) of the next kDepth - 1 rows are in flight while the
+    // current row is converted, so the bytes in flight per SM do not cost registers.  Every thread reads only what
+    // it copied itself, so a wait on its own copy groups is all the synchronisation there is.
+    constexpr int NV = int(sizeof(Tin)) * kVec / 16;                        // 16-byte pieces per row chunk
+    constexpr int kDepth = (sizeof(Tin) == 2 || RING == 2) ? RING : RING / 2;  // ring slots (32 KiB per block at most)
+    __shared__ uint4 ring[kDepth * NV * kThreads];
+    const uint32_t ring0 = uint32_t(__cvta_generic_to_shared(ring)) + threadIdx.x * 16u;
+    auto slot_addr = [&](int slot, int v) { return ring0 + uint32_t((slot * NV + v) * kThreads) * 16u; };
+    auto copy_row = [&](const Tin *row_src, int slot, bool valid) {          // one commit group per call, always
+        if (valid) {
+#pragma unroll
+            for (int v = 0; v < NV; v++)
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(slot_addr(slot, v)),
+                             "l"(reinterpret_cast<const char *>(row_src) + 16 * v) : "memory");
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    auto read_row = [&](int slot, Raw16<Tin> &r) {
+#pragma unroll
+        for (int v = 0; v < NV; v++) {
+            uint4 w;
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w)
+                         : "r"(slot_addr(slot, v)) : "memory");
+            set_piece(r, v, w);
+        }
+    };
+    if (whole) {
+#pragma unroll
+        for (int d = 0; d < kDepth - 1; d++) copy_row(src + int64_t(d) * src_step, d, int64_t(r0) + int64_t(d) * R < M);
+    }
     int q = 0;                                               // N-segment (weights only) the constants belong to
     int64_t q_end = 0;                                       // first row beyond it (0: no constants yet)
     SegConst cp, cn;
     int zp = 0;
     bool fast = false;
+    int slot = 0;                                            // ring slot of the current row
     for (int64_t row = r0; row < M; row += R) {
         if (row >= q_end) {                                  // (weights) the row entered another N-segment
             if (row_segments) {
@@ -359,9 +398,17 @@ quantize_kernel(const __grid_constant__ QuantParams prm)
             if (MODE == kZeroPoint) zp = __ldg(prm.zp + p);
             fast = whole && cp.fast && cn.fast && !(DUAL && CODE == SQ_CODE_INT8 && lo != -128);
         }
+        Raw16<Tin> cur;
+        if (whole) {
+            // row + (kDepth - 1) R goes into the slot the previous row has just left; then the oldest group, this
+            // row's, is complete once at most kDepth - 1 newer groups are pending
+            const int ahead = slot == 0 ? kDepth - 1 : slot - 1;
+            copy_row(src + int64_t(kDepth - 1) * src_step, ahead, row + int64_t(kDepth - 1) * R < M);
+            asm volatile("cp.async.wait_group %0;" ::"n"(kDepth - 1) : "memory");
+            if (fast) read_row(slot, cur);
+            slot = slot + 1 == kDepth ? 0 : slot + 1;
+        }
         if (fast) {
-            const bool more = row + R < M;
-            if (more) load16(src + src_step, nxt);           // next row in flight during the conversion
             uint32_t wp[4], wn[4];
 #pragma unroll
             for (int g4 = 0; g4 < 4; g4++) {
@@ -375,7 +422,6 @@ quantize_kernel(const __grid_constant__ QuantParams prm)
             }
             *reinterpret_cast<uint4 *>(dp) = make_uint4(wp[0], wp[1], wp[2], wp[3]);
             if (DUAL) *reinterpret_cast<uint4 *>(dn) = make_uint4(wn[0], wn[1], wn[2], wn[3]);
-            if (more) cur = nxt;
         } else {                                 // segment bound or end of row inside the chunk, or an extreme scale
             const int n = min(kVec, K - k0);
             int pp = p;
@@ -390,12 +436,12 @@ quantize_kernel(const __grid_constant__ QuantParams prm)
                 dp[i] = uint8_t(a);
                 if (DUAL) dn[i] = uint8_t(b);
             }
-            if (whole && row + R < M) load16(src + src_step, cur);
         }
         src += src_step;
         dp += dst_step;
         if (DUAL) dn += dst_step;
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");     // nothing of this thread's is in flight when it leaves
 }
 
 // ----------------------------------------------------------------------------- per-row scales (W4A8)
@@ -580,8 +626,14 @@ sq_status prepare_t(QuantLaunch &L)
     prm.V = int(V);
     prm.R = int(R);
     L.blocks = unsigned(blocks);
-    L.kernel = pre ? reinterpret_cast<const void *>(quantize_kernel<Tin, CODE, MODE, true>)
-                   : reinterpret_cast<const void *>(quantize_kernel<Tin, CODE, MODE, false>);
+    // fp32 input: 64-byte chunks, so half the depth for the same shared memory
+    const bool deep = iters >= 10 && sizeof(Tin) == 2;
+    if (pre)
+        L.kernel = deep ? reinterpret_cast<const void *>(quantize_kernel<Tin, CODE, MODE, true, 4>)
+                        : reinterpret_cast<const void *>(quantize_kernel<Tin, CODE, MODE, true, 2>);
+    else
+        L.kernel = deep ? reinterpret_cast<const void *>(quantize_kernel<Tin, CODE, MODE, false, 4>)
+                        : reinterpret_cast<const void *>(quantize_kernel<Tin, CODE, MODE, false, 2>);
     return SQ_OK;
 }
 
