@@ -501,6 +501,45 @@ def oracle_sample(specs, target_s=12.0, probe_rows=8):
                       f"{reps} pass(es), {t:.1f} s of CPU time"}, rows, t
 
 
+def library_8bit_peaks(dev):
+    """Context for the peak: what the vendor library's own dense int8 and fp8 GEMMs reach on this GPU (8192^3, best
+    of 10 single launches after warm-up, CUDA events; these are 1-2 ms kernels, far above the event timer's
+    resolution).  Denominator context only: nothing of the product path calls these."""
+    out = {}
+    n = 8192
+    ops = 2.0 * n * n * n
+
+    def best(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        return ops / (min(ts) * 1e-3) / 1e12
+
+    try:
+        a = torch.randint(-127, 128, (n, n), dtype=torch.int8, device=dev)
+        b = torch.randint(-127, 128, (n, n), dtype=torch.int8, device=dev).t()
+        out["int8_tops"] = round(best(lambda: torch._int_mm(a, b)), 1)
+    except Exception as e:
+        out["int8_tops"] = None
+        out["int8_error"] = f"{type(e).__name__}: {str(e)[:120]}"
+    try:
+        a8 = torch.randn((n, n), device=dev).to(torch.float8_e4m3fn)
+        b8 = torch.randn((n, n), device=dev).to(torch.float8_e4m3fn).t()
+        one = torch.ones((), device=dev)
+        out["fp8_tops"] = round(best(lambda: torch._scaled_mm(a8, b8, scale_a=one, scale_b=one, out_dtype=torch.bfloat16)), 1)
+    except Exception as e:
+        out["fp8_tops"] = None
+        out["fp8_error"] = f"{type(e).__name__}: {str(e)[:120]}"
+    torch.cuda.empty_cache()
+    return out
+
+
 def eight_bit_peaks(peaks):
     """Dense 8-bit tensor peaks (TOPS): measured bf16 burst and sustained figures x the nominal 8-bit : bf16
     ratio of 2, and the nominal figure itself."""
@@ -710,6 +749,10 @@ def run_ours(args):
     step_tops = exec_ops / (step_ms * 1e-3) / 1e12
     region_s = step_ms * 1e-3 * args.steps * reps
 
+    lib_peaks = None
+    if world == 1 and rank == 0 and not args.only_headline:
+        time.sleep(COOL_DOWN_S)
+        lib_peaks = library_8bit_peaks(dev)
     side = {}
     if world == 1 and rank == 0 and not args.only_headline:
         del layers
@@ -772,6 +815,9 @@ def run_ours(args):
                                         "ratio); burst because each launch is timed alone between its own events with L2 flushed",
                          "frac_definition": "sum over the step's GEMM launches of max(executed ops / peak, algorithmic bytes / "
                                             "measured HBM bandwidth), over their summed CUDA-event time",
+                         "library_gemm_8192": lib_peaks,
+                         "library_gemm_note": "the vendor library's dense int8 / fp8 GEMM at 8192^3 on this GPU (burst), for "
+                                              "context beside the derived peak; not part of the product path",
                          "algorithmic_ops_per_step": exec_ops, "avg_launch_us": round(gemm_ms * 1e3 / len(specs), 2),
                          "note": "8-bit integer / fp8 tensor ops counted as flops"},
             "quantize_roofline": {"bound": "hbm",
