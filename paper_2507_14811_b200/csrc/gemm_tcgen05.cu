@@ -413,7 +413,20 @@ struct TokenScale {
     float row_factor;
     const float *col_scale;      // already offset to the accumulator's K-segment
     int col_stride, N;
+    uint32_t col_smem;           // nonzero: shared address such that col_smem + 4 n holds column n's scale (this tile)
 };
+__device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t ld_shared_64(uint32_t addr)
+{
+    uint64_t v;
+    asm volatile("ld.shared.b64 %0, [%1];" : "=l"(v) : "r"(addr));
+    return v;
+}
 
 template <int KIND, bool GENERIC, bool INIT = false>
 __device__ __forceinline__ void scale_add_unit(uint64_t (&y2)[16], const uint32_t (&r)[32], int a, int Q, int q_lo,
@@ -425,17 +438,24 @@ __device__ __forceinline__ void scale_add_unit(uint64_t (&y2)[16], const uint32_
 #pragma unroll
             for (int j4 = 0; j4 < 8; j4++) ld_shared_2x64(bias_slab + uint32_t(16 * j4), y2[2 * j4], y2[2 * j4 + 1]);
         }
+        const uint64_t rf2 = pack_f32x2(ts->row_factor, ts->row_factor);
 #pragma unroll
         for (int j = 0; j < 16; j++) {
-            float cc[2];
+            uint64_t c2;
+            if (ts->col_smem) {                       // the tile's channel scales are staged in shared memory
+                c2 = mul_f32x2(rf2, ld_shared_64(ts->col_smem + uint32_t(nf + 2 * j) * 4u));
+            } else {
+                float cc[2];
 #pragma unroll
-            for (int t = 0; t < 2; t++) {
-                const int n = nf + 2 * j + t;
-                cc[t] = n < ts->N ? __fmul_rn(ts->row_factor, __ldg(ts->col_scale + size_t(n) * ts->col_stride)) : 0.0f;
+                for (int t = 0; t < 2; t++) {
+                    const int n = nf + 2 * j + t;
+                    cc[t] = n < ts->N ? __fmul_rn(ts->row_factor, __ldg(ts->col_scale + size_t(n) * ts->col_stride)) : 0.0f;
+                }
+                c2 = pack_f32x2(cc[0], cc[1]);
             }
             const uint64_t v2 = KIND == 0 ? pack_f32x2(__int2float_rn(int(r[2 * j])), __int2float_rn(int(r[2 * j + 1])))
                                           : pack_b32x2(r[2 * j], r[2 * j + 1]);
-            y2[j] = fma_f32x2(pack_f32x2(cc[0], cc[1]), v2, y2[j]);
+            y2[j] = fma_f32x2(c2, v2, y2[j]);
         }
         return;
     }
@@ -623,8 +643,10 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     float *sh_bias = reinterpret_cast<float *>(sh_stage + (GENERIC ? 0 : kStageBytes));     // [TILE_N], per tile
     float *sh_tab = sh_bias + kTileCols;                                                    // [nacc][Q], per launch
     int *sh_nb = reinterpret_cast<int *>(sh_tab + prm.nacc * prm.sb.Q);                     // [Q + 1]
-    SharedHeader *hdr = reinterpret_cast<SharedHeader *>(reinterpret_cast<uint8_t *>(sh_bias) +
-                                                         epi_table_bytes(prm.nacc, prm.sb.Q, kTileCols));
+    // (per-token mode, few K-segments) the tile's channel scales [P][kTileCols], refreshed per tile
+    float *sh_col = reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(sh_bias) +
+                                              epi_table_bytes(prm.nacc, prm.sb.Q, kTileCols));
+    SharedHeader *hdr = reinterpret_cast<SharedHeader *>(reinterpret_cast<uint8_t *>(sh_col) + prm.col_tab_bytes);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -840,14 +862,18 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
             sh_tab[i] = s_act * prm.s_w[p * Q + q];
         }
         // (per-token mode) this thread's token scale for accumulator a = p * NPOL + pol, and the channel scales of p
+        const bool col_staged = per_token && prm.col_tab_bytes != 0;
+        const uint32_t col_addr = smem_u32(sh_col);
+        int tile_n0 = 0;                                                 // first column of the current tile
         auto token_scale = [&](int a, int row_) -> TokenScale {
-            TokenScale t{0.0f, nullptr, 0, prm.N};
+            TokenScale t{0.0f, nullptr, 0, prm.N, 0u};
             if (per_token) {
                 const int p = a / NPOL;
                 const float *rs = (NPOL == 2 && (a & 1)) ? prm.row_neg : prm.row_pos;
                 t.row_factor = row_ < prm.M ? __ldg(rs + size_t(row_) * P + p) : 0.0f;
                 t.col_scale = prm.col_scale + p;
                 t.col_stride = P;
+                if (col_staged) t.col_smem = col_addr + uint32_t(p * kTileCols - tile_n0) * 4u;
             }
             return t;
         };
@@ -864,6 +890,13 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
 
             asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // previous tile's readers are done
             if (et < TILE_N) sh_bias[et] = bias_next;
+            if (GENERIC && col_staged) {                                     // this tile's channel scales, all K-segments
+                tile_n0 = n0;
+                for (int i = et; i < P * kTileCols; i += kEpiThreads) {
+                    const int pp = i / kTileCols, c = i - pp * kTileCols;
+                    sh_col[i] = n0 + c < prm.N ? __ldg(prm.col_scale + size_t(n0 + c) * P + pp) : 0.0f;
+                }
+            }
             bias_next = fetch_bias(tile + num_units);                        // lands during this tile's work
             if (WIDE) {
                 sh_bias[TILE_N + et] = bias_next1;                           // et < 256 = TILE_N for every epilogue thread
@@ -1210,7 +1243,10 @@ sq_status prepare_variant(const GemmArgs &g, GemmLaunch &L, int device, int sm_c
     if (!make_map(&L.tb, g.b, g.N, g.K, g.ldb, B_ROWS)) return SQ_ERR_CUDA;
 
     const uint32_t stage_bytes = NPOL * TILE_M * BLOCK_K + (WIDE ? 2 : 1) * B_ROWS * BLOCK_K;
-    const uint32_t tail = (GENERIC ? 0u : kStageBytes) + epi_table_bytes(prm.nacc, prm.sb.Q, kTileCols) + sizeof(SharedHeader);
+    // per-token mode: the tile's channel scales are staged in shared memory when there are few K-segments
+    prm.col_tab_bytes = (GENERIC && prm.col_scale && prm.sb.P <= 8) ? uint32_t(prm.sb.P) * kTileCols * 4u : 0u;
+    const uint32_t tail = (GENERIC ? 0u : kStageBytes) + epi_table_bytes(prm.nacc, prm.sb.Q, kTileCols) + prm.col_tab_bytes +
+                          sizeof(SharedHeader);
     int stages = int((kSmemBudget - 1024 - tail) / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     const int tune_stages = g_tune_stages.load(std::memory_order_relaxed);

@@ -131,6 +131,7 @@ struct KernelParams {
     SegBounds sb;
     const float *s_pos, *s_neg, *s_w, *bias;
     const float *row_pos, *row_neg, *col_scale;   // per-token [M][P] and per-channel [N][P] scales instead of the tables
+    uint32_t col_tab_bytes;                       // shared memory for the tile's channel scales (0: read from global)
     void *Y;
     long long ldy;     // elements
     int y_is_f32;
