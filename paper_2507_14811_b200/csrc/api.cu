@@ -1,4 +1,5 @@
-// C ABI: host-side validation and dispatch.  Every argument error is reported before any launch.
+// C ABI: host-side validation and dispatch.  Every argument error is reported before any launch.  A layer call
+// can also be prepared once (segquant_plan_layer) and replayed as two bare launches (segquant_plan_run).
 #include <atomic>
 #include <cstring>
 #include "sq_common.cuh"

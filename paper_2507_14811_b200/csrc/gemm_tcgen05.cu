@@ -28,6 +28,8 @@
 // Every wait on an mbarrier is bounded (SM cycle counter, about 2 s); on expiry the CTA records
 // which wait gave up in the status word, stops issuing work, lets its own copies land and leaves
 // normally.  No load uses cluster multicast.
+// Host side: prepare_gemm works out everything a launch needs (tile plan, kernel instantiation, tensor maps,
+// shared-memory size, grid) without launching; run_gemm is one cudaLaunchKernelExC from that.
 #include <atomic>
 #include <mutex>
 #include <vector>

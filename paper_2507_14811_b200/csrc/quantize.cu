@@ -1,9 +1,11 @@
 // Activation / weight quantization kernels (Sec. 3 uniform quantizer, Sec. 4.3.2 Q_dual and polarity
-// split, Sec. 4.2.2 one scale per segment).  HBM-streaming: every thread converts 16 consecutive
-// elements per row (128-bit loads, one 128-bit store per code matrix) and walks down the rows with that column
-// chunk.  The codes are those of "one IEEE fp32 division, round half to even, clip"; the common case computes
-// them with a handful of full-rate fp32 instructions per element (see SegConst) so that the pass stays memory
-// bound.
+// split, Sec. 4.2.2 one scale per segment; App. A zero-point quantizer as a mode; the act-to-linear prologue of
+// Sec. 4.3.2 compiled in on request; per-row scales and 4-bit packing for the W4A8 setting of App. B).
+// HBM-streaming: every thread converts 16 consecutive elements per row (the row pieces arrive through a
+// thread-private ring of asynchronous 16-byte copies in shared memory, one 128-bit store per code matrix goes out)
+// and walks down the rows with that column chunk.  The codes are those of "one IEEE fp32 division, round half to
+// even, clip"; the common case computes them with a handful of full-rate fp32 instructions per element (see
+// SegConst) so that the pass stays memory bound.
 #include <cuda_bf16.h>
 #include "sq_common.cuh"
 
