@@ -1406,6 +1406,9 @@ sq_status prepare_gemm(const GemmArgs &g, GemmLaunch *out)
         };
         if (score(tile_max / 2, 0.75) > score(tile_max, 1.0)) tile_n = tile_max / 2;
     }
+    // per-(token, channel) factors run in the checking variant, whose epilogue releases a full-TMEM accumulator set
+    // only at its end: keep two sets so that it overlaps the next tile's main loop
+    if (g.col_scale && 2 * tile_n * prm.nacc > kTmemCols && tile_n >= 64) tile_n >>= 1;
     if (tune_tile_n >= 32 && tune_tile_n <= tile_max && (tune_tile_n & (tune_tile_n - 1)) == 0)
         tile_n = tune_tile_n;
     prm.acc_stages = (2 * tile_n * prm.nacc <= kTmemCols) ? 2 : 1;
