@@ -879,8 +879,8 @@ def run_reference(args):
     import oracle as O
     from paper_2507_14811_b200 import workloads as WL
     specs = WL.WORKLOADS[args.workload]
-    steps, warmup = max(1, min(args.steps, 3)), max(0, min(args.warmup, 1))
-    rows = 16
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    rows = 128 if args.workload != "tiny_qkv" else 16      # per layer and step: the whole run stays within a minute or two
     prepared = []
     for spec in specs:
         data = WL.make_layer(spec, M=rows)
@@ -909,7 +909,11 @@ def run_reference(args):
             "steps": steps, "warmup": warmup, "ms_per_step": round(dt * 1e3, 3), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None,
             "dtype": "e4m3" if specs[0].code == "e4m3" else "int8", "data": "synthetic",
-            "config": {"workload": args.workload, "sample": sample},
+            "config": {"workload": args.workload,
+                       "layers": [f"{s.name} M={s.M} K={s.K} N={s.N} P={s.P} Q={s.Q} {'dual' if s.dual else 'single'} {s.code}"
+                                  for s in specs],
+                       "ops": "executed tensor ops: 4MNK for dual layers, 2MNK for single-scale layers",
+                       "sample": sample},
             "cpu_baseline": {"value": val, "unit": "TOPS", "cores": O.num_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
