@@ -845,10 +845,10 @@ def run_ours(args):
 # prefix of the GEMM kernel source the counters were taken with; once that file has changed the figure is stale
 # and the bench prints null.
 GEMM_DRAM_TRAFFIC = {
-    "sd3_mmdit": {"bytes": 41503488 + 39893504 + 23285760 + 56154368 + 122918656 + 14132736, "source_tag": "7b16cb28f185017f",
+    "sd3_mmdit": {"bytes": 41489408 + 39405824 + 23212032 + 56258304 + 123196160 + 14200320, "source_tag": "e4d7ceaf4da88663",
                   "from": "ncu --set full of the three GEMM launches of one eager step (bench.py --workload sd3_mmdit "
                           "--profile-steps 4); below the algorithmic bytes because part of Y is still in L2 when a kernel ends"},
-    "dit_xl2": {"bytes": 12757504 + 13824 + 24236800 + 0, "source_tag": "7b16cb28f185017f",
+    "dit_xl2": {"bytes": 12757760 + 17152 + 24237312 + 0, "source_tag": "e4d7ceaf4da88663",
                 "from": "ncu --set full of the two GEMM launches of one eager step (bench.py --workload dit_xl2 "
                         "--profile-steps 4); operands partly L2-resident from the quantize pass, Y stays in L2"},
 }
