@@ -134,7 +134,7 @@ sq_status segquant_quantize_act(const void *X, sq_dtype dt, int64_t M, int64_t K
  *   have stored it in), then x = a * mult[k] as one fp32 multiply (mult dev [K] fp32, or NULL), then the codes
  *   of segquant_quantize_act for x.  The activation never goes through device memory.
  *   Accuracy of the activation: evaluated in fp32 with relative error <= (|h| + 8) 2^-23 (SiLU) and
- *   (2 h^2 + 32) 2^-24 (GELU); where the exact value lies that close to a rounding boundary of dt the stored
+ *   (3 h^2 + 48) 2^-24 (GELU); where the exact value lies that close to a rounding boundary of dt the stored
  *   value, and with it the code, may be that of the neighbouring dt value.  With SQ_ACT_NONE the codes are exact.
  *   Everything else as for segquant_quantize_act. */
 sq_status segquant_quantize_act_fused(const void *H, sq_dtype dt, int64_t M, int64_t K, int64_t ld,

@@ -178,7 +178,7 @@ def test_per_channel_multiplier_codes_are_exact(code, dual, x_dtype):
 def act_rel_eps(h, act):
     """Relative error bound of the kernel's fp32 evaluation of the activation (stated in the C header)."""
     h = h.astype(np.float64)
-    return (np.abs(h) + 8.0) * 2.0 ** -23 if act == "silu" else (2.0 * h ** 2 + 32.0) * 2.0 ** -24
+    return (np.abs(h) + 8.0) * 2.0 ** -23 if act == "silu" else (3.0 * h ** 2 + 48.0) * 2.0 ** -24
 
 
 def stored_candidates(h, act, stored):
