@@ -107,7 +107,8 @@ __device__ __forceinline__ void quant1(float x, float sp, float sn, int zp, int 
 // GELU(h) = h Phi(h) with E = erfc(t), t = |h| / sqrt 2: h (1 - E / 2) for h >= 0, (h / 2) E below.
 // erfc(t) = exp(-t^2) g(t); the smooth factor g (the scaled complementary error function) is a degree-9
 // polynomial in z = (t - 2.5) / (t + 2.5), which maps [0, 9.6] into [-1, 0.59) (coefficients from a least-squares
-// fit of the relative error on Chebyshev nodes, 2^-29; beyond t = 9.6 the exponential has underflowed).  t^2 is
+// fit of the relative error on Chebyshev nodes, 2^-29, by gelu_coefficients.py; beyond t = 9.6 the exponential
+// has underflowed).  t^2 is
 // split into its rounded value s and the rounding error e = fma(t, t, -s), and exp(-t^2) = exp(-s) (1 - e) to
 // first order, so that the rounding of the square, which the exponential would amplify by t^2, does not count.
 // What remains is the hardware exponential's own error (|s| 2^-24 from the product with log2 e, one unit in the
