@@ -430,7 +430,7 @@ __device__ __forceinline__ uint64_t ld_shared_64(uint32_t addr)
     return v;
 }
 
-template <int KIND, bool GENERIC, bool INIT = false>
+template <int KIND, bool GENERIC, bool INIT = false, bool PT = false>
 __device__ __forceinline__ void scale_add_unit(uint64_t (&y2)[16], const uint32_t (&r)[32], int a, int Q, int q_lo,
                                                int q_hi, int nf, uint32_t tab_addr, uint32_t nb_addr,
                                                uint32_t bias_slab = 0, const TokenScale *ts = nullptr)
@@ -462,8 +462,10 @@ __device__ __forceinline__ void scale_add_unit(uint64_t (&y2)[16], const uint32_
         return;
     }
     if (!GENERIC || q_lo == q_hi) {
-        const float c = ld_shared_f32(tab_addr + uint32_t(a * Q + q_lo) * 4u);
-        const uint64_t c2 = pack_f32x2(c, c);
+        // PT (production variant of the per-token layer): the token's scale times the staged channel scales
+        const float c = PT ? ts->row_factor : ld_shared_f32(tab_addr + uint32_t(a * Q + q_lo) * 4u);
+        uint64_t c2 = pack_f32x2(c, c);
+        const uint64_t rf2 = c2;
 #pragma unroll
         for (int j4 = 0; j4 < 8; j4++) {
             uint64_t b0 = y2[2 * j4], b1 = y2[2 * j4 + 1];
@@ -471,6 +473,7 @@ __device__ __forceinline__ void scale_add_unit(uint64_t (&y2)[16], const uint32_
 #pragma unroll
             for (int t = 0; t < 2; t++) {
                 const int j = 2 * j4 + t;
+                if (PT) c2 = mul_f32x2(rf2, ld_shared_64(ts->col_smem + uint32_t(nf + 2 * j) * 4u));
                 const uint64_t v2 = KIND == 0 ? pack_f32x2(__int2float_rn(int(r[2 * j])), __int2float_rn(int(r[2 * j + 1])))
                                               : pack_b32x2(r[2 * j], r[2 * j + 1]);
                 y2[j] = fma_f32x2(c2, v2, t == 0 ? b0 : b1);
@@ -623,7 +626,9 @@ __device__ __forceinline__ void store_slab(const uint64_t (&y2)[16], const Param
 // weight tile).  A single-scale 256 x 256 tile asks for 64 bytes of operands per SM cycle, which is all the L2
 // path delivers; the wide tile asks for 48.  Each half has its own weight tile in the ring stage, its own
 // issuing thread and accumulator, and is released to its thread separately, like the polarities of a dual tile.
-template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ, bool WIDE = false>
+// PT = true: the production variant for layers with per-token and per-channel scales (W4A8): the tile's channel
+// scales are staged in shared memory and every factor is the token's scale times the channel's.
+template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ, bool WIDE = false, bool PT = false>
 // 384 threads = 12 warps, 3 on each SM sub-partition with 16 K registers: 168 registers per thread at launch
 __global__ void __launch_bounds__(kThreads, 1)
 segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_constant__ CUtensorMap tm_a_neg,
@@ -857,7 +862,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
         float bias_next1 = WIDE ? fetch_bias(unit, 1) : 0.0f;   // second half of a wide tile
         // dequantization factors c[a][q] = s_act[p][pol] * s_w[p][q], a = p * NPOL + pol (one fp32 multiply);
         // built here, off the producer's and the MMA issuer's path, and published by the first tile's barrier
-        const bool per_token = GENERIC && prm.col_scale != nullptr;      // factors per (token, channel), no table
+        const bool per_token = PT || (GENERIC && prm.col_scale != nullptr);      // factors per (token, channel), no table
         for (int i = et; i < nacc * Q && !per_token; i += kEpiThreads) {
             const int a = i / Q, q = i - a * Q, p = a / NPOL;
             const float s_act = (NPOL == 2 && (a & 1)) ? prm.s_neg[p] : prm.s_pos[p];
@@ -892,7 +897,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
 
             asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // previous tile's readers are done
             if (et < TILE_N) sh_bias[et] = bias_next;
-            if (GENERIC && col_staged) {                                     // this tile's channel scales, all K-segments
+            if ((GENERIC || PT) && col_staged) {                              // this tile's channel scales, all K-segments
                 tile_n0 = n0;
                 for (int i = et; i < P * kTileCols; i += kEpiThreads) {
                     const int pp = i / kTileCols, c = i - pp * kTileCols;
@@ -952,7 +957,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                         const int a = p * NPOL + pol;
                         const int nf = n0 + (slab0 + sl) * 32;
                         const TokenScale tk = token_scale(a, row);
-                        scale_add_unit<KIND, GENERIC>(y2[sl], buf[u % NB], a, Q, q_lo[sl], q_hi[sl], nf, tab_addr, nb_addr, 0, &tk);
+                        scale_add_unit<KIND, GENERIC, false, PT>(y2[sl], buf[u % NB], a, Q, q_lo[sl], q_hi[sl], nf, tab_addr, nb_addr, 0, &tk);
                         if (GENERIC && prm.acc_dump && row < prm.M)
                             dump_unit(prm.acc_dump, buf[u % NB], a, row, nf, prm.M, prm.N);
                     }
@@ -989,8 +994,9 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                         const int h = u >> 2, sl = u & 3;
                         const int c0 = h * TILE_N + (slab0 + sl) * 32, nf = n0 + c0;
                         const int q = seg_of_column(min(nf, prm.N - 1), Q, nb_addr, lane);
-                        scale_add_unit<KIND, false, true>(y2, hb[h][sl], 0, Q, q, q, nf, tab_addr, nb_addr,
-                                                          bias_addr + uint32_t(c0) * 4u);
+                        const TokenScale tk = token_scale(0, row);
+                        scale_add_unit<KIND, false, true, PT>(y2, hb[h][sl], 0, Q, q, q, nf, tab_addr, nb_addr,
+                                                              bias_addr + uint32_t(c0) * 4u, &tk);
                         store_slab<GENERIC>(y2, prm, row, nf, yo);
                         if (u == 1) {
                             tc_ld32(t_h1 + 64u, hb[1][2]);
@@ -1018,10 +1024,11 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                     for (int sl = 0; sl < 4; sl++) {
                         const int c0 = (slab0 + sl) * 32, nf = n0 + c0;
                         const int q = seg_of_column(nf, Q, nb_addr, lane);
-                        scale_add_unit<KIND, false, true>(y2, pb[sl], 0, Q, q, q, nf, tab_addr, nb_addr,
-                                                          bias_addr + uint32_t(c0) * 4u);
+                        const TokenScale tk0 = token_scale(0, row), tk1 = token_scale(1, row);
+                        scale_add_unit<KIND, false, true, PT>(y2, pb[sl], 0, Q, q, q, nf, tab_addr, nb_addr,
+                                                              bias_addr + uint32_t(c0) * 4u, &tk0);
                         if (sl == 0) tc_wait_ld();
-                        scale_add_unit<KIND, false>(y2, nbuf[sl], 1, Q, q, q, nf, tab_addr, nb_addr);
+                        scale_add_unit<KIND, false, false, PT>(y2, nbuf[sl], 1, Q, q, q, nf, tab_addr, nb_addr, 0, &tk1);
                         store_slab<GENERIC>(y2, prm, row, nf, yo);
                         if (sl == 0) {                        // registers of slab 0 are free: the last two negative units
                             tc_ld32(t_neg + 64u, nbuf[2]);
@@ -1063,11 +1070,11 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                             q_lo = seg_of_column(nf, Q, nb_addr, lane);
                             q_hi = GENERIC ? seg_of_column(min(nf + 31, prm.N - 1), Q, nb_addr, lane) : q_lo;
                             const TokenScale tk = token_scale(pol, row);
-                            scale_add_unit<KIND, GENERIC, true>(y2, buf[u % NB], pol, Q, q_lo, q_hi, nf, tab_addr, nb_addr,
-                                                                bias_addr + uint32_t(c0) * 4u, &tk);
+                            scale_add_unit<KIND, GENERIC, true, PT>(y2, buf[u % NB], pol, Q, q_lo, q_hi, nf, tab_addr, nb_addr,
+                                                                    bias_addr + uint32_t(c0) * 4u, &tk);
                         } else {
                             const TokenScale tk = token_scale(pol, row);
-                            scale_add_unit<KIND, GENERIC>(y2, buf[u % NB], pol, Q, q_lo, q_hi, nf, tab_addr, nb_addr, 0, &tk);
+                            scale_add_unit<KIND, GENERIC, false, PT>(y2, buf[u % NB], pol, Q, q_lo, q_hi, nf, tab_addr, nb_addr, 0, &tk);
                         }
                         if (GENERIC && prm.acc_dump && row < prm.M)
                             dump_unit(prm.acc_dump, buf[u % NB], pol, row, nf, prm.M, prm.N);
@@ -1100,7 +1107,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                             ld_shared_2x64(bias_addr + uint32_t(c0 + 4 * j4) * 4u, y2[2 * j4], y2[2 * j4 + 1]);
                     }
                     const TokenScale tk = token_scale(c_a, row);
-                    scale_add_unit<KIND, GENERIC>(y2, r, c_a, Q, q_lo, q_hi, nf, tab_addr, nb_addr, 0, &tk);
+                    scale_add_unit<KIND, GENERIC, false, PT>(y2, r, c_a, Q, q_lo, q_hi, nf, tab_addr, nb_addr, 0, &tk);
                     if (GENERIC && prm.acc_dump && row < prm.M) dump_unit(prm.acc_dump, r, c_a, row, nf, prm.M, prm.N);
                     if (++c_a < nacc) return;
                     c_a = 0;
@@ -1232,7 +1239,7 @@ sq_status kernel_facts(int device, Kern kern, size_t smem, int cg, const cudaLau
     return SQ_OK;
 }
 
-template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ, bool WIDE = false>
+template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ, bool WIDE = false, bool PT = false>
 sq_status prepare_variant(const GemmArgs &g, GemmLaunch &L, int device, int sm_count)
 {
     constexpr int kTileCols = TILE_N * (WIDE ? 2 : 1);
@@ -1246,7 +1253,7 @@ sq_status prepare_variant(const GemmArgs &g, GemmLaunch &L, int device, int sm_c
 
     const uint32_t stage_bytes = NPOL * TILE_M * BLOCK_K + (WIDE ? 2 : 1) * B_ROWS * BLOCK_K;
     // per-token mode: the tile's channel scales are staged in shared memory when there are few K-segments
-    prm.col_tab_bytes = (GENERIC && prm.col_scale && prm.sb.P <= 8) ? uint32_t(prm.sb.P) * kTileCols * 4u : 0u;
+    prm.col_tab_bytes = ((GENERIC || PT) && prm.col_scale && prm.sb.P <= 8) ? uint32_t(prm.sb.P) * kTileCols * 4u : 0u;
     const uint32_t tail = (GENERIC ? 0u : kStageBytes) + epi_table_bytes(prm.nacc, prm.sb.Q, kTileCols) + prm.col_tab_bytes +
                           sizeof(SharedHeader);
     int stages = int((kSmemBudget - 1024 - tail) / stage_bytes);
@@ -1259,7 +1266,7 @@ sq_status prepare_variant(const GemmArgs &g, GemmLaunch &L, int device, int sm_c
     prm.num_n_tiles = int((g.N + kTileCols - 1) / kTileCols);
     const size_t smem = 1024 + size_t(stages) * stage_bytes + tail;
 
-    auto kern = segquant_gemm_kernel<KIND, NPOL, TILE_N, CG, GENERIC, SEQ, WIDE>;
+    auto kern = segquant_gemm_kernel<KIND, NPOL, TILE_N, CG, GENERIC, SEQ, WIDE, PT>;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(unsigned(sm_count / CG * CG));
     cfg.blockDim = dim3(kThreads);
@@ -1290,14 +1297,27 @@ template <int KIND, int NPOL, int CG>
 sq_status prepare_tile(const GemmArgs &g, GemmLaunch &L, int tile_n, bool seq, int device, int sm_count)
 {
     KernelParams &prm = L.prm;
-    bool dbg = prm.y_is_f32 || prm.acc_dump != nullptr || prm.col_scale != nullptr;
+    bool dbg = prm.y_is_f32 || prm.acc_dump != nullptr;
     // the production variant writes Y with TMA stores: 16-byte aligned base and row pitch
     dbg = dbg || reinterpret_cast<uintptr_t>(g.Y) % 16 != 0 || (size_t(g.ldy) * 2) % 16 != 0;
     for (int q = 1; q < prm.sb.Q; q++) dbg = dbg || (prm.sb.nb[q] % 32 != 0);
+    // per-token x per-channel scales: the production variant stages a tile's channel scales in shared memory, which
+    // it does for up to 8 K-segments, int8 codes and CTA pairs; anything else runs the checking variant
+    const bool pt = prm.col_scale != nullptr;
+    if (pt && !(KIND == 0 && CG == 2 && prm.sb.P <= 8)) dbg = true;
     if (seq) {      // sequential K-segments: one tile width per polarity count
         constexpr int TN = NPOL == 1 ? 256 : 128;
-        return dbg ? prepare_variant<KIND, NPOL, TN, CG, true, true>(g, L, device, sm_count)
-                   : prepare_variant<KIND, NPOL, TN, CG, false, true>(g, L, device, sm_count);
+        if (dbg) return prepare_variant<KIND, NPOL, TN, CG, true, true>(g, L, device, sm_count);
+        if constexpr (KIND == 0 && CG == 2)
+            if (pt) return prepare_variant<KIND, NPOL, TN, CG, false, true, false, true>(g, L, device, sm_count);
+        return prepare_variant<KIND, NPOL, TN, CG, false, true>(g, L, device, sm_count);
+    }
+    if constexpr (KIND == 0 && CG == 2) {
+        if (pt && !dbg) {     // 256- and 128-column tiles only (the automatic choice never goes below for these layers)
+            if (tile_n == 256) return prepare_variant<KIND, NPOL, 256, CG, false, false, false, true>(g, L, device, sm_count);
+            if (tile_n == 128) return prepare_variant<KIND, NPOL, 128, CG, false, false, false, true>(g, L, device, sm_count);
+            dbg = true;
+        }
     }
     // single-scale layer, one K-segment, CTA pairs, at least two 256-column tiles: 256 x 512 tiles whose halves
     // share the activation tile; an odd number of 256-column tiles leaves one half idle, so then only when there
@@ -1408,7 +1428,8 @@ sq_status prepare_gemm(const GemmArgs &g, GemmLaunch *out)
     }
     // per-(token, channel) factors run in the checking variant, whose epilogue releases a full-TMEM accumulator set
     // only at its end: keep two sets so that it overlaps the next tile's main loop
-    if (g.col_scale && 2 * tile_n * prm.nacc > kTmemCols && tile_n >= 64) tile_n >>= 1;
+    const bool pt_generic = g.col_scale && (prm.y_is_f32 || prm.acc_dump || g.code != SQ_CODE_INT8 || cg != 2 || g.sb.P > 8);
+    if (pt_generic && 2 * tile_n * prm.nacc > kTmemCols && tile_n >= 64) tile_n >>= 1;
     if (tune_tile_n >= 32 && tune_tile_n <= tile_max && (tune_tile_n & (tune_tile_n - 1)) == 0)
         tile_n = tune_tile_n;
     prm.acc_stages = (2 * tile_n * prm.nacc <= kTmemCols) ? 2 : 1;
