@@ -61,6 +61,7 @@ constexpr uint32_t kSmemBudget = 227 * 1024;
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s
 constexpr uint32_t kStageBytesPerWarp = 32 * 64;       // one 32 x 32 bf16 output block per epilogue warp
 constexpr uint32_t kStageBytes = kEpiWarps * kStageBytesPerWarp;
+constexpr int kMaxTokenSegments = 32;                  // per-token layers: channel scales of up to 32 K-segments (32 KiB at 256 columns) are staged per tile
 constexpr int kMaxFactorTable = 2048;                  // (K-segments x polarities) x N-segments factors in shared memory
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -1253,7 +1254,7 @@ sq_status prepare_variant(const GemmArgs &g, GemmLaunch &L, int device, int sm_c
 
     const uint32_t stage_bytes = NPOL * TILE_M * BLOCK_K + (WIDE ? 2 : 1) * B_ROWS * BLOCK_K;
     // per-token mode: the tile's channel scales are staged in shared memory when there are few K-segments
-    prm.col_tab_bytes = ((GENERIC || PT) && prm.col_scale && prm.sb.P <= 8) ? uint32_t(prm.sb.P) * kTileCols * 4u : 0u;
+    prm.col_tab_bytes = ((GENERIC || PT) && prm.col_scale && prm.sb.P <= kMaxTokenSegments) ? uint32_t(prm.sb.P) * kTileCols * 4u : 0u;
     const uint32_t tail = (GENERIC ? 0u : kStageBytes) + epi_table_bytes(prm.nacc, prm.sb.Q, kTileCols) + prm.col_tab_bytes +
                           sizeof(SharedHeader);
     int stages = int((kSmemBudget - 1024 - tail) / stage_bytes);
@@ -1302,9 +1303,9 @@ sq_status prepare_tile(const GemmArgs &g, GemmLaunch &L, int tile_n, bool seq, i
     dbg = dbg || reinterpret_cast<uintptr_t>(g.Y) % 16 != 0 || (size_t(g.ldy) * 2) % 16 != 0;
     for (int q = 1; q < prm.sb.Q; q++) dbg = dbg || (prm.sb.nb[q] % 32 != 0);
     // per-token x per-channel scales: the production variant stages a tile's channel scales in shared memory, which
-    // it does for up to 8 K-segments, int8 codes and CTA pairs; anything else runs the checking variant
+    // it does for up to 32 K-segments, int8 codes and CTA pairs; anything else runs the checking variant
     const bool pt = prm.col_scale != nullptr;
-    if (pt && !(KIND == 0 && CG == 2 && prm.sb.P <= 8)) dbg = true;
+    if (pt && !(KIND == 0 && CG == 2 && prm.sb.P <= kMaxTokenSegments)) dbg = true;
     if (seq) {      // sequential K-segments: one tile width per polarity count
         constexpr int TN = NPOL == 1 ? 256 : 128;
         if (dbg) return prepare_variant<KIND, NPOL, TN, CG, true, true>(g, L, device, sm_count);
@@ -1428,7 +1429,7 @@ sq_status prepare_gemm(const GemmArgs &g, GemmLaunch *out)
     }
     // per-(token, channel) factors run in the checking variant, whose epilogue releases a full-TMEM accumulator set
     // only at its end: keep two sets so that it overlaps the next tile's main loop
-    const bool pt_generic = g.col_scale && (prm.y_is_f32 || prm.acc_dump || g.code != SQ_CODE_INT8 || cg != 2 || g.sb.P > 8);
+    const bool pt_generic = g.col_scale && (prm.y_is_f32 || prm.acc_dump || g.code != SQ_CODE_INT8 || cg != 2 || g.sb.P > kMaxTokenSegments);
     if (pt_generic && 2 * tile_n * prm.nacc > kTmemCols && tile_n >= 64) tile_n >>= 1;
     if (tune_tile_n >= 32 && tune_tile_n <= tile_max && (tune_tile_n & (tune_tile_n - 1)) == 0)
         tile_n = tune_tile_n;

@@ -305,6 +305,7 @@ def run_w4a8_parity(spec):
     ("w4_ragged", 129, 208, 200, [0, 96, 208]),
     ("w4_long_row", 70, 16384, 64, [0, 4096, 16384]),
     ("w4_heads", 260, 1536, 320, list(range(0, 1537, 64))),
+    ("w4_seg40", 140, 1280, 136, list(range(0, 1281, 32))),      # more K-segments than are staged: checking variant only
 ])
 def test_w4a8_layer_parity(case, dual):
     name, M, K, N, kb = case
