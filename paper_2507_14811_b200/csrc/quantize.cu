@@ -488,6 +488,30 @@ __device__ __forceinline__ float ord_dec(uint32_t u)
     return __uint_as_float((u & 0x80000000u) ? (u & 0x7FFFFFFFu) : ~u);
 }
 
+// largest and smallest of the 16 elements of a chunk (bf16: on packed pairs, two elements per instruction)
+__device__ __forceinline__ void chunk_extrema(const Raw16<float> &r, float &mx, float &mn)
+{
+    mx = -INFINITY; mn = INFINITY;
+#pragma unroll
+    for (int v = 0; v < 4; v++) {
+        mx = fmaxf(fmaxf(mx, r.v[v].x), fmaxf(r.v[v].y, fmaxf(r.v[v].z, r.v[v].w)));
+        mn = fminf(fminf(mn, r.v[v].x), fminf(r.v[v].y, fminf(r.v[v].z, r.v[v].w)));
+    }
+}
+__device__ __forceinline__ void chunk_extrema(const Raw16<__nv_bfloat16> &r, float &mx, float &mn)
+{
+    const uint32_t w[8] = {r.v[0].x, r.v[0].y, r.v[0].z, r.v[0].w, r.v[1].x, r.v[1].y, r.v[1].z, r.v[1].w};
+    __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162 *>(&w[0]), lo = hi;
+#pragma unroll
+    for (int i = 1; i < 8; i++) {
+        const __nv_bfloat162 x = *reinterpret_cast<const __nv_bfloat162 *>(&w[i]);
+        hi = __hmax2(hi, x);
+        lo = __hmin2(lo, x);
+    }
+    mx = fmaxf(__low2float(hi), __high2float(hi));
+    mn = fminf(__low2float(lo), __high2float(lo));
+}
+
 template <typename Tin, bool DUAL>
 __global__ void __launch_bounds__(kThreads)
 quantize_per_row_kernel(const Tin *__restrict__ X, int K, int64_t ld, const SegBounds sb, float q_max, float q_min_abs,
@@ -515,14 +539,8 @@ quantize_per_row_kernel(const Tin *__restrict__ X, int K, int64_t ld, const SegB
         if (k0 + kVec <= sb.kb[p + 1]) {
             seg[c] = p;
             load16(src + k0, raw[c]);
-            float mx = -INFINITY, mn = INFINITY;
-#pragma unroll
-            for (int g4 = 0; g4 < 4; g4++) {
-                float x[4];
-                get4(raw[c], g4, x);
-#pragma unroll
-                for (int i = 0; i < 4; i++) { mx = fmaxf(mx, x[i]); mn = fminf(mn, x[i]); }
-            }
+            float mx, mn;
+            chunk_extrema(raw[c], mx, mn);
             atomicMax(&sh_max[p], ord_enc(mx));
             atomicMin(&sh_min[p], ord_enc(mn));
         } else {
@@ -556,6 +574,8 @@ quantize_per_row_kernel(const Tin *__restrict__ X, int K, int64_t ld, const SegB
     __syncthreads();
     const int hi = int(q_max), lo = DUAL ? -int(q_min_abs) : -int(q_max);
     constexpr int MODE = DUAL ? kDual : kSingle;
+    SegConst cp, cn;
+    int const_seg = -1;
 #pragma unroll
     for (int c = 0; c < kRowChunks; c++) {
         const int k0 = (int(threadIdx.x) + c * int(blockDim.x)) * kVec;
@@ -564,8 +584,11 @@ quantize_per_row_kernel(const Tin *__restrict__ X, int K, int64_t ld, const SegB
         uint8_t *dn = DUAL ? c_neg + row * ldc + k0 : nullptr;
         bool done = false;
         if (seg[c] >= 0) {
-            const SegConst cp = seg_const(sh_sp[seg[c]]);
-            const SegConst cn = seg_const(DUAL ? sh_sn[seg[c]] : 1.0f);
+            if (seg[c] != const_seg) {              // constants are remade only when the chunk's K-segment changes
+                cp = seg_const(sh_sp[seg[c]]);
+                cn = seg_const(DUAL ? sh_sn[seg[c]] : 1.0f);
+                const_seg = seg[c];
+            }
             if (cp.fast && cn.fast && !(DUAL && lo != -128)) {
                 uint32_t wp[4], wn[4];
 #pragma unroll
