@@ -57,6 +57,8 @@ def lib():
         _lib.sqo_silu.argtypes = [C.c_double]
         _lib.sqo_gelu.restype = C.c_double
         _lib.sqo_gelu.argtypes = [C.c_double]
+        _lib.sqo_geglu.restype = C.c_double
+        _lib.sqo_geglu.argtypes = [C.c_double, C.c_double]
     return _lib
 
 
@@ -327,6 +329,20 @@ def activation(H, act: str, stored="bf16"):
     out = np.zeros(H.shape, np.float32)
     exact = np.zeros(H.shape, np.float64)
     lib().sqo_activation(_p(H), C.c_int64(H.size), C.c_int(ACT[act]), C.c_int(int(stored == "bf16")), _p(out), _p(exact))
+    return out, exact
+
+
+def activation_gated(H, stored="bf16"):
+    """GEGLU: H [M, 2K] -> H[:, :K] * GELU(H[:, K:]) in fp64, rounded once to the stored dtype.
+    Returns (fp32 array [M, K], fp64 exact values)."""
+    H = _f32(H)
+    M, K2 = H.shape
+    assert K2 % 2 == 0
+    K = K2 // 2
+    out = np.zeros((M, K), np.float32)
+    exact = np.zeros((M, K), np.float64)
+    lib().sqo_activation_gated(_p(H), C.c_int64(M), C.c_int64(K), C.c_int64(K2), C.c_int(int(stored == "bf16")), _p(out),
+                               C.c_int64(K), _p(exact))
     return out, exact
 
 

@@ -443,6 +443,30 @@ void sqo_activation(const float *H, int64_t n, int act, int stored_bf16, float *
     }
 }
 
+/* Gated GELU (App. B names GEGLU among the polarity-sensitive activations that feed DualScale layers, without a
+ * form; the form taken is that of the gated feed-forward: the 2K columns of the pre-activation row are two
+ * halves, value half first, gate half second, and a[k] = H[k] * GELU(H[K + k])).  The product is exact in fp64
+ * up to one rounding and, as above, the value is rounded ONCE to the stored dtype.                             */
+double sqo_geglu(double value, double gate) { return value * sqo_gelu(gate); }
+
+void sqo_activation_gated(const float *H, int64_t M, int64_t K, int64_t ld, int stored_bf16, float *out, int64_t ldo,
+                          double *exact)
+{
+    for (int64_t m = 0; m < M; m++)
+        for (int64_t k = 0; k < K; k++) {
+            double a = sqo_geglu((double)H[m * ld + k], (double)H[m * ld + K + k]);
+            if (exact) exact[m * ldo + k] = a;
+            if (stored_bf16) {
+                uint32_t bits = (uint32_t)sqo_bf16_from_f64(a) << 16;
+                float f;
+                memcpy(&f, &bits, 4);
+                out[m * ldo + k] = f;
+            } else {
+                out[m * ldo + k] = (float)a;
+            }
+        }
+}
+
 /* Per-channel multiplier in front of the quantizer (Sec. 4.2.2 last paragraph: SmoothQuant's migration, one
  * strength per segment; the multiplier m[k] = 1 / smoothing factor is made offline): out = fl32(x * m[k]).   */
 void sqo_smooth(const float *X, int64_t M, int64_t K, int64_t ld, const float *mult, float *out, int64_t ldo)

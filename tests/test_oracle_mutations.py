@@ -55,6 +55,9 @@ MUTATIONS = {
     "gelu_half_dropped": ("return 0.5 * h * erfc(-h / sqrt(2.0));", "return h * erfc(-h / sqrt(2.0));"),
     "gelu_tanh_like_argument": ("return 0.5 * h * erfc(-h / sqrt(2.0));", "return 0.5 * h * erfc(-h / 2.0);"),
     "activation_rounded_twice": ("uint32_t bits = (uint32_t)sqo_bf16_from_f64(a) << 16;", "uint32_t bits = (uint32_t)sqo_bf16_from_f64((double)(float)a + 1e-3 * a) << 16;"),
+    "geglu_halves_swapped": ("sqo_geglu((double)H[m * ld + k], (double)H[m * ld + K + k]);", "sqo_geglu((double)H[m * ld + K + k], (double)H[m * ld + k]);"),
+    "geglu_gate_through_silu": ("return value * sqo_gelu(gate);", "return value * sqo_silu(gate);"),
+    "geglu_gate_rounded_first": ("return value * sqo_gelu(gate);", "return value * (double)(float)sqo_gelu(gate) * (1.0 + 1e-3);"),
     "smooth_indexed_by_row": ("out[m * ldo + k] = X[m * ld + k] * mult[k];", "out[m * ldo + k] = X[m * ld + k] * mult[m % K];"),
     "per_row_uses_first_rows_scales": ("sqo_quantize_act_i8(X + m * ld, 1, K, ld, P, kb, s_pos + m * P,", "sqo_quantize_act_i8(X + m * ld, 1, K, ld, P, kb, s_pos,"),
     "per_row_scales_from_whole_matrix": ("sqo_calib_act(X + m * ld, 1, K, ld, P, kb, dual,", "sqo_calib_act(X, M, K, ld, P, kb, dual,"),

@@ -764,6 +764,46 @@ def test_activation_is_rounded_once_to_the_stored_dtype(act):
     assert np.array_equal(out32, exact32.astype(np.float32)) and np.array_equal(exact32, exact)
 
 
+def test_gated_gelu_against_library_and_identities():
+    """GEGLU (App. B): value half times GELU(gate half).  Pinned to torch's fp64 GELU on the chunked halves, to the
+    identity a(v, g) - a(v, -g) = v g, to a(v, 0) = 0 and a(1, g) = GELU(g), and to which half is the gate."""
+    r = rng(49)
+    M, K = 7, 24
+    H = torch.from_numpy(r.normal(0, 2.0, (M, 2 * K)).astype(np.float32)).to(torch.bfloat16).float().numpy()
+    out, exact = O.activation_gated(H, "f32")
+    value, gate = torch.from_numpy(H).double().chunk(2, dim=1)
+    want = (value * torch.nn.functional.gelu(gate)).numpy()
+    assert exact.shape == (M, K) and np.allclose(exact, want, rtol=1e-9, atol=1e-14)
+    assert np.array_equal(out, exact.astype(np.float32))
+    L = O.lib()
+    for v, g in [(0.7, 1.3), (-2.0, 0.4), (3.0, -2.5)]:
+        assert math.isclose(L.sqo_geglu(v, g) - L.sqo_geglu(v, -g), v * g, rel_tol=1e-13)
+        assert L.sqo_geglu(v, 0.0) == 0.0
+        assert L.sqo_geglu(1.0, g) == L.sqo_gelu(g)
+    # the gate is the SECOND half: a large negative gate closes the unit whatever the value half holds
+    Hc = H.copy()
+    Hc[:, K:] = -30.0
+    assert np.all(np.abs(O.activation_gated(Hc, "f32")[1]) < 1e-100)
+    Hc = H.copy()
+    Hc[:, :K] = -30.0
+    assert np.all(np.abs(O.activation_gated(Hc, "f32")[1])[H[:, K:] > 0.5] > 1e-3)
+    # rows do not mix
+    out1, _ = O.activation_gated(H[3:4], "f32")
+    assert np.array_equal(out1[0], out[3])
+
+
+def test_gated_gelu_is_rounded_once_to_the_stored_dtype():
+    H = torch.from_numpy(rng(50).normal(0, 2.5, (40, 128)).astype(np.float32)).to(torch.bfloat16).float().numpy()
+    out, exact = O.activation_gated(H, "bf16")
+    bits = out.view(np.uint32)
+    assert np.all((bits & 0xFFFF) == 0)
+    assert np.array_equal((bits >> 16).astype(np.uint16), O.bf16_bits(exact))
+    # rounding GELU(gate) to bf16 first and the product again (two roundings) gives different values somewhere
+    g16 = O.activation(H[:, 64:], "gelu", "bf16")[0].astype(np.float64)
+    twice = O.bf16_bits(H[:, :64].astype(np.float64) * g16)
+    assert np.any(twice != (bits >> 16).astype(np.uint16))
+
+
 def test_smoothing_multiplier_is_one_fp32_multiply():
     r = rng(48)
     X = r.normal(0, 1, (9, 40)).astype(np.float32)
