@@ -152,6 +152,9 @@ class BenchLayer:
             self.zp = {"s_x": s_x, "z_x": z_x, "codes": B.new_codes(self.M, spec.K, device),
                        "bias": B.segquant_fold_zero_point(L.Wq, L.seg, s_x, z_x, L.s_w, L.bias)}
         self.a_stage = torch.empty_like(self.X) if (spec.dual and self.act) else None
+        # gated GELU: the pre-activation row holds a value half and a gate half (timing only: any values do)
+        self.H2 = torch.cat([self.X, self.X], dim=1).contiguous() if self.act == "geglu" else None
+        self.g_stage = torch.empty_like(self.X) if self.act == "geglu" else None
         # the same layer as W4A8: per-channel 4-bit weights (kept packed), per-token activation scales
         self.w4 = None
         if spec.code == "int8" and spec.K <= 16384:
@@ -193,13 +196,18 @@ class BenchLayer:
         """Pre-activation -> activation -> codes in one pass.  Timing only: the layer's input stands in for the
         pre-activation (the cost does not depend on the values)."""
         L = self.layer
-        self.B.segquant_quantize_act_fused(self.X, L.seg, L.s_pos, L.s_neg, L.code, act=self.act, c_pos=self.c_pos,
+        H = self.H2 if self.act == "geglu" else self.X
+        self.B.segquant_quantize_act_fused(H, L.seg, L.s_pos, L.s_neg, L.code, act=self.act, c_pos=self.c_pos,
                                            c_neg=self.c_neg)
 
     def act_unfused(self):
         """The activation as its own elementwise pass (a library kernel, comparison only): reads the
         pre-activation, writes the activation that the quantize pass then reads."""
-        if self.act == "silu":
+        if self.act == "geglu":                                  # two library kernels: GELU of the gate half, the product
+            K = self.spec.K
+            torch.ops.aten.gelu.out(self.H2[:, K:], out=self.g_stage)
+            torch.mul(self.H2[:, :K], self.g_stage, out=self.a_stage)
+        elif self.act == "silu":
             torch.nn.functional.silu(self.X, inplace=False) if self.a_stage is None else torch.ops.aten.silu.out(self.X, out=self.a_stage)
         else:
             torch.ops.aten.gelu.out(self.X, out=self.a_stage)
@@ -252,7 +260,7 @@ class BenchLayer:
         for name in ("Wq", "s_w", "bias", "s_pos", "s_neg", "workspace"):
             t = getattr(self.layer, name)
             setattr(other.layer, name, None if t is None else t.clone())
-        for name in ("X", "c_pos", "c_neg", "Y", "a_stage"):
+        for name in ("X", "c_pos", "c_neg", "Y", "a_stage", "H2", "g_stage"):
             t = getattr(self, name)
             setattr(other, name, None if t is None else t.clone())
         if self.zp is not None:
@@ -608,7 +616,8 @@ def layer_table(specs, kt, peaks):
             r["fused_act"] = {"act": s.x_kind.partition("+")[2], "fused_quant_us": us(kt["q_fused"][i]),
                               "unfused_act_us": us(kt["act"][i]), "unfused_pair_us": us(kt["act"][i] + q * 1e3),
                               "fused_time_over_unfused_pair": round(kt["q_fused"][i] / (kt["act"][i] + q * 1e3), 3),
-                              "hbm_bytes_saved": 4 * s.M * s.K,
+                              # unfused: the activation is written and read again (gated: so is GELU(gate))
+                              "hbm_bytes_saved": (8 if s.x_kind.endswith("geglu") else 4) * s.M * s.K,
                               "note": "the unfused activation is a library elementwise kernel (comparison only)"}
     return rows
 
@@ -649,7 +658,7 @@ def measure_side_workload(name, dev, args, peaks):
     return out
 
 
-SIDE_WORKLOADS = ["flux", "dit_xl2", "sdxl_skip", "sdxl_sweep", "sd3_heads"]
+SIDE_WORKLOADS = ["flux", "dit_xl2", "sdxl_skip", "sdxl_sweep", "sd3_heads", "sdxl_geglu"]
 
 
 def run_ours(args):

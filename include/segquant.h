@@ -50,7 +50,7 @@ typedef enum {
 
 typedef enum { SQ_CODE_INT8 = 0, SQ_CODE_E4M3 = 1 } sq_code;   /* 8-bit code type */
 typedef enum { SQ_F32 = 0, SQ_BF16 = 1 } sq_dtype;             /* real-valued element type */
-typedef enum { SQ_ACT_NONE = 0, SQ_ACT_SILU = 1, SQ_ACT_GELU = 2 } sq_act;   /* activation in front of the quantizer */
+typedef enum { SQ_ACT_NONE = 0, SQ_ACT_SILU = 1, SQ_ACT_GELU = 2, SQ_ACT_GEGLU = 3 } sq_act;   /* activation in front of the quantizer */
 
 /* flags */
 #define SQ_FLAG_QMIN_SYM 1u  /* int8 DualScale: clamp the negative path to -127 instead of -128 */
@@ -136,6 +136,10 @@ sq_status segquant_quantize_act(const void *X, sq_dtype dt, int64_t M, int64_t K
  *   Accuracy of the activation: evaluated in fp32 with relative error <= (|h| + 8) 2^-23 (SiLU) and
  *   (3 h^2 + 48) 2^-24 (GELU); where the exact value lies that close to a rounding boundary of dt the stored
  *   value, and with it the code, may be that of the neighbouring dt value.  With SQ_ACT_NONE the codes are exact.
+ *   SQ_ACT_GEGLU (gated GELU; App. B names it without a form): H is [M, 2K] with ld >= 2K, value half in columns
+ *   [0, K), gate half in [K, 2K), a[k] = H[k] * GELU(H[K + k]) with relative error <= (3 g^2 + 49) 2^-24, g the
+ *   gate; K, mult, the segment table and the codes refer to the K outputs.  The gate half must start on a 16-byte
+ *   boundary: K a multiple of 8 (bf16) or 4 (fp32), else SQ_ERR_ALIGN.
  *   Everything else as for segquant_quantize_act. */
 sq_status segquant_quantize_act_fused(const void *H, sq_dtype dt, int64_t M, int64_t K, int64_t ld,
                                       const sq_segtable *seg, const float *s_pos, const float *s_neg,

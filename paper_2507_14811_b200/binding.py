@@ -173,13 +173,16 @@ def segquant_quantize_act(X: torch.Tensor, seg: SegTable, s_pos, s_neg, code: st
     return c_pos, (c_neg if s_neg is not None else None)
 
 
-SQ_ACT = {None: 0, "none": 0, "silu": 1, "gelu": 2}
+SQ_ACT = {None: 0, "none": 0, "silu": 1, "gelu": 2, "geglu": 3}
 
 
 def segquant_quantize_act_fused(H: torch.Tensor, seg: SegTable, s_pos, s_neg, code: str, act=None, mult=None,
                                 flags: int = 0, c_pos=None, c_neg=None):
-    """Activation function and / or per-channel multiplier in front of the quantizer, in one pass over H."""
+    """Activation function and / or per-channel multiplier in front of the quantizer, in one pass over H.
+    act="geglu": H is [M, 2K] (value half, gate half) and the codes are [M, K]."""
     M, K = H.shape
+    if act == "geglu":
+        K //= 2
     if c_pos is None:
         c_pos = new_codes(M, K, H.device)
     if s_neg is not None and c_neg is None:

@@ -181,9 +181,11 @@ sq_status segquant_quantize_act_fused(const void *H, sq_dtype dt, int64_t M, int
 {
     if (!s_pos || (s_neg && !c_neg)) return SQ_ERR_NULL;
     if (!valid_dt(dt) || !valid_code(code)) return SQ_ERR_UNSUPPORTED;
-    if (act != SQ_ACT_NONE && act != SQ_ACT_SILU && act != SQ_ACT_GELU) return SQ_ERR_UNSUPPORTED;
+    if (act != SQ_ACT_NONE && act != SQ_ACT_SILU && act != SQ_ACT_GELU && act != SQ_ACT_GEGLU) return SQ_ERR_UNSUPPORTED;
     sq_status st;
-    if ((st = check_matrix(H, M, K, ld, dt_size(dt))) != SQ_OK) return st;
+    const bool gated = act == SQ_ACT_GEGLU;                  // the row holds 2 K pre-activations: value half, gate half
+    if (gated && K > 0 && (K * int64_t(dt_size(dt))) % 16 != 0) return SQ_ERR_ALIGN;
+    if ((st = check_matrix(H, M, gated ? 2 * K : K, ld, dt_size(dt))) != SQ_OK) return st;
     if ((st = check_matrix(c_pos, M, K, ldc, 1)) != SQ_OK) return st;
     if (s_neg && (st = check_matrix(c_neg, M, K, ldc, 1)) != SQ_OK) return st;
     HostSeg hs = load_segtable(seg, K, seg && seg->nb && seg->Q >= 1 ? seg->nb[seg->Q] : 0);

@@ -151,6 +151,15 @@ __device__ __forceinline__ float pre1(float h, int act, float mult)
     }
     return __fmul_rn(a, mult);                                // the per-channel multiplier: one fp32 multiply
 }
+// Gated GELU (App. B lists GEGLU with SiLU and GELU): value * GELU(gate), the product in fp32 (one more rounding
+// on top of the GELU's error: relative error <= (3 g^2 + 49) 2^-24), rounded once to the stored dtype.
+template <typename Tin>
+__device__ __forceinline__ float pre_gated(float value, float gate, float mult)
+{
+    float a = __fmul_rn(value, gelu_f32(gate));
+    if (sizeof(Tin) == 2) a = __bfloat162float(__float2bfloat16_rn(a));
+    return __fmul_rn(a, mult);
+}
 
 // Per-segment constants of the fast form.  The quotient x / s is obtained from the correctly rounded
 // reciprocal r = RN(1/s) by one multiply and two FMAs,
@@ -336,15 +345,18 @@ __device__ __forceinline__ void quant4(const float (&x)[4], const SegConst &cp, 
 // (V chunks per row, R rows in flight over the whole grid), so that a warp reads 1 KiB (bf16) of consecutive
 // addresses per row, the per-segment constants are made once per thread, and the next row's loads are in
 // flight while the current row is converted.
-// PRE compiles in the act-to-linear prologue: activation function and per-channel multiplier in front of the
-// quantizer, so that the activation's output never goes through HBM.
+// PRE != 0 compiles in the act-to-linear prologue: activation function and per-channel multiplier in front of the
+// quantizer, so that the activation's output never goes through HBM.  PRE == 2 is the gated form: the row holds
+// 2 K pre-activations, the value half travels through the ring like any input and the gate half (K elements
+// further on) is fetched into registers one row ahead.
 // RING: depth of the shared-memory ring the rows travel through (see below); 4 when a thread has many rows to
 // walk (large inputs: more bytes in flight), 2 otherwise (less shared memory, more L1 for the copies).
-template <typename Tin, int CODE, int MODE, bool PRE, int RING>
+template <typename Tin, int CODE, int MODE, int PRE, int RING>
 __global__ void __launch_bounds__(kThreads, PRE ? 3 : kBlocksPerSm)
 quantize_kernel(const __grid_constant__ QuantParams prm)
 {
     constexpr bool DUAL = MODE == kDual;
+    constexpr bool GATED = PRE == 2;
     // Programmatic dependent launch: this kernel may be scheduled while the previous kernel of the stream
     // winds down, and lets the next one be scheduled while its own last blocks run; nothing in global
     // memory is touched before the previous kernel has completed.
@@ -406,6 +418,9 @@ quantize_kernel(const __grid_constant__ QuantParams prm)
 #pragma unroll
         for (int d = 0; d < kDepth - 1; d++) copy_row(src + int64_t(d) * src_step, d, int64_t(r0) + int64_t(d) * R < M);
     }
+    const Tin *gsrc = src + K;                               // (gated) this chunk of the gate half
+    Raw16<Tin> gate_next;
+    if (GATED && whole) load16(gsrc, gate_next);
     int q = 0;                                               // N-segment (weights only) the constants belong to
     int64_t q_end = 0;                                       // first row beyond it (0: no constants yet)
     SegConst cp, cn;
@@ -425,7 +440,11 @@ quantize_kernel(const __grid_constant__ QuantParams prm)
             if (MODE == kZeroPoint) zp = __ldg(prm.zp + p);
             fast = whole && cp.fast && cn.fast && !(DUAL && CODE == SQ_CODE_INT8 && lo != -128);
         }
-        Raw16<Tin> cur;
+        Raw16<Tin> cur, gate;
+        if (GATED && whole) {
+            gate = gate_next;
+            if (row + R < M) load16(gsrc + src_step, gate_next);
+        }
         if (whole) {
             // row + (kDepth - 1) R goes into the slot the previous row has just left; then the oldest group, this
             // row's, is complete once at most kDepth - 1 newer groups are pending
@@ -441,7 +460,12 @@ quantize_kernel(const __grid_constant__ QuantParams prm)
             for (int g4 = 0; g4 < 4; g4++) {
                 float x[4];
                 get4(cur, g4, x);
-                if (PRE) {
+                if (GATED) {
+                    float gt[4];
+                    get4(gate, g4, gt);
+#pragma unroll
+                    for (int i = 0; i < 4; i++) x[i] = pre_gated<Tin>(x[i], gt[i], mreg[PRE ? 4 * g4 + i : 0]);
+                } else if (PRE) {
 #pragma unroll
                     for (int i = 0; i < 4; i++) x[i] = pre1<Tin>(x[i], prm.act, mreg[PRE ? 4 * g4 + i : 0]);
                 }
@@ -457,7 +481,8 @@ quantize_kernel(const __grid_constant__ QuantParams prm)
                 while (pp + 1 < sb.P && k0 + i >= sb.kb[pp + 1]) pp++;
                 uint32_t a, b;
                 float x = load1(src + i);
-                if (PRE) x = pre1<Tin>(x, prm.act, prm.mult ? __ldg(prm.mult + k0 + i) : 1.0f);
+                if (GATED) x = pre_gated<Tin>(x, load1(gsrc + i), prm.mult ? __ldg(prm.mult + k0 + i) : 1.0f);
+                else if (PRE) x = pre1<Tin>(x, prm.act, prm.mult ? __ldg(prm.mult + k0 + i) : 1.0f);
                 quant1<CODE, MODE>(x, __ldg(prm.s_pos + pp * Qs + qq), DUAL ? __ldg(prm.s_neg + pp * Qs + qq) : 0.0f,
                                    MODE == kZeroPoint ? __ldg(prm.zp + pp) : 0, lo, hi, a, b);
                 dp[i] = uint8_t(a);
@@ -465,6 +490,7 @@ quantize_kernel(const __grid_constant__ QuantParams prm)
             }
         }
         src += src_step;
+        if (GATED) gsrc += src_step;
         dp += dst_step;
         if (DUAL) dn += dst_step;
     }
@@ -678,12 +704,15 @@ sq_status prepare_t(QuantLaunch &L)
     L.blocks = unsigned(blocks);
     // fp32 input: 64-byte chunks, so half the depth for the same shared memory
     const bool deep = iters >= 10 && sizeof(Tin) == 2;
-    if (pre)
-        L.kernel = deep ? reinterpret_cast<const void *>(quantize_kernel<Tin, CODE, MODE, true, 4>)
-                        : reinterpret_cast<const void *>(quantize_kernel<Tin, CODE, MODE, true, 2>);
+    if (prm.act == SQ_ACT_GEGLU)
+        L.kernel = deep ? reinterpret_cast<const void *>(quantize_kernel<Tin, CODE, MODE, 2, 4>)
+                        : reinterpret_cast<const void *>(quantize_kernel<Tin, CODE, MODE, 2, 2>);
+    else if (pre)
+        L.kernel = deep ? reinterpret_cast<const void *>(quantize_kernel<Tin, CODE, MODE, 1, 4>)
+                        : reinterpret_cast<const void *>(quantize_kernel<Tin, CODE, MODE, 1, 2>);
     else
-        L.kernel = deep ? reinterpret_cast<const void *>(quantize_kernel<Tin, CODE, MODE, false, 4>)
-                        : reinterpret_cast<const void *>(quantize_kernel<Tin, CODE, MODE, false, 2>);
+        L.kernel = deep ? reinterpret_cast<const void *>(quantize_kernel<Tin, CODE, MODE, 0, 4>)
+                        : reinterpret_cast<const void *>(quantize_kernel<Tin, CODE, MODE, 0, 2>);
     return SQ_OK;
 }
 

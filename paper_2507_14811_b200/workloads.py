@@ -82,6 +82,8 @@ def _draw_x(spec: LayerSpec, rows: int, g: torch.Generator) -> torch.Tensor:
         x = _gelu(pre)
     elif act == "silu":
         x = _silu(pre)
+    elif act == "geglu":                     # gated GELU: the segment-scaled draw is the value half
+        x = pre * _gelu(torch.randn((rows, spec.K), generator=g) * 1.5)
     elif act == "":
         x = pre
     else:
@@ -170,6 +172,15 @@ WORKLOADS: dict[str, list[LayerSpec]] = {
               x_kind="normal+silu", w_kind="plain", seed=4000, x_seg_std=[1.0, 8.0]),
     ],
 }
+
+# the output projection of a gated-GELU feed-forward (SDXL-like transformer blocks at 640 and 1280 channels,
+# 64 x 64 and 32 x 32 tokens, batch 2): its input is value * GELU(gate)
+WORKLOADS["sdxl_geglu"] = [
+    _spec("ff_out_640", 8192, 2560, 640, dual=True, code="int8", x_dtype="bf16",
+          x_kind="normal+geglu", w_kind="plain", seed=6000, x_seg_std=[1.5]),
+    _spec("ff_out_1280", 2048, 5120, 1280, dual=True, code="int8", x_dtype="bf16",
+          x_kind="normal+geglu", w_kind="plain", seed=6001, x_seg_std=[1.5]),
+]
 
 SDXL_SWEEP_M = [512, 1024, 2048, 4096, 8192, 16384, 32768, 65536]
 

@@ -258,6 +258,65 @@ def test_fused_activation_equals_the_unfused_pair_when_the_stored_values_agree(a
     assert agree > 0.999
 
 
+@pytest.mark.parametrize("code,dual,dtype", [("int8", True, "bf16"), ("int8", False, "bf16"), ("e4m3", True, "bf16"),
+                                             ("int8", True, "f32")])
+def test_fused_gated_gelu_codes_are_valid(code, dual, dtype):
+    """H [M, 2K] (value half, gate half) -> value * GELU(gate) -> stored dtype -> multiplier -> codes in one kernel
+    (App. B: GEGLU is one of the activations in front of DualScale layers).  Same validity rule as for the unary
+    activations, with the kernel's bound (3 g^2 + 49) 2^-24 on the relative error of the product."""
+    rs = np.random.default_rng(11)
+    M, K = 600, 448                                                   # 28 chunks per row; segments of 192 and 256
+    kb = [0, 192, K]
+    H = np.concatenate([rs.normal(0, 1.5, (M, 192)), rs.normal(0, 3.0, (M, K - 192)), rs.normal(0, 2.0, (M, K))],
+                       axis=1).astype(np.float32)
+    H[0, :8] = [0.0, -0.0, 5.0, -5.0, 1e-20, 100.0, -100.0, 3.0]
+    H[0, K:K + 8] = [1.0, 1.0, -9.0, 9.0, 1.0, -40.0, 40.0, 0.0]
+    if dtype == "bf16":
+        Hd = torch.from_numpy(H).to(torch.bfloat16)
+        H = Hd.float().numpy()
+    else:
+        Hd = torch.from_numpy(H)
+    mult = rs.uniform(0.5, 2.0, K).astype(np.float32)
+    qmax, qmin_abs = QRANGE[code]
+    a_ref, exact = O.activation_gated(H, dtype)
+    s_pos, s_neg = O.calib_act(O.smooth(a_ref[:256], mult), kb, dual, q_max=qmax, q_min_abs=qmin_abs)
+    seg = B.SegTable(kb, [0, 64])
+    c_pos, c_neg = B.segquant_quantize_act_fused(Hd.to(DEV), seg, torch.from_numpy(s_pos).to(DEV),
+                                                 torch.from_numpy(s_neg).to(DEV) if dual else None, code, act="geglu",
+                                                 mult=torch.from_numpy(mult).to(DEV))
+    torch.cuda.synchronize()
+    assert tuple(c_pos.shape) == (M, K)
+    dt = np.int8 if code == "int8" else np.uint8
+    g_pos = c_pos.cpu().numpy().view(dt)
+    g_neg = c_neg.cpu().numpy().view(dt) if dual else None
+    gate = H[:, K:].astype(np.float64)
+    eps = (3.0 * gate ** 2 + 49.0) * 2.0 ** -24
+    lo, hi = exact * (1 - np.sign(exact) * eps), exact * (1 + np.sign(exact) * eps)
+    if dtype == "bf16":
+        rnd = lambda v: (O.bf16_bits(v).astype(np.uint32) << 16).view(np.float32)
+    else:
+        rnd = lambda v: v.astype(np.float32)
+    tiny = np.abs(exact) < 2.0 ** -100
+    ok = np.zeros((M, K), bool)
+    first = None
+    for j, a in enumerate([a_ref, rnd(lo), rnd(hi), np.zeros_like(a_ref)]):
+        r_pos, r_neg = O.quantize_act(O.smooth(a, mult), kb, s_pos, s_neg, code=code, q_max=qmax, q_min_abs=qmin_abs)
+        same = (g_pos == r_pos) & ((g_neg == r_neg) if dual else True)
+        if first is None:
+            first = same
+        ok |= same if j < 3 else (same & tiny)
+    assert ok.all(), f"{(~ok).sum()} codes are neither the oracle's nor a neighbour's"
+    assert first.mean() > 0.999, f"only {first.mean():.5f} of the codes equal the oracle's"
+
+
+def test_fused_gated_gelu_rejects_a_gate_half_off_the_16_byte_grid():
+    H = torch.zeros(8, 2 * 36, dtype=torch.bfloat16, device=DEV)       # K = 36: the gate half starts at byte 72
+    seg = B.SegTable([0, 36], [0, 8])
+    s = torch.ones(1, device=DEV)
+    with pytest.raises(RuntimeError, match="ALIGN"):
+        B.segquant_quantize_act_fused(H, seg, s, s, "int8", act="geglu")
+
+
 # ------------------------------------------------------------------ W4A8: per-channel 4-bit weights, per-token scales
 
 def run_w4a8_parity(spec):
