@@ -152,6 +152,7 @@ class BenchLayer:
             self.zp = {"s_x": s_x, "z_x": z_x, "codes": B.new_codes(self.M, spec.K, device),
                        "bias": B.segquant_fold_zero_point(L.Wq, L.seg, s_x, z_x, L.s_w, L.bias)}
         self.a_stage = torch.empty_like(self.X) if (spec.dual and self.act) else None
+        self.ws_split = None
         # gated GELU: the pre-activation row holds a value half and a gate half (timing only: any values do)
         self.H2 = torch.cat([self.X, self.X], dim=1).contiguous() if self.act == "geglu" else None
         self.g_stage = torch.empty_like(self.X) if self.act == "geglu" else None
@@ -231,6 +232,23 @@ class BenchLayer:
         self.B.segquant_w4a8_gemm(self.c_pos, self.c_neg, w["w8"], self.seg4, w["s_pos"], w["s_neg"], w["s_w"],
                                   self.layer.bias, self.layer.workspace, Y=self.Y)
 
+    def gemm_split(self):
+        """The layer's GEMM with tiles split along K across CTA pairs (the larger workspace; forced, whatever the
+        automatic choice would be).  Timing only."""
+        if self.ws_split is None:
+            self.ws_split = self.B.new_workspace(self.X.device, split_for=(self.M, self.spec.N, self.spec.dual))
+        L = self.layer
+        self.B.segquant_set_tuning(0, 0, 0, 6)
+        try:
+            if L.dual:
+                self.B.segquant_dualscale_gemm(self.c_pos, self.c_neg, L.Wq, L.seg, L.code, L.s_pos, L.s_neg, L.s_w,
+                                               L.bias, self.ws_split, Y=self.Y)
+            else:
+                self.B.segquant_seglinear_gemm(self.c_pos, L.Wq, L.seg, L.code, L.s_pos, L.s_w, L.bias, self.ws_split,
+                                               Y=self.Y)
+        finally:
+            self.B.segquant_set_tuning(0, 0, 0, 0)
+
     def gemm_plain(self):
         """The same shape as a plain single-scale W8A8 layer (one code matrix): the denominator of the
         DualScale overhead.  Timing only; its output is not checked."""
@@ -260,7 +278,7 @@ class BenchLayer:
         for name in ("Wq", "s_w", "bias", "s_pos", "s_neg", "workspace"):
             t = getattr(self.layer, name)
             setattr(other.layer, name, None if t is None else t.clone())
-        for name in ("X", "c_pos", "c_neg", "Y", "a_stage", "H2", "g_stage"):
+        for name in ("X", "c_pos", "c_neg", "Y", "a_stage", "H2", "g_stage", "ws_split"):
             t = getattr(self, name)
             setattr(other, name, None if t is None else t.clone())
         if self.zp is not None:
@@ -307,7 +325,7 @@ def graph_time_per_launch(calls, rounds):
     return e0.elapsed_time(e1) * 1e3 / (rounds * len(calls))
 
 
-def time_kernels(layers, launches=48, max_copies=96, with_w4a8=True):
+def time_kernels(layers, launches=48, max_copies=96, with_w4a8=True, with_split=False):
     """Per-layer device time of each kernel, timed alone: a CUDA graph of >= `launches` launches of that one
     kernel, launch i on copy i mod C of the layer's device buffers, C chosen so that the copies the kernel walks
     through are at least twice the L2 capacity (every launch finds its operands in HBM).  A single launch between
@@ -315,7 +333,7 @@ def time_kernels(layers, launches=48, max_copies=96, with_w4a8=True):
     event pair around one small kernel reads 6-8 us more than the kernel's own span.
     Returns lists (quantize_us, gemm_us, plain_us | None, unsegmented_us | None, copies)."""
     out = {"q": [], "g": [], "plain": [], "unseg": [], "copies": [], "q_plain": [], "q_zp": [], "g_zp": [], "q_fused": [],
-           "act": [], "w4_q": [], "w4_unpack": [], "w4_g": []}
+           "act": [], "w4_q": [], "w4_unpack": [], "w4_g": [], "g_split": []}
     for bl in layers:
         s = bl.spec
         foot = min(quant_bytes(s, bl.M), gemm_bytes(s, bl.M))
@@ -334,6 +352,8 @@ def time_kernels(layers, launches=48, max_copies=96, with_w4a8=True):
         fused = s.dual and bl.act
         out["q_fused"].append(graph_time_per_launch([c.quantize_fused_act for c in copies], rounds) if fused else None)
         out["act"].append(graph_time_per_launch([c.act_unfused for c in copies], rounds) if fused else None)
+        split = with_split and s.P == 1 and bl.M > 128
+        out["g_split"].append(graph_time_per_launch([c.gemm_split for c in copies], rounds) if split else None)
         w4 = bl.w4 is not None and with_w4a8
         out["w4_q"].append(graph_time_per_launch([c.w4_quantize for c in copies], rounds) if w4 else None)
         out["w4_unpack"].append(graph_time_per_launch([c.w4_unpack for c in copies], rounds) if w4 else None)
@@ -612,6 +632,10 @@ def layer_table(specs, kt, peaks):
                          "gemm_us": us(kt["w4_g"][i]), "layer_time_over_w8a8_layer": round(w4_us / layer_us, 3),
                          "note": "per-channel 4-bit weights kept packed and unpacked in front of the GEMM, per-token "
                                  "activation scales; the GEMM runs the variant with per-(token, channel) factors"}
+        if kt["g_split"][i] is not None:
+            r["split_tiles"] = {"gemm_us": us(kt["g_split"][i]), "time_over_whole_tiles": round(kt["g_split"][i] / (g * 1e3), 3),
+                                "note": "K loops cut across CTA pairs with the partial sums exchanged through the larger "
+                                        "workspace, forced for this measurement; the automatic choice is the other column"}
         if kt["q_fused"][i] is not None:
             r["fused_act"] = {"act": s.x_kind.partition("+")[2], "fused_quant_us": us(kt["q_fused"][i]),
                               "unfused_act_us": us(kt["act"][i]), "unfused_pair_us": us(kt["act"][i] + q * 1e3),
@@ -636,7 +660,7 @@ def measure_side_workload(name, dev, args, peaks):
     specs = WL.WORKLOADS[name]
     layers = [BenchLayer(s, dev) for s in specs]
     time.sleep(COOL_DOWN_S)                    # the power state of the previous long region must not leak in
-    kt = time_kernels(layers, with_w4a8=name in ("dit_xl2", "sd3_heads"))
+    kt = time_kernels(layers, with_w4a8=name in ("dit_xl2", "sd3_heads"), with_split=name in ("dit_xl2", "sdxl_geglu"))
     for bl in layers:
         bl.layer.check_status()
     sets, set_bytes, n_sets = buffer_sets(layers)

@@ -74,6 +74,19 @@ typedef struct {
  * once by the caller after allocating it.  Two calls that may run concurrently need two workspaces. */
 size_t segquant_workspace_bytes(void);
 
+/* Optional larger workspace for the GEMM entry points (and the plan): with at least this many bytes -- zero-filled
+ * once, like the small one -- a layer with ONE K-segment whose output tiles would leave a good part of the GPU idle
+ * (fewer tiles than SM pairs, or a small last wave) is computed with SPLIT tiles: the K loop of every tile is cut so
+ * that all SM pairs get the same number of K-blocks, the CTAs that worked on part of a tile leave their raw
+ * accumulators in this workspace, and the last of them to finish adds them up (exact int32 sums for int8 codes;
+ * fp32 sums in the order of the K ranges for e4m3, within the tolerance of the fp32 epilogue) and runs the usual
+ * epilogue (Sec. 4.2.2 / 4.3.2 products unchanged: the accumulators are the same sums).  Nothing waits inside the
+ * kernel.  The size depends on the device (its SM count; about 38 MB on a 148-SM GPU) and weakly on M and N
+ * (dual != 0 for the DualScale entry point).  Returns 0 if the device cannot be queried.  The counters in it are
+ * left at zero by every completed launch; after SQ_ERR_TIMEOUT zero-fill the workspace again.  Layers that do not
+ * qualify, and smaller workspaces, run exactly as before. */
+size_t segquant_split_workspace_bytes(int64_t M, int64_t N, int dual);
+
 /* Step "calibration" -- Sec. 4.3.2 scale formula (s_- = |min x| / |q_min|, s_+ = max x / q_max),
  * strict min/max (App. B, Dual Scale Sensitivity Analysis), one scalar per segment (App. B,
  * per-tensor 8-bit scheme; Sec. 4.2.2 "independently within each segment").
@@ -307,7 +320,8 @@ sq_status segquant_last_device_status(void *workspace, void *stream, uint32_t *d
  * segments pass through tensor memory one after the other, running sums in registers), 1 (all
  * accumulators of a tile resident in tensor memory; at most 16 of them), 2 (sequential) or 4
  * (automatic, but single-scale layers keep 256 x 256 tiles instead of 256 x 512 ones) or 5 (256 x 512
- * tiles for single-scale layers even where the automatic choice expects no gain from them).
+ * tiles for single-scale layers even where the automatic choice expects no gain from them), 6 (split
+ * tiles wherever the layer and the workspace allow them) or 7 (never split tiles).
  * Process-wide (atomic words read when a launch or a plan is prepared); meant for benchmarking sweeps and
  * tests only: production callers leave everything automatic.  Values the layer cannot use are replaced by the
  * automatic choice. */

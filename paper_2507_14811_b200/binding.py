@@ -29,6 +29,7 @@ EXPORTS = [
     "segquant_status_string", "segquant_quantize_act_fused", "segquant_calib_zero_point",
     "segquant_quantize_act_zero_point", "segquant_fold_zero_point", "segquant_plan_layer", "segquant_plan_run",
     "segquant_quantize_per_row", "segquant_pack_w4", "segquant_unpack_w4", "segquant_w4a8_gemm",
+    "segquant_split_workspace_bytes",
 ]
 
 
@@ -53,6 +54,8 @@ def lib():
             raise RuntimeError(f"{LIB_PATH} not found: build it with `python -m paper_2507_14811_b200.build`")
         L = C.CDLL(LIB_PATH)
         L.segquant_workspace_bytes.restype = C.c_size_t
+        L.segquant_split_workspace_bytes.restype = C.c_size_t
+        L.segquant_split_workspace_bytes.argtypes = [C.c_int64, C.c_int64, C.c_int]
         L.segquant_layer_scratch_bytes.restype = C.c_size_t
         L.segquant_layer_scratch_bytes.argtypes = [C.c_int64, C.c_int64, C.c_int]
         L.segquant_launch_count.restype = C.c_uint64
@@ -111,9 +114,19 @@ def workspace_bytes() -> int:
     return int(lib().segquant_workspace_bytes())
 
 
-def new_workspace(device="cuda") -> torch.Tensor:
-    """Zero-filled, 256-byte aligned device scratch for the calls below."""
-    return torch.zeros(workspace_bytes(), dtype=torch.uint8, device=device)
+def split_workspace_bytes(M: int, N: int, dual: bool) -> int:
+    """Size of the larger workspace that lets the GEMM calls split tiles for an [M, N] output (current device)."""
+    return int(lib().segquant_split_workspace_bytes(C.c_int64(M), C.c_int64(N), C.c_int(int(dual))))
+
+
+def new_workspace(device="cuda", split_for=None) -> torch.Tensor:
+    """Zero-filled, 256-byte aligned device scratch for the calls below.  split_for=(M, N, dual) makes it large
+    enough for the GEMM calls to split tiles of such a layer."""
+    n = workspace_bytes()
+    if split_for is not None:
+        with torch.cuda.device(device):
+            n = max(n, split_workspace_bytes(*split_for))
+    return torch.zeros(n, dtype=torch.uint8, device=device)
 
 
 def segquant_calib_scales(X: torch.Tensor, seg: SegTable, code: str, is_weight: bool, dual: bool,

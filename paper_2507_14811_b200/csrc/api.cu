@@ -95,6 +95,10 @@ static sq_status gemm_args(const void *a_pos, const void *a_neg, int dual, int64
     g.Y = Y; g.y_dtype = y_dtype; g.ldy = ldy;
     g.acc_dump = acc_dump;
     g.status = static_cast<uint32_t *>(workspace);
+    if (ws_bytes > kWsBytes) {           // a larger workspace: room for the partial sums of split tiles
+        g.sk_scratch = static_cast<uint8_t *>(workspace) + kWsBytes;
+        g.sk_bytes = ws_bytes - kWsBytes;
+    }
     return SQ_OK;
 }
 
@@ -126,6 +130,12 @@ using namespace sq;
 extern "C" {
 
 size_t segquant_workspace_bytes(void) { return kWsBytes; }
+
+size_t segquant_split_workspace_bytes(int64_t M, int64_t N, int dual)
+{
+    const size_t extra = gemm_split_scratch_bytes(M, N, dual);
+    return extra ? kWsBytes + extra : 0;
+}
 
 sq_status segquant_calib_scales(const void *X, sq_dtype dt, int64_t rows, int64_t K, int64_t ld,
                                 const sq_segtable *seg, sq_code code, int is_weight, int dual, uint32_t flags,

@@ -315,7 +315,59 @@ struct SharedHeader {
     uint64_t tmem_empty[2];
     uint32_t tmem_base;
     uint32_t abort_flag;
+    uint32_t sk_flag;            // (split tiles) the arrival count the CTA's thread 0 read, for the other epilogue threads
 };
+
+// Split tiles (SK variants): the work of a launch is the sequence of all (tile, K-block) units, tile-major, cut
+// into one contiguous range per CTA pair: pair c takes units [c U / C, (c + 1) U / C).  A range is walked as
+// segments (tile, K-blocks k0 .. k1 - 1); a segment that is not a whole tile is a PARTIAL one.  Every role of a
+// CTA walks the same sequence.
+struct SkWalk {
+    int u, u_begin, u_end, kblocks;
+};
+__device__ __forceinline__ int sk_bound(int c, int total_units, int pairs)
+{
+    return int((long long)c * total_units / pairs);
+}
+__device__ __forceinline__ SkWalk sk_range(int pair, int pairs, int num_tiles, int kblocks)
+{
+    const int total = num_tiles * kblocks;
+    SkWalk w;
+    w.u_begin = sk_bound(pair, total, pairs);
+    w.u_end = sk_bound(pair + 1, total, pairs);
+    w.u = w.u_begin;
+    w.kblocks = kblocks;
+    return w;
+}
+__device__ __forceinline__ bool sk_next(SkWalk &w, int &tile, int &k0, int &k1)
+{
+    if (w.u >= w.u_end) return false;
+    tile = w.u / w.kblocks;
+    k0 = w.u - tile * w.kblocks;
+    const int rem = w.u_end - w.u;
+    k1 = k0 + rem < w.kblocks ? k0 + rem : w.kblocks;
+    w.u += k1 - k0;
+    return true;
+}
+// the pair whose range holds unit x: the largest c with c U / C <= x
+__device__ __forceinline__ int sk_owner(int x, int total_units, int pairs)
+{
+    return int((((long long)x + 1) * pairs - 1) / total_units);
+}
+// barrier 1 of the 256 epilogue threads, returning the AND of their predicates
+__device__ __forceinline__ bool epilogue_all(bool pred)
+{
+    uint32_t r;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %1, 0;\n\tbar.red.and.pred q, 1, 256, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+                 : "=r"(r) : "r"(uint32_t(pred)) : "memory");
+    return r != 0;
+}
+__device__ __forceinline__ uint4 ld_global_cg_16(const uint4 *p)
+{
+    uint4 v;
+    asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
 
 // where-codes written to the status word when a wait expires
 enum : uint32_t { kWhereProducer = 0x100, kWhereMmaFull = 0x200, kWhereMmaTmem = 0x300, kWhereEpilogue = 0x400 };
@@ -629,7 +681,12 @@ __device__ __forceinline__ void store_slab(const uint64_t (&y2)[16], const Param
 // issuing thread and accumulator, and is released to its thread separately, like the polarities of a dual tile.
 // PT = true: the production variant for layers with per-token and per-channel scales (W4A8): the tile's channel
 // scales are staged in shared memory and every factor is the token's scale times the channel's.
-template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ, bool WIDE = false, bool PT = false>
+// SK = true (one K-segment, CTA pairs, layers whose tile count fills the machine badly): the K loops of the tiles
+// are cut so that every CTA pair gets the same number of K-blocks (SkWalk above).  A CTA that has worked on part
+// of a tile's K range writes its raw accumulators (exact int32 sums, or fp32 ones) to a slot of the caller's
+// workspace and counts itself in on the tile's counter; the CTA whose count completes the tile adds the slots up,
+// in the order of the K ranges, and runs the tile's epilogue.  Nobody waits for anybody.
+template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ, bool WIDE = false, bool PT = false, bool SK = false>
 // 384 threads = 12 warps, 3 on each SM sub-partition with 16 K registers: 168 registers per thread at launch
 __global__ void __launch_bounds__(kThreads, 1)
 segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_constant__ CUtensorMap tm_a_neg,
@@ -645,6 +702,7 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     constexpr int kTileCols = TILE_N * kHalves;          // output columns of a tile
     constexpr int kIssuers = (NPOL == 2 || WIDE) ? 2 : 1;
     static_assert(!WIDE || (NPOL == 1 && TILE_N == 256 && CG == 2 && !GENERIC && !SEQ), "wide single-scale tile");
+    static_assert(!SK || (CG == 2 && !GENERIC && !SEQ && !WIDE && !PT && NPOL * TILE_N == 256), "split tiles");
     constexpr uint32_t stage_bytes = NPOL * a_bytes + kHalves * b_bytes;
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t *sh_stage = smem + size_t(prm.stages) * stage_bytes;      // 1 KiB aligned: stages are multiples of 1 KiB
@@ -708,7 +766,8 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
     // (barrier tmem_empty[0] = positive accumulator free, tmem_empty[1] = negative one): the epilogue reads all
     // positive columns first, and the thread that issues the positive MMAs starts the next tile as soon as they
     // are in registers, ahead of the negative thread by at most the depth of the ring.
-    constexpr bool kSplitRel = (NPOL == 2 && TILE_N == 256 && !SEQ && !GENERIC) || WIDE;
+    constexpr bool kSplitRel = (NPOL == 2 && TILE_N == 256 && !SEQ && !GENERIC && !SK) || WIDE;
+    const int sk_pairs = min(num_units, num_tiles * prm.sk_kblocks);    // (SK) pairs that have a range
 
     // The producer and the MMA issuer are single threads: their loops are kept to a few dozen
     // instructions per K-block (ring slot and phase advance incrementally, descriptors by addition).
@@ -725,7 +784,29 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
             const uint32_t ring0 = smem_u32(smem);
             uint32_t s = 0, ph = 0, issued = 0;
             bool ok = true;
-            for (int tile = unit; tile < num_tiles && ok; tile += num_units) {
+            if constexpr (SK) {
+                SkWalk w = sk_range(unit, sk_pairs, num_tiles, prm.sk_kblocks);
+                int tile = 0, k0 = 0, k1 = 0;
+                while (ok && unit < sk_pairs && sk_next(w, tile, k0, k1)) {
+                    const int m0 = (tile / prm.num_n_tiles) * (TILE_M * CG) + int(rank) * TILE_M;
+                    const int n0 = (tile % prm.num_n_tiles) * kTileCols + int(rank) * B_ROWS;
+                    for (int kbi = k0; kbi < k1; kbi++) {
+                        if (!mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag, prm.status, kWhereProducer)) {
+                            ok = false;
+                            break;
+                        }
+                        const uint32_t dst = ring0 + s * stage_bytes;
+                        if (rank == 0) mbar_expect_tx(full0 + 8 * s, CG * stage_bytes);
+                        const uint32_t bar = full0_sig + 8 * s;
+                        tma_load_2d<CG>(dst, &tm_a_pos, bar, kbi * BLOCK_K, m0);
+                        if (NPOL == 2) tma_load_2d<CG>(dst + a_bytes, &tm_a_neg, bar, kbi * BLOCK_K, m0);
+                        tma_load_2d<CG>(dst + NPOL * a_bytes, &tm_b, bar, kbi * BLOCK_K, n0);
+                        issued++;
+                        if (++s == stages) { s = 0; ph ^= 1; }
+                    }
+                }
+            }
+            for (int tile = unit; !SK && tile < num_tiles && ok; tile += num_units) {
                 const int m0 = (tile / prm.num_n_tiles) * (TILE_M * CG) + int(rank) * TILE_M;
                 const int n0 = (tile % prm.num_n_tiles) * kTileCols + int(rank) * B_ROWS;
                 for (uint32_t p = 0; p < P && ok; p++) {
@@ -780,7 +861,36 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                                         : (uint64_t(NPOL * a_bytes) >> 4) - pol * (uint64_t(a_bytes) >> 4);
             uint32_t s = 0, ph = 0, as = 0, aph = 0;
             bool ok = true;
-            for (int tile = unit; tile < num_tiles && ok; tile += num_units) {
+            if constexpr (SK) {
+                SkWalk w = sk_range(unit, sk_pairs, num_tiles, prm.sk_kblocks);
+                int tile = 0, k0 = 0, k1 = 0;
+                while (ok && unit < sk_pairs && sk_next(w, tile, k0, k1)) {
+                    if (!mbar_wait(smem_u32(&hdr->tmem_empty[as]), aph ^ 1, abort_flag, prm.status, kWhereMmaTmem)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t d0 = tmem_base + as * acc_cols + pol * TILE_N;
+                    uint32_t accumulate = 0;                       // a segment starts from zero wherever it begins in K
+                    for (int kbi = k0; kbi < k1; kbi++) {
+                        if (!mbar_wait(full0 + 8 * s, ph, abort_flag, prm.status, kWhereMmaFull)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint64_t da = desc0 + s * kStageDesc;
+                        const int rem = prm.K - kbi * BLOCK_K;
+                        const int nk = rem >= BLOCK_K ? BLOCK_K / MMA_K : (rem + MMA_K - 1) / MMA_K;
+                        issue_kblock<KIND, 1, TILE_N, CG>(d0, da, da + b_off, idesc, nk, accumulate);
+                        accumulate = 1;
+                        tc_commit<CG>(empty0 + 8 * s);
+                        if (++s == stages) { s = 0; ph ^= 1; }
+                    }
+                    if (ok) tc_commit<CG>(smem_u32(&hdr->tmem_full[as]));
+                    if (++as == acc_stages) { as = 0; aph ^= 1; }
+                }
+            }
+            for (int tile = unit; !SK && tile < num_tiles && ok; tile += num_units) {
                 if (!SEQ) {
                     const uint32_t bar = smem_u32(&hdr->tmem_empty[kSplitRel ? pol : as]);
                     if (!mbar_wait(bar, aph ^ 1, abort_flag, prm.status, kWhereMmaTmem)) {
@@ -859,7 +969,8 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
             return n < prm.N ? __ldg(prm.bias + n) : 0.0f;
         };
         grid_dependency_wait();                     // scales, bias and Y may belong to the previous kernel
-        float bias_next = fetch_bias(unit);
+        SkWalk skw = sk_range(SK ? unit : 0, SK ? max(sk_pairs, 1) : 1, SK ? num_tiles : 0, SK ? prm.sk_kblocks : 1);
+        float bias_next = fetch_bias(SK ? (unit < sk_pairs ? skw.u_begin / max(prm.sk_kblocks, 1) : num_tiles) : unit);
         float bias_next1 = WIDE ? fetch_bias(unit, 1) : 0.0f;   // second half of a wide tile
         // dequantization factors c[a][q] = s_act[p][pol] * s_w[p][q], a = p * NPOL + pol (one fp32 multiply);
         // built here, off the producer's and the MMA issuer's path, and published by the first tile's barrier
@@ -890,7 +1001,19 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
         YOut yo{&tm_y, smem_u32(sh_stage) + uint32_t(ew) * kStageBytesPerWarp, lane, 0};
         uint32_t as = 0, aph = 0;
         bool ok = true;
-        for (int tile = unit; tile < num_tiles; tile += num_units) {
+        int tile = unit - num_units;
+        while (true) {
+            int sk_k0 = 0, sk_k1 = 0, next_tile = 0;          // (SK) this segment's K-blocks; the tile after this one
+            if constexpr (SK) {
+                if (unit >= sk_pairs || !sk_next(skw, tile, sk_k0, sk_k1)) break;
+                SkWalk peek = skw;
+                int pk0, pk1;
+                if (!sk_next(peek, next_tile, pk0, pk1)) next_tile = num_tiles;
+            } else {
+                tile += num_units;
+                if (tile >= num_tiles) break;
+                next_tile = tile + num_units;
+            }
             const int m0 = (tile / prm.num_n_tiles) * (TILE_M * CG) + int(rank) * TILE_M;
             const int n0 = (tile % prm.num_n_tiles) * kTileCols;
             const int row = m0 + lane_grp * 32 + lane;
@@ -905,10 +1028,10 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                     sh_col[i] = n0 + c < prm.N ? __ldg(prm.col_scale + size_t(n0 + c) * P + pp) : 0.0f;
                 }
             }
-            bias_next = fetch_bias(tile + num_units);                        // lands during this tile's work
+            bias_next = fetch_bias(next_tile);                               // lands during this tile's work
             if (WIDE) {
                 sh_bias[TILE_N + et] = bias_next1;                           // et < 256 = TILE_N for every epilogue thread
-                bias_next1 = fetch_bias(tile + num_units, 1);
+                bias_next1 = fetch_bias(next_tile, 1);
             }
             asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
 
@@ -973,10 +1096,127 @@ segquant_gemm_kernel(const __grid_constant__ CUtensorMap tm_a_pos, const __grid_
                 const uint32_t cur_as = as, cur_aph = aph;
                 if (++as == uint32_t(prm.acc_stages)) { as = 0; aph ^= 1; }
                 if (ok) ok = mbar_wait(smem_u32(&hdr->tmem_full[cur_as]), cur_aph, abort_flag, prm.status, kWhereEpilogue);
+                if constexpr (SK) ok = epilogue_all(ok);    // the barriers below need all 256 threads or none
                 if (!ok) continue;                  // keep the named barriers balanced, do no more work
                 tc_fence_after();
                 const uint32_t t_row = tmem_base + (uint32_t(lane_grp * 32) << 16) + cur_as * acc_cols;
                 constexpr bool kEvenSplit = kSlabsPerWarp * kColGroups == kSlabs;
+                if constexpr (SK) {
+                    const int kbt = prm.sk_kblocks;
+                    if (!(sk_k0 == 0 && sk_k1 == kbt)) {
+                        // ---- part of a tile's K range.  n pairs share the tile; the one that holds its first K-blocks
+                        // (the OWNER; that segment is the last of its range, the others' segments the first of theirs)
+                        // normally finds the other n - 1 partial sums waiting and finishes the tile from its own
+                        // accumulators in TMEM plus their slots.  Counter protocol, without any waiting: a non-owner
+                        // writes its slot, then adds 1; the owner adds 1 first, and if that did not read n - 1 it
+                        // writes its slot too and adds 1 again.  Whoever brings the count to n + 1 (or the owner
+                        // reading n - 1) finishes the tile, from the slots alone in the first case.
+                        static_assert(!SK || kEvenSplit, "split tiles: every warp has the same number of slabs");
+                        constexpr int kUnits = kSlabsPerWarp * NPOL;
+                        constexpr size_t kSlotBytes = size_t(NPOL) * TILE_M * TILE_N * 4;   // one CTA's accumulators
+                        const int total = num_tiles * kbt, tile_u0 = tile * kbt;
+                        // slot 0 of a pair: the segment that starts the pair's range; slot 1: its other partial one
+                        auto slot_of = [&](int pair, int seg_u0) {
+                            const int sl = seg_u0 == sk_bound(pair, total, sk_pairs) ? 0 : 1;
+                            return reinterpret_cast<uint4 *>(prm.sk_slots + size_t((pair * 2 + sl) * 2 + int(rank)) * kSlotBytes) + et;
+                        };
+                        const uint32_t t_warp = t_row + uint32_t(slab0 * 32);
+                        uint32_t *cnt = prm.sk_counters + tile * 2 + int(rank);
+                        const int c_first = sk_owner(tile_u0, total, sk_pairs), c_last = sk_owner(tile_u0 + kbt - 1, total, sk_pairs);
+                        const int sharers = c_last - c_first + 1;
+                        auto count_in = [&]() -> int {             // all 256 threads; returns the count before this arrival
+                            asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+                            if (et == 0) {
+                                const uint32_t before = atomicAdd(cnt, 1u);
+                                __threadfence();
+                                st_shared_volatile_u32(smem_u32(&hdr->sk_flag), before);
+                            }
+                            asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+                            return int(ld_shared_volatile_u32(smem_u32(&hdr->sk_flag)));
+                        };
+                        bool from_tmem = false;                    // finishing with this CTA's own sums still in TMEM
+                        bool finish = false;
+                        if (sk_k0 == 0) {
+                            from_tmem = finish = count_in() == sharers - 1;
+                        }
+                        if (!from_tmem) {
+                            uint4 *mine = slot_of(unit, tile_u0 + sk_k0);
+                            uint32_t buf[2][32];
+                            tc_ld32(t_warp, buf[0]);
+#pragma unroll
+                            for (int u = 0; u < kUnits; u++) {
+                                tc_wait_ld();
+                                if (u + 1 < kUnits)
+                                    tc_ld32(t_warp + uint32_t(((u + 1) % NPOL) * TILE_N + ((u + 1) / NPOL) * 32), buf[(u + 1) & 1]);
+                                else
+                                    release(cur_as);
+#pragma unroll
+                                for (int j = 0; j < 8; j++)          // 512 consecutive bytes per warp and store
+                                    st_global_16(mine + (u * 8 + j) * kEpiThreads,
+                                                 make_uint4(buf[u & 1][4 * j], buf[u & 1][4 * j + 1], buf[u & 1][4 * j + 2], buf[u & 1][4 * j + 3]));
+                            }
+                            __threadfence();
+                            finish = count_in() == sharers;         // n + 1 arrivals with this one
+                        }
+                        if (!finish) continue;
+                        // ---- this CTA completes the tile: the sums of the K ranges in ascending order, then the usual
+                        // epilogue.  The counter goes back to zero for the next launch.
+                        if (et == 0) *cnt = 0u;
+#pragma unroll 1
+                        for (int sl = 0; sl < kSlabsPerWarp; sl++) {
+                            const int c0 = (slab0 + sl) * 32, nf = n0 + c0;
+                            const int q = seg_of_column(nf, Q, nb_addr, lane);
+                            uint64_t y2[16];
+#pragma unroll
+                            for (int pol = 0; pol < NPOL; pol++) {
+                                const int u = sl * NPOL + pol;
+                                uint32_t acc[32];
+                                if (from_tmem) {                   // the owner's range is the first in K (c_first == unit)
+                                    tc_ld32(t_warp + uint32_t(pol * TILE_N + sl * 32), acc);
+                                    tc_wait_ld();
+                                } else {
+#pragma unroll
+                                    for (int j = 0; j < 32; j++) acc[j] = 0u;
+                                }
+                                // two slots' loads (16 of 16 bytes) are in flight before the first add
+                                for (int c = c_first + (from_tmem ? 1 : 0); c <= c_last; c += 2) {
+                                    const bool two = c + 1 <= c_last;
+                                    const uint4 *src0 = slot_of(c, max(sk_bound(c, total, sk_pairs), tile_u0)) + u * 8 * kEpiThreads;
+                                    const uint4 *src1 = two ? slot_of(c + 1, max(sk_bound(c + 1, total, sk_pairs), tile_u0)) + u * 8 * kEpiThreads
+                                                            : src0;
+                                    uint4 v[2][8];
+#pragma unroll
+                                    for (int j = 0; j < 8; j++) v[0][j] = ld_global_cg_16(src0 + j * kEpiThreads);
+                                    if (two) {
+#pragma unroll
+                                        for (int j = 0; j < 8; j++) v[1][j] = ld_global_cg_16(src1 + j * kEpiThreads);
+                                    }
+#pragma unroll
+                                    for (int h = 0; h < 2; h++) {
+                                        if (h == 1 && !two) break;
+#pragma unroll
+                                        for (int j = 0; j < 8; j++) {
+                                            const uint32_t w[4] = {v[h][j].x, v[h][j].y, v[h][j].z, v[h][j].w};
+#pragma unroll
+                                            for (int t = 0; t < 4; t++)
+                                                acc[4 * j + t] = KIND == 0 ? acc[4 * j + t] + w[t]
+                                                                           : __float_as_uint(__uint_as_float(acc[4 * j + t]) + __uint_as_float(w[t]));
+                                        }
+                                    }
+                                }
+                                const TokenScale tk = token_scale(pol, row);
+                                if (pol == 0)
+                                    scale_add_unit<KIND, false, true, false>(y2, acc, 0, Q, q, q, nf, tab_addr, nb_addr,
+                                                                             bias_addr + uint32_t(c0) * 4u, &tk);
+                                else
+                                    scale_add_unit<KIND, false, false, false>(y2, acc, pol, Q, q, q, nf, tab_addr, nb_addr, 0, &tk);
+                            }
+                            store_slab<GENERIC>(y2, prm, row, nf, yo);
+                        }
+                        if (from_tmem) release(cur_as);
+                        continue;
+                    }
+                }
                 if constexpr (WIDE) {
                     // two independent 256-column halves, four slabs of each per warp: all units of half 0 first
                     // (then its accumulator goes back), two of half 1, and the last two of half 1 into the
@@ -1240,7 +1480,14 @@ sq_status kernel_facts(int device, Kern kern, size_t smem, int cg, const cudaLau
     return SQ_OK;
 }
 
-template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ, bool WIDE = false, bool PT = false>
+// Split tiles hold 256 accumulator columns per CTA (two sets fit in TMEM, and a CTA's partial sums are 128 KiB):
+// 256-column tiles for single-scale layers, 128-column tiles for dual ones.  (256-column dual tiles were measured
+// too: twice the partial sums to exchange, one accumulator set, slower on every shape tried.)
+constexpr int sk_tile_n(int npol) { return npol == 2 ? 128 : 256; }
+constexpr size_t kSkSlotBytes = size_t(TILE_M) * 256 * 4;                  // one CTA's accumulators of such a tile
+inline size_t sk_counter_bytes(int64_t tiles) { return size_t((tiles * 2 * 4 + 255) / 256 * 256); }
+
+template <int KIND, int NPOL, int TILE_N, int CG, bool GENERIC, bool SEQ, bool WIDE = false, bool PT = false, bool SK = false>
 sq_status prepare_variant(const GemmArgs &g, GemmLaunch &L, int device, int sm_count)
 {
     constexpr int kTileCols = TILE_N * (WIDE ? 2 : 1);
@@ -1267,7 +1514,7 @@ sq_status prepare_variant(const GemmArgs &g, GemmLaunch &L, int device, int sm_c
     prm.num_n_tiles = int((g.N + kTileCols - 1) / kTileCols);
     const size_t smem = 1024 + size_t(stages) * stage_bytes + tail;
 
-    auto kern = segquant_gemm_kernel<KIND, NPOL, TILE_N, CG, GENERIC, SEQ, WIDE, PT>;
+    auto kern = segquant_gemm_kernel<KIND, NPOL, TILE_N, CG, GENERIC, SEQ, WIDE, PT, SK>;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(unsigned(sm_count / CG * CG));
     cfg.blockDim = dim3(kThreads);
@@ -1288,6 +1535,20 @@ sq_status prepare_variant(const GemmArgs &g, GemmLaunch &L, int device, int sm_c
     const int tiles = prm.num_m_tiles * prm.num_n_tiles;
     L.kernel = reinterpret_cast<const void *>(kern);
     L.grid = unsigned((tiles < units ? tiles : units) * CG);
+    if (SK) {
+        // every pair gets the same share of all (tile, K-block) units; two slots per pair and CTA for its partial
+        // segments, one counter per tile and CTA of the pair
+        static_assert(!SK || size_t(NPOL) * TILE_M * TILE_N * 4 == kSkSlotBytes, "slot size");
+        const int64_t kblocks = (g.K + BLOCK_K - 1) / BLOCK_K, total = int64_t(tiles) * kblocks;
+        if (total > 0x3FFFFFFF) return SQ_ERR_UNSUPPORTED;
+        const int pairs = int(total < units ? total : units);
+        const size_t need = sk_counter_bytes(tiles) + size_t(pairs) * 4 * kSkSlotBytes;
+        if (!g.sk_scratch || g.sk_bytes < need) return SQ_ERR_WORKSPACE;
+        prm.sk_counters = static_cast<uint32_t *>(g.sk_scratch);
+        prm.sk_slots = static_cast<uint8_t *>(g.sk_scratch) + sk_counter_bytes(tiles);
+        prm.sk_kblocks = int(kblocks);
+        L.grid = unsigned(pairs * CG);
+    }
     L.cluster = CG;
     L.smem = smem;
     L.device = device;
@@ -1328,8 +1589,32 @@ sq_status prepare_tile(const GemmArgs &g, GemmLaunch &L, int tile_n, bool seq, i
     const int64_t n256 = (g.N + 255) / 256, m_pairs = (g.M + 2 * TILE_M - 1) / (2 * TILE_M), units = sm_count / 2;
     const int64_t waves_256 = (m_pairs * n256 + units - 1) / units;
     const int64_t waves_wide = (m_pairs * ((n256 + 1) / 2) + units - 1) / units;
-    if (NPOL == 1 && CG == 2 && !dbg && tile_n == 256 && prm.sb.P == 1 && tune_seq != 4 &&
-        (n256 % 2 == 0 || n256 >= 9) && (tune_seq == 5 || 2 * waves_wide * 94 < waves_256 * 100)) {
+    const bool wide = NPOL == 1 && CG == 2 && !dbg && tile_n == 256 && prm.sb.P == 1 && tune_seq != 4 &&
+                      (n256 % 2 == 0 || n256 >= 9) && (tune_seq == 5 || 2 * waves_wide * 94 < waves_256 * 100);
+    // Split tiles: one K-segment, CTA pairs, production output, and a tile count that leaves a good part of the
+    // last wave idle.  Time in K-blocks of 256 accumulator columns: whole tiles take waves x K-blocks; split
+    // tiles take their even share plus the exchange of partial sums (a fixed part and one slot read per pair
+    // that shares a tile, in K-block times; measured).  segment_mode 6 forces the split where it is possible, 7 forbids it.
+    if constexpr (CG == 2) {
+        if (!dbg && !pt && prm.sb.P == 1 && g.sk_scratch && tune_seq != 7) {
+            constexpr int TN = sk_tile_n(NPOL);
+            constexpr double kSkFixup = 30.0, kSkPerSharer = 10.0;
+            const int64_t pairs = sm_count / 2, m_tiles = (g.M + 2 * TILE_M - 1) / (2 * TILE_M);
+            const int64_t kblocks = (g.K + BLOCK_K - 1) / BLOCK_K;
+            const int64_t tiles_sk = m_tiles * ((g.N + TN - 1) / TN), tiles_dp = m_tiles * ((g.N + tile_n - 1) / tile_n);
+            double t_dp = double((tiles_dp + pairs - 1) / pairs) * double(kblocks) * (double(tile_n * NPOL) / 256.0);
+            if (wide) t_dp = double(2 * waves_wide) * 0.94 * double(kblocks);
+            // the CTA that completes a tile reads one slot per pair that worked on it
+            const double sharers = double(pairs) / double(tiles_sk) + 1.0;
+            const double t_sk = double(tiles_sk * kblocks) / double(pairs) + kSkFixup + kSkPerSharer * (sharers < 2.0 ? 2.0 : sharers);
+            const size_t need = sk_counter_bytes(tiles_sk) + size_t(pairs) * 4 * kSkSlotBytes;
+            if (g.sk_bytes >= need && tiles_sk * kblocks >= 2 && (tune_seq == 6 || t_sk < 0.9 * t_dp)) {
+                prm.acc_stages = 2;
+                return prepare_variant<KIND, NPOL, TN, 2, false, false, false, false, true>(g, L, device, sm_count);
+            }
+        }
+    }
+    if (wide) {
         prm.acc_stages = 1;
         return prepare_variant<KIND, 1, 256, 2, false, false, true>(g, L, device, sm_count);
     }
@@ -1357,6 +1642,16 @@ sq_status prepare_kind(const GemmArgs &g, GemmLaunch &L, int npol, int cg, int t
 }
 
 }  // namespace
+
+size_t gemm_split_scratch_bytes(int64_t M, int64_t N, int dual)
+{
+    int dev = 0, sm_count = 0;
+    if (M <= 0 || N <= 0 || cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count < 2)
+        return 0;
+    const int64_t tiles = ((M + 2 * TILE_M - 1) / (2 * TILE_M)) * ((N + sk_tile_n(dual ? 2 : 1) - 1) / sk_tile_n(dual ? 2 : 1));
+    return sk_counter_bytes(tiles) + size_t(sm_count / 2) * 4 * kSkSlotBytes;
+}
 
 void set_gemm_tuning(int tile_n, int stages, int cta_group, int segment_mode)
 {

@@ -120,6 +120,8 @@ struct GemmArgs {
     int64_t ldy;
     void *acc_dump;
     uint32_t *status;
+    void *sk_scratch;            // split tiles: zero-filled device scratch behind the workspace's fixed part, or nullptr
+    size_t sk_bytes;
 };
 // Parameters of the GEMM kernel (by value, constant bank).
 struct KernelParams {
@@ -138,6 +140,9 @@ struct KernelParams {
     int y_wide;        // rows of Y are 32-byte aligned: 256-bit stores allowed
     void *acc_dump;
     uint32_t *status;
+    uint32_t *sk_counters;       // split tiles: arrivals per (tile, CTA of the pair), zero between launches
+    uint8_t *sk_slots;           // split tiles: per (pair, slot, CTA) one CTA's raw accumulators
+    int sk_kblocks;              // split tiles: K-blocks per tile (0: tiles are not split)
 };
 
 // A GEMM launch worked out ahead of time: kernel instantiation, tensor maps, parameters, grid.
@@ -153,5 +158,7 @@ sq_status prepare_gemm(const GemmArgs &g, GemmLaunch *out);    // launches nothi
 sq_status run_gemm(const GemmLaunch &l, cudaStream_t st);      // one launch, no queries
 sq_status launch_gemm(const GemmArgs &g, cudaStream_t st);     // prepare + run
 void set_gemm_tuning(int tile_n, int stages, int cta_group, int segment_mode);
+// bytes behind the workspace's fixed part that let prepare_gemm split tiles for an [M, N] output on the current device
+size_t gemm_split_scratch_bytes(int64_t M, int64_t N, int dual);
 
 }  // namespace sq

@@ -32,6 +32,11 @@ class SegQuantLinear:
                                                          self.workspace, self.flags)
         return self.s_pos, self.s_neg
 
+    def allow_split_tiles(self, M: int):
+        """Replaces the workspace by the larger one with which the GEMM may split tiles along K for inputs of up
+        to M rows (used where the layer's output has too few tiles to fill the GPU; see the C header)."""
+        self.workspace = B.new_workspace(self.device, split_for=(M, self.N, self.dual))
+
     def scratch_for(self, M: int) -> torch.Tensor:
         need = B.layer_scratch_bytes(M, self.K, self.dual)
         if self._scratch is None or self._scratch.numel() < need:

@@ -22,8 +22,9 @@ def custom_spec(name, M, K, N, kb, nb, dual, code, x_dtype="bf16", x_kind="norma
                         x_kind=x_kind, w_kind=w_kind, seed=seed, cal_rows=cal_rows, x_seg_std=x_seg_std or [])
 
 
-def run_parity(spec, rows=None, flags=0, tile_n=0, cta_group=0, segment_mode=0):
-    """Full element-by-element parity of one layer.  rows: optional subset of rows the oracle computes."""
+def run_parity(spec, rows=None, flags=0, tile_n=0, cta_group=0, segment_mode=0, split=False):
+    """Full element-by-element parity of one layer.  rows: optional subset of rows the oracle computes.
+    split: give the layer the larger workspace, with which the bf16 call may split tiles along K."""
     data = WL.make_layer(spec)
     qmin_sym = bool(flags & B.SQ_FLAG_QMIN_SYM)
     s_pos, s_neg, s_w, Wq, (qmax, qmin_abs) = oracle_scales(data, qmin_sym)
@@ -31,6 +32,8 @@ def run_parity(spec, rows=None, flags=0, tile_n=0, cta_group=0, segment_mode=0):
     B.segquant_set_tuning(tile_n, 0, cta_group, segment_mode)
     try:
         layer = SegQuantLinear(data.W, data.bias, spec.kb, spec.nb, spec.dual, spec.code, DEV, flags)
+        if split:
+            layer.allow_split_tiles(spec.M)
         g_pos, g_neg = layer.calibrate(data.X_cal)
         # --- scales: bit-exact
         assert np.array_equal(layer.s_w.cpu().numpy().reshape(spec.P, spec.Q), s_w)
@@ -45,6 +48,21 @@ def run_parity(spec, rows=None, flags=0, tile_n=0, cta_group=0, segment_mode=0):
         Ybf = layer.forward(Xd)                       # the one-call path, bf16 output
         layer.check_status()
         torch.cuda.synchronize()
+        if split:
+            # partial sums went through the workspace, every tile counter is back at zero, and a second call
+            # (which finds the slots of the first) gives the same bytes; so does the unsplit kernel for int8
+            ws = layer.workspace[B.workspace_bytes():]
+            assert int(ws.count_nonzero()) > 0, "the layer did not split any tile"
+            n_tiles = -(-spec.M // 256) * -(-spec.N // (128 if spec.dual else 256))
+            assert int(ws[:8 * n_tiles].count_nonzero()) == 0
+            assert torch.equal(layer.forward(Xd), Ybf)
+            B.segquant_set_tuning(tile_n, 0, cta_group, 7)
+            Y_whole = layer.forward(Xd)
+            layer.check_status()
+            if spec.code == "int8":
+                assert torch.equal(Y_whole, Ybf)
+            else:
+                assert (Y_whole.float() - Ybf.float()).abs().max() <= 0.02 * Ybf.float().abs().max()
     finally:
         B.segquant_set_tuning(0, 0, 0, 0)
 
@@ -58,6 +76,7 @@ def run_parity(spec, rows=None, flags=0, tile_n=0, cta_group=0, segment_mode=0):
     if spec.dual:
         assert np.array_equal(c_neg.cpu().numpy().view(dt)[sel], res.c_neg)
     # --- accumulators
+    acc_extra = 0.0
     npol = 2 if spec.dual else 1
     acc = dump.cpu().numpy().reshape(spec.P, npol, spec.M, spec.N)[:, :, sel]
     nacc = spec.P * npol
@@ -69,18 +88,24 @@ def run_parity(spec, rows=None, flags=0, tile_n=0, cta_group=0, segment_mode=0):
     else:
         # e4m3: tensor-core fp32 accumulation against exact sums; judged against the sum of |products|
         mag = lambda c: (np.asarray(c, np.uint8) & 0x7F)
+        q_of_n = np.searchsorted(np.asarray(spec.nb), np.arange(spec.N), side="right") - 1
         for pol, (cx, ref) in enumerate([(res.c_pos, res.acc_pos), (res.c_neg, res.acc_neg)][:npol]):
             abs_sum = O.accumulate(mag(cx), mag(Wq), spec.kb, code="e4m3")
             err = np.abs(acc[:, pol].astype(np.float64) - ref)
-            assert np.all(err <= 1e-3 * np.abs(ref) + 1e-5 * abs_sum), \
+            allow = 1e-3 * np.abs(ref) + 1e-5 * abs_sum
+            assert np.all(err <= allow), \
                 f"e4m3 accumulator error {np.max(err / np.maximum(abs_sum, 1e-30)):.3g} of sum|prod|"
+            if split:      # the split kernel adds fp32 partial sums: its accumulators get the same allowance again
+                s_act = (s_pos, s_neg)[pol].astype(np.float64)
+                c = s_act[:, None] * s_w.reshape(spec.P, spec.Q).astype(np.float64)[:, q_of_n]      # [P, N]
+                acc_extra = acc_extra + (c[:, None, :] * allow).sum(0)
         # epilogue is judged on the accumulators the GPU produced
         a_pos = acc[:, 0].astype(np.float64)
         a_neg = acc[:, 1].astype(np.float64) if spec.dual else None
         y64, y_abs = O.dequant(a_pos, a_neg, spec.nb, s_pos, s_neg, s_w, to_f32_np(data.bias), with_abs=True)
     # --- epilogue
     check_fp32_output(Y32[torch.as_tensor(sel, device=DEV)], y64, y_abs, nacc)
-    check_bf16_output(Ybf[torch.as_tensor(sel, device=DEV)], y64, y_abs, nacc)
+    check_bf16_output(Ybf[torch.as_tensor(sel, device=DEV)], y64, y_abs, nacc, extra=acc_extra)
     return res
 
 
@@ -153,6 +178,23 @@ def test_wide_single_scale_tiles(case):
     finally:
         B.segquant_set_tuning(0, 0, 0, 0)
     assert torch.equal(Y_wide, Y_narrow)
+
+
+@pytest.mark.parametrize("case", [
+    # layers with one K-segment whose K loops are cut across CTA pairs (the larger workspace; forced here): fewer
+    # tiles than pairs (every tile shared by several pairs), a few more tiles than pairs, ragged M / N / K,
+    # a K of two blocks (most pairs get one block or none), several N-segments, both code types and polarities
+    ("split_few_tiles_dual", 512, 4608, 256, [0, 256], True, "int8"),
+    ("split_one_tile_single", 200, 9216, 256, [0, 256], False, "int8"),
+    ("split_ragged_dual", 1300, 1072, 392, [0, 128, 392], True, "int8"),
+    ("split_ragged_single", 2100, 2000, 776, [0, 512, 776], False, "int8"),
+    ("split_short_k", 2560, 256, 1280, [0, 1280], True, "int8"),
+    ("split_e4m3_dual", 700, 3072, 384, [0, 384], True, "e4m3"),
+    ("split_e4m3_single", 520, 2048, 520, [0, 520], False, "e4m3"),
+])
+def test_split_tiles(case):
+    name, M, K, N, nb, dual, code = case
+    run_parity(custom_spec(name, M, K, N, [0, K], nb, dual, code, seed=71), segment_mode=6, split=True)
 
 
 @pytest.mark.parametrize("cta_group", [1, 2])
