@@ -325,7 +325,31 @@ def graph_time_per_launch(calls, rounds):
     return e0.elapsed_time(e1) * 1e3 / (rounds * len(calls))
 
 
-def time_kernels(layers, launches=48, max_copies=96, with_w4a8=True, with_split=False):
+def library_gemm_same_shape(spec, M, n_copies, rounds, dev):
+    """Context only: the vendor library's plain dense GEMM on the layer's shape (int8 -> int32, or e4m3 -> bf16 with
+    unit scales; no segment scales, no bias, one code matrix), timed like the product's kernels: a CUDA graph of
+    launches over rotating operand copies.  M is rounded up to a multiple of 8 for the library.  Returns
+    microseconds per launch, or None where the library refuses the shape."""
+    Mp = -(-M // 8) * 8
+    try:
+        if spec.code == "int8":
+            sets = [(torch.randint(-127, 128, (Mp, spec.K), dtype=torch.int8, device=dev),
+                     torch.randint(-127, 128, (spec.N, spec.K), dtype=torch.int8, device=dev).t()) for _ in range(n_copies)]
+            calls = [(lambda a=a, b=b: torch._int_mm(a, b)) for a, b in sets]
+        else:
+            one = torch.ones((), device=dev)
+            sets = [(torch.randn((Mp, spec.K), device=dev).to(torch.float8_e4m3fn),
+                     torch.randn((spec.N, spec.K), device=dev).to(torch.float8_e4m3fn).t()) for _ in range(n_copies)]
+            calls = [(lambda a=a, b=b: torch._scaled_mm(a, b, scale_a=one, scale_b=one, out_dtype=torch.bfloat16))
+                     for a, b in sets]
+        t = graph_time_per_launch(calls, rounds)
+    except Exception:
+        t = None
+    torch.cuda.empty_cache()
+    return t
+
+
+def time_kernels(layers, launches=48, max_copies=96, with_w4a8=True, with_split=False, with_library=True):
     """Per-layer device time of each kernel, timed alone: a CUDA graph of >= `launches` launches of that one
     kernel, launch i on copy i mod C of the layer's device buffers, C chosen so that the copies the kernel walks
     through are at least twice the L2 capacity (every launch finds its operands in HBM).  A single launch between
@@ -333,7 +357,7 @@ def time_kernels(layers, launches=48, max_copies=96, with_w4a8=True, with_split=
     event pair around one small kernel reads 6-8 us more than the kernel's own span.
     Returns lists (quantize_us, gemm_us, plain_us | None, unsegmented_us | None, copies)."""
     out = {"q": [], "g": [], "plain": [], "unseg": [], "copies": [], "q_plain": [], "q_zp": [], "g_zp": [], "q_fused": [],
-           "act": [], "w4_q": [], "w4_unpack": [], "w4_g": [], "g_split": []}
+           "act": [], "w4_q": [], "w4_unpack": [], "w4_g": [], "g_split": [], "lib": []}
     for bl in layers:
         s = bl.spec
         foot = min(quant_bytes(s, bl.M), gemm_bytes(s, bl.M))
@@ -360,6 +384,8 @@ def time_kernels(layers, launches=48, max_copies=96, with_w4a8=True, with_split=
         out["w4_g"].append(graph_time_per_launch([c.w4_gemm for c in copies], rounds) if w4 else None)
         del copies
         torch.cuda.empty_cache()
+        out["lib"].append(library_gemm_same_shape(s, bl.M, min(n, 24), max(1, -(-launches // min(n, 24))), bl.X.device)
+                          if with_library else None)
     return out
 
 
@@ -632,6 +658,13 @@ def layer_table(specs, kt, peaks):
                          "gemm_us": us(kt["w4_g"][i]), "layer_time_over_w8a8_layer": round(w4_us / layer_us, 3),
                          "note": "per-channel 4-bit weights kept packed and unpacked in front of the GEMM, per-token "
                                  "activation scales; the GEMM runs the variant with per-(token, channel) factors"}
+        if kt["lib"][i] is not None:
+            ours = kt["plain"][i] if s.dual else g * 1e3           # the single-code-matrix GEMM of this shape
+            r["library_gemm_same_shape"] = {
+                "us": us(kt["lib"][i]), "ours_single_scale_us": us(ours), "ours_over_library": round(ours / kt["lib"][i], 3),
+                "note": "vendor library's plain dense GEMM of this M, K, N (int8 -> int32 or e4m3 -> bf16, no segment "
+                        "scales, no bias), same timing method; ours is the single-scale GEMM with its dequantizing "
+                        "epilogue; context, not part of the product path"}
         if kt["g_split"][i] is not None:
             r["split_tiles"] = {"gemm_us": us(kt["g_split"][i]), "time_over_whole_tiles": round(kt["g_split"][i] / (g * 1e3), 3),
                                 "note": "K loops cut across CTA pairs with the partial sums exchanged through the larger "

@@ -554,6 +554,44 @@ def test_degenerate_all_nonnegative_input():
     check_fp32_output(Y, res.y64, res.y_abs, 2)
 
 
+def test_host_threads_with_their_own_streams_and_workspaces():
+    """Two host threads prepare and launch different layers at the same time, each on its own stream with its own
+    layer object (workspace included): the library's shared state (tensor-map encoder, per-kernel attributes and
+    occupancy caches) is guarded, so both get the bytes of their serial runs."""
+    import threading
+    specs = [custom_spec("thr_a", 700, 512, 520, [0, 256, 512], [0, 256, 520], True, "int8", seed=81),
+             custom_spec("thr_b", 1300, 384, 1032, [0, 384], [0, 1032], False, "e4m3", seed=82)]
+    jobs = []
+    for sp in specs:
+        data = WL.make_layer(sp)
+        layer = SegQuantLinear(data.W, data.bias, sp.kb, sp.nb, sp.dual, sp.code, DEV)
+        layer.calibrate(data.X_cal)
+        Xd = data.X.to(DEV)
+        jobs.append((layer, Xd, layer.forward(Xd).clone()))
+    torch.cuda.synchronize()
+    errors = []
+
+    def work(layer, Xd, want):
+        try:
+            st = torch.cuda.Stream()
+            with torch.cuda.stream(st):
+                for _ in range(40):
+                    Y = layer.forward(Xd)
+                st.synchronize()
+                layer.check_status()
+                if not torch.equal(Y, want):
+                    errors.append("output differs from the serial run")
+        except Exception as e:                      # surfaced in the main thread below
+            errors.append(repr(e))
+
+    threads = [threading.Thread(target=work, args=j) for j in jobs]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+
+
 def test_repeated_calls_are_deterministic():
     spec = custom_spec("det", 300, 512, 384, [0, 256, 512], [0, 384], True, "int8")
     data = WL.make_layer(spec)
