@@ -327,6 +327,13 @@ sq_status segquant_last_device_status(void *workspace, void *stream, uint32_t *d
  * automatic choice. */
 sq_status segquant_set_tuning(int tile_n, int stages, int cta_group, int segment_mode);
 
+/* The fused activation of segquant_quantize_act_fused has two implementations with identical results: one that
+ * evaluates SiLU / GELU per element, and, for bf16 inputs, one that looks the stored activation up in a table of
+ * all 65536 bf16 values which every thread block builds in shared memory first (about 9 us per launch, then one
+ * load per element).  fused_table_mode: 0 automatic (the table from 8 Mi elements up for GELU, 16 Mi for SiLU), 1 the table wherever it
+ * applies, 2 never.  Process-wide and for tests and sweeps, like segquant_set_tuning. */
+sq_status segquant_set_quantize_tuning(int fused_table_mode);
+
 /* Text of the CUDA error behind the most recent SQ_ERR_CUDA of a GEMM launch ("no error" if none). */
 const char *segquant_last_cuda_error(void);
 

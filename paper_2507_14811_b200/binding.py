@@ -29,7 +29,7 @@ EXPORTS = [
     "segquant_status_string", "segquant_quantize_act_fused", "segquant_calib_zero_point",
     "segquant_quantize_act_zero_point", "segquant_fold_zero_point", "segquant_plan_layer", "segquant_plan_run",
     "segquant_quantize_per_row", "segquant_pack_w4", "segquant_unpack_w4", "segquant_w4a8_gemm",
-    "segquant_split_workspace_bytes",
+    "segquant_split_workspace_bytes", "segquant_set_quantize_tuning",
 ]
 
 
@@ -112,6 +112,10 @@ def _check(status, where):
 
 def workspace_bytes() -> int:
     return int(lib().segquant_workspace_bytes())
+
+
+def segquant_set_quantize_tuning(fused_table_mode: int = 0):
+    _check(lib().segquant_set_quantize_tuning(C.c_int(fused_table_mode)), "segquant_set_quantize_tuning")
 
 
 def split_workspace_bytes(M: int, N: int, dual: bool) -> int:

@@ -516,6 +516,13 @@ sq_status segquant_last_device_status(void *workspace, void *stream, uint32_t *d
     return SQ_ERR_TIMEOUT;
 }
 
+sq_status segquant_set_quantize_tuning(int fused_table_mode)
+{
+    if (fused_table_mode < 0 || fused_table_mode > 2) return SQ_ERR_UNSUPPORTED;
+    set_quantize_table_mode(fused_table_mode);
+    return SQ_OK;
+}
+
 sq_status segquant_set_tuning(int tile_n, int stages, int cta_group, int segment_mode)
 {
     set_gemm_tuning(tile_n, stages, cta_group, segment_mode);

@@ -7,6 +7,7 @@
 // even, clip"; the common case computes them with a handful of full-rate fp32 instructions per element (see
 // SegConst) so that the pass stays memory bound.
 #include <cuda_bf16.h>
+#include <atomic>
 #include "sq_common.cuh"
 
 namespace sq {
@@ -139,7 +140,9 @@ __device__ __forceinline__ float gelu_f32(float h)
     float E = __fmul_rn(__expf(-s), g);
     E = fmaf(-E, e, E);                                   // exp(-(s + e)) = exp(-s) (1 - e) to first order
     const float half = __fmul_rn(0.5f, h);
-    return h >= 0.0f ? fmaf(-half, E, h) : __fmul_rn(half, E);
+    const float v = h >= 0.0f ? fmaf(-half, E, h) : __fmul_rn(half, E);
+    // beyond t = 13.5 the exponential has long underflowed: h or -0, also where t^2 overflows or h is infinite
+    return t >= 13.5f ? (h >= 0.0f ? h : -0.0f) : v;
 }
 template <typename Tin>
 __device__ __forceinline__ float pre1(float h, int act, float mult)
@@ -497,6 +500,140 @@ quantize_kernel(const __grid_constant__ QuantParams prm)
     asm volatile("cp.async.wait_group 0;" ::: "memory");     // nothing of this thread's is in flight when it leaves
 }
 
+// ----------------------------------------------------------------------------- fused activation by table (bf16 inputs)
+// A bf16 pre-activation has 65536 possible values, so the stored activation bf16(act(h)) is a table of 128 KiB.
+// Every CTA (1024 threads, one per SM) builds the table in its shared memory with the same silu_f32 / gelu_f32 as
+// the arithmetic variant (a few evaluations per thread: most bit patterns need none), after which an element costs one
+// shared-memory load instead of about 30 instructions: the fused pass stops being bound by the ALUs.  Results are
+// those of the arithmetic variant bit for bit.  Used for large inputs: a launch of this kernel costs about 9 us
+// more than the other's (the table, and a CTA that fills the SM cannot start under the previous kernel's tail).
+// (Not for the gated form: its product is rounded once, from the unrounded GELU, which a bf16 table does not hold.)
+// The rest is quantize_kernel's scheme: thread g owns column chunk g % V of rows g / V, g / V + R, ...; the rows
+// travel through a thread-private ring of kTableDepth slots behind the table.
+constexpr int kTableThreads = 1024;
+constexpr int kTableDepth = 3;
+constexpr size_t kTableBytes = 65536 * 2;
+constexpr size_t kTableSmem = kTableBytes + size_t(kTableDepth) * 2 * kTableThreads * 16;      // 224 KiB
+
+template <int CODE, int MODE>
+__global__ void __launch_bounds__(kTableThreads, 1)
+quantize_table_kernel(const __grid_constant__ QuantParams prm)
+{
+    constexpr bool DUAL = MODE == kDual;
+    extern __shared__ __align__(16) uint8_t table_smem[];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const uint32_t tab0 = uint32_t(__cvta_generic_to_shared(table_smem));
+    // Most bit patterns need no evaluation, because silu_f32 / gelu_f32 return a value known in advance there
+    // (a warp's 32 consecutive patterns share sign and exponent, so the branch is uniform):
+    //   2^-124 <= |h| < 2^-26: both give h / 2 after the rounding to bf16 (the sigmoid / Phi factor is 1/2 to
+    //                          far below a bf16 half-step);
+    //   h >= 32 (SiLU), h >= 16 (GELU): h itself (exp(-h), erfc(h / sqrt 2) are below fp32's resolution of 1);
+    //   h <= -128 (SiLU), h <= -16 (GELU): -0 (the exponential has underflowed to zero).
+    // NaN and infinities go through the functions.  The test that compares this variant with the arithmetic one
+    // on all 65536 patterns holds these statements to the bit.
+    const bool is_silu = prm.act == 1;
+    for (uint32_t b = threadIdx.x; b < 65536u; b += kTableThreads) {
+        const uint32_t e = (b >> 7) & 0xFFu, neg = b >> 15;
+        uint32_t out;
+        if (e >= 3u && e <= 100u) {
+            out = b - 0x80u;                                  // exponent - 1
+        } else if (e != 255u && !neg && e >= (is_silu ? 132u : 131u)) {
+            out = b;
+        } else if (e != 255u && neg && e >= (is_silu ? 134u : 131u)) {
+            out = 0x8000u;
+        } else {
+            const float h = __uint_as_float(b << 16);
+            const float a = is_silu ? silu_f32(h) : gelu_f32(h);
+            const __nv_bfloat16 r = __float2bfloat16_rn(a);
+            out = *reinterpret_cast<const unsigned short *>(&r);
+        }
+        reinterpret_cast<unsigned short *>(table_smem)[b] = static_cast<unsigned short>(out);
+    }
+    __syncthreads();
+    auto lookup = [&](uint32_t bits16) -> float {       // bits of a bf16 pre-activation -> stored activation as fp32
+        uint32_t v;
+        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(tab0 + (bits16 << 1)));
+        return __uint_as_float(v << 16);
+    };
+
+    const SegBounds &sb = prm.sb;
+    const int64_t M = prm.M;
+    const int R = prm.R;
+    const uint32_t g = blockIdx.x * kTableThreads + threadIdx.x;
+    const uint32_t r0 = g / uint32_t(prm.V);
+    if (r0 >= uint32_t(R) || int64_t(r0) >= M) return;
+    const int k0 = int(g - r0 * uint32_t(prm.V)) * kVec;     // the host checked: every chunk lies in one K-segment
+    int p = 0;
+    while (p + 1 < sb.P && k0 >= sb.kb[p + 1]) p++;
+
+    using Tin = __nv_bfloat16;
+    const Tin *src = static_cast<const Tin *>(prm.X) + int64_t(r0) * prm.ld + k0;
+    uint8_t *dp = prm.c_pos + int64_t(r0) * prm.ldc + k0;
+    uint8_t *dn = DUAL ? prm.c_neg + int64_t(r0) * prm.ldc + k0 : nullptr;
+    const int64_t src_step = int64_t(R) * prm.ld, dst_step = int64_t(R) * prm.ldc;
+    float mreg[kVec];
+#pragma unroll
+    for (int i = 0; i < kVec; i++) mreg[i] = prm.mult ? __ldg(prm.mult + k0 + i) : 1.0f;
+    const SegConst cp = seg_const(__ldg(prm.s_pos + p));
+    const SegConst cn = seg_const(DUAL ? __ldg(prm.s_neg + p) : 1.0f);
+    const bool fast = cp.fast && cn.fast && !(DUAL && CODE == SQ_CODE_INT8 && prm.lo != -128);
+
+    const uint32_t ring0 = tab0 + uint32_t(kTableBytes) + threadIdx.x * 16u;
+    auto slot_addr = [&](int slot, int v) { return ring0 + uint32_t((slot * 2 + v) * kTableThreads) * 16u; };
+    auto copy_row = [&](const Tin *row_src, int slot, bool valid) {          // one commit group per call, always
+        if (valid) {
+#pragma unroll
+            for (int v = 0; v < 2; v++)
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(slot_addr(slot, v)),
+                             "l"(reinterpret_cast<const char *>(row_src) + 16 * v) : "memory");
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+#pragma unroll
+    for (int d = 0; d < kTableDepth - 1; d++) copy_row(src + int64_t(d) * src_step, d, int64_t(r0) + int64_t(d) * R < M);
+    int slot = 0;
+    for (int64_t row = r0; row < M; row += R) {
+        const int ahead = slot == 0 ? kTableDepth - 1 : slot - 1;
+        copy_row(src + int64_t(kTableDepth - 1) * src_step, ahead, row + int64_t(kTableDepth - 1) * R < M);
+        asm volatile("cp.async.wait_group %0;" ::"n"(kTableDepth - 1) : "memory");
+        uint32_t w[8];
+#pragma unroll
+        for (int v = 0; v < 2; v++)
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w[4 * v]), "=r"(w[4 * v + 1]), "=r"(w[4 * v + 2]), "=r"(w[4 * v + 3])
+                         : "r"(slot_addr(slot, v)) : "memory");
+        slot = slot + 1 == kTableDepth ? 0 : slot + 1;
+        uint32_t wp[4], wn[4];
+#pragma unroll
+        for (int g4 = 0; g4 < 4; g4++) {
+            float x[4];
+#pragma unroll
+            for (int i = 0; i < 4; i++) {
+                const uint32_t word = w[2 * g4 + (i >> 1)];
+                x[i] = __fmul_rn(lookup((i & 1) ? (word >> 16) : (word & 0xFFFFu)), mreg[4 * g4 + i]);
+            }
+            if (fast) {
+                quant4<CODE, MODE>(x, cp, cn, float(prm.hi), 0, wp[g4], wn[g4]);
+            } else {
+                wp[g4] = wn[g4] = 0u;
+#pragma unroll
+                for (int i = 0; i < 4; i++) {
+                    uint32_t a, b;
+                    quant1<CODE, MODE>(x[i], cp.s, cn.s, 0, prm.lo, prm.hi, a, b);
+                    wp[g4] |= (a & 0xFFu) << (8 * i);
+                    wn[g4] |= (b & 0xFFu) << (8 * i);
+                }
+            }
+        }
+        *reinterpret_cast<uint4 *>(dp) = make_uint4(wp[0], wp[1], wp[2], wp[3]);
+        if (DUAL) *reinterpret_cast<uint4 *>(dn) = make_uint4(wn[0], wn[1], wn[2], wn[3]);
+        src += src_step;
+        dp += dst_step;
+        if (DUAL) dn += dst_step;
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+
 // ----------------------------------------------------------------------------- per-row scales (W4A8)
 // App. B "Extra Hyperparameter Settings": 4-bit weights are quantized per channel, activations dynamically per
 // token.  One CTA per row: the row is read once into registers (up to kRowChunks 16-element chunks per thread),
@@ -725,7 +862,54 @@ sq_status prepare_mode(QuantLaunch &L, sq_code code, int mode)
     return mode == kDual ? prepare_t<Tin, SQ_CODE_E4M3, kDual>(L) : prepare_t<Tin, SQ_CODE_E4M3, kSingle>(L);
 }
 
+// The table variant of the fused activation: bf16 input, SiLU or GELU, every 16-element chunk inside one K-segment,
+// and enough elements for the table's set-up time not to count.  Returns false where it does not apply.
+std::atomic<int> g_table_mode{0};        // test hook: 0 automatic, 1 always where possible, 2 never
+constexpr int64_t kTableMinSilu = int64_t(16) << 20, kTableMinGelu = int64_t(8) << 20;   // measured break-even points
+bool prepare_table(QuantLaunch &L, sq_dtype dt, sq_code code, int mode)
+{
+    QuantParams &prm = L.prm;
+    const int tm = g_table_mode.load(std::memory_order_relaxed);
+    if (tm == 2 || dt != SQ_BF16 || mode == kZeroPoint || prm.row_segments) return false;
+    if (prm.act != SQ_ACT_SILU && prm.act != SQ_ACT_GELU) return false;
+    if (prm.K % kVec != 0) return false;
+    for (int p = 1; p < prm.sb.P; p++)
+        if (prm.sb.kb[p] % kVec != 0) return false;
+    if (tm != 1 && prm.M * int64_t(prm.K) < (prm.act == SQ_ACT_SILU ? kTableMinSilu : kTableMinGelu)) return false;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        return false;
+    const int64_t V = prm.K / kVec;
+    const int64_t threads = int64_t(sms) * kTableThreads;                 // one CTA per SM
+    int64_t iters = (prm.M * V + threads - 1) / threads;
+    if (iters < 1) iters = 1;
+    const int64_t R = (prm.M + iters - 1) / iters;
+    const int64_t blocks = (R * V + kTableThreads - 1) / kTableThreads;
+    if (blocks > 0x7FFFFFFF || R * V > 0xFFFFFFFFll || V > 0x7FFFFFFF || R > 0x7FFFFFFF) return false;
+    const void *kern = nullptr;
+    if (code == SQ_CODE_INT8)
+        kern = mode == kDual ? reinterpret_cast<const void *>(quantize_table_kernel<SQ_CODE_INT8, kDual>)
+                             : reinterpret_cast<const void *>(quantize_table_kernel<SQ_CODE_INT8, kSingle>);
+    else
+        kern = mode == kDual ? reinterpret_cast<const void *>(quantize_table_kernel<SQ_CODE_E4M3, kDual>)
+                             : reinterpret_cast<const void *>(quantize_table_kernel<SQ_CODE_E4M3, kSingle>);
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kTableSmem)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return false;
+    }
+    prm.V = int(V);
+    prm.R = int(R);
+    L.blocks = unsigned(blocks);
+    L.kernel = kern;
+    L.threads = kTableThreads;
+    L.smem = unsigned(kTableSmem);
+    return true;
+}
+
 }  // namespace
+
+void set_quantize_table_mode(int mode) { g_table_mode.store(mode, std::memory_order_relaxed); }
 
 sq_status prepare_quantize(const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld, const SegBounds &sb,
                            const float *s_pos, const float *s_neg, const int32_t *zero_point, int row_segments,
@@ -734,6 +918,8 @@ sq_status prepare_quantize(const void *X, sq_dtype dt, int64_t M, int64_t K, int
 {
     QuantParams &prm = out->prm;
     prm = QuantParams{};
+    out->threads = 0;
+    out->smem = 0;
     prm.X = X; prm.M = M; prm.K = int(K); prm.ld = ld;
     prm.sb = sb;
     prm.s_pos = s_pos; prm.s_neg = s_neg; prm.zp = zero_point;
@@ -744,6 +930,7 @@ sq_status prepare_quantize(const void *X, sq_dtype dt, int64_t M, int64_t K, int
     prm.c_pos = static_cast<uint8_t *>(c_pos); prm.c_neg = static_cast<uint8_t *>(c_neg); prm.ldc = ldc;
     prm.act = act; prm.mult = mult;
     const int mode = zero_point ? kZeroPoint : (s_neg ? kDual : kSingle);
+    if (prepare_table(*out, dt, code, mode)) return SQ_OK;
     return dt == SQ_F32 ? prepare_mode<float>(*out, code, mode) : prepare_mode<__nv_bfloat16>(*out, code, mode);
 }
 
@@ -751,7 +938,8 @@ sq_status run_quantize(const QuantLaunch &L, cudaStream_t st)
 {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(L.blocks);
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(L.threads ? L.threads : unsigned(kThreads));
+    cfg.dynamicSmemBytes = L.smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

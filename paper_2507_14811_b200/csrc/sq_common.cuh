@@ -75,6 +75,8 @@ struct QuantLaunch {
     QuantParams prm;
     const void *kernel;
     unsigned blocks;
+    unsigned threads;         // 0: the kernel's default block size
+    unsigned smem;            // dynamic shared memory
 };
 
 // zero_point != nullptr selects the App. A asymmetric quantizer (int8); act / mult: optional activation
@@ -89,6 +91,7 @@ sq_status prepare_quantize(const void *X, sq_dtype dt, int64_t M, int64_t K, int
                            sq_code code, float q_max, float q_min_abs, int act, const float *mult,
                            void *c_pos, void *c_neg, int64_t ldc, QuantLaunch *out);    // launches nothing
 sq_status run_quantize(const QuantLaunch &l, cudaStream_t st);                          // one launch, no queries
+void set_quantize_table_mode(int mode);      // fused activation by table: 0 automatic, 1 wherever possible, 2 never (tests)
 
 // One scale per (row, K-segment) from the row's own extrema, written to s_pos / s_neg [rows][P], and the int8 codes
 // quantized with them (per-token activations, q_max 127; per-channel 4-bit weights, q_max 7).

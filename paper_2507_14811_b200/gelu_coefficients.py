@@ -37,7 +37,8 @@ def gelu_f32(h, coef):
     E = (np.exp(-s.astype(np.float64)).astype(f32) * g).astype(f32)
     E = (E - E * e).astype(f32)
     half = (f32(0.5) * h).astype(f32)
-    return np.where(h >= 0, (h - half * E).astype(f32), (half * E).astype(f32))
+    v = np.where(h >= 0, (h - half * E).astype(f32), (half * E).astype(f32))
+    return np.where(t >= f32(13.5), np.where(h >= 0, h, f32(-0.0)), v)      # the kernel's cut-off beyond the underflow
 
 
 if __name__ == "__main__":

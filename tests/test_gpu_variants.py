@@ -196,19 +196,22 @@ def stored_candidates(h, act, stored):
     return cands, tiny
 
 
+@pytest.mark.parametrize("table", [2, 1])
 @pytest.mark.parametrize("act", ["silu", "gelu"])
 @pytest.mark.parametrize("code,dual", [("int8", True), ("int8", False), ("e4m3", True)])
-def test_fused_activation_codes_are_valid(act, code, dual):
+def test_fused_activation_codes_are_valid(act, code, dual, table):
     """H (bf16 pre-activation) -> act -> bf16 -> (multiplier) -> codes in one kernel.  The oracle evaluates the
     activation in fp64 and rounds once; a GPU code must be the oracle's code, or the code of the neighbouring
     bf16 value where the exact activation lies within the kernel's stated error bound of a bf16 rounding
-    boundary.  Almost every element must take the first branch."""
+    boundary.  Almost every element must take the first branch.  table: 2 = the activation evaluated per element,
+    1 = looked up in the table of all bf16 values that the kernel builds in shared memory."""
     rs = np.random.default_rng(9)
     spec = custom_spec("fact", 700, 512, 64, [0, 192, 512], [0, 64], dual, code, x_kind="normal", seed=63,
                        x_seg_std=[1.5, 3.0])
     data = WL.make_layer(spec)
     H = to_f32_np(data.X)
     H[0, :12] = [0.0, -0.0, 11.5, -11.5, 30.0, -30.0, -60.0, -100.0, 1e-20, -1e-20, 88.0, -88.0]
+    H[1, :4] = [1e30, -1e30, 1e19, -1e19]                    # far beyond any activation: the codes saturate, no NaN
     Hb = torch.from_numpy(H).to(torch.bfloat16)
     H = Hb.float().numpy()
     mult = rs.uniform(0.5, 2.0, spec.K).astype(np.float32)
@@ -216,10 +219,14 @@ def test_fused_activation_codes_are_valid(act, code, dual):
     cal, _ = O.activation(to_f32_np(data.X_cal), act, "bf16")
     s_pos, s_neg = O.calib_act(O.smooth(cal, mult), spec.kb, dual, q_max=qmax, q_min_abs=qmin_abs)
     seg = B.SegTable(spec.kb, spec.nb)
-    c_pos, c_neg = B.segquant_quantize_act_fused(Hb.to(DEV), seg, torch.from_numpy(s_pos).to(DEV),
-                                                 torch.from_numpy(s_neg).to(DEV) if dual else None, code, act=act,
-                                                 mult=torch.from_numpy(mult).to(DEV))
-    torch.cuda.synchronize()
+    B.segquant_set_quantize_tuning(table)
+    try:
+        c_pos, c_neg = B.segquant_quantize_act_fused(Hb.to(DEV), seg, torch.from_numpy(s_pos).to(DEV),
+                                                     torch.from_numpy(s_neg).to(DEV) if dual else None, code, act=act,
+                                                     mult=torch.from_numpy(mult).to(DEV))
+        torch.cuda.synchronize()
+    finally:
+        B.segquant_set_quantize_tuning(0)
     dt = np.int8 if code == "int8" else np.uint8
     g_pos = c_pos.cpu().numpy().view(dt)
     g_neg = c_neg.cpu().numpy().view(dt) if dual else None
@@ -237,6 +244,44 @@ def test_fused_activation_codes_are_valid(act, code, dual):
             ok |= same & tiny
     assert ok.all(), f"{(~ok).sum()} codes are neither the oracle's nor a neighbour's"
     assert first.mean() > 0.999, f"only {first.mean():.5f} of the codes equal the oracle's"
+
+
+@pytest.mark.parametrize("act", ["silu", "gelu"])
+@pytest.mark.parametrize("case", [
+    # M, K, kb, dual, code, scale: several rows per thread, a thread count that is no multiple of the block, two
+    # K-segments, both code types, every bf16 bit pattern as input, and scales outside the fast quantizer's range
+    (5000, 1024, [0, 1024], True, "int8", None),
+    (333, 208, [0, 96, 208], False, "int8", None),
+    (700, 512, [0, 192, 512], True, "e4m3", None),
+    (4096, 16, [0, 16], True, "int8", None),
+    (300, 256, [0, 256], True, "int8", 1e-30),
+    (300, 256, [0, 256], False, "e4m3", 1e32),
+])
+def test_fused_activation_table_equals_the_per_element_evaluation(act, case):
+    """The two implementations of the fused activation give the same bytes on every input, all 65536 bf16 bit
+    patterns (NaNs and infinities included) among them."""
+    M, K, kb, dual, code, scale = case
+    g = torch.Generator().manual_seed(91)
+    H = (torch.randn((M, K), generator=g) * 2.5).to(torch.bfloat16)
+    bits = torch.arange(65536, dtype=torch.int32).to(torch.int16).view(torch.bfloat16)
+    H.view(-1)[:65536] = bits[: H.numel()] if H.numel() < 65536 else bits
+    P = len(kb) - 1
+    s_val = [0.02 * (p + 1) for p in range(P)] if scale is None else [scale] * P
+    sp = torch.tensor(s_val, dtype=torch.float32, device=DEV)
+    sn = (sp * 0.5) if dual else None
+    mult = (torch.rand(K, generator=g) + 0.5).to(DEV)
+    seg = B.SegTable(kb, [0, 64])
+    outs = []
+    try:
+        for mode in (2, 1):
+            B.segquant_set_quantize_tuning(mode)
+            outs.append(B.segquant_quantize_act_fused(H.to(DEV), seg, sp, sn, code, act=act, mult=mult))
+        torch.cuda.synchronize()
+    finally:
+        B.segquant_set_quantize_tuning(0)
+    assert torch.equal(outs[0][0], outs[1][0])
+    if dual:
+        assert torch.equal(outs[0][1], outs[1][1])
 
 
 @pytest.mark.parametrize("act", ["silu", "gelu"])
