@@ -132,7 +132,9 @@ sq_status segquant_calib_scales_static(const void *X, sq_dtype dt, int64_t rows,
  *   e4m3 codes: "round" is the round-to-nearest-even cast to e4m3 (finite, max 448, subnormals
  *   kept), saturating; a result of -0 is stored as +0.
  *   X [M,K] dev (dtype dt, ld elements); c_pos, c_neg [M,K] dev, 1 byte per code, leading dimension
- *   ldc bytes.  Alignment: X, c_pos, c_neg 16 bytes; ld*sizeof(dt) and ldc multiples of 16 bytes. */
+ *   ldc bytes.  Alignment: X, c_pos, c_neg 16 bytes; ld*sizeof(dt) and ldc multiples of 16 bytes.
+ *   Inputs must be finite: every finite x, however large, gets the clipped code of the definition; the codes of
+ *   infinities and NaNs are unspecified (an int8 DualScale +inf sets both of its codes). */
 sq_status segquant_quantize_act(const void *X, sq_dtype dt, int64_t M, int64_t K, int64_t ld,
                                 const sq_segtable *seg, const float *s_pos, const float *s_neg,
                                 sq_code code, uint32_t flags, void *c_pos, void *c_neg, int64_t ldc,
