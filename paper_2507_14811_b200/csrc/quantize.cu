@@ -522,7 +522,6 @@ quantize_table_kernel(const __grid_constant__ QuantParams prm)
     constexpr bool DUAL = MODE == kDual;
     extern __shared__ __align__(16) uint8_t table_smem[];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint32_t tab0 = uint32_t(__cvta_generic_to_shared(table_smem));
     // Most bit patterns need no evaluation, because silu_f32 / gelu_f32 return a value known in advance there
     // (a warp's 32 consecutive patterns share sign and exponent, so the branch is uniform):
@@ -550,6 +549,8 @@ quantize_table_kernel(const __grid_constant__ QuantParams prm)
         }
         reinterpret_cast<unsigned short *>(table_smem)[b] = static_cast<unsigned short>(out);
     }
+    // the table depends on nothing in memory: it is built before the wait for the previous kernel of the stream
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     __syncthreads();
     auto lookup = [&](uint32_t bits16) -> float {       // bits of a bf16 pre-activation -> stored activation as fp32
         uint32_t v;
