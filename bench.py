@@ -715,7 +715,7 @@ def measure_side_workload(name, dev, args, peaks):
     return out
 
 
-SIDE_WORKLOADS = ["flux", "dit_xl2", "sdxl_skip", "sdxl_sweep", "sd3_heads", "sdxl_geglu"]
+SIDE_WORKLOADS = ["flux", "dit_xl2", "sdxl_skip", "sdxl_sweep", "sd3_heads", "sdxl_geglu", "modulation_small_m"]
 
 
 def run_ours(args):

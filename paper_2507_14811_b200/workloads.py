@@ -182,6 +182,17 @@ WORKLOADS["sdxl_geglu"] = [
           x_kind="normal+geglu", w_kind="plain", seed=6001, x_seg_std=[1.5]),
 ]
 
+# the modulation layers at the row count they have in the real models (one conditioning vector per sample, batch 8
+# and batch 1) instead of the token count of the benchmark configurations: bound by streaming the weights
+WORKLOADS["modulation_small_m"] = [
+    _spec("flux_modulation_M8", 8, 3072, 18432, Q=6, dual=True, code="e4m3", x_dtype="bf16",
+          x_kind="student_t4+silu", w_kind="segment_ladder", seed=3002),
+    _spec("flux_modulation_M1", 1, 3072, 18432, Q=6, dual=True, code="e4m3", x_dtype="bf16",
+          x_kind="student_t4+silu", w_kind="segment_ladder", seed=3002),
+    _spec("dit_adaln_M8", 8, 1152, 6912, Q=6, dual=True, code="int8", x_dtype="bf16",
+          x_kind="normal+silu", w_kind="segment_ladder", seed=1000),
+]
+
 SDXL_SWEEP_M = [512, 1024, 2048, 4096, 8192, 16384, 32768, 65536]
 
 # input segmentation by attention heads: the head-merge reshape in front of an attention output projection
