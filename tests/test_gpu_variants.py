@@ -354,6 +354,26 @@ def test_fused_gated_gelu_codes_are_valid(code, dual, dtype):
     assert first.mean() > 0.999, f"only {first.mean():.5f} of the codes equal the oracle's"
 
 
+def test_fused_gated_gelu_ragged_row_and_segment_bound_inside_a_chunk():
+    """K = 40 (a row tail of 8 elements) with a K-segment bound at 24: every chunk takes the per-element path, and
+    the gate half starts at byte 80 of the row."""
+    rs = np.random.default_rng(12)
+    M, K, kb = 33, 40, [0, 24, 40]
+    H = torch.from_numpy(rs.normal(0, 2.0, (M, 2 * K)).astype(np.float32)).to(torch.bfloat16)
+    Hn = H.float().numpy()
+    a_ref, exact = O.activation_gated(Hn, "bf16")
+    s_pos, s_neg = O.calib_act(a_ref, kb, True)
+    seg = B.SegTable(kb, [0, 8])
+    c_pos, c_neg = B.segquant_quantize_act_fused(H.to(DEV), seg, torch.from_numpy(s_pos).to(DEV),
+                                                 torch.from_numpy(s_neg).to(DEV), "int8", act="geglu")
+    torch.cuda.synchronize()
+    r_pos, r_neg = O.quantize_act(a_ref, kb, s_pos, s_neg, code="int8")
+    same = (c_pos.cpu().numpy().view(np.int8) == r_pos) & (c_neg.cpu().numpy().view(np.int8) == r_neg)
+    assert same.mean() > 0.995                       # the rest: stored values one bf16 step apart (checked above at size)
+    assert np.all(np.abs(c_pos.cpu().numpy().view(np.int8).astype(int) - r_pos) <= 1)
+    assert np.all(np.abs(c_neg.cpu().numpy().view(np.int8).astype(int) - r_neg) <= 1)
+
+
 def test_fused_gated_gelu_rejects_a_gate_half_off_the_16_byte_grid():
     H = torch.zeros(8, 2 * 36, dtype=torch.bfloat16, device=DEV)       # K = 36: the gate half starts at byte 72
     seg = B.SegTable([0, 36], [0, 8])
