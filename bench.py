@@ -715,7 +715,7 @@ def measure_side_workload(name, dev, args, peaks):
     return out
 
 
-SIDE_WORKLOADS = ["flux", "dit_xl2", "sdxl_skip", "sdxl_sweep", "sd3_heads", "sdxl_geglu", "modulation_small_m"]
+SIDE_WORKLOADS = ["flux", "dit_xl2", "sdxl_skip", "sdxl_sweep", "sd3_heads", "sdxl_geglu", "modulation_small_m", "sd3_qkv_768x2"]
 
 
 def run_ours(args):

@@ -193,6 +193,12 @@ WORKLOADS["modulation_small_m"] = [
           x_kind="normal+silu", w_kind="segment_ladder", seed=1000),
 ]
 
+# the other reading of the joint-QKV configuration: 1536 input channels as two concatenated streams of 768
+WORKLOADS["sd3_qkv_768x2"] = [
+    _spec("joint_qkv_768x2", 8858, 1536, 4608, P=2, Q=3, dual=False, code="int8", x_dtype="bf16",
+          x_kind="normal", w_kind="plain", seed=2000, x_seg_std=[1.0, 5.0]),
+]
+
 SDXL_SWEEP_M = [512, 1024, 2048, 4096, 8192, 16384, 32768, 65536]
 
 # input segmentation by attention heads: the head-merge reshape in front of an attention output projection
