@@ -623,7 +623,9 @@ def test_reduced_benchmark_layers(wl, idx, M, K, N):
 
 @pytest.mark.parametrize("wl,idx", [("dit_xl2", 0), ("dit_xl2", 1), ("sd3_mmdit", 0), ("sd3_mmdit", 1),
                                     ("sd3_mmdit", 2), ("flux", 0), ("flux", 1), ("flux", 2), ("sdxl_skip", 0),
-                                    ("sdxl_sweep", 0), ("sdxl_sweep", 7), ("sd3_heads", 0), ("sd3_heads", 1)])
+                                    ("sdxl_sweep", 0), ("sdxl_sweep", 7), ("sd3_heads", 0), ("sd3_heads", 1),
+                                    ("sdxl_geglu", 0), ("sdxl_geglu", 1), ("sd3_qkv_768x2", 0),
+                                    ("modulation_small_m", 0), ("modulation_small_m", 1), ("modulation_small_m", 2)])
 def test_full_size_layers_every_row(wl, idx):
     """Every benchmark layer at its full size, in the launch configuration the benchmark times (automatic tile
     plan): codes, accumulators (dumped by the checking variant of the kernel) and both outputs (fp32 from the
