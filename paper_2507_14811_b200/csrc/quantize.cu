@@ -703,10 +703,6 @@ quantize_per_row_kernel(const Tin *__restrict__ X, int K, int64_t ld, const SegB
         if (k0 + kVec <= sb.kb[p + 1]) {
             seg[c] = p;
             load16(src + k0, raw[c]);
-            float mx, mn;
-            chunk_extrema(raw[c], mx, mn);
-            atomicMax(&sh_max[p], ord_enc(mx));
-            atomicMin(&sh_min[p], ord_enc(mn));
         } else {
             seg[c] = -1;
             const int n = min(kVec, K - k0);
@@ -716,6 +712,30 @@ quantize_per_row_kernel(const Tin *__restrict__ X, int K, int64_t ld, const SegB
                 atomicMax(&sh_max[p], ord_enc(x));
                 atomicMin(&sh_min[p], ord_enc(x));
             }
+        }
+    }
+    // Extrema: where the 32 chunks of a warp lie in one K-segment (512 consecutive columns: the usual case) they are
+    // reduced with shuffles and one lane updates the shared words; same-address shared atomics from every thread
+    // serialise, and were most of this kernel's time.  Every lane takes part in the votes and shuffles.
+#pragma unroll
+    for (int c = 0; c < kRowChunks; c++) {
+        float mx = -INFINITY, mn = INFINITY;
+        if (seg[c] >= 0) chunk_extrema(raw[c], mx, mn);
+        const int s0 = __shfl_sync(0xFFFFFFFFu, seg[c], 0);
+        const bool uniform = __all_sync(0xFFFFFFFFu, seg[c] == s0) && s0 >= 0;
+        if (uniform) {
+#pragma unroll
+            for (int o = 16; o >= 1; o >>= 1) {
+                mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+                mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, o));
+            }
+            if ((threadIdx.x & 31) == 0) {
+                atomicMax(&sh_max[s0], ord_enc(mx));
+                atomicMin(&sh_min[s0], ord_enc(mn));
+            }
+        } else if (seg[c] >= 0) {
+            atomicMax(&sh_max[seg[c]], ord_enc(mx));
+            atomicMin(&sh_min[seg[c]], ord_enc(mn));
         }
     }
     __syncthreads();
