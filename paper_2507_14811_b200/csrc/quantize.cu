@@ -688,8 +688,16 @@ quantize_per_row_kernel(const Tin *__restrict__ X, int K, int64_t ld, const SegB
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int64_t row = blockIdx.x;
     const int P = sb.P;
-    for (int i = threadIdx.x; i < P; i += blockDim.x) { sh_max[i] = 0u; sh_min[i] = 0xFFFFFFFFu; }
-    __syncthreads();
+    // One K-segment (the usual case) needs ONE block barrier: every warp leaves its extrema in a slot, and after the
+    // barrier every thread reduces the slots and computes the scales itself.  Several K-segments go through
+    // shared-memory words per segment (three barriers).
+    const bool one = P == 1;
+    __shared__ float sh_wmax[kThreads / 32], sh_wmin[kThreads / 32];
+    float one_sp = 1.0f, one_sn = 1.0f, tail_mx = -INFINITY, tail_mn = INFINITY;
+    if (!one) {
+        for (int i = threadIdx.x; i < P; i += blockDim.x) { sh_max[i] = 0u; sh_min[i] = 0xFFFFFFFFu; }
+        __syncthreads();
+    }
     const Tin *src = X + row * ld;
     Raw16<Tin> raw[kRowChunks];
     int seg[kRowChunks];                            // K-segment of a whole chunk, -1: straddles a bound or the row end
@@ -709,11 +717,47 @@ quantize_per_row_kernel(const Tin *__restrict__ X, int K, int64_t ld, const SegB
             for (int i = 0; i < n; i++) {
                 while (p + 1 < P && k0 + i >= sb.kb[p + 1]) p++;
                 const float x = load1(src + k0 + i);
-                atomicMax(&sh_max[p], ord_enc(x));
-                atomicMin(&sh_min[p], ord_enc(x));
+                if (one) {
+                    tail_mx = fmaxf(tail_mx, x);
+                    tail_mn = fminf(tail_mn, x);
+                } else {
+                    atomicMax(&sh_max[p], ord_enc(x));
+                    atomicMin(&sh_min[p], ord_enc(x));
+                }
             }
         }
     }
+    if (one) {
+        float mx = tail_mx, mn = tail_mn;
+#pragma unroll
+        for (int c = 0; c < kRowChunks; c++) {
+            if (seg[c] >= 0) {
+                float cx, cm;
+                chunk_extrema(raw[c], cx, cm);
+                mx = fmaxf(mx, cx);
+                mn = fminf(mn, cm);
+            }
+        }
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) {
+            mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+            mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, o));
+        }
+        if ((threadIdx.x & 31) == 0) { sh_wmax[threadIdx.x >> 5] = mx; sh_wmin[threadIdx.x >> 5] = mn; }
+        __syncthreads();
+        mx = sh_wmax[0]; mn = sh_wmin[0];
+        for (int w = 1; w < int(blockDim.x >> 5); w++) { mx = fmaxf(mx, sh_wmax[w]); mn = fminf(mn, sh_wmin[w]); }
+        if (DUAL) {
+            const float h = fmaxf(mx, 0.0f), l = fmaxf(-mn, 0.0f);
+            one_sp = h > 0.0f ? __fdiv_rn(h, q_max) : 1.0f;
+            one_sn = l > 0.0f ? __fdiv_rn(l, q_min_abs) : 1.0f;
+            if (threadIdx.x == 0) s_neg[row] = one_sn;
+        } else {
+            const float a = fmaxf(fabsf(mx), fabsf(mn));
+            one_sp = a > 0.0f ? __fdiv_rn(a, q_max) : 1.0f;
+        }
+        if (threadIdx.x == 0) s_pos[row] = one_sp;
+    } else {
     // Extrema: where the 32 chunks of a warp lie in one K-segment (512 consecutive columns: the usual case) they are
     // reduced with shuffles and one lane updates the shared words; same-address shared atomics from every thread
     // serialise, and were most of this kernel's time.  Every lane takes part in the votes and shuffles.
@@ -756,6 +800,7 @@ quantize_per_row_kernel(const Tin *__restrict__ X, int K, int64_t ld, const SegB
         sh_sn[p] = sn;
     }
     __syncthreads();
+    }
     const int hi = int(q_max), lo = DUAL ? -int(q_min_abs) : -int(q_max);
     constexpr int MODE = DUAL ? kDual : kSingle;
     SegConst cp, cn;
@@ -769,8 +814,8 @@ quantize_per_row_kernel(const Tin *__restrict__ X, int K, int64_t ld, const SegB
         bool done = false;
         if (seg[c] >= 0) {
             if (seg[c] != const_seg) {              // constants are remade only when the chunk's K-segment changes
-                cp = seg_const(sh_sp[seg[c]]);
-                cn = seg_const(DUAL ? sh_sn[seg[c]] : 1.0f);
+                cp = seg_const(one ? one_sp : sh_sp[seg[c]]);
+                cn = seg_const(DUAL ? (one ? one_sn : sh_sn[seg[c]]) : 1.0f);
                 const_seg = seg[c];
             }
             if (cp.fast && cn.fast && !(DUAL && lo != -128)) {
@@ -792,7 +837,7 @@ quantize_per_row_kernel(const Tin *__restrict__ X, int K, int64_t ld, const SegB
             for (int i = 0; i < n; i++) {
                 while (p + 1 < P && k0 + i >= sb.kb[p + 1]) p++;
                 uint32_t a, b;
-                quant1<SQ_CODE_INT8, MODE>(load1(src + k0 + i), sh_sp[p], sh_sn[p], 0, lo, hi, a, b);
+                quant1<SQ_CODE_INT8, MODE>(load1(src + k0 + i), one ? one_sp : sh_sp[p], one ? one_sn : sh_sn[p], 0, lo, hi, a, b);
                 dp[i] = uint8_t(a);
                 if (DUAL) dn[i] = uint8_t(b);
             }
