@@ -1576,6 +1576,16 @@ sq_status prepare_tile(const GemmArgs &g, GemmLaunch &L, int tile_n, bool seq, i
     }
     if constexpr (KIND == 0 && CG == 2) {
         if (pt && !dbg) {     // 256- and 128-column tiles only (the automatic choice never goes below for these layers)
+            if constexpr (NPOL == 1) {      // single-scale, one K-segment: 256 x 512 tiles under the rule given further down
+                const int tune = g_tune_seq.load(std::memory_order_relaxed);
+                const int64_t n256w = (g.N + 255) / 256, mp = (g.M + 2 * TILE_M - 1) / (2 * TILE_M), un = sm_count / 2;
+                const int64_t w256 = (mp * n256w + un - 1) / un, wwide = (mp * ((n256w + 1) / 2) + un - 1) / un;
+                if (tile_n == 256 && prm.sb.P == 1 && tune != 4 && (n256w % 2 == 0 || n256w >= 9) &&
+                    (tune == 5 || 2 * wwide * 94 < w256 * 100)) {
+                    prm.acc_stages = 1;
+                    return prepare_variant<KIND, 1, 256, 2, false, false, true, true>(g, L, device, sm_count);
+                }
+            }
             if (tile_n == 256) return prepare_variant<KIND, NPOL, 256, CG, false, false, false, true>(g, L, device, sm_count);
             if (tile_n == 128) return prepare_variant<KIND, NPOL, 128, CG, false, false, false, true>(g, L, device, sm_count);
             dbg = true;

@@ -437,6 +437,17 @@ def test_w4a8_layer_parity(case, dual):
                                 x_seg_std=[1.0 + (i % 7) for i in range(len(kb) - 1)]))
 
 
+@pytest.mark.parametrize("N", [776, 1000, 2048])
+def test_w4a8_single_scale_layer_on_wide_tiles(N):
+    """The 256 x 512 tiles of single-scale layers with per-(token, channel) factors (forced here; the automatic
+    choice takes them on large layers): a ragged last tile, a second half of 8 columns, exact multiples."""
+    B.segquant_set_tuning(256, 0, 2, 5)
+    try:
+        run_w4a8_parity(custom_spec("w4_wide", 700, 384, N, [0, 384], [0, N], False, "int8", seed=83))
+    finally:
+        B.segquant_set_tuning(0, 0, 0, 0)
+
+
 def test_w4a8_tokens_of_very_different_magnitude_and_degenerate_rows():
     """Per-token scales: tokens spread over five orders of magnitude, an all-zero token, a token without
     negative values; fp32 input."""
