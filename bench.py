@@ -911,10 +911,10 @@ def run_ours(args):
 # prefix of the GEMM kernel source the counters were taken with; once that file has changed the figure is stale
 # and the bench prints null.
 GEMM_DRAM_TRAFFIC = {
-    "sd3_mmdit": {"bytes": 41490688 + 39781120 + 23208192 + 56429568 + 123241216 + 15425024, "source_tag": "de837fa16b5dbafb",
+    "sd3_mmdit": {"bytes": 41489920 + 39200512 + 23266048 + 59767040 + 122890496 + 14484224, "source_tag": "377849a5a34f92d9",
                   "from": "ncu --set full of the three GEMM launches of one eager step (bench.py --workload sd3_mmdit "
                           "--profile-steps 4); below the algorithmic bytes because part of Y is still in L2 when a kernel ends"},
-    "dit_xl2": {"bytes": 12757760 + 17152 + 24236800 + 0, "source_tag": "de837fa16b5dbafb",
+    "dit_xl2": {"bytes": 12758272 + 15872 + 24237312 + 0, "source_tag": "377849a5a34f92d9",
                 "from": "ncu --set full of the two GEMM launches of one eager step (bench.py --workload dit_xl2 "
                         "--profile-steps 4); operands partly L2-resident from the quantize pass, Y stays in L2"},
 }
